@@ -1,0 +1,116 @@
+"""ctypes front end of ``hgemm_oracle.c`` -- TEST INFRASTRUCTURE, not product code.
+
+The arithmetic lives in the C file; this module only compiles it with gcc, loads
+it, and marshals numpy arrays.  fp16 matrices travel as ``uint16`` bit patterns so
+that no half-precision type of numpy, the compiler or CUDA takes part in the
+oracle's arithmetic (paper section 2.3, Eq. 1: a CPU reference on widened inputs;
+here widened to fp64).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hgemm_oracle.c")
+_LIB = os.path.join(_HERE, "libhgemm_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP over rows only). Returns the .so path."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            cmd = ["gcc", "-O2", "-fopenmp", "-fno-fast-math", "-ffp-contract=off", "-shared", "-fPIC",
+                   "-o", tmp, _SRC, "-lm"]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        i64, p = ctypes.c_int64, ctypes.c_void_p
+        lib.oracle_f16_bits_to_f64.restype = ctypes.c_double
+        lib.oracle_f16_bits_to_f64.argtypes = [ctypes.c_uint16]
+        lib.oracle_f64_to_f16_bits_rne.restype = ctypes.c_uint16
+        lib.oracle_f64_to_f16_bits_rne.argtypes = [ctypes.c_double]
+        lib.oracle_f64_to_f16_bits_rne_array.restype = None
+        lib.oracle_f64_to_f16_bits_rne_array.argtypes = [i64, p, p]
+        lib.oracle_f16_bits_to_f64_array.restype = None
+        lib.oracle_f16_bits_to_f64_array.argtypes = [i64, p, p]
+        lib.oracle_hgemm_full.restype = ctypes.c_int
+        lib.oracle_hgemm_full.argtypes = [i64, i64, i64, p, i64, p, i64, p]
+        lib.oracle_hgemm_sampled.restype = ctypes.c_int
+        lib.oracle_hgemm_sampled.argtypes = [i64, p, i64, p, i64, i64, p, p, p]
+        lib.oracle_max_threads.restype = ctypes.c_int
+        lib.oracle_max_threads.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def _bits(x: np.ndarray) -> np.ndarray:
+    """Accept uint16 bit patterns (or a float16 array, reinterpreted) as C-contiguous uint16."""
+    x = np.asarray(x)
+    if x.dtype == np.float16:
+        x = x.view(np.uint16)
+    if x.dtype != np.uint16:
+        raise TypeError(f"fp16 matrices are passed as uint16 bit patterns, got {x.dtype}")
+    return np.ascontiguousarray(x)
+
+
+def max_threads() -> int:
+    return int(_load().oracle_max_threads())
+
+
+def f16_bits_to_f64(bits) -> np.ndarray:
+    b = _bits(np.atleast_1d(bits))
+    out = np.empty(b.shape, dtype=np.float64)
+    _load().oracle_f16_bits_to_f64_array(b.size, b.ctypes.data, out.ctypes.data)
+    return out
+
+
+def f64_to_f16_bits(x) -> np.ndarray:
+    v = np.ascontiguousarray(np.atleast_1d(x), dtype=np.float64)
+    out = np.empty(v.shape, dtype=np.uint16)
+    _load().oracle_f64_to_f16_bits_rne_array(v.size, v.ctypes.data, out.ctypes.data)
+    return out
+
+
+def hgemm_full(a_bits, b_bits) -> np.ndarray:
+    """C_ref (fp64, M x N) for A (M x K) and B (N x K), both as fp16 bit patterns."""
+    a, b = _bits(a_bits), _bits(b_bits)
+    if a.ndim != 2 or b.ndim != 2 or a.shape[1] != b.shape[1]:
+        raise ValueError(f"need A (M,K) and B (N,K); got {a.shape} and {b.shape}")
+    m, k = a.shape
+    n = b.shape[0]
+    c = np.empty((m, n), dtype=np.float64)
+    _load().oracle_hgemm_full(m, n, k, a.ctypes.data, k, b.ctypes.data, k, c.ctypes.data)
+    return c
+
+
+def hgemm_sampled(a_bits, b_bits, ii, jj) -> np.ndarray:
+    """C_ref[ii[t], jj[t]] (fp64) -- ii indexes rows of ``a_bits``, jj rows of ``b_bits``."""
+    a, b = _bits(a_bits), _bits(b_bits)
+    if a.ndim != 2 or b.ndim != 2 or a.shape[1] != b.shape[1]:
+        raise ValueError(f"need A (*,K) and B (*,K); got {a.shape} and {b.shape}")
+    ii = np.ascontiguousarray(ii, dtype=np.int64)
+    jj = np.ascontiguousarray(jj, dtype=np.int64)
+    if ii.shape != jj.shape or ii.ndim != 1:
+        raise ValueError("ii and jj must be 1-D and of equal length")
+    if ii.size and (ii.min() < 0 or ii.max() >= a.shape[0] or jj.min() < 0 or jj.max() >= b.shape[0]):
+        raise IndexError("sample index out of range")
+    out = np.empty(ii.shape, dtype=np.float64)
+    _load().oracle_hgemm_sampled(a.shape[1], a.ctypes.data, a.shape[1], b.ctypes.data, b.shape[1],
+                                 ii.size, ii.ctypes.data, jj.ctypes.data, out.ctypes.data)
+    return out

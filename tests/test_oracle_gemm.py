@@ -1,0 +1,154 @@
+"""Pins for the oracle's triple loop (CPU only).
+
+Each test fixes the loop against something the mathematics decides, chosen so that
+a dropped term, a wrong index or a transposed operand fails at least one:
+exact int64 arithmetic on integer inputs, identity / permutation / rank-1 closed
+forms on non-square shapes, a library fp64 matmul, exact rationals on tiny shapes.
+"""
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_02551_b200 import inputs
+
+
+def _f16_exact(bits):
+    """Independent decode: numpy float16 -> python float (exact)."""
+    return np.asarray(bits, dtype=np.uint16).view(np.float16).astype(np.float64)
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (64, 192, 320), (37, 53, 1000), (8, 16, 12288)])
+def test_integer_inputs_match_int64(oracle_lib, M, N, K):
+    a, b = inputs.make_ab(M, N, K, dist="int5")
+    ai = a.to(torch.int64).numpy()
+    bi = b.to(torch.int64).numpy()
+    want = ai @ bi.T                                       # exact integer arithmetic
+    got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    assert got.shape == (M, N)
+    assert np.array_equal(got, want.astype(np.float64))
+    assert np.abs(want).max() > 0
+    # the rounded result is the integer itself wherever it is representable
+    small = np.abs(want) <= 2048
+    assert np.array_equal(_f16_exact(oracle_lib.f64_to_f16_bits(got.ravel()))[small.ravel()],
+                          want.astype(np.float64).ravel()[small.ravel()])
+
+
+def test_identity_returns_b_transposed(oracle_lib):
+    K = M = 96
+    N = 40
+    b = inputs.draw(7, inputs.TAG_B, N, K, "uniform")
+    eye = torch.eye(M, K, dtype=torch.float16)
+    got = oracle_lib.hgemm_full(inputs.bits(eye), inputs.bits(b))
+    assert np.array_equal(got, b.double().numpy().T)
+
+
+def test_permutation_selects_columns(oracle_lib):
+    M, N, K = 50, 70, 90
+    rng = np.random.default_rng(3)
+    pi = rng.permutation(K)[:M]
+    a = torch.zeros(M, K, dtype=torch.float16)
+    a[torch.arange(M), torch.from_numpy(pi)] = 1.0
+    b = inputs.draw(11, inputs.TAG_B, N, K, "uniform")
+    got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    want = b.double().numpy()[:, pi].T                     # C[i][j] = B[j][pi(i)]
+    assert np.array_equal(got, want)
+
+
+def test_rank1_one_hot_k(oracle_lib):
+    M, N, K, k0 = 33, 65, 128, 77
+    u = inputs.draw(5, 1, M, 1, "uniform")[:, 0]
+    v = inputs.draw(5, 2, N, 1, "uniform")[:, 0]
+    a = torch.zeros(M, K, dtype=torch.float16)
+    b = torch.zeros(N, K, dtype=torch.float16)
+    a[:, k0] = u
+    b[:, k0] = v
+    got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    want = np.outer(u.double().numpy(), v.double().numpy())  # exact: 22-bit products
+    assert np.array_equal(got, want)
+    got16 = oracle_lib.f64_to_f16_bits(got.ravel())
+    want16 = want.astype(np.float16).view(np.uint16).ravel()
+    assert np.array_equal(got16, want16)
+
+
+@pytest.mark.parametrize("K", [64, 4096, 12288])
+def test_rank1_constant_along_k(oracle_lib, K):
+    M, N = 24, 40
+    vals = np.array([0.5, 1.0, 2.0, -0.5, -1.0, -2.0])
+    rng = np.random.default_rng(K)
+    u = rng.choice(vals, M)
+    v = rng.choice(vals, N)
+    a = torch.from_numpy(np.repeat(u[:, None], K, 1)).to(torch.float16)
+    b = torch.from_numpy(np.repeat(v[:, None], K, 1)).to(torch.float16)
+    got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    assert np.array_equal(got, K * np.outer(u, v))         # every partial sum is exact
+
+
+@pytest.mark.parametrize("dist", ["uniform", "normal"])
+def test_library_fp64_matmul(oracle_lib, dist):
+    M, N, K = 70, 90, 2048
+    a, b = inputs.make_ab(M, N, K, dist=dist)
+    got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    want = torch.matmul(a.double(), b.double().T).numpy()  # other summation order, fp64
+    scale = (a.double().abs() @ b.double().abs().T).numpy()
+    assert np.all(np.abs(got - want) <= 1e-12 * scale + 1e-300)
+
+
+def test_tiny_shapes_exact_rationals(oracle_lib):
+    for (M, N, K) in [(1, 1, 1), (2, 3, 5), (4, 7, 8), (8, 8, 8), (3, 2, 17)]:
+        a, b = inputs.make_ab(M, N, K, dist="uniform", seed=100 + M + N + K)
+        af = [[Fraction(float(x)) for x in row] for row in a.tolist()]
+        bf = [[Fraction(float(x)) for x in row] for row in b.tolist()]
+        got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+        for i in range(M):
+            for j in range(N):
+                exact = sum(af[i][k] * bf[j][k] for k in range(K))
+                # K <= 17 terms of <= 22 bits each: the fp64 sum is exact
+                assert Fraction(float(got[i, j])) == exact, (M, N, K, i, j)
+
+
+def test_sampled_equals_full_and_handles_gathered_rows(oracle_lib):
+    M, N, K = 45, 77, 256
+    a, b = inputs.make_ab(M, N, K)
+    full = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    ii, jj, row, col = inputs.sample_indices(99, M, N, n=500)
+    got = oracle_lib.hgemm_sampled(inputs.bits(a), inputs.bits(b), ii, jj)
+    assert np.array_equal(got, full[ii, jj])
+    # gathered form: only the needed rows are drawn
+    ui, inv_i = np.unique(ii, return_inverse=True)
+    uj, inv_j = np.unique(jj, return_inverse=True)
+    s = inputs.shape_seed(M, N, K)
+    ag = inputs.draw(s, inputs.TAG_A, M, K, row_index=ui)
+    bg = inputs.draw(s, inputs.TAG_B, N, K, row_index=uj)
+    assert torch.equal(ag, a[torch.from_numpy(ui)])
+    got2 = oracle_lib.hgemm_sampled(inputs.bits(ag), inputs.bits(bg), inv_i, inv_j)
+    assert np.array_equal(got2, got)
+    with pytest.raises(IndexError):
+        oracle_lib.hgemm_sampled(inputs.bits(a), inputs.bits(b), [M], [0])
+
+
+def test_empty_and_degenerate(oracle_lib):
+    z = oracle_lib.hgemm_full(np.zeros((0, 8), np.uint16), np.zeros((5, 8), np.uint16))
+    assert z.shape == (0, 5)
+    z = oracle_lib.hgemm_full(np.zeros((3, 0), np.uint16), np.zeros((5, 0), np.uint16))
+    assert z.shape == (3, 5) and not z.any()               # empty sum = 0
+    with pytest.raises(ValueError):
+        oracle_lib.hgemm_full(np.zeros((3, 4), np.uint16), np.zeros((5, 6), np.uint16))
+    with pytest.raises(TypeError):
+        oracle_lib.hgemm_full(np.zeros((3, 4), np.float32), np.zeros((5, 4), np.float32))
+
+
+def test_paper_style_binary_exact_match(oracle_lib):
+    """Section 2.3 "Exact Match with binary Inputs": {0,1} inputs give non-negative integer
+    sums; every entry below 2048 is exactly representable in fp16."""
+    M, N, K = 64, 64, 8192
+    p = inputs.binary_p(K)
+    a, b = inputs.make_ab(M, N, K, dist="binary", p=p)
+    got = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    want = (a.to(torch.int64) @ b.to(torch.int64).T).numpy()
+    assert np.array_equal(got, want)
+    frac_checkable = np.mean((want > 0) & (want < 2048))
+    assert frac_checkable > 0.9
+    r16 = _f16_exact(oracle_lib.f64_to_f16_bits(got.ravel())).reshape(M, N)
+    assert np.array_equal(r16[want < 2048], want[want < 2048].astype(np.float64))
