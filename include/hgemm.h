@@ -1,0 +1,147 @@
+/*
+ * hgemm.h -- C ABI of the B200 (sm_100a) half-precision GEMM library.
+ *
+ * Operation (paper section 2.1 "HGEMM": C = alpha*A*B + beta*C with alpha = 1,
+ * beta = 0; operand layout of the "TN" baseline, appendix Listing 6):
+ *
+ *     C[i][j] = fp16_rn( sum_{k<K} A[i][k] * B[j][k] ),   i < M, j < N
+ *
+ *   A : M x K fp16, row-major, dense (row stride K)           -- device memory
+ *   B : N x K fp16, K-contiguous (the K x N operand stored     -- device memory
+ *       column-major), dense (row stride K)
+ *   C : M x N fp16, row-major, dense (row stride N)            -- device memory
+ *
+ * Products are exact, sums are accumulated in fp32 on the tensor cores
+ * (the paper allows fp16 or fp32 accumulators, section 1), and each result is
+ * rounded once to fp16, round-to-nearest-even.  C is overwritten, never read.
+ *
+ * Conventions
+ *   - All functions return a status; nothing throws across the boundary; out
+ *     parameters are written only on HGEMM_OK.
+ *   - Pointers passed to hgemm_run are DEVICE pointers on the context's device,
+ *     16-byte aligned; the caller owns A, B, C; A and B must not overlap C.
+ *   - Shapes: M, N, K >= 1, K % 8 == 0 and N % 8 == 0 (rows must be multiples of
+ *     16 bytes); anything else makes hgemm_plan return HGEMM_ERR_UNSUPPORTED.
+ *     There is no fallback path.
+ *   - hgemm_run is asynchronous on the given stream.  It creates no stream,
+ *     allocates nothing and never synchronises (the timing rules of paper
+ *     section 2.4 "Avoiding Timing Measurement Hacking" forbid side streams);
+ *     its return value is the launch status only.  The context's device must be
+ *     the calling thread's current device.
+ *   - A plan owns its split-K workspace: one plan must not run on two streams at
+ *     the same time.  Plans are not thread-safe; use one per thread.
+ */
+#ifndef HGEMM_H_
+#define HGEMM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hgemm_ctx_s hgemm_ctx_t;   /* opaque; one per device; owns its plans */
+typedef struct hgemm_plan_s hgemm_plan_t; /* opaque; owned by its context */
+
+typedef enum {
+    HGEMM_OK = 0,
+    HGEMM_ERR_INVALID_ARG = 1, /* null pointer, misaligned pointer, non-positive size */
+    HGEMM_ERR_UNSUPPORTED = 2, /* shape or configuration the kernels cannot run */
+    HGEMM_ERR_ALLOC = 3,       /* host or device allocation failed */
+    HGEMM_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (see hgemm_last_cuda_error) */
+    HGEMM_ERR_ARCH = 5,        /* the device is not compute capability 10.0 */
+    HGEMM_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (see hgemm_last_device_status) */
+} hgemm_status_t;
+
+/* Kernel families (section 5.1 of the paper picks a different kernel structure
+ * for small and for large shapes; the families here are this library's own). */
+enum {
+    HGEMM_FAMILY_UMMA_1CTA = 0, /* persistent, warp-specialised, 128 x block_n tiles, one CTA per tile */
+    HGEMM_FAMILY_UMMA_2CTA = 1  /* the same with CTA pairs: 256 x block_n tiles, B split across the pair */
+};
+
+enum {
+    HGEMM_EPILOGUE_DIRECT = 0, /* registers -> 16-byte global stores */
+    HGEMM_EPILOGUE_TMA = 1     /* registers -> swizzled shared memory -> TMA store */
+};
+
+/* One point of the per-shape configuration space (the paper's BM/BN/BK, stage
+ * count and block-swizzle stride of sections 5.2 and 6, plus split-K). */
+typedef struct {
+    int32_t family;       /* HGEMM_FAMILY_* */
+    int32_t block_m;      /* 128 (1-CTA) or 256 (2-CTA pair) */
+    int32_t block_n;      /* multiple of 32 in [32, 256] */
+    int32_t block_k;      /* 64 (one 128-byte swizzle span of fp16) */
+    int32_t stages;       /* shared-memory ring depth, 2..12, bounded by shared memory */
+    int32_t split_k;      /* >= 1; K slices reduced in slice order (deterministic) */
+    int32_t raster_group; /* m-tiles per raster group (>= 1): tile order for L2 reuse */
+    int32_t epilogue;     /* HGEMM_EPILOGUE_* (split_k > 1 always finishes with direct stores) */
+    int32_t reserved[8];  /* must be zero */
+} hgemm_config_t;
+
+/* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the
+ * device has compute capability 10.0.  Allocates a 4-byte device status word. */
+hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device);
+
+/* Free the context, every plan it still owns and their workspaces. */
+hgemm_status_t hgemm_destroy(hgemm_ctx_t *ctx);
+
+/* Plan one (M, N, K): picks a configuration (tuned table, else heuristic) and
+ * allocates the split-K workspace if the configuration needs one.  May call
+ * cudaMalloc/cudaMemset (synchronising); call it outside timed regions and
+ * outside stream capture. */
+hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_plan_t **out);
+
+/* Launch C = A * B^T for the plan's shape on `stream` (a cudaStream_t, may be
+ * NULL for the default stream).  A, B, C: device pointers as described above. */
+hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream);
+
+/* Free one plan early (hgemm_destroy frees the rest). */
+hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan);
+
+/* Read / override the plan's configuration (tuner, tests).  set_config returns
+ * HGEMM_ERR_UNSUPPORTED, leaving the plan unchanged, if the configuration is
+ * illegal for the shape or does not fit shared/tensor memory; it may reallocate
+ * the workspace (synchronising). */
+hgemm_status_t hgemm_plan_get_config(const hgemm_plan_t *plan, hgemm_config_t *out);
+hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *cfg);
+
+/* The heuristic the planner falls back to, as a pure host function (no GPU
+ * needed): configuration for (M, N, K) on a device with `num_sms` SMs. */
+hgemm_status_t hgemm_heuristic_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
+
+/* Check a configuration against a shape without a GPU: HGEMM_OK if legal. */
+hgemm_status_t hgemm_validate_config(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg);
+
+/* Dynamic shared memory (bytes) and split-K workspace (bytes) a configuration needs. */
+int64_t hgemm_config_smem_bytes(const hgemm_config_t *cfg);
+int64_t hgemm_config_workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg);
+
+/* Number of kernels the last hgemm_run of this plan launched (1). */
+int32_t hgemm_plan_launches_per_run(const hgemm_plan_t *plan);
+
+/* Every device-side wait is bounded; when one runs out the kernel records
+ * (role << 24 | barrier index << 8 | stage) in the context's status word, drains
+ * and returns.  This call synchronises the device, reads the word into *code
+ * (0 = no event), clears it, and returns HGEMM_ERR_TIMEOUT if it was non-zero. */
+hgemm_status_t hgemm_last_device_status(hgemm_ctx_t *ctx, uint32_t *code);
+
+/* Wait budget of the bounded waits, in SM clock cycles (default 2e9, about a
+ * second).  Affects plans created afterwards and later hgemm_run calls. */
+hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles);
+
+/* Test hook for the timeout path: launches one small kernel on `stream` whose
+ * only wait is on a barrier that nothing signals, with the context's wait
+ * budget.  The kernel returns by itself; hgemm_last_device_status then reports
+ * HGEMM_ERR_TIMEOUT.  Nothing faults or hangs. */
+hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
+
+/* cudaError_t (as int) of the last failing CUDA call made through this context. */
+int32_t hgemm_last_cuda_error(const hgemm_ctx_t *ctx);
+
+const char *hgemm_status_string(hgemm_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HGEMM_H_ */

@@ -1,0 +1,422 @@
+// C ABI of the HGEMM library (see include/hgemm.h): contexts, plans, tensor maps, launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/hgemm.h"
+#include "hgemm_kernel.cuh"
+#include "hgemm_planner.h"
+
+using hgemm_dev::KernelParams;
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct hgemm_ctx_s {
+    int device = 0;
+    int num_sms = 0;
+    uint32_t *d_status = nullptr;
+    long long wait_budget = 2000000000LL;
+    encode_tiled_fn encode = nullptr;
+    int last_cuda_error = 0;
+    std::vector<hgemm_plan_s *> plans;
+};
+
+struct hgemm_plan_s {
+    hgemm_ctx_s *ctx = nullptr;
+    int64_t M = 0, N = 0, K = 0;
+    hgemm_config_t cfg;
+    KernelParams params;
+    int grid = 0;
+    int smem = 0;
+    void *workspace = nullptr;
+    int64_t workspace_bytes = 0;
+    uint32_t *counters = nullptr;
+    int64_t counter_bytes = 0;
+    // tensor maps depend on the pointers: cached for the last (A, B, C) seen
+    const void *cached_a = nullptr, *cached_b = nullptr;
+    void *cached_c = nullptr;
+    CUtensorMap tmap_a, tmap_b, tmap_c;
+};
+
+namespace {
+
+hgemm_status_t cuda_fail(hgemm_ctx_s *ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda_error = int(e);
+    (void)cudaGetLastError();
+    return HGEMM_ERR_CUDA;
+}
+
+int32_t pow2_at_least(int32_t x)
+{
+    int32_t p = 32;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+uint32_t make_idesc(int m, int n)
+{
+    // tcgen05 instruction descriptor, kind::f16: D = fp32, A = B = fp16, both K-major, dense
+    uint32_t d = 0;
+    d |= 1u << 4;                      // [4,6)   D format: 1 = fp32
+    d |= 0u << 7;                      // [7,10)  A format: 0 = fp16
+    d |= 0u << 10;                     // [10,13) B format: 0 = fp16
+    d |= 0u << 15;                     // [15]    A major: 0 = K
+    d |= 0u << 16;                     // [16]    B major: 0 = K
+    d |= uint32_t(n >> 3) << 17;       // [17,23) N >> 3
+    d |= uint32_t(m >> 4) << 24;       // [24,29) M >> 4
+    return d;
+}
+
+// Applies a validated configuration to a plan: derived kernel parameters, workspace.
+hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
+{
+    hgemm_ctx_s *ctx = pl->ctx;
+    const int cg = hgemm_host::cta_group_of(cfg);
+    const int64_t ws = hgemm_host::workspace_bytes(pl->M, pl->N, pl->K, cfg);
+    const int64_t cb = hgemm_host::counter_bytes(pl->M, pl->N, cfg);
+    if (ws > pl->workspace_bytes) {
+        if (pl->workspace) cudaFree(pl->workspace);
+        pl->workspace = nullptr;
+        pl->workspace_bytes = 0;
+        cudaError_t e = cudaMalloc(&pl->workspace, size_t(ws));
+        if (e != cudaSuccess) {
+            cuda_fail(ctx, e);
+            return HGEMM_ERR_ALLOC;
+        }
+        pl->workspace_bytes = ws;
+    }
+    if (cb > pl->counter_bytes) {
+        if (pl->counters) cudaFree(pl->counters);
+        pl->counters = nullptr;
+        pl->counter_bytes = 0;
+        cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&pl->counters), size_t(cb));
+        if (e != cudaSuccess) {
+            cuda_fail(ctx, e);
+            return HGEMM_ERR_ALLOC;
+        }
+        pl->counter_bytes = cb;
+    }
+    if (pl->counters) {
+        cudaError_t e = cudaMemset(pl->counters, 0, size_t(pl->counter_bytes));
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+
+    pl->cfg = cfg;
+    KernelParams &p = pl->params;
+    std::memset(&p, 0, sizeof(p));
+    p.M = int32_t(pl->M);
+    p.N = int32_t(pl->N);
+    p.K = int32_t(pl->K);
+    p.tiles_m = int32_t((pl->M + 128 * cg - 1) / (128 * cg));
+    p.tiles_n = int32_t((pl->N + cfg.block_n - 1) / cfg.block_n);
+    p.split_k = cfg.split_k;
+    p.total_work = p.tiles_m * p.tiles_n * p.split_k;
+    p.kblocks = int32_t((pl->K + 63) / 64);
+    p.block_n = cfg.block_n;
+    p.stages = cfg.stages;
+    p.raster_group = std::min(cfg.raster_group, p.tiles_m);
+    p.tmem_cols = pow2_at_least(2 * cfg.block_n);
+    p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1) ? 1 : 0;
+    p.idesc = make_idesc(128 * cg, cfg.block_n);
+    p.workspace = static_cast<float *>(pl->workspace);
+    p.counters = pl->counters;
+    p.status = ctx->d_status;
+    p.C = nullptr;
+    p.wait_budget = ctx->wait_budget;
+    const int units = std::max(1, ctx->num_sms / cg);
+    pl->grid = cg * std::min(p.total_work, units);
+    // Always ask for the whole opt-in shared memory: it keeps a second CTA off the SM, so two
+    // CTAs can never wait on each other's tensor-memory allocation.
+    pl->smem = int(hgemm_host::kSmemOptInBytes);
+    pl->cached_a = pl->cached_b = nullptr;
+    pl->cached_c = nullptr;
+    return HGEMM_OK;
+}
+
+bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_inner,
+               uint32_t box_outer, CUtensorMapSwizzle swizzle)
+{
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {inner * 2};   // bytes between rows
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda_error = int(r);
+        return false;
+    }
+    return true;
+}
+
+} // namespace
+
+extern "C" {
+
+const char *hgemm_status_string(hgemm_status_t s)
+{
+    switch (s) {
+    case HGEMM_OK: return "ok";
+    case HGEMM_ERR_INVALID_ARG: return "invalid argument";
+    case HGEMM_ERR_UNSUPPORTED: return "unsupported shape or configuration";
+    case HGEMM_ERR_ALLOC: return "allocation failed";
+    case HGEMM_ERR_CUDA: return "CUDA call failed";
+    case HGEMM_ERR_ARCH: return "device is not compute capability 10.0";
+    case HGEMM_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
+{
+    if (!out || device < 0) return HGEMM_ERR_INVALID_ARG;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (device >= count) return HGEMM_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    if (prop.major != 10 || prop.minor != 0) return HGEMM_ERR_ARCH;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    e = cudaSetDevice(device);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+
+    hgemm_ctx_s *ctx = new (std::nothrow) hgemm_ctx_s;
+    if (!ctx) return HGEMM_ERR_ALLOC;
+    ctx->device = device;
+    ctx->num_sms = prop.multiProcessorCount;
+    hgemm_status_t st = HGEMM_OK;
+    do {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+            st = cuda_fail(ctx, e);
+            break;
+        }
+        ctx->encode = reinterpret_cast<encode_tiled_fn>(fn);
+        e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 256);
+        if (e != cudaSuccess) {
+            cuda_fail(ctx, e);
+            st = HGEMM_ERR_ALLOC;
+            break;
+        }
+        e = cudaMemset(ctx->d_status, 0, 256);
+        if (e != cudaSuccess) {
+            st = cuda_fail(ctx, e);
+            break;
+        }
+        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(hgemm_host::kSmemOptInBytes));
+        if (e != cudaSuccess) {
+            st = cuda_fail(ctx, e);
+            break;
+        }
+        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 int(hgemm_host::kSmemOptInBytes));
+        if (e != cudaSuccess) {
+            st = cuda_fail(ctx, e);
+            break;
+        }
+    } while (false);
+    cudaSetDevice(prev);
+    if (st != HGEMM_OK) {
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        delete ctx;
+        return st;
+    }
+    *out = ctx;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan)
+{
+    if (!plan) return HGEMM_ERR_INVALID_ARG;
+    hgemm_ctx_s *ctx = plan->ctx;
+    if (ctx) {
+        auto it = std::find(ctx->plans.begin(), ctx->plans.end(), plan);
+        if (it != ctx->plans.end()) ctx->plans.erase(it);
+    }
+    if (plan->workspace) cudaFree(plan->workspace);
+    if (plan->counters) cudaFree(plan->counters);
+    delete plan;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_destroy(hgemm_ctx_t *ctx)
+{
+    if (!ctx) return HGEMM_ERR_INVALID_ARG;
+    while (!ctx->plans.empty()) hgemm_plan_destroy(ctx->plans.back());
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_heuristic_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out)
+{
+    if (!out) return HGEMM_ERR_INVALID_ARG;
+    hgemm_config_t c;
+    const hgemm_status_t s = hgemm_host::heuristic(M, N, K, num_sms, &c);
+    if (s == HGEMM_OK) *out = c;
+    return s;
+}
+
+hgemm_status_t hgemm_validate_config(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg)
+{
+    if (!cfg) return HGEMM_ERR_INVALID_ARG;
+    return hgemm_host::validate(M, N, K, *cfg);
+}
+
+int64_t hgemm_config_smem_bytes(const hgemm_config_t *cfg)
+{
+    return cfg ? hgemm_host::smem_bytes(*cfg) : -1;
+}
+
+int64_t hgemm_config_workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg)
+{
+    return cfg ? hgemm_host::workspace_bytes(M, N, K, *cfg) + hgemm_host::counter_bytes(M, N, *cfg) : -1;
+}
+
+hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_plan_t **out)
+{
+    if (!ctx || !out) return HGEMM_ERR_INVALID_ARG;
+    hgemm_status_t s = hgemm_host::validate_shape(M, N, K);
+    if (s != HGEMM_OK) return s;
+    hgemm_config_t cfg;
+    if (!hgemm_host::table_lookup(M, N, K, &cfg)) {
+        s = hgemm_host::heuristic(M, N, K, ctx->num_sms, &cfg);
+        if (s != HGEMM_OK) return s;
+    }
+    hgemm_plan_s *pl = new (std::nothrow) hgemm_plan_s;
+    if (!pl) return HGEMM_ERR_ALLOC;
+    pl->ctx = ctx;
+    pl->M = M;
+    pl->N = N;
+    pl->K = K;
+    s = apply_config(pl, cfg);
+    if (s != HGEMM_OK) {
+        if (pl->workspace) cudaFree(pl->workspace);
+        if (pl->counters) cudaFree(pl->counters);
+        delete pl;
+        return s;
+    }
+    ctx->plans.push_back(pl);
+    *out = pl;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_plan_get_config(const hgemm_plan_t *plan, hgemm_config_t *out)
+{
+    if (!plan || !out) return HGEMM_ERR_INVALID_ARG;
+    *out = plan->cfg;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *cfg)
+{
+    if (!plan || !cfg) return HGEMM_ERR_INVALID_ARG;
+    const hgemm_status_t s = hgemm_host::validate(plan->M, plan->N, plan->K, *cfg);
+    if (s != HGEMM_OK) return s;
+    cudaError_t e = cudaDeviceSynchronize();   // the old workspace may still be in use
+    if (e != cudaSuccess) return cuda_fail(plan->ctx, e);
+    return apply_config(plan, *cfg);
+}
+
+int32_t hgemm_plan_launches_per_run(const hgemm_plan_t *plan)
+{
+    return plan ? 1 : 0;
+}
+
+hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream)
+{
+    if (!plan || !A || !B || !C) return HGEMM_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15u)
+        return HGEMM_ERR_INVALID_ARG;
+    hgemm_ctx_s *ctx = plan->ctx;
+    const hgemm_config_t &cfg = plan->cfg;
+    const int cg = hgemm_host::cta_group_of(cfg);
+
+    if (A != plan->cached_a || B != plan->cached_b || C != plan->cached_c) {
+        const uint64_t M = uint64_t(plan->M), N = uint64_t(plan->N), K = uint64_t(plan->K);
+        if (!encode_2d(ctx, &plan->tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
+        if (!encode_2d(ctx, &plan->tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
+            return HGEMM_ERR_CUDA;
+        if (!encode_2d(ctx, &plan->tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return HGEMM_ERR_CUDA;
+        plan->cached_a = A;
+        plan->cached_b = B;
+        plan->cached_c = C;
+    }
+    plan->params.C = static_cast<__half *>(C);
+    plan->params.wait_budget = ctx->wait_budget;
+
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof(lc));
+    lc.gridDim = dim3(unsigned(plan->grid), 1, 1);
+    lc.blockDim = dim3(hgemm_dev::kThreads, 1, 1);
+    lc.dynamicSmemBytes = size_t(plan->smem);
+    lc.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = unsigned(cg);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    cudaError_t e;
+    if (cg == 1)
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, plan->tmap_a, plan->tmap_b, plan->tmap_c, plan->params);
+    else
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2>, plan->tmap_a, plan->tmap_b, plan->tmap_c, plan->params);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_last_device_status(hgemm_ctx_t *ctx, uint32_t *code)
+{
+    if (!ctx || !code) return HGEMM_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    uint32_t v = 0;
+    e = cudaMemcpy(&v, ctx->d_status, 4, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (v != 0) {
+        e = cudaMemset(ctx->d_status, 0, 4);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    *code = v;
+    return v ? HGEMM_ERR_TIMEOUT : HGEMM_OK;
+}
+
+hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles)
+{
+    if (!ctx || cycles < 1) return HGEMM_ERR_INVALID_ARG;
+    ctx->wait_budget = cycles;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream)
+{
+    if (!ctx) return HGEMM_ERR_INVALID_ARG;
+    hgemm_dev::hgemm_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, ctx->wait_budget);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return HGEMM_OK;
+}
+
+int32_t hgemm_last_cuda_error(const hgemm_ctx_t *ctx)
+{
+    return ctx ? ctx->last_cuda_error : 0;
+}
+
+} // extern "C"

@@ -1,0 +1,167 @@
+// Host-only planner (see hgemm_planner.h).  No CUDA calls in this file.
+#include "hgemm_planner.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+
+namespace hgemm_host {
+
+namespace {
+constexpr int64_t kATileBytes = 128 * 64 * 2;
+constexpr int64_t kStagingBytes = 16384;
+constexpr int64_t kCtrlBytes = 512;
+constexpr int64_t kAlignSlack = 1024;
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+} // namespace
+
+int64_t stage_bytes(const hgemm_config_t &c)
+{
+    return kATileBytes + int64_t(c.block_n / cta_group_of(c)) * 64 * 2;
+}
+
+int64_t smem_bytes(const hgemm_config_t &c)
+{
+    return kAlignSlack + int64_t(c.stages) * stage_bytes(c) + kStagingBytes + kCtrlBytes;
+}
+
+int32_t max_stages(int32_t family, int32_t block_n)
+{
+    hgemm_config_t c;
+    std::memset(&c, 0, sizeof(c));
+    c.family = family;
+    c.block_n = block_n;
+    const int64_t room = kSmemOptInBytes - kAlignSlack - kStagingBytes - kCtrlBytes;
+    return int32_t(std::min<int64_t>(12, room / stage_bytes(c)));
+}
+
+int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c)
+{
+    (void)K;
+    if (c.split_k <= 1) return 0;
+    const int cg = cta_group_of(c);
+    const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
+    return tiles * c.split_k * cg * 128 * int64_t(c.block_n) * 4;
+}
+
+int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c)
+{
+    if (c.split_k <= 1) return 0;
+    const int cg = cta_group_of(c);
+    const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
+    return tiles * cg * 4 * 4;
+}
+
+hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K)
+{
+    if (M < 1 || N < 1 || K < 1) return HGEMM_ERR_INVALID_ARG;
+    if (M > kMaxDim || N > kMaxDim || K > kMaxDim) return HGEMM_ERR_UNSUPPORTED;
+    if ((K % 8) != 0 || (N % 8) != 0) return HGEMM_ERR_UNSUPPORTED;   // rows must be multiples of 16 bytes
+    return HGEMM_OK;
+}
+
+hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c)
+{
+    const hgemm_status_t s = validate_shape(M, N, K);
+    if (s != HGEMM_OK) return s;
+    if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA) return HGEMM_ERR_UNSUPPORTED;
+    const int cg = cta_group_of(c);
+    if (c.block_m != 128 * cg || c.block_k != 64) return HGEMM_ERR_UNSUPPORTED;
+    if (c.block_n < 32 || c.block_n > 256 || (c.block_n % 32) != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (c.stages < 1 || c.stages > 12) return HGEMM_ERR_UNSUPPORTED;
+    if (smem_bytes(c) > kSmemOptInBytes) return HGEMM_ERR_UNSUPPORTED;
+    if (c.split_k < 1 || c.split_k > ceil_div(K, 64)) return HGEMM_ERR_UNSUPPORTED;
+    if (c.raster_group < 1) return HGEMM_ERR_UNSUPPORTED;
+    if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA) return HGEMM_ERR_UNSUPPORTED;
+    for (int i = 0; i < 8; ++i)
+        if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+    const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
+    if (tiles * c.split_k >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
+    if (workspace_bytes(M, N, K, c) > kMaxWorkspaceBytes) return HGEMM_ERR_UNSUPPORTED;
+    return HGEMM_OK;
+}
+
+double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c)
+{
+    // Rough machine model, in SM clock cycles.  Constants are fitted by eye to measurements
+    // on a B200; the tuned table overrides this wherever it has an entry.
+    const double kMacPerClk = 4096.0;        // fp16 MACs per clock per SM
+    const double kSmFillBytesPerClk = 90.0;  // L2 -> one SM's shared memory
+    const double kL2BytesPerClk = 5500.0;    // L2 -> all SMs together
+    const double kHbmBytesPerClk = 3400.0;   // HBM, all SMs together
+    const double kFillLatency = 1800.0;      // first k-block of a work item: TMA round trip
+    const double kLaunch = 3000.0;
+
+    const int cg = cta_group_of(c);
+    const int64_t bm = 128 * cg;
+    const int64_t tiles = ceil_div(M, bm) * ceil_div(N, c.block_n);
+    const int64_t work = tiles * c.split_k;
+    const int64_t units = std::max(1, num_sms / cg);
+    const int64_t waves = ceil_div(work, units);
+    const int64_t kb = ceil_div(K, 64);
+    const int64_t kb_per = ceil_div(kb, c.split_k);
+    const double cta_bytes_kb = double(stage_bytes(c));
+    const double mma_kb = 128.0 * c.block_n * 64.0 / kMacPerClk;
+    const double fill_kb = cta_bytes_kb / kSmFillBytesPerClk;
+    const double concurrent_ctas = double(std::min(work, units)) * cg;
+    const double l2_kb = concurrent_ctas * cta_bytes_kb / kL2BytesPerClk;
+    const double t_kb = std::max(mma_kb, std::max(fill_kb, l2_kb));
+    const double epilogue = 2.5 * c.block_n + 400.0;
+    double t = double(waves) * (double(kb_per) * t_kb + 0.25 * kFillLatency) + 0.75 * kFillLatency + epilogue;
+    double bytes = 2.0 * (double(M) * K + double(N) * K + double(M) * N);
+    if (c.split_k > 1) {
+        const double partial = 128.0 * c.block_n * 4.0;
+        t += partial / 64.0 + double(c.split_k) * partial / 128.0 + 1500.0;   // park + ordered reduce by the last slice
+        bytes += 2.0 * double(work) * cg * partial;
+    }
+    t = std::max(t, bytes / kHbmBytesPerClk);
+    return t + kLaunch;
+}
+
+hgemm_status_t heuristic(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out)
+{
+    const hgemm_status_t s = validate_shape(M, N, K);
+    if (s != HGEMM_OK) return s;
+    if (num_sms < 2) num_sms = 148;
+    static const int32_t kSplits[] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64};
+    const int64_t kb = ceil_div(K, 64);
+    hgemm_config_t best;
+    double best_t = 0.0;
+    bool have = false;
+    for (int family = 0; family < 2; ++family) {
+        const int cg = family == HGEMM_FAMILY_UMMA_2CTA ? 2 : 1;
+        for (int32_t bn = 32; bn <= 256; bn += 32) {
+            if (bn > 32 && bn - 32 >= N) break;   // a wider tile would only add padding
+            for (int32_t split : kSplits) {
+                if (split > kb) break;
+                hgemm_config_t c;
+                std::memset(&c, 0, sizeof(c));
+                c.family = family;
+                c.block_m = 128 * cg;
+                c.block_n = bn;
+                c.block_k = 64;
+                c.split_k = split;
+                c.epilogue = HGEMM_EPILOGUE_DIRECT;
+                c.stages = std::max(1, std::min<int32_t>(max_stages(family, bn), 8));
+                const int64_t units = std::max(1, num_sms / cg);
+                const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, bn);
+                if (split > 1 && tiles * split > 2 * units) break;   // split-K only to fill an under-full machine
+                const double g = std::sqrt(double(units) * bn / (128.0 * cg));
+                c.raster_group = int32_t(std::max<int64_t>(1, std::min<int64_t>(ceil_div(M, 128 * cg), int64_t(g + 0.5))));
+                if (validate(M, N, K, c) != HGEMM_OK) continue;
+                const double t = estimate_cycles(M, N, K, num_sms, c);
+                if (!have || t < best_t) {
+                    best = c;
+                    best_t = t;
+                    have = true;
+                }
+            }
+        }
+    }
+    if (!have) return HGEMM_ERR_UNSUPPORTED;
+    *out = best;
+    return HGEMM_OK;
+}
+
+} // namespace hgemm_host

@@ -1,0 +1,37 @@
+// Host-only planner: legality of a configuration, its resource needs, and the heuristic
+// choice for a shape.  Pure functions, no CUDA calls, so they can be tested without a GPU.
+//
+// The configuration space is the paper's per-shape hyper-parameter space (sections 5.2 and
+// 6: BM/BN/BK, stage count, block-swizzle stride) restated for tcgen05 tiles, plus split-K
+// (which the paper does not use; skinny large-K shapes need it to fill 148 SMs).
+#pragma once
+
+#include <stdint.h>
+
+#include "../../include/hgemm.h"
+
+namespace hgemm_host {
+
+constexpr int64_t kSmemOptInBytes = 232448;   // 227 KB per CTA on sm_100
+constexpr int64_t kMaxWorkspaceBytes = int64_t(2) << 30;
+constexpr int64_t kMaxDim = int64_t(1) << 22;
+
+inline int cta_group_of(const hgemm_config_t &c) { return c.family == HGEMM_FAMILY_UMMA_2CTA ? 2 : 1; }
+
+int64_t stage_bytes(const hgemm_config_t &c);
+int64_t smem_bytes(const hgemm_config_t &c);
+int32_t max_stages(int32_t family, int32_t block_n);
+int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c);
+int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c);
+hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K);
+hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c);
+hgemm_status_t heuristic(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
+
+// Estimated run time (arbitrary but consistent units: SM clock cycles) of a configuration;
+// the heuristic picks the minimum over its candidate set.
+double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c);
+
+// Tuned table (generated on the box by the tuner; may be empty).  Returns true on a hit.
+bool table_lookup(int64_t M, int64_t N, int64_t K, hgemm_config_t *out);
+
+} // namespace hgemm_host

@@ -1,0 +1,210 @@
+"""Thin ctypes binding of ``libhgemm.so`` (the C ABI declared in ``include/hgemm.h``).
+
+Argument marshalling only: every step of the GEMM runs in the library's CUDA
+kernels.  PyTorch appears here only as the owner of device memory and streams
+(``tensor.data_ptr()``, ``torch.cuda.current_stream().cuda_stream``).  There is no
+fallback: if the library is missing or a call fails, this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libhgemm.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(7)
+FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA = 0, 1
+EPILOGUE_DIRECT, EPILOGUE_TMA = 0, 1
+
+# every symbol include/hgemm.h declares
+EXPORTS = [
+    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_plan_destroy",
+    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config",
+    "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
+    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe",
+    "hgemm_last_cuda_error", "hgemm_status_string",
+]
+
+
+class HgemmError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (status {status})")
+
+
+class Config(ctypes.Structure):
+    """Mirror of ``hgemm_config_t``."""
+    _fields_ = [("family", ctypes.c_int32), ("block_m", ctypes.c_int32), ("block_n", ctypes.c_int32),
+                ("block_k", ctypes.c_int32), ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32),
+                ("raster_group", ctypes.c_int32), ("epilogue", ctypes.c_int32), ("reserved", ctypes.c_int32 * 8)]
+
+    def as_dict(self) -> dict:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
+
+    @classmethod
+    def make(cls, family=FAMILY_UMMA_1CTA, block_n=128, stages=4, split_k=1, raster_group=8,
+             epilogue=EPILOGUE_DIRECT) -> "Config":
+        c = cls()
+        c.family = family
+        c.block_m = 256 if family == FAMILY_UMMA_2CTA else 128
+        c.block_n = block_n
+        c.block_k = 64
+        c.stages = stages
+        c.split_k = split_k
+        c.raster_group = raster_group
+        c.epilogue = epilogue
+        return c
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2512_02551_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        i32, i64, p = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
+        cfgp = ctypes.POINTER(Config)
+        sig = {
+            "hgemm_create": (i32, [ctypes.POINTER(p), ctypes.c_int]),
+            "hgemm_destroy": (i32, [p]),
+            "hgemm_plan": (i32, [p, i64, i64, i64, ctypes.POINTER(p)]),
+            "hgemm_run": (i32, [p, p, p, p, p]),
+            "hgemm_plan_destroy": (i32, [p]),
+            "hgemm_plan_get_config": (i32, [p, cfgp]),
+            "hgemm_plan_set_config": (i32, [p, cfgp]),
+            "hgemm_heuristic_config": (i32, [i64, i64, i64, i32, cfgp]),
+            "hgemm_validate_config": (i32, [i64, i64, i64, cfgp]),
+            "hgemm_config_smem_bytes": (i64, [cfgp]),
+            "hgemm_config_workspace_bytes": (i64, [i64, i64, i64, cfgp]),
+            "hgemm_plan_launches_per_run": (i32, [p]),
+            "hgemm_last_device_status": (i32, [p, ctypes.POINTER(ctypes.c_uint32)]),
+            "hgemm_set_wait_budget": (i32, [p, i64]),
+            "hgemm_debug_timeout_probe": (i32, [p, p]),
+            "hgemm_last_cuda_error": (i32, [p]),
+            "hgemm_status_string": (ctypes.c_char_p, [i32]),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().hgemm_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != OK:
+        raise HgemmError(status, what)
+
+
+def heuristic_config(M: int, N: int, K: int, num_sms: int = 148) -> Config:
+    c = Config()
+    _check(lib().hgemm_heuristic_config(M, N, K, num_sms, ctypes.byref(c)), f"hgemm_heuristic_config({M},{N},{K})")
+    return c
+
+
+def validate_config(M: int, N: int, K: int, cfg: Config) -> int:
+    return int(lib().hgemm_validate_config(M, N, K, ctypes.byref(cfg)))
+
+
+def config_smem_bytes(cfg: Config) -> int:
+    return int(lib().hgemm_config_smem_bytes(ctypes.byref(cfg)))
+
+
+def config_workspace_bytes(M: int, N: int, K: int, cfg: Config) -> int:
+    return int(lib().hgemm_config_workspace_bytes(M, N, K, ctypes.byref(cfg)))
+
+
+class Context:
+    """``hgemm_create`` / ``hgemm_destroy``."""
+
+    def __init__(self, device: int = 0):
+        self._h = ctypes.c_void_p()
+        _check(lib().hgemm_create(ctypes.byref(self._h), int(device)), f"hgemm_create(device={device})")
+        self.device = int(device)
+
+    def plan(self, M: int, N: int, K: int) -> "Plan":
+        return Plan(self, M, N, K)
+
+    def set_wait_budget(self, cycles: int) -> None:
+        _check(lib().hgemm_set_wait_budget(self._h, int(cycles)), "hgemm_set_wait_budget")
+
+    def last_device_status(self) -> tuple[int, int]:
+        """(status, code); synchronises the device."""
+        code = ctypes.c_uint32(0)
+        st = lib().hgemm_last_device_status(self._h, ctypes.byref(code))
+        return int(st), int(code.value)
+
+    def debug_timeout_probe(self, stream: int = 0) -> None:
+        _check(lib().hgemm_debug_timeout_probe(self._h, ctypes.c_void_p(stream)), "hgemm_debug_timeout_probe")
+
+    def last_cuda_error(self) -> int:
+        return int(lib().hgemm_last_cuda_error(self._h))
+
+    def close(self) -> None:
+        if self._h:
+            lib().hgemm_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+
+class Plan:
+    """``hgemm_plan`` / ``hgemm_run`` / ``hgemm_plan_destroy``."""
+
+    def __init__(self, ctx: Context, M: int, N: int, K: int):
+        self.ctx = ctx
+        self.shape = (int(M), int(N), int(K))
+        self._h = ctypes.c_void_p()
+        _check(lib().hgemm_plan(ctx._h, int(M), int(N), int(K), ctypes.byref(self._h)), f"hgemm_plan({M},{N},{K})")
+        self._run = lib().hgemm_run
+
+    @property
+    def config(self) -> Config:
+        c = Config()
+        _check(lib().hgemm_plan_get_config(self._h, ctypes.byref(c)), "hgemm_plan_get_config")
+        return c
+
+    def set_config(self, cfg: Config) -> None:
+        _check(lib().hgemm_plan_set_config(self._h, ctypes.byref(cfg)), f"hgemm_plan_set_config({cfg.as_dict()})")
+
+    def try_set_config(self, cfg: Config) -> int:
+        return int(lib().hgemm_plan_set_config(self._h, ctypes.byref(cfg)))
+
+    @property
+    def launches_per_run(self) -> int:
+        return int(lib().hgemm_plan_launches_per_run(self._h))
+
+    def run_ptr(self, a_ptr: int, b_ptr: int, c_ptr: int, stream: int = 0) -> None:
+        """``hgemm_run`` on raw device pointers and a raw ``cudaStream_t``."""
+        st = self._run(self._h, a_ptr, b_ptr, c_ptr, stream)
+        if st != OK:
+            raise HgemmError(st, f"hgemm_run{self.shape}")
+
+    def run(self, A, B, C, stream=None) -> None:
+        """``hgemm_run`` on torch CUDA tensors: A (M,K), B (N,K), C (M,N), fp16, contiguous."""
+        import torch
+        M, N, K = self.shape
+        for t, shp, name in ((A, (M, K), "A"), (B, (N, K), "B"), (C, (M, N), "C")):
+            if t.dtype != torch.float16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shp:
+                raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
+        s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
+        self.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+
+    def close(self) -> None:
+        if self._h and self.ctx._h:
+            lib().hgemm_plan_destroy(self._h)
+        self._h = ctypes.c_void_p()

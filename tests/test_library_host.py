@@ -1,0 +1,92 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, and its planner returns legal configurations."""
+import os
+import re
+
+import pytest
+
+from paper_2512_02551_b200 import build as hbuild
+from paper_2512_02551_b200 import hgemm
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+GRID = [64, 128, 256, 512, 1024, 2048, 4096, 8192, 12288]
+
+
+@pytest.fixture(scope="module")
+def lib():
+    hbuild.build()
+    return hgemm.lib()
+
+
+def test_header_symbols_are_exported(lib):
+    text = open(os.path.join(ROOT, "include", "hgemm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(hgemm_[a-z_]+)\s*\(", text))
+    assert declared == set(hgemm.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    seen = {hgemm.status_string(s) for s in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+
+
+def test_shape_rules(lib):
+    for bad in [(0, 64, 64), (64, 0, 64), (64, 64, 0), (-1, 64, 64)]:
+        with pytest.raises(hgemm.HgemmError) as e:
+            hgemm.heuristic_config(*bad)
+        assert e.value.status == hgemm.ERR_INVALID_ARG
+    for unsup in [(64, 64, 60), (64, 60, 64), (64, 64, 1 << 23)]:
+        with pytest.raises(hgemm.HgemmError) as e:
+            hgemm.heuristic_config(*unsup)
+        assert e.value.status == hgemm.ERR_UNSUPPORTED
+    hgemm.heuristic_config(1, 8, 8)          # smallest legal shape
+
+
+def test_heuristic_is_legal_over_the_grid(lib):
+    for M in GRID:
+        for N in GRID:
+            for K in GRID:
+                c = hgemm.heuristic_config(M, N, K)
+                assert hgemm.validate_config(M, N, K, c) == hgemm.OK, (M, N, K, c.as_dict())
+                assert hgemm.config_smem_bytes(c) <= 232448
+                assert c.split_k <= (K + 63) // 64
+                if c.split_k > 1:
+                    assert hgemm.config_workspace_bytes(M, N, K, c) > 0
+                else:
+                    assert hgemm.config_workspace_bytes(M, N, K, c) == 0
+
+
+def test_validate_rejects_illegal_configs(lib):
+    M = N = K = 1024
+    ok = hgemm.Config.make(block_n=128, stages=4)
+    assert hgemm.validate_config(M, N, K, ok) == hgemm.OK
+    for kw in [dict(block_n=48), dict(block_n=288), dict(block_n=0), dict(stages=0), dict(stages=13),
+               dict(block_n=256, stages=5), dict(split_k=0), dict(split_k=17), dict(raster_group=0),
+               dict(epilogue=2), dict(family=2)]:
+        c = hgemm.Config.make(**{**dict(block_n=128, stages=4), **kw})
+        assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED, kw
+    c = hgemm.Config.make(block_n=128, stages=4)
+    c.block_m = 256                           # wrong for the 1-CTA family
+    assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
+    c = hgemm.Config.make(block_n=128, stages=4)
+    c.reserved[3] = 1
+    assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
+    pair = hgemm.Config.make(family=hgemm.FAMILY_UMMA_2CTA, block_n=256, stages=6)
+    assert hgemm.validate_config(M, N, K, pair) == hgemm.OK
+    assert hgemm.config_smem_bytes(pair) == 1024 + 6 * (16384 + 128 * 128) + 16384 + 512
+
+
+def test_workspace_size(lib):
+    c = hgemm.Config.make(block_n=64, stages=4, split_k=8)
+    # one 128 x 64 fp32 partial per slice + 4 counters of 4 bytes for the single tile
+    assert hgemm.config_workspace_bytes(64, 64, 8192, c) == 8 * 128 * 64 * 4 + 16
+
+
+def test_no_gpu_create_fails_loudly(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(hgemm.HgemmError):
+        hgemm.Context(0)
