@@ -96,6 +96,15 @@ hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hge
  * NULL for the default stream).  A, B, C: device pointers as described above. */
 hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream);
 
+/* The same operation on HOST buffers (paper section 2.3 builds its inputs on the
+ * CPU): copies A and B to device staging owned by the plan, runs, copies C back,
+ * all enqueued on `stream`.  A_host, B_host, C_host are HOST pointers with the
+ * layouts above; with page-locked memory the call is asynchronous and the result
+ * is in C_host once the stream has been synchronised, with pageable memory the
+ * copies block.  The first call on a plan allocates the staging (cudaMalloc,
+ * synchronising): make it outside timed regions.  HGEMM_ERR_ALLOC if that fails. */
+hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void *B_host, void *C_host, void *stream);
+
 /* Free one plan early (hgemm_destroy frees the rest). */
 hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan);
 

@@ -39,10 +39,17 @@ struct hgemm_plan_s {
     int64_t workspace_bytes = 0;
     uint32_t *counters = nullptr;
     int64_t counter_bytes = 0;
-    // tensor maps depend on the pointers: cached for the last (A, B, C) seen
-    const void *cached_a = nullptr, *cached_b = nullptr;
-    void *cached_c = nullptr;
-    CUtensorMap tmap_a, tmap_b, tmap_c;
+    // tensor maps depend on the pointers: a small cache keyed by (A, B, C), round-robin replacement
+    struct MapEntry {
+        const void *a = nullptr, *b = nullptr;
+        void *c = nullptr;
+        CUtensorMap tmap_a, tmap_b, tmap_c;
+    };
+    static constexpr int kMapCache = 64;
+    MapEntry maps[kMapCache];
+    int maps_used = 0, maps_next = 0;
+    // device staging of hgemm_run_host (allocated by its first call)
+    void *stage_a = nullptr, *stage_b = nullptr, *stage_c = nullptr;
 };
 
 namespace {
@@ -136,8 +143,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     // Always ask for the whole opt-in shared memory: it keeps a second CTA off the SM, so two
     // CTAs can never wait on each other's tensor-memory allocation.
     pl->smem = int(hgemm_host::kSmemOptInBytes);
-    pl->cached_a = pl->cached_b = nullptr;
-    pl->cached_c = nullptr;
+    pl->maps_used = pl->maps_next = 0;   // the B box depends on the configuration
     return HGEMM_OK;
 }
 
@@ -250,6 +256,9 @@ hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan)
     }
     if (plan->workspace) cudaFree(plan->workspace);
     if (plan->counters) cudaFree(plan->counters);
+    if (plan->stage_a) cudaFree(plan->stage_a);
+    if (plan->stage_b) cudaFree(plan->stage_b);
+    if (plan->stage_c) cudaFree(plan->stage_c);
     delete plan;
     return HGEMM_OK;
 }
@@ -347,15 +356,29 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     const hgemm_config_t &cfg = plan->cfg;
     const int cg = hgemm_host::cta_group_of(cfg);
 
-    if (A != plan->cached_a || B != plan->cached_b || C != plan->cached_c) {
+    hgemm_plan_s::MapEntry *me = nullptr;
+    for (int i = 0; i < plan->maps_used; ++i) {
+        hgemm_plan_s::MapEntry &e = plan->maps[i];
+        if (e.a == A && e.b == B && e.c == C) {
+            me = &e;
+            break;
+        }
+    }
+    if (!me) {
+        hgemm_plan_s::MapEntry &e = plan->maps[plan->maps_next];
+        e.a = e.b = nullptr;
+        e.c = nullptr;
         const uint64_t M = uint64_t(plan->M), N = uint64_t(plan->N), K = uint64_t(plan->K);
-        if (!encode_2d(ctx, &plan->tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
-        if (!encode_2d(ctx, &plan->tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
+        if (!encode_2d(ctx, &e.tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
+        if (!encode_2d(ctx, &e.tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
             return HGEMM_ERR_CUDA;
-        if (!encode_2d(ctx, &plan->tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return HGEMM_ERR_CUDA;
-        plan->cached_a = A;
-        plan->cached_b = B;
-        plan->cached_c = C;
+        if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return HGEMM_ERR_CUDA;
+        e.a = A;
+        e.b = B;
+        e.c = C;
+        me = &e;
+        plan->maps_next = (plan->maps_next + 1) % hgemm_plan_s::kMapCache;
+        plan->maps_used = std::min(plan->maps_used + 1, int(hgemm_plan_s::kMapCache));
     }
     plan->params.C = static_cast<__half *>(C);
     plan->params.wait_budget = ctx->wait_budget;
@@ -375,9 +398,39 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     lc.numAttrs = 1;
     cudaError_t e;
     if (cg == 1)
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, plan->tmap_a, plan->tmap_b, plan->tmap_c, plan->params);
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, me->tmap_a, me->tmap_b, me->tmap_c, plan->params);
     else
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2>, plan->tmap_a, plan->tmap_b, plan->tmap_c, plan->params);
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2>, me->tmap_a, me->tmap_b, me->tmap_c, plan->params);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void *B_host, void *C_host, void *stream)
+{
+    if (!plan || !A_host || !B_host || !C_host) return HGEMM_ERR_INVALID_ARG;
+    hgemm_ctx_s *ctx = plan->ctx;
+    const size_t a_bytes = size_t(plan->M) * size_t(plan->K) * 2, b_bytes = size_t(plan->N) * size_t(plan->K) * 2,
+                 c_bytes = size_t(plan->M) * size_t(plan->N) * 2;
+    if (!plan->stage_a) {
+        cudaError_t e = cudaMalloc(&plan->stage_a, a_bytes);
+        if (e == cudaSuccess) e = cudaMalloc(&plan->stage_b, b_bytes);
+        if (e == cudaSuccess) e = cudaMalloc(&plan->stage_c, c_bytes);
+        if (e != cudaSuccess) {
+            if (plan->stage_a) cudaFree(plan->stage_a);
+            if (plan->stage_b) cudaFree(plan->stage_b);
+            plan->stage_a = plan->stage_b = plan->stage_c = nullptr;
+            cuda_fail(ctx, e);
+            return HGEMM_ERR_ALLOC;
+        }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(plan->stage_a, A_host, a_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = cudaMemcpyAsync(plan->stage_b, B_host, b_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const hgemm_status_t s = hgemm_run(plan, plan->stage_a, plan->stage_b, plan->stage_c, stream);
+    if (s != HGEMM_OK) return s;
+    e = cudaMemcpyAsync(C_host, plan->stage_c, c_bytes, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;
 }

@@ -19,7 +19,7 @@ EPILOGUE_DIRECT, EPILOGUE_TMA = 0, 1
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
-    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_plan_destroy",
+    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe",
@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_destroy": (i32, [p]),
             "hgemm_plan": (i32, [p, i64, i64, i64, ctypes.POINTER(p)]),
             "hgemm_run": (i32, [p, p, p, p, p]),
+            "hgemm_run_host": (i32, [p, p, p, p, p]),
             "hgemm_plan_destroy": (i32, [p]),
             "hgemm_plan_get_config": (i32, [p, cfgp]),
             "hgemm_plan_set_config": (i32, [p, cfgp]),
@@ -203,6 +204,18 @@ class Plan:
                 raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
         s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
         self.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+
+    def run_host(self, A, B, C, stream=None) -> None:
+        """``hgemm_run_host`` on torch CPU tensors (pinned for an asynchronous call)."""
+        import torch
+        M, N, K = self.shape
+        for t, shp, name in ((A, (M, K), "A"), (B, (N, K), "B"), (C, (M, N), "C")):
+            if t.dtype != torch.float16 or t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shp:
+                raise ValueError(f"{name} must be a contiguous host fp16 tensor of shape {shp}")
+        s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
+        st = lib().hgemm_run_host(self._h, A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+        if st != OK:
+            raise HgemmError(st, f"hgemm_run_host{self.shape}")
 
     def close(self) -> None:
         if self._h and self.ctx._h:

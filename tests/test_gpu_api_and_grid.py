@@ -1,0 +1,111 @@
+"""GPU tests of the C-ABI's error behaviour, the bounded-wait status path, and the full 729-shape grid."""
+import ctypes
+import os
+import time
+
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2512_02551_b200 import hgemm, inputs  # noqa: E402
+
+GRID = [64, 128, 256, 512, 1024, 2048, 4096, 8192, 12288]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    assert torch.cuda.is_available(), "these tests need a B200"
+    c = hgemm.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import gpu_util
+    return gpu_util
+
+
+def test_library_is_loaded_from_the_tree():
+    path = hgemm.LIB_PATH
+    assert os.path.exists(path)
+    with open("/proc/self/maps") as f:
+        hgemm.lib()
+        assert any(os.path.basename(path) in line for line in f.read().splitlines())
+
+
+def test_argument_errors(ctx):
+    L = hgemm.lib()
+    plan = ctx.plan(256, 256, 256)
+    A, B = inputs.make_ab(256, 256, 256, device="cuda")
+    C = torch.empty(256, 256, dtype=torch.float16, device="cuda")
+    a, b, c = A.data_ptr(), B.data_ptr(), C.data_ptr()
+    assert L.hgemm_run(None, a, b, c, None) == hgemm.ERR_INVALID_ARG
+    assert L.hgemm_run(plan._h, None, b, c, None) == hgemm.ERR_INVALID_ARG
+    assert L.hgemm_run(plan._h, a + 2, b, c, None) == hgemm.ERR_INVALID_ARG       # not 16-byte aligned
+    assert L.hgemm_run(plan._h, a, b, c + 8, None) == hgemm.ERR_INVALID_ARG
+    out = ctypes.c_void_p()
+    assert L.hgemm_plan(ctx._h, 64, 64, 60, ctypes.byref(out)) == hgemm.ERR_UNSUPPORTED and not out.value
+    assert L.hgemm_plan(ctx._h, 64, 60, 64, ctypes.byref(out)) == hgemm.ERR_UNSUPPORTED
+    assert L.hgemm_plan(ctx._h, 0, 64, 64, ctypes.byref(out)) == hgemm.ERR_INVALID_ARG
+    assert L.hgemm_plan(None, 64, 64, 64, ctypes.byref(out)) == hgemm.ERR_INVALID_ARG
+    assert L.hgemm_create(ctypes.byref(out), 99) == hgemm.ERR_INVALID_ARG
+    bad = hgemm.Config.make(block_n=48)
+    before = plan.config.as_dict()
+    assert plan.try_set_config(bad) == hgemm.ERR_UNSUPPORTED
+    assert plan.config.as_dict() == before                                         # plan unchanged
+    plan.run(A, B, C)                                                              # still usable
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    plan.close()
+
+
+def test_plan_tracks_new_pointers(ctx, gu):
+    """Tensor maps are cached per (A, B, C); a call with other buffers must re-encode them."""
+    M, N, K = 384, 256, 512
+    plan = ctx.plan(M, N, K)
+    for seed in (1, 2, 3):
+        A, B = inputs.make_ab(M, N, K, "int5", "cuda", seed=seed)
+        C, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+        assert torch.equal(C.float(), A.float() @ B.float().T)
+    plan.close()
+
+
+def test_run_on_a_side_stream(ctx, gu):
+    M, N, K = 512, 512, 1024
+    A, B = inputs.make_ab(M, N, K, "int5", "cuda")
+    C = torch.zeros(M, N, dtype=torch.float16, device="cuda")
+    plan = ctx.plan(M, N, K)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        plan.run(A, B, C)              # picks up the current (side) stream
+    s.synchronize()
+    assert torch.equal(C.float(), A.float() @ B.float().T)
+    plan.close()
+
+
+def test_bounded_wait_reports_timeout_and_context_survives(ctx, gu):
+    """A wait on a barrier that nothing signals runs out, the kernel returns, the host reads a
+    status, and the context keeps working (no fault, no hang)."""
+    ctx.set_wait_budget(2_000_000)                 # about a millisecond
+    t0 = time.time()
+    ctx.debug_timeout_probe()
+    st, code = ctx.last_device_status()
+    assert st == hgemm.ERR_TIMEOUT and (code >> 24) == 4
+    assert time.time() - t0 < 5.0
+    assert ctx.last_device_status() == (hgemm.OK, 0)          # the word is cleared by the read
+    ctx.set_wait_budget(2_000_000_000)
+    gu.check_shape(ctx, 256, 256, 256, "uniform")
+
+
+def test_full_grid_default_plans(ctx, gu):
+    """All 729 grid shapes with the plan the library picks: full-output oracle check up to 2048^3
+    by volume, 4096 samples + one row + one column above."""
+    worst = 0.0
+    for M in GRID:
+        for N in GRID:
+            for K in GRID:
+                rep = gu.check_shape(ctx, M, N, K, "uniform")
+                worst = max(worst, rep["max_err_over_bound"])
+    assert worst < 1.0

@@ -1,0 +1,226 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the fp64 CPU oracle.
+
+Bar: bit-exact on inputs whose sums are exactly representable (paper section 2.3, "Exact
+Match", generalised to signed small integers because this library accumulates in fp32);
+|C - C_ref| <= 2^-10 |C_ref| + 1e-3 sqrt(K) elementwise on random inputs, plus the
+scale-aware checks of oracle/acceptance.py.
+"""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2512_02551_b200 import hgemm, inputs  # noqa: E402
+
+F1, F2 = hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA
+DIRECT, TMA = hgemm.EPILOGUE_DIRECT, hgemm.EPILOGUE_TMA
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    assert torch.cuda.is_available(), "these tests need a B200"
+    c = hgemm.Context(0)
+    yield c
+    c.close()
+
+
+@pytest.fixture(scope="module")
+def gu():
+    import gpu_util
+    return gpu_util
+
+
+def _cfg(family=F1, bn=128, stages=4, split=1, raster=8, epi=DIRECT):
+    return hgemm.Config.make(family=family, block_n=bn, stages=stages, split_k=split, raster_group=raster, epilogue=epi)
+
+
+VARIANTS = [(F1, DIRECT), (F1, TMA), (F2, DIRECT), (F2, TMA)]
+
+
+# ---- configuration 1: single 128^3 GEMM, random and integer-valued -------------------------------
+
+@pytest.mark.parametrize("family,epi", VARIANTS)
+def test_config1_128_cubed(ctx, gu, family, epi):
+    import oracle
+    M = N = K = 128
+    cfg = _cfg(family, 128, 4, 1, 1, epi)
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    rep = gu.assert_close_full(C, A, B, "128^3 uniform")
+    assert rep["rel_frobenius"] < 3e-4
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), "128^3 integers")
+    plan.close()
+
+
+def test_default_plan_128_cubed(ctx, gu):
+    gu.check_shape(ctx, 128, 128, 128, "uniform")
+
+
+# ---- closed forms, bit for bit, every family and split factor ---------------------------------------
+
+@pytest.mark.parametrize("family,epi", VARIANTS)
+@pytest.mark.parametrize("split", [1, 3])
+def test_exact_closed_forms(ctx, gu, family, epi, split):
+    import oracle
+    M, N, K = 200, 136, 320          # ragged in M and N, 5 k-blocks
+    cfg = _cfg(family, 64, 3, split, 2, epi)
+    rng = np.random.default_rng(7)
+    # permutation: C[i][j] = B[j][pi(i)]
+    pi = rng.permutation(K)[:M]
+    A = torch.zeros(M, K, dtype=torch.float16)
+    A[torch.arange(M), torch.from_numpy(pi)] = 1.0
+    B = inputs.draw(3, inputs.TAG_B, N, K, "uniform")
+    C, _, plan = gu.run_gemm(ctx, A.cuda(), B.cuda(), cfg)
+    gu.assert_exact(C, B.double().numpy()[:, pi].T, "permutation")
+    # rank-1, one-hot k: C[i][j] = fp16(u_i v_j)
+    u = inputs.draw(5, 1, M, 1, "uniform")[:, 0]
+    v = inputs.draw(5, 2, N, 1, "uniform")[:, 0]
+    A = torch.zeros(M, K, dtype=torch.float16)
+    B = torch.zeros(N, K, dtype=torch.float16)
+    A[:, 77] = u
+    B[:, 77] = v
+    C, _, _ = gu.run_gemm(ctx, A.cuda(), B.cuda(), plan=plan)
+    gu.assert_exact(C, np.outer(u.double().numpy(), v.double().numpy()), "rank-1 one-hot")
+    # rank-1 constant along k with power-of-two entries: C[i][j] = K u_i v_j, all partial sums exact
+    vals = np.array([0.5, 1.0, 2.0, -0.5, -1.0, -2.0])
+    uu, vv = rng.choice(vals, M), rng.choice(vals, N)
+    A = torch.from_numpy(np.repeat(uu[:, None], K, 1)).to(torch.float16)
+    B = torch.from_numpy(np.repeat(vv[:, None], K, 1)).to(torch.float16)
+    C, _, _ = gu.run_gemm(ctx, A.cuda(), B.cuda(), plan=plan)
+    gu.assert_exact(C, K * np.outer(uu, vv), "rank-1 constant")
+    # integers in {-2..2}
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    C, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(C, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), "integers")
+    plan.close()
+
+
+def test_identity_returns_b_transposed(ctx, gu):
+    M = K = 256
+    N = 96
+    B = inputs.draw(9, inputs.TAG_B, N, K, "uniform", "cuda")
+    A = torch.eye(M, K, dtype=torch.float16, device="cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B)
+    assert torch.equal(C, B.T.contiguous())
+    plan.close()
+
+
+def test_paper_style_binary_exact_match(ctx, gu):
+    """Section 2.3: {0,1} inputs, exact equality required wherever the reference is below 2048."""
+    import oracle
+    M, N, K = 256, 192, 8192
+    for seed in (1, 2, 3):
+        A, B = inputs.make_ab(M, N, K, "binary", "cuda", seed=seed, p=inputs.binary_p(K))
+        C, _, plan = gu.run_gemm(ctx, A, B)
+        ref = oracle.hgemm_full(inputs.bits(A), inputs.bits(B))
+        got = gu.bits_to_f64(gu.c_bits(C))
+        small = ref < 2048
+        assert small.mean() > 0.9 and np.array_equal(got[small], ref[small])
+        plan.close()
+
+
+# ---- unit shapes: one tile, ring wrap-around, tails, many tiles per CTA, tile widths -------------------
+
+UNIT_CASES = [
+    # M, N, K, bn, stages, split, raster
+    (128, 128, 64, 128, 4, 1, 1),       # one tile, one k-block
+    (128, 128, 1024, 128, 3, 1, 1),     # ring wraps five times
+    (128, 32, 64, 32, 1, 1, 1),         # narrowest tile, single stage
+    (8, 8, 8, 32, 2, 1, 1),             # smallest legal shape: tails in all three dimensions
+    (100, 136, 72, 64, 4, 1, 1),        # ragged M, N and K
+    (130, 264, 200, 256, 4, 1, 1),      # one row / one column group past a tile edge
+    (384, 416, 192, 96, 4, 1, 2),       # tile width that is not a power of two
+    (640, 480, 256, 160, 2, 1, 3),
+    (1024, 2048, 128, 32, 10, 1, 4),    # 512 tiles on 148 SMs: several tiles per CTA, accumulators alternate
+    (2048, 2048, 64, 64, 2, 1, 16),
+    (64, 64, 2048, 64, 4, 4, 1),        # split-K
+    (300, 200, 1000, 96, 4, 16, 1),     # one k-block per slice
+    (512, 384, 640, 128, 4, 3, 2),      # uneven slices (10 k-blocks over 3)
+]
+
+
+@pytest.mark.parametrize("family", [F1, F2])
+@pytest.mark.parametrize("case", UNIT_CASES, ids=lambda c: "x".join(map(str, c[:3])) + f"-bn{c[3]}s{c[4]}k{c[5]}")
+def test_unit_shapes(ctx, gu, family, case):
+    import oracle
+    M, N, K, bn, stages, split, raster = case
+    for epi in (DIRECT, TMA):
+        cfg = _cfg(family, bn, stages, split, raster, epi)
+        A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+        C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+        gu.assert_close_full(C, A, B, f"{case} family={family} epi={epi}")
+        Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+        Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+        gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"{case} integers")
+        plan.close()
+        if split > 1:
+            break                         # split-K always finishes with direct stores
+
+
+# ---- configuration 2: square sweep ---------------------------------------------------------------------
+
+@pytest.mark.parametrize("S", [1024, 2048, 4096, 8192])
+def test_config2_square(ctx, gu, S):
+    rep = gu.check_shape(ctx, S, S, S, "uniform")
+    assert rep["rel_frobenius"] < 3e-4
+
+
+@pytest.mark.parametrize("family,bn,stages,epi", [(F1, 256, 4, TMA), (F1, 256, 4, DIRECT), (F2, 256, 6, TMA),
+                                                   (F2, 256, 4, DIRECT), (F2, 224, 4, TMA)])
+def test_config2_bench_configurations_4096(ctx, gu, family, bn, stages, epi):
+    """The launch configurations the benchmark times on 4096^3, checked on samples + one row + one column."""
+    gu.check_shape(ctx, 4096, 4096, 4096, "uniform", _cfg(family, bn, stages, 1, 4, epi))
+
+
+# ---- configuration 3: skinny LLM projections, N(0,1)/sqrt(K) ----------------------------------------------
+
+@pytest.mark.parametrize("NK", [(4096, 4096), (12288, 4096), (4096, 12288)])
+@pytest.mark.parametrize("M", [64, 128, 256])
+def test_config3_skinny(ctx, gu, M, NK):
+    N, K = NK
+    rep = gu.check_shape(ctx, M, N, K, "normal")
+    assert rep["rel_frobenius"] < 3e-4
+
+
+# ---- configuration 4: small M, N with large K; split-K determinism ------------------------------------------
+
+@pytest.mark.parametrize("K", [8192, 12288])
+@pytest.mark.parametrize("MN", [64, 256, 512])
+def test_config4_small_mn_large_k(ctx, gu, MN, K):
+    gu.check_shape(ctx, MN, MN, K, "uniform")
+
+
+@pytest.mark.parametrize("family", [F1, F2])
+@pytest.mark.parametrize("MN,K,bn,split", [(64, 8192, 64, 8), (64, 12288, 32, 48), (256, 12288, 128, 12),
+                                            (512, 8192, 128, 6), (512, 12288, 256, 16)])
+def test_split_k_is_deterministic(ctx, gu, family, MN, K, bn, split):
+    """Every split-K configuration reproduces its own bits run after run, with other work in flight
+    to perturb the order in which slices finish."""
+    cfg = _cfg(family, bn, 4, split, 1, DIRECT)
+    A, B = inputs.make_ab(MN, MN, K, "uniform", "cuda")
+    C0, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    gu.assert_close_full(C0, A, B, f"split-K {cfg.as_dict()}")
+    ref_bits = C0.view(torch.int16).clone()
+    noise = torch.empty(1 << 24, device="cuda")
+    side = torch.cuda.Stream()
+    for it in range(10):
+        C = torch.empty_like(C0)
+        with torch.cuda.stream(side):
+            for _ in range(it % 3 + 1):
+                noise.normal_()
+        plan.run(A, B, C)
+        torch.cuda.synchronize()
+        assert torch.equal(C.view(torch.int16), ref_bits), f"run {it} differs"
+    plan.close()
+
+
+# ---- the input generator draws the same bits on both devices --------------------------------------------------
+
+def test_generator_matches_across_devices():
+    for dist in ("uniform", "int5", "binary"):
+        a = inputs.draw(77, inputs.TAG_A, 513, 264, dist, "cpu")
+        b = inputs.draw(77, inputs.TAG_A, 513, 264, dist, "cuda")
+        assert torch.equal(a, b.cpu()), dist
