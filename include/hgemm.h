@@ -145,6 +145,14 @@ hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles);
  * HGEMM_ERR_TIMEOUT.  Nothing faults or hangs. */
 hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
 
+/* Instrumentation: when `device_buf` (DEVICE pointer to 8 uint64, or NULL to switch
+ * it off) is set, CTA 0 of every later launch of this plan writes nanosecond
+ * %globaltimer stamps of its pipeline events: 0 kernel entry, 1 set-up done,
+ * 2 first TMA load issued, 3 first k-block landed, 4 last MMA issued, 5 first
+ * accumulator ready, 6 epilogue done, 7 tensor memory freed.  The caller owns the
+ * buffer. */
+hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
+
 /* cudaError_t (as int) of the last failing CUDA call made through this context. */
 int32_t hgemm_last_cuda_error(const hgemm_ctx_t *ctx);
 

@@ -35,6 +35,7 @@ struct hgemm_plan_s {
     KernelParams params;
     int grid = 0;
     int smem = 0;
+    unsigned long long *trace = nullptr;
     void *workspace = nullptr;
     int64_t workspace_bytes = 0;
     uint32_t *counters = nullptr;
@@ -382,6 +383,7 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     }
     plan->params.C = static_cast<__half *>(C);
     plan->params.wait_budget = ctx->wait_budget;
+    plan->params.trace = plan->trace;
 
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof(lc));
@@ -432,6 +434,13 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
     if (s != HGEMM_OK) return s;
     e = cudaMemcpyAsync(C_host, plan->stage_c, c_bytes, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf)
+{
+    if (!plan) return HGEMM_ERR_INVALID_ARG;
+    plan->trace = static_cast<unsigned long long *>(device_buf);
     return HGEMM_OK;
 }
 

@@ -64,7 +64,17 @@ struct KernelParams {
     uint32_t *status;             // device status word (0 = fine)
     __half *C;
     long long wait_budget;        // clock cycles a wait may take before the kernel gives up
+    unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
 };
+
+__device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
+{
+    if (p.trace != nullptr && blockIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[slot] = t;
+    }
+}
 
 // -------------------------------------------------------------------------------------
 // bounded wait
@@ -189,6 +199,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     // ---- set-up -----------------------------------------------------------------------
     if (threadIdx.x == 0) {
+        trace_stamp(p, 0);
         *abort_flag = 0u;
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(bar_full + 8 * s, CTA_GROUP);   // one arrive.expect_tx per CTA of the pair
@@ -215,6 +226,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
+    if (threadIdx.x == 0) trace_stamp(p, 1);
 
     // ---- roles ------------------------------------------------------------------------
     if (warp == 0) {
@@ -247,6 +259,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         tma_load_2d_pair(a_dst, &tmap_a, k0, a_row, fb);
                         tma_load_2d_pair(b_dst, &tmap_b, k0, b_row, fb);
                     }
+                    if (w == unit && kb == 0) trace_stamp(p, 2);
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
@@ -269,6 +282,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int32_t kb = 0; kb < it.kb_count; ++kb) {
                     ok = mbar_wait(bar_full + 8 * s, ph, ctl, status_code(kRoleMma, 0, s));
                     if (!ok) break;
+                    if (w == unit && kb == 0) trace_stamp(p, 3);
                     tc_fence_after_sync();
                     const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
                     const uint64_t a_desc = make_smem_desc_sw128(a_addr);
@@ -289,6 +303,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
+                if (w == unit) trace_stamp(p, 4);
                 if constexpr (CTA_GROUP == 1) {
                     umma_commit<1>(bar_tmem_full + 8 * acc);
                 } else {
@@ -314,6 +329,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
             ok = __all_sync(0xffffffffu, ok);   // the warp-wide tensor-memory loads below need the whole warp
             if (!ok) break;
+            if (w == unit && threadIdx.x == 64) trace_stamp(p, 5);
             tc_fence_after_sync();
             const int32_t row0 = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;  // first row of this CTA's 128
             const int32_t grow = row0 + static_cast<int32_t>(row_in_tile);          // this thread's global row
@@ -438,6 +454,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         // shared memory must stay valid until the last TMA stores have read it
         if (lane == 0) bulk_wait_group<0>();
+        if (threadIdx.x == 64) trace_stamp(p, 6);
     }
 
     // ---- teardown (every thread, also after an abort) ----------------------------------
@@ -454,6 +471,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         tc_fence_after_sync();
         tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+        if (lane == 0) trace_stamp(p, 7);
     }
 }
 

@@ -22,7 +22,7 @@ EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
-    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe",
+    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace",
     "hgemm_last_cuda_error", "hgemm_status_string",
 ]
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_last_device_status": (i32, [p, ctypes.POINTER(ctypes.c_uint32)]),
             "hgemm_set_wait_budget": (i32, [p, i64]),
             "hgemm_debug_timeout_probe": (i32, [p, p]),
+            "hgemm_debug_set_trace": (i32, [p, p]),
             "hgemm_last_cuda_error": (i32, [p]),
             "hgemm_status_string": (ctypes.c_char_p, [i32]),
         }
@@ -204,6 +205,9 @@ class Plan:
                 raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
         s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
         self.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+
+    def set_trace(self, device_ptr: int) -> None:
+        _check(lib().hgemm_debug_set_trace(self._h, ctypes.c_void_p(device_ptr)), "hgemm_debug_set_trace")
 
     def run_host(self, A, B, C, stream=None) -> None:
         """``hgemm_run_host`` on torch CPU tensors (pinned for an asynchronous call)."""
