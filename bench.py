@@ -132,7 +132,9 @@ def run_reference(args) -> None:
     import oracle
     from paper_2512_02551_b200 import inputs
     oracle.build()
-    rows = 96
+    # rows of C per shape per step, sized so that warm-up + steps end within about a minute
+    per_row_macs = sum(S * S for S in SWEEP)
+    rows = max(1, min(96, int(60.0 * 15e9 / ((args.steps + args.warmup) * per_row_macs))))
     slabs = [(S, *oracle_slab(oracle, inputs, S, rows)) for S in SWEEP]
     macs = sum(rows * S * S for S in SWEEP)
     for _ in range(max(args.warmup, 1) if args.warmup else 0):
@@ -213,7 +215,7 @@ def run_ours(args) -> None:
             else:
                 w["plan"].run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), stream.cuda_stream)
 
-    def timed(fn, steps, warmup, sampler=None):
+    def timed(fn, steps, warmup, sampler=None, label="hgemm_timed_region"):
         for i in range(warmup):
             fn(i)
         barrier()
@@ -223,11 +225,13 @@ def run_ours(args) -> None:
             time.sleep(0.25)
             t0w = time.time()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.nvtx.range_push(label)
         e0.record(stream)
         for i in range(steps):
             fn(warmup + i)
         e1.record(stream)
         barrier()
+        torch.cuda.nvtx.range_pop()
         t1w = time.time()
         ms = e0.elapsed_time(e1)
         if dist is not None:
@@ -319,7 +323,7 @@ def run_ours(args) -> None:
         for plan, hA, hB, hC in host:
             plan.run_host(hA, hB, hC, stream.cuda_stream)
     e2e_steps = max(3, min(args.steps, 10))
-    e2e_ms, _, _ = timed(e2e_step, e2e_steps, 2)
+    e2e_ms, _, _ = timed(e2e_step, e2e_steps, 2, label="hgemm_e2e_region")
     e2e_value = world * step_flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
     # the result that came back is the GEMM's (spot check against the device-resident run)
     if rank == 0:

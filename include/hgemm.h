@@ -60,6 +60,14 @@ enum {
     HGEMM_FAMILY_UMMA_2CTA = 1  /* the same with CTA pairs: 256 x block_n tiles, B split across the pair */
 };
 
+/* Where the fp32 partial sums of a split-K tile meet.  Both sum the slices in slice
+ * order 0..S-1, so a configuration reproduces its own bits run after run. */
+enum {
+    HGEMM_SPLIT_WORKSPACE = 0, /* partials parked in a global workspace; any family; split_k <= 64 */
+    HGEMM_SPLIT_CLUSTER = 1    /* the slices of a tile form one thread-block cluster and are summed through
+                                  distributed shared memory; 1-CTA family only; split_k in [2, 16] */
+};
+
 enum {
     HGEMM_EPILOGUE_DIRECT = 0, /* registers -> 16-byte global stores */
     HGEMM_EPILOGUE_TMA = 1     /* registers -> swizzled shared memory -> TMA store */
@@ -71,12 +79,13 @@ typedef struct {
     int32_t family;       /* HGEMM_FAMILY_* */
     int32_t block_m;      /* 128 (1-CTA) or 256 (2-CTA pair) */
     int32_t block_n;      /* multiple of 32 in [32, 256] */
-    int32_t block_k;      /* 64 (one 128-byte swizzle span of fp16) */
+    int32_t block_k;      /* K extent of a pipeline stage: 64 or 128 (one or two 128-byte swizzle spans) */
     int32_t stages;       /* shared-memory ring depth, 2..12, bounded by shared memory */
     int32_t split_k;      /* >= 1; K slices reduced in slice order (deterministic) */
     int32_t raster_group; /* m-tiles per raster group (>= 1): tile order for L2 reuse */
     int32_t epilogue;     /* HGEMM_EPILOGUE_* (split_k > 1 always finishes with direct stores) */
-    int32_t reserved[8];  /* must be zero */
+    int32_t split_mode;   /* HGEMM_SPLIT_* : how the K slices of a tile are summed (ignored when split_k == 1) */
+    int32_t reserved[7];  /* must be zero */
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the
@@ -122,6 +131,10 @@ hgemm_status_t hgemm_heuristic_config(int64_t M, int64_t N, int64_t K, int32_t n
 /* Check a configuration against a shape without a GPU: HGEMM_OK if legal. */
 hgemm_status_t hgemm_validate_config(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg);
 
+/* The planner's cost model: estimated SM clock cycles of one run (a ranking aid for
+ * the tuner, not a prediction); negative if the configuration is illegal. */
+double hgemm_estimate_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t *cfg);
+
 /* Dynamic shared memory (bytes) and split-K workspace (bytes) a configuration needs. */
 int64_t hgemm_config_smem_bytes(const hgemm_config_t *cfg);
 int64_t hgemm_config_workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg);
@@ -145,13 +158,21 @@ hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles);
  * HGEMM_ERR_TIMEOUT.  Nothing faults or hangs. */
 hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
 
-/* Instrumentation: when `device_buf` (DEVICE pointer to 8 uint64, or NULL to switch
+/* Instrumentation: when `device_buf` (DEVICE pointer to 24 uint64, or NULL to switch
  * it off) is set, CTA 0 of every later launch of this plan writes nanosecond
  * %globaltimer stamps of its pipeline events: 0 kernel entry, 1 set-up done,
  * 2 first TMA load issued, 3 first k-block landed, 4 last MMA issued, 5 first
- * accumulator ready, 6 epilogue done, 7 tensor memory freed.  The caller owns the
- * buffer. */
+ * accumulator ready, 6 epilogue done, 7 tensor memory freed; and SM-clock totals:
+ * 8/9/10 MMA thread waiting for data / issuing MMAs / committing, 11/12 producer
+ * waiting for a free stage / issuing loads, 13 MMA thread waiting for a free
+ * accumulator, 15 k-blocks processed; and for split-K stamps 16 partial parked,
+ * 17 all slices arrived, 18 share reduced.  The caller owns the buffer. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
+
+/* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan
+ * issue no TMA loads, bit 1 no MMAs (the pipeline still runs; C is garbage).
+ * 0 restores normal operation. */
+hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask);
 
 /* cudaError_t (as int) of the last failing CUDA call made through this context. */
 int32_t hgemm_last_cuda_error(const hgemm_ctx_t *ctx);

@@ -34,8 +34,10 @@ struct hgemm_plan_s {
     hgemm_config_t cfg;
     KernelParams params;
     int grid = 0;
+    int cluster_dim = 1;
     int smem = 0;
     unsigned long long *trace = nullptr;
+    uint32_t debug_skip = 0;
     void *workspace = nullptr;
     int64_t workspace_bytes = 0;
     uint32_t *counters = nullptr;
@@ -88,6 +90,31 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
 {
     hgemm_ctx_s *ctx = pl->ctx;
     const int cg = hgemm_host::cta_group_of(cfg);
+    // the slices of a tile wait for each other: each needs its own SM (or SM pair)
+    if (cfg.split_k > 1 && cfg.split_k > ctx->num_sms / cg) return HGEMM_ERR_UNSUPPORTED;
+    const bool cluster_split = cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER;
+    if (cluster_split) {
+        // can the device place a cluster of split_k CTAs of this kernel at all?
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof(lc));
+        lc.gridDim = dim3(unsigned(cfg.split_k), 1, 1);
+        lc.blockDim = dim3(hgemm_dev::kThreads, 1, 1);
+        lc.dynamicSmemBytes = size_t(hgemm_host::kSmemOptInBytes);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = unsigned(cfg.split_k);
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        int clusters = 0;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1>, &lc);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            return HGEMM_ERR_UNSUPPORTED;
+        }
+        if (clusters < 1) return HGEMM_ERR_UNSUPPORTED;
+    }
     const int64_t ws = hgemm_host::workspace_bytes(pl->M, pl->N, pl->K, cfg);
     const int64_t cb = hgemm_host::counter_bytes(pl->M, pl->N, cfg);
     if (ws > pl->workspace_bytes) {
@@ -127,7 +154,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.tiles_n = int32_t((pl->N + cfg.block_n - 1) / cfg.block_n);
     p.split_k = cfg.split_k;
     p.total_work = p.tiles_m * p.tiles_n * p.split_k;
-    p.kblocks = int32_t((pl->K + 63) / 64);
+    p.block_k = cfg.block_k;
+    p.kblocks = int32_t((pl->K + cfg.block_k - 1) / cfg.block_k);
     p.block_n = cfg.block_n;
     p.stages = cfg.stages;
     p.raster_group = std::min(cfg.raster_group, p.tiles_m);
@@ -137,10 +165,13 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.workspace = static_cast<float *>(pl->workspace);
     p.counters = pl->counters;
     p.status = ctx->d_status;
+    p.cluster_split = cluster_split ? 1 : 0;
     p.C = nullptr;
     p.wait_budget = ctx->wait_budget;
     const int units = std::max(1, ctx->num_sms / cg);
-    pl->grid = cg * std::min(p.total_work, units);
+    // cluster split-K is not persistent: one CTA per (tile, slice), the hardware schedules the clusters
+    pl->grid = cluster_split ? p.total_work : cg * std::min(p.total_work, units);
+    pl->cluster_dim = cluster_split ? cfg.split_k : cg;
     // Always ask for the whole opt-in shared memory: it keeps a second CTA off the SM, so two
     // CTAs can never wait on each other's tensor-memory allocation.
     pl->smem = int(hgemm_host::kSmemOptInBytes);
@@ -230,6 +261,11 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             st = cuda_fail(ctx, e);
             break;
         }
+        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) {
+            st = cuda_fail(ctx, e);
+            break;
+        }
         e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(hgemm_host::kSmemOptInBytes));
         if (e != cudaSuccess) {
@@ -286,6 +322,12 @@ hgemm_status_t hgemm_validate_config(int64_t M, int64_t N, int64_t K, const hgem
 {
     if (!cfg) return HGEMM_ERR_INVALID_ARG;
     return hgemm_host::validate(M, N, K, *cfg);
+}
+
+double hgemm_estimate_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t *cfg)
+{
+    if (!cfg || hgemm_host::validate(M, N, K, *cfg) != HGEMM_OK) return -1.0;
+    return hgemm_host::estimate_cycles(M, N, K, num_sms, *cfg);
 }
 
 int64_t hgemm_config_smem_bytes(const hgemm_config_t *cfg)
@@ -384,6 +426,7 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     plan->params.C = static_cast<__half *>(C);
     plan->params.wait_budget = ctx->wait_budget;
     plan->params.trace = plan->trace;
+    plan->params.debug_skip = plan->debug_skip;
 
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof(lc));
@@ -393,7 +436,7 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     lc.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = unsigned(cg);
+    attr[0].val.clusterDim.x = unsigned(plan->cluster_dim);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     lc.attrs = attr;
@@ -441,6 +484,13 @@ hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf)
 {
     if (!plan) return HGEMM_ERR_INVALID_ARG;
     plan->trace = static_cast<unsigned long long *>(device_buf);
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask)
+{
+    if (!plan || mask > 3u) return HGEMM_ERR_INVALID_ARG;
+    plan->debug_skip = mask;
     return HGEMM_OK;
 }
 

@@ -1,16 +1,17 @@
 // The persistent, warp-specialised tcgen05 HGEMM kernel (all kernel families are
 // instances of this one template).
 //
-// Structure per CTA (192 threads):
+// Structure per CTA (320 threads):
 //   warp 0      TMA producer: fills a ring of shared-memory stages with 64-wide
 //               k-blocks of A (128 rows) and B (block_n rows, or block_n/2 in a pair)
 //   warp 1      allocates tensor memory; one thread issues tcgen05.mma into one of two
 //               fp32 accumulators (double-buffered so the epilogue of tile t overlaps
 //               the main loop of tile t+1)
-//   warps 2..5  epilogue: tensor memory -> registers -> fp16 -> global (direct 16-byte
-//               stores, or swizzled shared memory + TMA store); with split-K the fp32
-//               partial goes to a workspace and the last slice to finish sums all
-//               slices of its tile in slice order.
+//   warps 2..9  epilogue: tensor memory -> registers -> fp16 -> global (direct 16-byte
+//               stores, or swizzled shared memory + TMA store); with split-K each slice
+//               parks its fp32 partial in a workspace, waits (bounded) for the other
+//               slices of its tile, and sums its share of the tile over all slices in
+//               slice order.
 // This is the tiled structure of the paper's section 2.1 (global -> shared -> tensor
 // core main loop over K, then an epilogue) mapped onto Blackwell: TMA in place of
 // cp.async, tensor memory in place of register accumulators, a persistent tile loop in
@@ -34,14 +35,14 @@ namespace hgemm_dev {
 using namespace hgemm_ptx;
 
 constexpr int kBlockM = 128;          // rows of one CTA's accumulator (UMMA M per CTA)
-constexpr int kBlockK = 64;           // fp16 elements per k-block = one 128-byte swizzle span
+constexpr int kSubK = 64;             // fp16 elements of one sub-tile row = one 128-byte swizzle span
 constexpr int kUmmaK = 16;            // K of one tcgen05.mma.kind::f16
 constexpr int kMaxStages = 12;
-constexpr int kThreads = 192;
-constexpr int kATileBytes = kBlockM * kBlockK * 2;           // 16 KB
+constexpr int kThreads = 320;          // producer warp + MMA warp + 8 epilogue warps
+constexpr int kATileBytes = kBlockM * kSubK * 2;             // 16 KB: one 128 x 64 sub-tile of A
 constexpr int kStoreBoxRows = 32, kStoreBoxCols = 32;        // TMA-store box: one warp's 32 x 32 chunk
 constexpr int kStagingBytesPerWarp = 2 * kStoreBoxRows * kStoreBoxCols * 2;  // two 2 KB buffers
-constexpr int kStagingBytes = 4 * kStagingBytesPerWarp;      // 16 KB
+constexpr int kStagingBytes = 8 * kStagingBytesPerWarp;      // 32 KB
 constexpr int kCtrlBytes = 512;       // barriers, tensor-memory base, abort flag
 
 // Status-word roles
@@ -52,19 +53,22 @@ struct KernelParams {
     int32_t tiles_m, tiles_n;     // tiles_m counts block_m-row tiles (256 rows for a pair)
     int32_t total_work;           // tiles_m * tiles_n * split_k
     int32_t split_k;
-    int32_t kblocks;              // ceil(K / 64)
+    int32_t kblocks;              // ceil(K / block_k)
+    int32_t block_k;              // K extent of one pipeline stage: 64 or 128 (one or two 64-wide sub-tiles)
     int32_t block_n;
     int32_t stages;
     int32_t raster_group;
     int32_t tmem_cols;            // power of two >= 2 * block_n
     int32_t epilogue_tma;         // 1: TMA-store epilogue (only when split_k == 1)
+    int32_t cluster_split;        // 1: the split_k slices of a tile are one cluster and reduce through shared memory
     uint32_t idesc;               // tcgen05 instruction descriptor
-    float *workspace;             // split-K partials: [work item][chunk][col][128 rows]
-    uint32_t *counters;           // split-K arrival counters: [tile][cta of pair][row quarter]
+    float *workspace;             // split-K partials: [work item][cta of pair][chunk][128 rows][32 cols]
+    uint32_t *counters;           // split-K counters: [tile][cta of pair][arrived, finished]
     uint32_t *status;             // device status word (0 = fine)
     __half *C;
     long long wait_budget;        // clock cycles a wait may take before the kernel gives up
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
+    uint32_t debug_skip;          // instrumentation: bit 0 = issue no TMA loads, bit 1 = issue no MMAs (results are garbage)
 };
 
 __device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
@@ -173,8 +177,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint8_t *smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
 
     const int32_t b_rows = p.block_n / CTA_GROUP;            // B rows this CTA stages per k-block
-    const uint32_t b_tile_bytes = static_cast<uint32_t>(b_rows) * kBlockK * 2;
-    const uint32_t stage_bytes = kATileBytes + b_tile_bytes;
+    const int32_t subs = p.block_k / kSubK;                  // 64-wide sub-tiles per stage (1 or 2)
+    const uint32_t b_sub_bytes = static_cast<uint32_t>(b_rows) * kSubK * 2;
+    const uint32_t a_stage_bytes = static_cast<uint32_t>(subs) * kATileBytes;
+    const uint32_t stage_bytes = a_stage_bytes + static_cast<uint32_t>(subs) * b_sub_bytes;   // [A sub-tiles | B sub-tiles]
     const uint32_t staging_base = smem_base + static_cast<uint32_t>(p.stages) * stage_bytes;
     const uint32_t ctrl_base = staging_base + kStagingBytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl_base - smem_base);
@@ -187,8 +193,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     volatile uint32_t *tmem_base_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 16 * kMaxStages + 32);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 16 * kMaxStages + 36);
 
-    const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t lane = threadIdx.x & 31;
+    // the warp index through a shuffle: a value the compiler knows to be warp-uniform
+    const uint32_t warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);
+    const uint32_t lane = lane_id();
     const uint32_t cta_rank = (CTA_GROUP == 2) ? cluster_ctarank() : 0u;
     const bool is_leader = (cta_rank == 0);
     const int32_t unit = (CTA_GROUP == 2) ? static_cast<int32_t>(blockIdx.x >> 1) : static_cast<int32_t>(blockIdx.x);
@@ -207,7 +214,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tmem_full + 8 * a, 1);              // one tcgen05.commit
-            mbar_init(bar_tmem_empty + 8 * a, 4 * CTA_GROUP); // one arrive per epilogue warp (of both CTAs)
+            mbar_init(bar_tmem_empty + 8 * a, 8 * CTA_GROUP); // one arrive per epilogue warp (of both CTAs)
         }
         fence_mbar_init();
         prefetch_tensormap(&tmap_a);
@@ -229,94 +236,128 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     if (threadIdx.x == 0) trace_stamp(p, 1);
 
     // ---- roles ------------------------------------------------------------------------
+    // Producer and MMA loops are executed by their whole warp with warp-uniform control flow (the
+    // wait results are voted), and only the single-thread instructions are predicated on lane 0:
+    // TMA and tcgen05 instructions take their operands from uniform registers, so operands the
+    // compiler can prove warp-uniform cost nothing to issue, while per-thread ones each need a move.
     if (warp == 0) {
-        if (lane == 0) {
-            // ===== TMA producer =====
-            int s = 0;
-            uint32_t ph = 0;
-            const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, 0) : bar_full;
-            bool ok = true;
-            for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
-                const WorkItem it = decode_work(w, p, kBlockMTotal);
-                const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
-                const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * b_rows;
-                for (int32_t kb = 0; kb < it.kb_count; ++kb) {
-                    ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, ctl, status_code(kRoleProducer, 0, s));
-                    if (!ok) break;
-                    const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
-                    const uint32_t b_dst = a_dst + kATileBytes;
-                    const int32_t k0 = (it.kb_begin + kb) * kBlockK;
-                    if constexpr (CTA_GROUP == 1) {
-                        mbar_arrive_expect_tx(bar_full + 8 * s, stage_bytes);
-                        tma_load_2d(a_dst, &tmap_a, k0, a_row, bar_full + 8 * s);
-                        tma_load_2d(b_dst, &tmap_b, k0, b_row, bar_full + 8 * s);
-                    } else {
-                        // both CTAs of the pair announce their bytes on the leader's barrier; the peer's
-                        // remote arrive is relaxed (it orders nothing: the data arrives through TMA)
-                        const uint32_t fb = full_leader + 8 * s;
-                        if (is_leader) mbar_arrive_expect_tx(bar_full + 8 * s, stage_bytes);
-                        else mbar_arrive_expect_tx_cluster_relaxed(fb, stage_bytes);
-                        tma_load_2d_pair(a_dst, &tmap_a, k0, a_row, fb);
-                        tma_load_2d_pair(b_dst, &tmap_b, k0, b_row, fb);
+        // ===== TMA producer =====
+        int s = 0;
+        uint32_t ph = 0;
+        const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, 0) : bar_full;
+        const bool tr = p.trace != nullptr && blockIdx.x == 0;
+        const uint32_t leader = (lane == 0) ? 1u : 0u;     // the lane that issues the loads
+        long long t_wait = 0, t_work = 0;
+        bool ok = true;
+        for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
+            const WorkItem it = decode_work(w, p, kBlockMTotal);
+            const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
+            const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * b_rows;
+            for (int32_t kb = 0; kb < it.kb_count; ++kb) {
+                const long long c0 = tr ? clock64() : 0;
+                ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, ctl, status_code(kRoleProducer, 0, s));
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const long long c1 = tr ? clock64() : 0;
+                const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
+                const uint32_t b_dst = a_dst + a_stage_bytes;
+                const int32_t k0 = (it.kb_begin + kb) * p.block_k;
+                const uint32_t fb = full_leader + 8 * s;      // the (leader's) full barrier of this stage
+                if (p.debug_skip & 1u) {
+                    if (lane == 0) {
+                        if (is_leader) mbar_arrive(bar_full + 8 * s);
+                        else mbar_arrive_cluster(fb);
                     }
-                    if (w == unit && kb == 0) trace_stamp(p, 2);
-                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                } else if constexpr (CTA_GROUP == 1) {
+                    mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                    for (int32_t sub = 0; sub < subs; ++sub) {
+                        tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, bar_full + 8 * s);
+                        tma_load_2d_if(leader, b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, bar_full + 8 * s);
+                    }
+                } else {
+                    // both CTAs of the pair announce their bytes on the leader's barrier; the peer's
+                    // remote arrive is relaxed (it orders nothing: the data arrives through TMA)
+                    if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, stage_bytes);
+                    for (int32_t sub = 0; sub < subs; ++sub) {
+                        tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                        tma_load_2d_pair_if(leader, b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, fb);
+                    }
                 }
+                if (w == unit && kb == 0 && lane == 0) trace_stamp(p, 2);
+                if (tr) { t_wait += c1 - c0; t_work += clock64() - c1; }
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
+        if (tr && lane == 0) { p.trace[11] = t_wait; p.trace[12] = t_work; }
     } else if (warp == 1) {
-        if (lane == 0 && is_leader) {
+        if (is_leader) {
             // ===== MMA issuer =====
             int s = 0;
             uint32_t ph = 0;
             uint32_t local_tile = 0;
+            const bool tr = p.trace != nullptr && blockIdx.x == 0;
+            const uint32_t leader = (lane == 0) ? 1u : 0u; // the lane that issues every MMA and commit
+            long long t_wait = 0, t_issue = 0, t_commit = 0, t_acc = 0, n_kb = 0;
+            const uint64_t desc_a0 = make_smem_desc_sw128(smem_base);
+            const uint64_t desc_b0 = make_smem_desc_sw128(smem_base + a_stage_bytes);
+            const uint32_t desc_stage_step = stage_bytes >> 4;
+            const bool issue_mma = !(p.debug_skip & 2u);
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
                 const WorkItem it = decode_work(w, p, kBlockMTotal);
                 const uint32_t acc = local_tile & 1u;
                 const uint32_t acc_ph = (local_tile >> 1) & 1u;
+                const long long ca = tr ? clock64() : 0;
                 ok = mbar_wait(bar_tmem_empty + 8 * acc, acc_ph ^ 1u, ctl, status_code(kRoleMma, 1, acc));
+                ok = __all_sync(0xffffffffu, ok);
+                if (tr) t_acc += clock64() - ca;
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * static_cast<uint32_t>(p.block_n);
                 for (int32_t kb = 0; kb < it.kb_count; ++kb) {
+                    const long long c0 = tr ? clock64() : 0;
                     ok = mbar_wait(bar_full + 8 * s, ph, ctl, status_code(kRoleMma, 0, s));
+                    ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    if (w == unit && kb == 0) trace_stamp(p, 3);
+                    const long long c1 = tr ? clock64() : 0;
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_base + static_cast<uint32_t>(s) * stage_bytes;
-                    const uint64_t a_desc = make_smem_desc_sw128(a_addr);
-                    const uint64_t b_desc = make_smem_desc_sw128(a_addr + kATileBytes);
+                    const uint64_t a_desc = desc_a0 + static_cast<uint64_t>(static_cast<uint32_t>(s) * desc_stage_step);
+                    const uint64_t b_desc = desc_b0 + static_cast<uint64_t>(static_cast<uint32_t>(s) * desc_stage_step);
+                    if (w == unit && kb == 0 && lane == 0) trace_stamp(p, 3);
+                    if (issue_mma) {
+                        for (int32_t sub = 0; sub < subs; ++sub) {
+                            const uint64_t a_sub = a_desc + static_cast<uint64_t>(static_cast<uint32_t>(sub) * (kATileBytes >> 4));
+                            const uint64_t b_sub = b_desc + static_cast<uint64_t>(static_cast<uint32_t>(sub) * (b_sub_bytes >> 4));
 #pragma unroll
-                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
-                        umma_f16<CTA_GROUP>(d_tmem, a_desc + 2u * k, b_desc + 2u * k, p.idesc,
-                                            (kb | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < kSubK / kUmmaK; ++k) {
+                                // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
+                                umma_f16_if<CTA_GROUP>(leader, d_tmem, a_sub + 2u * k, b_sub + 2u * k, p.idesc,
+                                                       (kb | sub | k) != 0 ? 1u : 0u);
+                            }
+                        }
                     }
+                    const long long c2 = tr ? clock64() : 0;
                     // free the stage (in both CTAs of a pair) once these MMAs have read it
-                    if constexpr (CTA_GROUP == 1) {
-                        umma_commit<1>(bar_empty + 8 * s);
-                    } else {
-                        umma_commit<2>(mapa(bar_empty + 8 * s, 0));
-                        umma_commit<2>(mapa(bar_empty + 8 * s, 1));
-                    }
+                    umma_commit_if<CTA_GROUP>(leader, bar_empty + 8 * s);
+                    if (tr) { t_wait += c1 - c0; t_issue += c2 - c1; t_commit += clock64() - c2; ++n_kb; }
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                if (w == unit) trace_stamp(p, 4);
-                if constexpr (CTA_GROUP == 1) {
-                    umma_commit<1>(bar_tmem_full + 8 * acc);
-                } else {
-                    umma_commit<2>(mapa(bar_tmem_full + 8 * acc, 0));
-                    umma_commit<2>(mapa(bar_tmem_full + 8 * acc, 1));
-                }
+                if (w == unit && lane == 0) trace_stamp(p, 4);
+                umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc);
             }
+            if (tr && lane == 0) { p.trace[8] = t_wait; p.trace[9] = t_issue; p.trace[10] = t_commit; p.trace[13] = t_acc; p.trace[15] = n_kb; }
         }
     } else {
-        // ===== epilogue (warps 2..5) =====
+        // ===== epilogue (warps 2..9) =====
+        // Two warps share each tensor-memory lane quarter (a warp may only touch lanes
+        // 32 * (warp % 4) .. + 31) and take alternate 32-column chunks of the accumulator.
+        const uint32_t ew = warp - 2u;                              // 0..7
         const uint32_t q = warp & 3u;                               // tensor-memory lane quarter of this warp
+        const uint32_t first_chunk = ew >> 2;                       // chunks first_chunk, first_chunk + 2, ...
         const uint32_t row_in_tile = q * 32u + lane;                // accumulator row = tensor-memory lane
-        const uint32_t staging = staging_base + (warp - 2u) * kStagingBytesPerWarp;
+        const uint32_t staging = staging_base + ew * kStagingBytesPerWarp;
         const uint32_t tmem_empty_leader = (CTA_GROUP == 2) ? mapa(bar_tmem_empty, 0) : bar_tmem_empty;
         const int32_t chunks = p.block_n / 32;
         uint32_t local_tile = 0;
@@ -335,126 +376,231 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int32_t grow = row0 + static_cast<int32_t>(row_in_tile);          // this thread's global row
             const uint32_t t_addr = tmem_base + ((q * 32u) << 16) + acc * static_cast<uint32_t>(p.block_n);
 
-            if (p.split_k == 1) {
-                for (int32_t c = 0; c < chunks; ++c) {
-                    uint32_t v[32];
-                    const int32_t col0 = it.n0 + c * 32;
-                    if (p.epilogue_tma) {
-                        const uint32_t buf = staging + (store_count & 1u) * (kStagingBytesPerWarp / 2);
-                        // the buffer written two stores ago must have been read by its TMA store
-                        if (lane == 0) bulk_wait_group_read<1>();
-                        __syncwarp();
-                        tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
-                        tmem_ld_wait();
-                        // row `lane` of the 32 x 32 box is 64 bytes; 64-byte swizzle: 16-byte chunk j of
-                        // row r lives at chunk j ^ ((r >> 1) & 3)
-                        const uint32_t row_addr = buf + lane * 64u;
-                        const uint32_t sw = (lane >> 1) & 3u;
+            // One 32-column chunk of this thread's row, converted and sent to C.
+            auto emit_chunk = [&](const uint32_t (&v)[32], int32_t c) {
+                const int32_t col0 = it.n0 + c * 32;
+                if (p.epilogue_tma) {
+                    const uint32_t buf = staging + (store_count & 1u) * (kStagingBytesPerWarp / 2);
+                    // the buffer written two stores ago must have been read by its TMA store
+                    if (lane == 0) bulk_wait_group_read<1>();
+                    __syncwarp();
+                    // row `lane` of the 32 x 32 box is 64 bytes; 64-byte swizzle: 16-byte chunk j of
+                    // row r lives at chunk j ^ ((r >> 1) & 3)
+                    const uint32_t row_addr = buf + lane * 64u;
+                    const uint32_t sw = (lane >> 1) & 3u;
 #pragma unroll
-                        for (uint32_t j = 0; j < 4; ++j) {
-                            st_shared_v4(row_addr + ((j ^ sw) << 4),
-                                         pack_half2_rn(v[8 * j + 0], v[8 * j + 1]), pack_half2_rn(v[8 * j + 2], v[8 * j + 3]),
-                                         pack_half2_rn(v[8 * j + 4], v[8 * j + 5]), pack_half2_rn(v[8 * j + 6], v[8 * j + 7]));
-                        }
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                            if (box_row < p.M && col0 < p.N) {
-                                tma_store_2d(&tmap_c, col0, box_row, buf);
-                            }
-                            bulk_commit_group();
-                        }
-                        ++store_count;
-                    } else {
-                        tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
-                        tmem_ld_wait();
-                        if (grow < p.M) {
-                            __half *dst = p.C + static_cast<size_t>(grow) * p.N + col0;
+                    for (uint32_t j = 0; j < 4; ++j) {
+                        st_shared_v4(row_addr + ((j ^ sw) << 4),
+                                     pack_half2_rn(v[8 * j + 0], v[8 * j + 1]), pack_half2_rn(v[8 * j + 2], v[8 * j + 3]),
+                                     pack_half2_rn(v[8 * j + 4], v[8 * j + 5]), pack_half2_rn(v[8 * j + 6], v[8 * j + 7]));
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
+                        if (box_row < p.M && col0 < p.N) tma_store_2d(&tmap_c, col0, box_row, buf);
+                        bulk_commit_group();
+                    }
+                    ++store_count;
+                } else if (grow < p.M) {
+                    __half *dst = p.C + static_cast<size_t>(grow) * p.N + col0;
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                if (col0 + 8 * j + 8 <= p.N) {
-                                    uint4 o;
-                                    o.x = pack_half2_rn(v[8 * j + 0], v[8 * j + 1]);
-                                    o.y = pack_half2_rn(v[8 * j + 2], v[8 * j + 3]);
-                                    o.z = pack_half2_rn(v[8 * j + 4], v[8 * j + 5]);
-                                    o.w = pack_half2_rn(v[8 * j + 6], v[8 * j + 7]);
-                                    *reinterpret_cast<uint4 *>(dst + 8 * j) = o;
-                                }
-                            }
+                    for (int j = 0; j < 4; ++j) {
+                        if (col0 + 8 * j + 8 <= p.N) {
+                            uint4 o;
+                            o.x = pack_half2_rn(v[8 * j + 0], v[8 * j + 1]);
+                            o.y = pack_half2_rn(v[8 * j + 2], v[8 * j + 3]);
+                            o.z = pack_half2_rn(v[8 * j + 4], v[8 * j + 5]);
+                            o.w = pack_half2_rn(v[8 * j + 6], v[8 * j + 7]);
+                            *reinterpret_cast<uint4 *>(dst + 8 * j) = o;
                         }
                     }
                 }
-                // accumulator drained: hand it back to the MMA issuer
+            };
+            auto release_accumulator = [&]() {
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) {
                     if constexpr (CTA_GROUP == 1) mbar_arrive(bar_tmem_empty + 8 * acc);
                     else mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
                 }
-            } else {
-                // ---- split-K: park the fp32 partial, the last slice to arrive reduces in slice order ----
-                const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
-                // one slot per (work item, CTA of the pair); layout [chunk][col][128 rows] so a warp's
-                // 32 rows of one column are one 128-byte line
-                float *slot = p.workspace + (static_cast<size_t>(w) * CTA_GROUP + cta_rank) * slot_floats;
-                for (int32_t c = 0; c < chunks; ++c) {
+            };
+
+            if (p.split_k == 1) {
+                // software pipeline: the load of the next chunk is in flight while this one is stored
+                uint32_t va[32], vb[32];
+                int32_t c = static_cast<int32_t>(first_chunk);
+                if (c < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, va);
+                while (c < chunks) {
+                    tmem_ld_wait();
+                    if (c + 2 < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c + 2) * 32u, vb);
+                    else release_accumulator();                    // every load of this warp has completed
+                    emit_chunk(va, c);
+                    c += 2;
+                    if (c >= chunks) break;
+                    tmem_ld_wait();
+                    if (c + 2 < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c + 2) * 32u, va);
+                    else release_accumulator();
+                    emit_chunk(vb, c);
+                    c += 2;
+                }
+                if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load (block_n == 32)
+            } else if (CTA_GROUP == 1 && p.cluster_split) {
+                // ---- split-K inside a cluster: stage the fp32 partial in this CTA's shared memory -------
+                // The stage ring is free: this CTA has exactly one work item, every load has landed and
+                // every MMA has completed.  Layout: float4 unit u = (chunk * 8 + column group) * 128 + row,
+                // so a warp's 32 rows of one column group are 512 contiguous bytes (no bank conflicts).
+                for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        __stcg(slot + (static_cast<size_t>(c) * 32 + j) * kBlockM + row_in_tile, __uint_as_float(v[j]));
+                    for (int g = 0; g < 8; ++g)
+                        st_shared_v4(smem_base + ((static_cast<uint32_t>(c) * 8u + g) * kBlockM + row_in_tile) * 16u,
+                                     v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                 }
-                tc_fence_before_sync();
+                release_accumulator();
+            } else {
+                // ---- split-K through a global workspace ---------------------------------------------------
+                // 1. park this slice's fp32 partial in the workspace: slot layout [chunk][128 rows][32 cols]
+                const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
+                float *slot = p.workspace + (static_cast<size_t>(w) * CTA_GROUP + cta_rank) * slot_floats;
+                for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
+                    tmem_ld_wait();
+                    if (grow < p.M && it.n0 + c * 32 < p.N) {
+                        float4 *dst = reinterpret_cast<float4 *>(slot + (static_cast<size_t>(c) * kBlockM + row_in_tile) * 32);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            __stcg(dst + j, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                        __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+                    }
+                }
+                release_accumulator();
+                if (w == unit && threadIdx.x == 64) trace_stamp(p, 16);
+                // 2. announce it, then wait (bounded) until every slice of this tile has done the same.
+                //    All slices of a tile are in flight together: the grid never exceeds the SM count, one
+                //    CTA per SM, and work items are handed out in tile order.
+                uint32_t *ctr = p.counters + (static_cast<size_t>(it.tile) * CTA_GROUP + cta_rank) * 2;
+                const uint32_t target = 8u * static_cast<uint32_t>(p.split_k);
                 __threadfence();
                 __syncwarp();
-                uint32_t prev = 0;
-                uint32_t *counter = p.counters + (static_cast<size_t>(it.tile) * CTA_GROUP + cta_rank) * 4 + q;
                 if (lane == 0) {
-                    if constexpr (CTA_GROUP == 1) mbar_arrive(bar_tmem_empty + 8 * acc);
-                    else mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
-                    prev = atomicAdd(counter, 1u);
-                    __threadfence();
-                }
-                prev = __shfl_sync(0xffffffffu, prev, 0);
-                if (prev == static_cast<uint32_t>(p.split_k) - 1u) {
-                    __threadfence();
-                    // all slices of this tile quarter are in the workspace: sum them in slice order
-                    const size_t first_slot = static_cast<size_t>(it.tile) * p.split_k;
-                    for (int32_t c = 0; c < chunks; ++c) {
-                        float accv[32];
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) accv[j] = 0.0f;
-                        for (int32_t sl = 0; sl < p.split_k; ++sl) {
-                            const float *src = p.workspace + ((first_slot + sl) * CTA_GROUP + cta_rank) * slot_floats;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                accv[j] += __ldcg(src + (static_cast<size_t>(c) * 32 + j) * kBlockM + row_in_tile);
+                    atomicAdd(ctr, 1u);
+                    const long long t0 = clock64();
+                    while (true) {
+                        uint32_t seen;
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(ctr) : "memory");
+                        if (seen >= target) break;
+                        if (*abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > p.wait_budget) {
+                            *abort_flag = 1u;
+                            atomicCAS(p.status, 0u, status_code(kRoleEpilogue, 3, it.slice));
+                            ok = false;
+                            break;
                         }
-                        const int32_t col0 = it.n0 + c * 32;
-                        if (grow < p.M) {
-                            __half *dst = p.C + static_cast<size_t>(grow) * p.N + col0;
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                if (col0 + 8 * j + 8 <= p.N) {
-                                    uint4 o;
-                                    o.x = pack_half2_rn(__float_as_uint(accv[8 * j + 0]), __float_as_uint(accv[8 * j + 1]));
-                                    o.y = pack_half2_rn(__float_as_uint(accv[8 * j + 2]), __float_as_uint(accv[8 * j + 3]));
-                                    o.z = pack_half2_rn(__float_as_uint(accv[8 * j + 4]), __float_as_uint(accv[8 * j + 5]));
-                                    o.w = pack_half2_rn(__float_as_uint(accv[8 * j + 6]), __float_as_uint(accv[8 * j + 7]));
-                                    *reinterpret_cast<uint4 *>(dst + 8 * j) = o;
-                                }
-                            }
-                        }
+                        __nanosleep(40);
                     }
-                    if (lane == 0) *counter = 0u;   // ready for the next run of this plan
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (w == unit && threadIdx.x == 64) trace_stamp(p, 17);
+                __threadfence();
+                // 3. every slice reduces its share of the tile.  A unit is four consecutive columns of one
+                //    row (one float4 per slice); slice s owns the contiguous unit range
+                //    [s U / S, (s + 1) U / S), so neighbouring threads read neighbouring addresses.  Each
+                //    unit is summed over the slices in slice order 0..S-1, up to 8 loads in flight.
+                const size_t first_slot = static_cast<size_t>(it.tile) * p.split_k;
+                const size_t slice_stride = static_cast<size_t>(CTA_GROUP) * slot_floats;
+                const float *tile_ws = p.workspace + (first_slot * CTA_GROUP + cta_rank) * slot_floats;
+                const int64_t units = static_cast<int64_t>(chunks) * kBlockM * 8;
+                const int32_t u_begin = static_cast<int32_t>(units * it.slice / p.split_k);
+                const int32_t u_end = static_cast<int32_t>(units * (it.slice + 1) / p.split_k);
+                for (int32_t u = u_begin + static_cast<int32_t>(ew * 32u + lane); u < u_end; u += 256) {
+                    const int32_t c = u >> 10, r = (u >> 3) & 127, g = u & 7;   // chunk, row, column group
+                    const int32_t orow = row0 + r, col = it.n0 + c * 32 + g * 4;
+                    if (orow >= p.M || col >= p.N) continue;
+                    const float4 *src = reinterpret_cast<const float4 *>(tile_ws) + u;   // [chunk][row][8 float4]
+                    float4 sum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    for (int32_t sl0 = 0; sl0 < p.split_k; sl0 += 8) {
+                        float4 x[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (sl0 + j < p.split_k)
+                                x[j] = __ldcg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(src) +
+                                                                               static_cast<size_t>(sl0 + j) * slice_stride));
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (sl0 + j < p.split_k) {
+                                sum.x += x[j].x; sum.y += x[j].y; sum.z += x[j].z; sum.w += x[j].w;
+                            }
+                    }
+                    uint2 o;
+                    o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
+                    o.y = pack_half2_rn(__float_as_uint(sum.z), __float_as_uint(sum.w));
+                    *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
+                }
+                // 4. the last warp of the last slice to finish re-arms the counters for the next launch
+                __syncwarp();
+                if (w == unit && threadIdx.x == 64) trace_stamp(p, 18);
+                if (lane == 0) {
+                    const uint32_t d = atomicAdd(ctr + 1, 1u);
+                    if (d == target - 1u) {
+                        ctr[0] = 0u;
+                        ctr[1] = 0u;
+                        __threadfence();
+                    }
                 }
             }
         }
         // shared memory must stay valid until the last TMA stores have read it
         if (lane == 0) bulk_wait_group<0>();
         if (threadIdx.x == 64) trace_stamp(p, 6);
+    }
+
+    // ---- cluster split-K: sum the slices through distributed shared memory -----------------
+    if constexpr (CTA_GROUP == 1) {
+        if (p.cluster_split) {
+            // every thread of every CTA of the cluster takes part in both barriers, also after an abort
+            cluster_arrive();
+            cluster_wait();
+            if (warp >= 2 && *abort_flag == 0u) {
+                const WorkItem it = decode_work(unit, p, kBlockMTotal);
+                const uint32_t ew = warp - 2u;
+                const int32_t chunks = p.block_n / 32;
+                // slice s sums the contiguous unit range [s U / S, (s + 1) U / S) over all slices, in
+                // slice order; the partial of slice r sits at the same offset in CTA r of the cluster
+                const int64_t units = static_cast<int64_t>(chunks) * 8 * kBlockM;
+                const int32_t u_begin = static_cast<int32_t>(units * it.slice / p.split_k);
+                const int32_t u_end = static_cast<int32_t>(units * (it.slice + 1) / p.split_k);
+                for (int32_t u = u_begin + static_cast<int32_t>(ew * 32u + lane); u < u_end; u += 256) {
+                    const int32_t c = u >> 10, g = (u >> 7) & 7, r = u & 127;
+                    const int32_t orow = it.m0 + r, col = it.n0 + c * 32 + g * 4;
+                    if (orow >= p.M || col >= p.N) continue;
+                    const uint32_t local = smem_base + static_cast<uint32_t>(u) * 16u;
+                    float4 sum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    for (int32_t sl0 = 0; sl0 < p.split_k; sl0 += 8) {
+                        float4 x[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (sl0 + j < p.split_k) x[j] = ld_shared_cluster_v4(mapa(local, static_cast<uint32_t>(sl0 + j)));
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (sl0 + j < p.split_k) {
+                                sum.x += x[j].x; sum.y += x[j].y; sum.z += x[j].z; sum.w += x[j].w;
+                            }
+                    }
+                    uint2 o;
+                    o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
+                    o.y = pack_half2_rn(__float_as_uint(sum.z), __float_as_uint(sum.w));
+                    *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
+                }
+            }
+            // nobody leaves while a peer may still read its shared memory
+            cluster_arrive();
+            cluster_wait();
+        }
     }
 
     // ---- teardown (every thread, also after an abort) ----------------------------------

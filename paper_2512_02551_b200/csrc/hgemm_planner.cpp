@@ -9,7 +9,7 @@ namespace hgemm_host {
 
 namespace {
 constexpr int64_t kATileBytes = 128 * 64 * 2;
-constexpr int64_t kStagingBytes = 16384;
+constexpr int64_t kStagingBytes = 32768;
 constexpr int64_t kCtrlBytes = 512;
 constexpr int64_t kAlignSlack = 1024;
 
@@ -18,7 +18,8 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 int64_t stage_bytes(const hgemm_config_t &c)
 {
-    return kATileBytes + int64_t(c.block_n / cta_group_of(c)) * 64 * 2;
+    const int64_t subs = c.block_k / 64;
+    return subs * (kATileBytes + int64_t(c.block_n / cta_group_of(c)) * 64 * 2);
 }
 
 int64_t smem_bytes(const hgemm_config_t &c)
@@ -26,12 +27,13 @@ int64_t smem_bytes(const hgemm_config_t &c)
     return kAlignSlack + int64_t(c.stages) * stage_bytes(c) + kStagingBytes + kCtrlBytes;
 }
 
-int32_t max_stages(int32_t family, int32_t block_n)
+int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k)
 {
     hgemm_config_t c;
     std::memset(&c, 0, sizeof(c));
     c.family = family;
     c.block_n = block_n;
+    c.block_k = block_k;
     const int64_t room = kSmemOptInBytes - kAlignSlack - kStagingBytes - kCtrlBytes;
     return int32_t(std::min<int64_t>(12, room / stage_bytes(c)));
 }
@@ -39,7 +41,7 @@ int32_t max_stages(int32_t family, int32_t block_n)
 int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c)
 {
     (void)K;
-    if (c.split_k <= 1) return 0;
+    if (c.split_k <= 1 || c.split_mode == HGEMM_SPLIT_CLUSTER) return 0;
     const int cg = cta_group_of(c);
     const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
     return tiles * c.split_k * cg * 128 * int64_t(c.block_n) * 4;
@@ -47,10 +49,10 @@ int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
 
 int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c)
 {
-    if (c.split_k <= 1) return 0;
+    if (c.split_k <= 1 || c.split_mode == HGEMM_SPLIT_CLUSTER) return 0;
     const int cg = cta_group_of(c);
     const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
-    return tiles * cg * 4 * 4;
+    return tiles * cg * 2 * 4;
 }
 
 hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K)
@@ -67,15 +69,23 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     if (s != HGEMM_OK) return s;
     if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA) return HGEMM_ERR_UNSUPPORTED;
     const int cg = cta_group_of(c);
-    if (c.block_m != 128 * cg || c.block_k != 64) return HGEMM_ERR_UNSUPPORTED;
+    if (c.block_m != 128 * cg || (c.block_k != 64 && c.block_k != 128)) return HGEMM_ERR_UNSUPPORTED;
     if (c.block_n < 32 || c.block_n > 256 || (c.block_n % 32) != 0) return HGEMM_ERR_UNSUPPORTED;
     if (c.stages < 1 || c.stages > 12) return HGEMM_ERR_UNSUPPORTED;
     if (smem_bytes(c) > kSmemOptInBytes) return HGEMM_ERR_UNSUPPORTED;
-    if (c.split_k < 1 || c.split_k > ceil_div(K, 64)) return HGEMM_ERR_UNSUPPORTED;
+    if (c.split_k < 1 || c.split_k > ceil_div(K, c.block_k)) return HGEMM_ERR_UNSUPPORTED;
+    // the slices of one tile wait for each other, so they must all be resident at once
+    if (c.split_k > kMaxSplitK) return HGEMM_ERR_UNSUPPORTED;
     if (c.raster_group < 1) return HGEMM_ERR_UNSUPPORTED;
     if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA) return HGEMM_ERR_UNSUPPORTED;
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 7; ++i)
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) return HGEMM_ERR_UNSUPPORTED;
+    if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) {
+        if (cg != 1 || c.split_k > 16) return HGEMM_ERR_UNSUPPORTED;
+        // the fp32 partial (128 x block_n) is staged in the shared-memory ring once the main loop is done
+        if (int64_t(c.stages) * stage_bytes(c) < int64_t(128) * c.block_n * 4) return HGEMM_ERR_UNSUPPORTED;
+    }
     const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
     if (tiles * c.split_k >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
     if (workspace_bytes(M, N, K, c) > kMaxWorkspaceBytes) return HGEMM_ERR_UNSUPPORTED;
@@ -99,10 +109,13 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     const int64_t work = tiles * c.split_k;
     const int64_t units = std::max(1, num_sms / cg);
     const int64_t waves = ceil_div(work, units);
-    const int64_t kb = ceil_div(K, 64);
+    const int64_t kb = ceil_div(K, c.block_k);
     const int64_t kb_per = ceil_div(kb, c.split_k);
     const double cta_bytes_kb = double(stage_bytes(c));
-    const double mma_kb = 128.0 * c.block_n * 64.0 / kMacPerClk;
+    // issuing one MMA costs the issuing thread about 70 cycles whatever its width, plus a fixed
+    // wait + commit per stage: narrow tiles are issue-bound
+    const double subs = c.block_k / 64.0;
+    const double mma_kb = std::max(128.0 * c.block_n * c.block_k / kMacPerClk, subs * 4.0 * 70.0 + 180.0);
     const double fill_kb = cta_bytes_kb / kSmFillBytesPerClk;
     const double concurrent_ctas = double(std::min(work, units)) * cg;
     const double l2_kb = concurrent_ctas * cta_bytes_kb / kL2BytesPerClk;
@@ -112,8 +125,12 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     double bytes = 2.0 * (double(M) * K + double(N) * K + double(M) * N);
     if (c.split_k > 1) {
         const double partial = 128.0 * c.block_n * 4.0;
-        t += partial / 64.0 + double(c.split_k) * partial / 128.0 + 1500.0;   // park + ordered reduce by the last slice
-        bytes += 2.0 * double(work) * cg * partial;
+        if (c.split_mode == HGEMM_SPLIT_CLUSTER) {
+            t += partial / 64.0 + partial / 96.0 + 2500.0;                      // stage in shared memory, two cluster barriers, pull
+        } else {
+            t += partial / 64.0 + partial / 48.0 + 9000.0;                      // park, signal, wait, pull through L2
+            bytes += 2.0 * double(work) * cg * partial;
+        }
     }
     t = std::max(t, bytes / kHbmBytesPerClk);
     return t + kLaunch;
@@ -135,18 +152,21 @@ hgemm_status_t heuristic(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm
             if (bn > 32 && bn - 32 >= N) break;   // a wider tile would only add padding
             for (int32_t split : kSplits) {
                 if (split > kb) break;
+                for (int mode = 0; mode < 2; ++mode) {
+                if (mode == 1 && (split == 1 || split > 16 || family != HGEMM_FAMILY_UMMA_1CTA)) continue;
                 hgemm_config_t c;
                 std::memset(&c, 0, sizeof(c));
+                c.split_mode = mode;
                 c.family = family;
                 c.block_m = 128 * cg;
                 c.block_n = bn;
-                c.block_k = 64;
+                c.block_k = (K >= 1024 && split == 1) ? 128 : 64;
                 c.split_k = split;
-                c.epilogue = HGEMM_EPILOGUE_DIRECT;
-                c.stages = std::max(1, std::min<int32_t>(max_stages(family, bn), 8));
+                c.epilogue = split == 1 ? HGEMM_EPILOGUE_TMA : HGEMM_EPILOGUE_DIRECT;
+                c.stages = std::max(1, std::min<int32_t>(max_stages(family, bn, c.block_k), 8));
                 const int64_t units = std::max(1, num_sms / cg);
                 const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, bn);
-                if (split > 1 && tiles * split > 2 * units) break;   // split-K only to fill an under-full machine
+                if (split > 1 && tiles * split > 2 * units) continue;   // split-K only to fill an under-full machine
                 const double g = std::sqrt(double(units) * bn / (128.0 * cg));
                 c.raster_group = int32_t(std::max<int64_t>(1, std::min<int64_t>(ceil_div(M, 128 * cg), int64_t(g + 0.5))));
                 if (validate(M, N, K, c) != HGEMM_OK) continue;
@@ -155,6 +175,7 @@ hgemm_status_t heuristic(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm
                     best = c;
                     best_t = t;
                     have = true;
+                }
                 }
             }
         }

@@ -15,12 +15,13 @@ namespace hgemm_host {
 constexpr int64_t kSmemOptInBytes = 232448;   // 227 KB per CTA on sm_100
 constexpr int64_t kMaxWorkspaceBytes = int64_t(2) << 30;
 constexpr int64_t kMaxDim = int64_t(1) << 22;
+constexpr int32_t kMaxSplitK = 64;            // at most this many slices per tile (all co-resident)
 
 inline int cta_group_of(const hgemm_config_t &c) { return c.family == HGEMM_FAMILY_UMMA_2CTA ? 2 : 1; }
 
 int64_t stage_bytes(const hgemm_config_t &c);
 int64_t smem_bytes(const hgemm_config_t &c);
-int32_t max_stages(int32_t family, int32_t block_n);
+int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k);
 int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c);
 int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c);
 hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K);

@@ -147,6 +147,15 @@ __device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank)
     return r;
 }
 
+// 16-byte load from the shared memory of any CTA of the cluster (address from mapa).
+__device__ __forceinline__ float4 ld_shared_cluster_v4(uint32_t cluster_addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ void cluster_arrive()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -229,6 +238,14 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
         asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// The same arrival delivered to the barrier at this shared-memory offset in every CTA of the
+// cluster named in cta_mask (used by a CTA pair to free a stage in both CTAs at once).
+__device__ __forceinline__ void umma_commit_pair_multicast(uint32_t bar, uint16_t cta_mask)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(cta_mask) : "memory");
+}
+
 // Whole warp: thread t reads 32 consecutive fp32 columns of tensor-memory lane (base lane + t).
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -247,6 +264,81 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
 __device__ __forceinline__ void tmem_ld_wait()
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// ---- predicated single-thread forms ------------------------------------------------------
+// The same instructions, executed by the whole warp in convergent code with a per-thread
+// predicate (true in one lane).  Predicating inside the asm block instead of branching in C++
+// keeps the surrounding code warp-uniform, so the compiler can hold the operands (descriptors,
+// barrier and shared-memory addresses, coordinates) in uniform registers, where TMA and tcgen05
+// instructions read them, instead of moving them there before every instruction.
+
+__device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t pred, uint32_t bar, uint32_t bytes)
+{
+    asm volatile(
+        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t}"
+        ::"r"(pred), "r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed_if(uint32_t pred, uint32_t cluster_bar, uint32_t bytes)
+{
+    asm volatile(
+        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "@e mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%1], %2;\n\t}"
+        ::"r"(pred), "r"(cluster_bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_2d_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%1], [%2, {%3, %4}], [%5];\n\t}"
+        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_2d_pair_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "@e cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%1], [%2, {%3, %4}], [%5];\n\t}"
+        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+template <int CTA_GROUP>
+__device__ __forceinline__ void umma_f16_if(uint32_t pred, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    if constexpr (CTA_GROUP == 1)
+        asm volatile(
+            "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 e, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "@e tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t}"
+            ::"r"(pred), "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 e, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "@e tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %4, p;\n\t}"
+            ::"r"(pred), "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+}
+
+template <int CTA_GROUP>
+__device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar)
+{
+    if constexpr (CTA_GROUP == 1)
+        asm volatile(
+            "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+            "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
+            ::"r"(pred), "r"(bar) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+            "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%1], %2;\n\t}"
+            ::"r"(pred), "r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
 }
 
 // ---- small helpers ------------------------------------------------------------------

@@ -16,13 +16,14 @@ LIB_PATH = os.path.join(HERE, "libhgemm.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(7)
 FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA = 0, 1
 EPILOGUE_DIRECT, EPILOGUE_TMA = 0, 1
+SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_plan_destroy",
-    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config",
+    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
-    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace",
+    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
 ]
 
@@ -37,23 +38,25 @@ class Config(ctypes.Structure):
     """Mirror of ``hgemm_config_t``."""
     _fields_ = [("family", ctypes.c_int32), ("block_m", ctypes.c_int32), ("block_n", ctypes.c_int32),
                 ("block_k", ctypes.c_int32), ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32),
-                ("raster_group", ctypes.c_int32), ("epilogue", ctypes.c_int32), ("reserved", ctypes.c_int32 * 8)]
+                ("raster_group", ctypes.c_int32), ("epilogue", ctypes.c_int32), ("split_mode", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 7)]
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
 
     @classmethod
     def make(cls, family=FAMILY_UMMA_1CTA, block_n=128, stages=4, split_k=1, raster_group=8,
-             epilogue=EPILOGUE_DIRECT) -> "Config":
+             epilogue=EPILOGUE_DIRECT, block_k=64, split_mode=0) -> "Config":
         c = cls()
         c.family = family
         c.block_m = 256 if family == FAMILY_UMMA_2CTA else 128
         c.block_n = block_n
-        c.block_k = 64
+        c.block_k = block_k
         c.stages = stages
         c.split_k = split_k
         c.raster_group = raster_group
         c.epilogue = epilogue
+        c.split_mode = split_mode
         return c
 
 
@@ -81,6 +84,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan_set_config": (i32, [p, cfgp]),
             "hgemm_heuristic_config": (i32, [i64, i64, i64, i32, cfgp]),
             "hgemm_validate_config": (i32, [i64, i64, i64, cfgp]),
+            "hgemm_estimate_config": (ctypes.c_double, [i64, i64, i64, i32, cfgp]),
             "hgemm_config_smem_bytes": (i64, [cfgp]),
             "hgemm_config_workspace_bytes": (i64, [i64, i64, i64, cfgp]),
             "hgemm_plan_launches_per_run": (i32, [p]),
@@ -88,6 +92,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_set_wait_budget": (i32, [p, i64]),
             "hgemm_debug_timeout_probe": (i32, [p, p]),
             "hgemm_debug_set_trace": (i32, [p, p]),
+            "hgemm_debug_set_skip": (i32, [p, ctypes.c_uint32]),
             "hgemm_last_cuda_error": (i32, [p]),
             "hgemm_status_string": (ctypes.c_char_p, [i32]),
         }
@@ -116,6 +121,10 @@ def heuristic_config(M: int, N: int, K: int, num_sms: int = 148) -> Config:
 
 def validate_config(M: int, N: int, K: int, cfg: Config) -> int:
     return int(lib().hgemm_validate_config(M, N, K, ctypes.byref(cfg)))
+
+
+def estimate_config(M: int, N: int, K: int, cfg: Config, num_sms: int = 148) -> float:
+    return float(lib().hgemm_estimate_config(M, N, K, num_sms, ctypes.byref(cfg)))
 
 
 def config_smem_bytes(cfg: Config) -> int:
@@ -208,6 +217,9 @@ class Plan:
 
     def set_trace(self, device_ptr: int) -> None:
         _check(lib().hgemm_debug_set_trace(self._h, ctypes.c_void_p(device_ptr)), "hgemm_debug_set_trace")
+
+    def set_skip(self, mask: int) -> None:
+        _check(lib().hgemm_debug_set_skip(self._h, int(mask)), "hgemm_debug_set_skip")
 
     def run_host(self, A, B, C, stream=None) -> None:
         """``hgemm_run_host`` on torch CPU tensors (pinned for an asynchronous call)."""

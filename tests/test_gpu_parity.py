@@ -134,7 +134,7 @@ UNIT_CASES = [
     (130, 264, 200, 256, 4, 1, 1),      # one row / one column group past a tile edge
     (384, 416, 192, 96, 4, 1, 2),       # tile width that is not a power of two
     (640, 480, 256, 160, 2, 1, 3),
-    (1024, 2048, 128, 32, 10, 1, 4),    # 512 tiles on 148 SMs: several tiles per CTA, accumulators alternate
+    (1024, 2048, 128, 32, 9, 1, 4),     # 512 tiles on 148 SMs: several tiles per CTA, accumulators alternate
     (2048, 2048, 64, 64, 2, 1, 16),
     (64, 64, 2048, 64, 4, 4, 1),        # split-K
     (300, 200, 1000, 96, 4, 16, 1),     # one k-block per slice

@@ -52,7 +52,7 @@ def test_heuristic_is_legal_over_the_grid(lib):
                 assert hgemm.validate_config(M, N, K, c) == hgemm.OK, (M, N, K, c.as_dict())
                 assert hgemm.config_smem_bytes(c) <= 232448
                 assert c.split_k <= (K + 63) // 64
-                if c.split_k > 1:
+                if c.split_k > 1 and c.split_mode == hgemm.SPLIT_WORKSPACE:
                     assert hgemm.config_workspace_bytes(M, N, K, c) > 0
                 else:
                     assert hgemm.config_workspace_bytes(M, N, K, c) == 0
@@ -63,7 +63,7 @@ def test_validate_rejects_illegal_configs(lib):
     ok = hgemm.Config.make(block_n=128, stages=4)
     assert hgemm.validate_config(M, N, K, ok) == hgemm.OK
     for kw in [dict(block_n=48), dict(block_n=288), dict(block_n=0), dict(stages=0), dict(stages=13),
-               dict(block_n=256, stages=5), dict(split_k=0), dict(split_k=17), dict(raster_group=0),
+               dict(block_n=256, stages=5), dict(split_k=0), dict(split_k=17), dict(block_k=32), dict(block_k=256), dict(raster_group=0),
                dict(epilogue=2), dict(family=2)]:
         c = hgemm.Config.make(**{**dict(block_n=128, stages=4), **kw})
         assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED, kw
@@ -73,15 +73,20 @@ def test_validate_rejects_illegal_configs(lib):
     c = hgemm.Config.make(block_n=128, stages=4)
     c.reserved[3] = 1
     assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
+    # cluster split-K: 1-CTA family only, at most 16 slices, the ring must hold the fp32 partial
+    assert hgemm.validate_config(M, N, 4096, hgemm.Config.make(block_n=128, stages=4, split_k=8, split_mode=1)) == hgemm.OK
+    for kw in [dict(family=1, split_k=4), dict(split_k=32), dict(block_n=256, stages=2, split_k=4)]:
+        c = hgemm.Config.make(**{**dict(block_n=128, stages=4, split_mode=1), **kw})
+        assert hgemm.validate_config(M, N, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
     pair = hgemm.Config.make(family=hgemm.FAMILY_UMMA_2CTA, block_n=256, stages=6)
     assert hgemm.validate_config(M, N, K, pair) == hgemm.OK
-    assert hgemm.config_smem_bytes(pair) == 1024 + 6 * (16384 + 128 * 128) + 16384 + 512
+    assert hgemm.config_smem_bytes(pair) == 1024 + 6 * (16384 + 128 * 128) + 32768 + 512
 
 
 def test_workspace_size(lib):
     c = hgemm.Config.make(block_n=64, stages=4, split_k=8)
-    # one 128 x 64 fp32 partial per slice + 4 counters of 4 bytes for the single tile
-    assert hgemm.config_workspace_bytes(64, 64, 8192, c) == 8 * 128 * 64 * 4 + 16
+    # one 128 x 64 fp32 partial per slice + 2 counters of 4 bytes for the single tile
+    assert hgemm.config_workspace_bytes(64, 64, 8192, c) == 8 * 128 * 64 * 4 + 8
 
 
 def test_no_gpu_create_fails_loudly(lib):
