@@ -50,7 +50,8 @@ typedef enum {
     HGEMM_ERR_ALLOC = 3,       /* host or device allocation failed */
     HGEMM_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (see hgemm_last_cuda_error) */
     HGEMM_ERR_ARCH = 5,        /* the device is not compute capability 10.0 */
-    HGEMM_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (see hgemm_last_device_status) */
+    HGEMM_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out (see hgemm_last_device_status) */
+    HGEMM_ERR_SCRATCH_LIMIT = 7 /* hgemm_run_splitk_static: the call needs more scratch than the built-in buffer holds */
 } hgemm_status_t;
 
 /* Kernel families (section 5.1 of the paper picks a different kernel structure
@@ -113,6 +114,42 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
  * copies block.  The first call on a plan allocates the staging (cudaMalloc,
  * synchronising): make it outside timed regions.  HGEMM_ERR_ALLOC if that fails. */
 hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void *B_host, void *C_host, void *stream);
+
+/* Split-K GEMM for callers that must not allocate.  (The paper has no counterpart:
+ * this entry point exists for deployment, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a serving
+ * process whose memory was frozen at start-up, a callback inside another library, a
+ * job under a fixed-footprint policy.  hgemm_create and hgemm_plan call cudaMalloc,
+ * so such callers cannot use them; this function needs neither a context nor a plan
+ * and calls no cudaMalloc, cudaFree or any other allocating routine.  The split-K
+ * partial sums, the arrival counters and the status word live in one static device
+ * array inside the library: 8 MiB of partial sums plus a 4 KiB control page, held by
+ * every GPU that loads the library until the process exits.
+ *
+ * Same operation and layouts as hgemm_run (A: M x K, B: N x K, C: M x N, fp16, DEVICE
+ * pointers, 16-byte aligned, caller-owned) on the calling thread's CURRENT device,
+ * with the 1-CTA kernel family, tile width `block_n` (multiple of 32 in [32, 256]),
+ * 64-wide K stages and `split_k` K slices summed in slice order through that array
+ * (split_k == 1 is allowed and uses no scratch).  Asynchronous on `stream`.
+ *
+ * Limits and errors, checked before anything is launched:
+ *   - ceil(M/128) * ceil(N/block_n) * split_k * 128 * block_n * 4 bytes of partial sums
+ *     must fit in 8 MiB and the tile count in the control page (at most 480 tiles),
+ *     else HGEMM_ERR_SCRATCH_LIMIT;
+ *   - split_k <= min(64, ceil(K/64), SM count); shape rules as for hgemm_plan, else
+ *     HGEMM_ERR_UNSUPPORTED / HGEMM_ERR_INVALID_ARG; HGEMM_ERR_ARCH off sm_100.
+ *
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) and sets the kernel's shared-memory limit; make that first
+ * call before any stream capture begins.  Every call shares the one array, which
+ * keeps the previous call's contents: the function clears the control page on
+ * `stream` before each launch (the partial sums need no clearing), and two calls that
+ * overlap on the GPU -- different streams, or different threads -- race on it.
+ * Serialise them.  A bounded wait that runs out leaves C undefined; this variant has
+ * no status read-back. */
+hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t K, int32_t block_n, int32_t split_k,
+                                       const void *A, const void *B, void *C, void *stream);
 
 /* Free one plan early (hgemm_destroy frees the rest). */
 hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan);

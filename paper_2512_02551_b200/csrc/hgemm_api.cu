@@ -210,6 +210,7 @@ const char *hgemm_status_string(hgemm_status_t s)
     case HGEMM_ERR_CUDA: return "CUDA call failed";
     case HGEMM_ERR_ARCH: return "device is not compute capability 10.0";
     case HGEMM_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case HGEMM_ERR_SCRATCH_LIMIT: return "the call needs more scratch memory than the library's built-in buffer holds";
     }
     return "unknown status";
 }

@@ -13,14 +13,14 @@ import os
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhgemm.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_SCRATCH_LIMIT = range(8)
 FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA = 0, 1
 EPILOGUE_DIRECT, EPILOGUE_TMA = 0, 1
 SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
-    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_plan_destroy",
+    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
@@ -79,6 +79,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan": (i32, [p, i64, i64, i64, ctypes.POINTER(p)]),
             "hgemm_run": (i32, [p, p, p, p, p]),
             "hgemm_run_host": (i32, [p, p, p, p, p]),
+            "hgemm_run_splitk_static": (i32, [i64, i64, i64, i32, i32, p, p, p, p]),
             "hgemm_plan_destroy": (i32, [p]),
             "hgemm_plan_get_config": (i32, [p, cfgp]),
             "hgemm_plan_set_config": (i32, [p, cfgp]),
@@ -133,6 +134,13 @@ def config_smem_bytes(cfg: Config) -> int:
 
 def config_workspace_bytes(M: int, N: int, K: int, cfg: Config) -> int:
     return int(lib().hgemm_config_workspace_bytes(M, N, K, ctypes.byref(cfg)))
+
+
+def run_splitk_static(M: int, N: int, K: int, block_n: int, split_k: int, a_ptr: int, b_ptr: int, c_ptr: int,
+                      stream: int = 0) -> int:
+    """``hgemm_run_splitk_static`` on raw device pointers: the split-K GEMM whose scratch memory is a
+    static array inside the library, for callers that may not allocate.  Returns the status."""
+    return int(lib().hgemm_run_splitk_static(M, N, K, block_n, split_k, a_ptr, b_ptr, c_ptr, stream))
 
 
 class Context:

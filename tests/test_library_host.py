@@ -28,8 +28,8 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_status_strings(lib):
-    seen = {hgemm.status_string(s) for s in range(7)}
-    assert len(seen) == 7 and "ok" in seen
+    seen = {hgemm.status_string(s) for s in range(8)}
+    assert len(seen) == 8 and "ok" in seen
 
 
 def test_shape_rules(lib):
