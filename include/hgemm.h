@@ -189,6 +189,14 @@ hgemm_status_t hgemm_last_device_status(hgemm_ctx_t *ctx, uint32_t *code);
  * second).  Affects plans created afterwards and later hgemm_run calls. */
 hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles);
 
+/* hgemm_run launches with programmatic stream serialisation (on by default): the
+ * kernel may become resident, and run the set-up that touches no global memory,
+ * while the kernel ahead of it in the stream is still finishing; it waits for that
+ * kernel's completion before its first global-memory access, so stream order is
+ * kept for every buffer.  Back-to-back calls then overlap launch latency and set-up
+ * with the previous call's tail.  enabled = 0 restores plain stream-ordered launches. */
+hgemm_status_t hgemm_set_dependent_launch(hgemm_ctx_t *ctx, int32_t enabled);
+
 /* Test hook for the timeout path: launches one small kernel on `stream` whose
  * only wait is on a barrier that nothing signals, with the context's wait
  * budget.  The kernel returns by itself; hgemm_last_device_status then reports
@@ -197,7 +205,7 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
 
 /* Instrumentation: when `device_buf` (DEVICE pointer to 24 uint64, or NULL to switch
  * it off) is set, CTA 0 of every later launch of this plan writes nanosecond
- * %globaltimer stamps of its pipeline events: 0 kernel entry, 1 set-up done,
+ * %globaltimer stamps of its pipeline events: 0 dependencies met, 1 set-up done,
  * 2 first TMA load issued, 3 first k-block landed, 4 last MMA issued, 5 first
  * accumulator ready, 6 epilogue done, 7 tensor memory freed; and SM-clock totals:
  * 8/9/10 MMA thread waiting for data / issuing MMAs / committing, 11/12 producer

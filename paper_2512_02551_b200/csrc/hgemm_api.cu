@@ -25,6 +25,7 @@ struct hgemm_ctx_s {
     long long wait_budget = 2000000000LL;
     encode_tiled_fn encode = nullptr;
     int last_cuda_error = 0;
+    bool dependent_launch = true;
     std::vector<hgemm_plan_s *> plans;
 };
 
@@ -435,13 +436,17 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     lc.blockDim = dim3(hgemm_dev::kThreads, 1, 1);
     lc.dynamicSmemBytes = size_t(plan->smem);
     lc.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = unsigned(plan->cluster_dim);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // programmatic stream serialisation: this launch may become resident before the kernel ahead of
+    // it in the stream has finished; the kernel itself waits for that kernel before it touches memory
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = 1;
+    lc.numAttrs = ctx->dependent_launch ? 2 : 1;
     cudaError_t e;
     if (cg == 1)
         e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, me->tmap_a, me->tmap_b, me->tmap_c, plan->params);
@@ -515,6 +520,13 @@ hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles)
 {
     if (!ctx || cycles < 1) return HGEMM_ERR_INVALID_ARG;
     ctx->wait_budget = cycles;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_set_dependent_launch(hgemm_ctx_t *ctx, int32_t enabled)
+{
+    if (!ctx) return HGEMM_ERR_INVALID_ARG;
+    ctx->dependent_launch = enabled != 0;
     return HGEMM_OK;
 }
 

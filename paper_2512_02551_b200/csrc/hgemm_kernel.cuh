@@ -205,8 +205,12 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     WaitCtl ctl{abort_flag, p.status, p.wait_budget};
 
     // ---- set-up -----------------------------------------------------------------------
+    // Programmatic dependent launch: the next kernel in the stream may become resident (on SMs this
+    // grid does not occupy, or as its CTAs retire) and run its own set-up while this grid works.
+    // Nothing below touches global memory until grid_dependency_wait() has returned, so a dependent
+    // launch never sees or disturbs the data of the kernel before it.
+    grid_launch_dependents();
     if (threadIdx.x == 0) {
-        trace_stamp(p, 0);
         *abort_flag = 0u;
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(bar_full + 8 * s, CTA_GROUP);   // one arrive.expect_tx per CTA of the pair
@@ -232,7 +236,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         cluster_wait();
     }
     tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_base_slot;
+    grid_dependency_wait();          // from here on global memory may be read and written
+    if (threadIdx.x == 0) trace_stamp(p, 0);
+    // broadcast through a shuffle so that the compiler knows the address is warp-uniform
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_base_slot, 0);
     if (threadIdx.x == 0) trace_stamp(p, 1);
 
     // ---- roles ------------------------------------------------------------------------

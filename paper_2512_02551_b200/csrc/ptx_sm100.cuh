@@ -130,6 +130,22 @@ __device__ __forceinline__ void fence_proxy_async_smem()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// ---- programmatic dependent launch -------------------------------------------------
+
+// Lets the next kernel in the stream (if it was launched with programmatic stream
+// serialisation) become resident once every CTA of this grid has executed this or exited.
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Blocks until every kernel this grid depends on has completed and its memory operations are
+// visible.  Returns at once when the grid was launched without a programmatic dependency.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- cluster --------------------------------------------------------------------
 
 __device__ __forceinline__ uint32_t cluster_ctarank()
@@ -276,7 +292,7 @@ __device__ __forceinline__ void tmem_ld_wait()
 __device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t pred, uint32_t bar, uint32_t bytes)
 {
     asm volatile(
-        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
         "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t}"
         ::"r"(pred), "r"(bar), "r"(bytes) : "memory");
 }
@@ -284,7 +300,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t pred, uint32_t
 __device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed_if(uint32_t pred, uint32_t cluster_bar, uint32_t bytes)
 {
     asm volatile(
-        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
         "@e mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%1], %2;\n\t}"
         ::"r"(pred), "r"(cluster_bar), "r"(bytes) : "memory");
 }
@@ -292,7 +308,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed_if(uint32_
 __device__ __forceinline__ void tma_load_2d_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
 {
     asm volatile(
-        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
         "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%1], [%2, {%3, %4}], [%5];\n\t}"
         ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
         : "memory");
@@ -301,7 +317,7 @@ __device__ __forceinline__ void tma_load_2d_if(uint32_t pred, uint32_t dst, cons
 __device__ __forceinline__ void tma_load_2d_pair_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
 {
     asm volatile(
-        "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
         "@e cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
         " [%1], [%2, {%3, %4}], [%5];\n\t}"
         ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
@@ -314,13 +330,13 @@ __device__ __forceinline__ void umma_f16_if(uint32_t pred, uint32_t d_tmem, uint
 {
     if constexpr (CTA_GROUP == 1)
         asm volatile(
-            "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 e, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
             "@e tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t}"
             ::"r"(pred), "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
     else
         asm volatile(
-            "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 e, %0, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
             "@e tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %4, p;\n\t}"
             ::"r"(pred), "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
@@ -331,12 +347,12 @@ __device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar)
 {
     if constexpr (CTA_GROUP == 1)
         asm volatile(
-            "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+            "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
             "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
             ::"r"(pred), "r"(bar) : "memory");
     else
         asm volatile(
-            "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %0, 0;\n\t"
+            "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
             "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%1], %2;\n\t}"
             ::"r"(pred), "r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
 }

@@ -23,7 +23,7 @@ EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
-    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
+    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
 ]
 
@@ -91,6 +91,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan_launches_per_run": (i32, [p]),
             "hgemm_last_device_status": (i32, [p, ctypes.POINTER(ctypes.c_uint32)]),
             "hgemm_set_wait_budget": (i32, [p, i64]),
+            "hgemm_set_dependent_launch": (i32, [p, i32]),
             "hgemm_debug_timeout_probe": (i32, [p, p]),
             "hgemm_debug_set_trace": (i32, [p, p]),
             "hgemm_debug_set_skip": (i32, [p, ctypes.c_uint32]),
@@ -156,6 +157,9 @@ class Context:
 
     def set_wait_budget(self, cycles: int) -> None:
         _check(lib().hgemm_set_wait_budget(self._h, int(cycles)), "hgemm_set_wait_budget")
+
+    def set_dependent_launch(self, enabled: bool) -> None:
+        _check(lib().hgemm_set_dependent_launch(self._h, 1 if enabled else 0), "hgemm_set_dependent_launch")
 
     def last_device_status(self) -> tuple[int, int]:
         """(status, code); synchronises the device."""
