@@ -31,8 +31,12 @@ def gu():
     return gpu_util
 
 
-def _cfg(family=F1, bn=128, stages=4, split=1, raster=8, epi=DIRECT):
-    return hgemm.Config.make(family=family, block_n=bn, stages=stages, split_k=split, raster_group=raster, epilogue=epi)
+WORKSPACE, CLUSTER = hgemm.SPLIT_WORKSPACE, hgemm.SPLIT_CLUSTER
+
+
+def _cfg(family=F1, bn=128, stages=4, split=1, raster=8, epi=DIRECT, bk=64, mode=WORKSPACE):
+    return hgemm.Config.make(family=family, block_n=bn, stages=stages, split_k=split, raster_group=raster, epilogue=epi,
+                             block_k=bk, split_mode=mode)
 
 
 VARIANTS = [(F1, DIRECT), (F1, TMA), (F2, DIRECT), (F2, TMA)]
@@ -141,6 +145,20 @@ UNIT_CASES = [
     (512, 384, 640, 128, 4, 3, 2),      # uneven slices (10 k-blocks over 3)
 ]
 
+# M, N, K, bn, stages, split, raster, block_k, split mode: 128-wide K stages and cluster split-K
+UNIT_CASES_WIDE = [
+    (128, 128, 64, 128, 2, 1, 1, 128, WORKSPACE),     # K shorter than one stage: second sub-tile all zero-fill
+    (256, 256, 1024, 256, 2, 1, 1, 128, WORKSPACE),   # ring wraps
+    (100, 136, 200, 64, 4, 1, 1, 128, WORKSPACE),     # ragged everywhere, K = 1.56 stages
+    (640, 480, 1152, 160, 2, 1, 3, 128, WORKSPACE),
+    (300, 200, 1000, 96, 3, 4, 1, 128, WORKSPACE),    # split-K over 128-wide stages (8 stages over 4 slices)
+    (64, 64, 4096, 64, 4, 8, 1, 64, CLUSTER),         # one tile, eight slices in one cluster
+    (100, 136, 520, 32, 4, 9, 1, 64, CLUSTER),        # more slices than a portable cluster (non-portable size 9)
+    (512, 384, 640, 128, 4, 3, 2, 64, CLUSTER),       # uneven slices
+    (300, 200, 1000, 96, 3, 4, 1, 128, CLUSTER),
+    (256, 512, 12288, 256, 4, 16, 1, 64, CLUSTER),    # largest cluster, widest tile (128 KB partial in shared memory)
+]
+
 
 @pytest.mark.parametrize("family", [F1, F2])
 @pytest.mark.parametrize("case", UNIT_CASES, ids=lambda c: "x".join(map(str, c[:3])) + f"-bn{c[3]}s{c[4]}k{c[5]}")
@@ -158,6 +176,49 @@ def test_unit_shapes(ctx, gu, family, case):
         plan.close()
         if split > 1:
             break                         # split-K always finishes with direct stores
+
+
+@pytest.mark.parametrize("case", UNIT_CASES_WIDE, ids=lambda c: "x".join(map(str, c[:3])) + f"-bn{c[3]}s{c[4]}k{c[5]}bk{c[7]}m{c[8]}")
+def test_unit_shapes_wide_stages_and_cluster_split(ctx, gu, case):
+    import oracle
+    M, N, K, bn, stages, split, raster, bk, mode = case
+    for family in ((F1,) if mode == CLUSTER else (F1, F2)):
+        cfg = _cfg(family, bn, stages, split, raster, TMA if split == 1 else DIRECT, bk, mode)
+        A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+        C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+        gu.assert_close_full(C, A, B, f"{case} family={family}")
+        Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+        Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+        gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"{case} integers")
+        plan.close()
+
+
+def test_dependent_launch_keeps_stream_order(ctx, gu):
+    """Launches may become resident before the kernel ahead of them has finished.  A chain in which each
+    GEMM consumes the previous GEMM's output must still see stream order: C1 = A B1^T, C2 = C1 B2^T."""
+    import oracle
+    M, K1, N1, N2 = 512, 64, 64, 384
+    A = inputs.draw(1, inputs.TAG_A, M, K1, "int5", "cuda")
+    B1 = inputs.draw(2, inputs.TAG_B, N1, K1, "int5", "cuda")
+    B2 = inputs.draw(3, inputs.TAG_B, N2, N1, "int5", "cuda")
+    c1_ref = oracle.hgemm_full(inputs.bits(A), inputs.bits(B1))                 # |c| <= 256: exact in fp16
+    c1_bits = oracle.f64_to_f16_bits(c1_ref.ravel()).reshape(M, N1)
+    c2_ref = oracle.hgemm_full(c1_bits, inputs.bits(B2))                        # sums < 2^24: exact in fp32
+    p1, p2 = ctx.plan(M, N1, K1), ctx.plan(M, N2, N1)
+    for enabled in (True, False):
+        ctx.set_dependent_launch(enabled)
+        for rep in range(25):
+            C1 = torch.zeros(M, N1, dtype=torch.float16, device="cuda")
+            C2 = torch.zeros(M, N2, dtype=torch.float16, device="cuda")
+            p1.run(A, B1, C1)
+            p2.run(C1, B2, C2)
+            p1.run(A, B1, C1)                                                   # overwrites what p2 is reading from? no: same values
+            torch.cuda.synchronize()
+            gu.assert_exact(C2, c2_ref, f"chain, dependent launch {enabled}, repetition {rep}")
+    ctx.set_dependent_launch(True)
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    p1.close()
+    p2.close()
 
 
 # ---- configuration 2: square sweep ---------------------------------------------------------------------
@@ -193,13 +254,15 @@ def test_config4_small_mn_large_k(ctx, gu, MN, K):
     gu.check_shape(ctx, MN, MN, K, "uniform")
 
 
-@pytest.mark.parametrize("family", [F1, F2])
+@pytest.mark.parametrize("family,mode", [(F1, WORKSPACE), (F2, WORKSPACE), (F1, CLUSTER)])
 @pytest.mark.parametrize("MN,K,bn,split", [(64, 8192, 64, 8), (64, 12288, 32, 48), (256, 12288, 128, 12),
                                             (512, 8192, 128, 6), (512, 12288, 256, 16)])
-def test_split_k_is_deterministic(ctx, gu, family, MN, K, bn, split):
+def test_split_k_is_deterministic(ctx, gu, family, mode, MN, K, bn, split):
     """Every split-K configuration reproduces its own bits run after run, with other work in flight
     to perturb the order in which slices finish."""
-    cfg = _cfg(family, bn, 4, split, 1, DIRECT)
+    if mode == CLUSTER and split > 16:
+        pytest.skip("a cluster holds at most 16 slices")
+    cfg = _cfg(family, bn, 4, split, 1, DIRECT, 64, mode)
     A, B = inputs.make_ab(MN, MN, K, "uniform", "cuda")
     C0, _, plan = gu.run_gemm(ctx, A, B, cfg)
     gu.assert_close_full(C0, A, B, f"split-K {cfg.as_dict()}")
