@@ -211,7 +211,8 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
  * 8/9/10 MMA thread waiting for data / issuing MMAs / committing, 11/12 producer
  * waiting for a free stage / issuing loads, 13 MMA thread waiting for a free
  * accumulator, 15 k-blocks processed; and for split-K stamps 16 partial parked,
- * 17 all slices arrived, 18 share reduced.  The caller owns the buffer. */
+ * 17 all slices arrived, 18 share reduced; for cluster split-K 19 cluster gathered,
+ * 20 share reduced, 21 cluster released.  The caller owns the buffer. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan

@@ -26,6 +26,7 @@ struct hgemm_ctx_s {
     encode_tiled_fn encode = nullptr;
     int last_cuda_error = 0;
     bool dependent_launch = true;
+    bool tma_3d = true;
     std::vector<hgemm_plan_s *> plans;
 };
 
@@ -167,6 +168,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.counters = pl->counters;
     p.status = ctx->d_status;
     p.cluster_split = cluster_split ? 1 : 0;
+    p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d) ? 1 : 0;
     p.C = nullptr;
     p.wait_budget = ctx->wait_budget;
     const int units = std::max(1, ctx->num_sms / cg);
@@ -189,6 +191,25 @@ bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t in
     cuuint32_t estr[2] = {1, 1};
     CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda_error = int(r);
+        return false;
+    }
+    return true;
+}
+
+// A and B as 3-D tensors {64, rows, K / 64}: element (x, y, z) = row y, column 64 z + x.  A box
+// {64, rows, 2} then lands as two consecutive 64-wide sub-tiles, which is the layout of a 128-wide stage.
+// Only valid when K is a multiple of 64 (dimension 0 must not run past the end of a row).
+bool encode_3d_ksub(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t K, uint64_t rows, uint32_t box_rows)
+{
+    cuuint64_t dims[3] = {64, rows, K / 64};
+    cuuint64_t strides[2] = {K * 2, 128};   // bytes: next row, next 64-wide sub-tile
+    cuuint32_t box[3] = {64, box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         ctx->last_cuda_error = int(r);
@@ -414,9 +435,14 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
         e.a = e.b = nullptr;
         e.c = nullptr;
         const uint64_t M = uint64_t(plan->M), N = uint64_t(plan->N), K = uint64_t(plan->K);
-        if (!encode_2d(ctx, &e.tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
-        if (!encode_2d(ctx, &e.tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
-            return HGEMM_ERR_CUDA;
+        if (plan->params.tma_3d) {
+            if (!encode_3d_ksub(ctx, &e.tmap_a, A, K, M, 128)) return HGEMM_ERR_CUDA;
+            if (!encode_3d_ksub(ctx, &e.tmap_b, B, K, N, uint32_t(cfg.block_n / cg))) return HGEMM_ERR_CUDA;
+        } else {
+            if (!encode_2d(ctx, &e.tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
+            if (!encode_2d(ctx, &e.tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
+                return HGEMM_ERR_CUDA;
+        }
         if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return HGEMM_ERR_CUDA;
         e.a = A;
         e.b = B;

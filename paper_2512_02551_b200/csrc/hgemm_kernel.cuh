@@ -28,6 +28,8 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "ptx_sm100.cuh"
 
 namespace hgemm_dev {
@@ -60,6 +62,7 @@ struct KernelParams {
     int32_t raster_group;
     int32_t tmem_cols;            // power of two >= 2 * block_n
     int32_t epilogue_tma;         // 1: TMA-store epilogue (only when split_k == 1)
+    int32_t tma_3d;               // 1: the A and B maps are 3-D {64, rows, K / 64}: one load per operand per stage
     int32_t cluster_split;        // 1: the split_k slices of a tile are one cluster and reduce through shared memory
     uint32_t idesc;               // tcgen05 instruction descriptor
     float *workspace;             // split-K partials: [work item][cta of pair][chunk][128 rows][32 cols]
@@ -275,6 +278,19 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (is_leader) mbar_arrive(bar_full + 8 * s);
                         else mbar_arrive_cluster(fb);
                     }
+                } else if (p.tma_3d) {
+                    // one instruction per operand: dimension 2 of the map counts 64-wide K sub-tiles
+                    const int32_t ksub = k0 / kSubK;
+                    if constexpr (CTA_GROUP == 1) {
+                        mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                        tma_load_3d_if(leader, a_dst, &tmap_a, 0, a_row, ksub, bar_full + 8 * s);
+                        tma_load_3d_if(leader, b_dst, &tmap_b, 0, b_row, ksub, bar_full + 8 * s);
+                    } else {
+                        if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                        else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, stage_bytes);
+                        tma_load_3d_pair_if(leader, a_dst, &tmap_a, 0, a_row, ksub, fb);
+                        tma_load_3d_pair_if(leader, b_dst, &tmap_b, 0, b_row, ksub, fb);
+                    }
                 } else if constexpr (CTA_GROUP == 1) {
                     mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
                     for (int32_t sub = 0; sub < subs; ++sub) {
@@ -453,20 +469,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load (block_n == 32)
             } else if (CTA_GROUP == 1 && p.cluster_split) {
-                // ---- split-K inside a cluster: stage the fp32 partial in this CTA's shared memory -------
-                // The stage ring is free: this CTA has exactly one work item, every load has landed and
-                // every MMA has completed.  Layout: float4 unit u = (chunk * 8 + column group) * 128 + row,
-                // so a warp's 32 rows of one column group are 512 contiguous bytes (no bank conflicts).
-                for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
-                    uint32_t v[32];
-                    tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        st_shared_v4(smem_base + ((static_cast<uint32_t>(c) * 8u + g) * kBlockM + row_in_tile) * 16u,
-                                     v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                }
-                release_accumulator();
+                // split-K inside a cluster: the accumulator is complete; the exchange below needs every
+                // thread of the CTA, so it happens after the role branches
             } else {
                 // ---- split-K through a global workspace ---------------------------------------------------
                 // 1. park this slice's fp32 partial in the workspace: slot layout [chunk][128 rows][32 cols]
@@ -567,36 +571,59 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 
     // ---- cluster split-K: sum the slices through distributed shared memory -----------------
+    // The S slices of a tile are the S CTAs of one cluster.  The tile's float4 units
+    // u = (chunk * 8 + column group) * 128 + row are dealt out in contiguous shares of `cap` units:
+    // CTA o owns [o cap, (o + 1) cap).  Every CTA pushes each unit of its fp32 partial into the owner's
+    // shared memory (slot = the pusher's slice index), and after a cluster barrier every owner adds
+    // the S slots of each of its units in slice order and stores fp16.  Both barriers are taken by
+    // every thread of every CTA of the cluster, also after an abort.
     if constexpr (CTA_GROUP == 1) {
         if (p.cluster_split) {
-            // every thread of every CTA of the cluster takes part in both barriers, also after an abort
+            // barrier 1: every CTA has finished its main loop (its epilogue warps arrive only after the last
+            // MMA has completed), so the stage rings are free to receive
             cluster_arrive();
             cluster_wait();
-            if (warp >= 2 && *abort_flag == 0u) {
-                const WorkItem it = decode_work(unit, p, kBlockMTotal);
+            const WorkItem it = decode_work(unit, p, kBlockMTotal);
+            const int32_t chunks = p.block_n / 32;
+            const uint32_t units = static_cast<uint32_t>(chunks) * 8u * kBlockM;
+            const uint32_t cap = (units + static_cast<uint32_t>(p.split_k) - 1u) / static_cast<uint32_t>(p.split_k);
+            const bool live = *abort_flag == 0u;
+            if (threadIdx.x == 64) trace_stamp(p, 19);
+            if (warp >= 2 && live) {
+                const uint32_t ew = warp - 2u, q = warp & 3u;
+                const uint32_t row_in_tile = q * 32u + lane;
+                const uint32_t t_addr = tmem_base + ((q * 32u) << 16);      // the only work item used accumulator 0
+                tc_fence_after_sync();
+                for (int32_t c = static_cast<int32_t>(ew >> 2); c < chunks; c += 2) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (uint32_t g = 0; g < 8; ++g) {
+                        const uint32_t u = (static_cast<uint32_t>(c) * 8u + g) * kBlockM + row_in_tile;
+                        const uint32_t owner = u / cap, li = u - owner * cap;
+                        const uint32_t dst = smem_base + (static_cast<uint32_t>(it.slice) * cap + li) * 16u;
+                        st_shared_cluster_v4(mapa(dst, owner), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    }
+                }
+            }
+            // barrier 2: every push has landed (release / acquire at cluster scope)
+            cluster_arrive();
+            cluster_wait();
+            if (threadIdx.x == 64) trace_stamp(p, 20);
+            if (warp >= 2 && live) {
                 const uint32_t ew = warp - 2u;
-                const int32_t chunks = p.block_n / 32;
-                // slice s sums the contiguous unit range [s U / S, (s + 1) U / S) over all slices, in
-                // slice order; the partial of slice r sits at the same offset in CTA r of the cluster
-                const int64_t units = static_cast<int64_t>(chunks) * 8 * kBlockM;
-                const int32_t u_begin = static_cast<int32_t>(units * it.slice / p.split_k);
-                const int32_t u_end = static_cast<int32_t>(units * (it.slice + 1) / p.split_k);
-                for (int32_t u = u_begin + static_cast<int32_t>(ew * 32u + lane); u < u_end; u += 256) {
-                    const int32_t c = u >> 10, g = (u >> 7) & 7, r = u & 127;
+                const uint32_t own_begin = static_cast<uint32_t>(it.slice) * cap;
+                const uint32_t own_count = own_begin >= units ? 0u : min(cap, units - own_begin);
+                for (uint32_t li = ew * 32u + lane; li < own_count; li += 256u) {
+                    const uint32_t u = own_begin + li;
+                    const int32_t c = static_cast<int32_t>(u >> 10), g = static_cast<int32_t>((u >> 7) & 7u), r = static_cast<int32_t>(u & 127u);
                     const int32_t orow = it.m0 + r, col = it.n0 + c * 32 + g * 4;
                     if (orow >= p.M || col >= p.N) continue;
-                    const uint32_t local = smem_base + static_cast<uint32_t>(u) * 16u;
                     float4 sum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    for (int32_t sl0 = 0; sl0 < p.split_k; sl0 += 8) {
-                        float4 x[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (sl0 + j < p.split_k) x[j] = ld_shared_cluster_v4(mapa(local, static_cast<uint32_t>(sl0 + j)));
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (sl0 + j < p.split_k) {
-                                sum.x += x[j].x; sum.y += x[j].y; sum.z += x[j].z; sum.w += x[j].w;
-                            }
+                    for (int32_t sl = 0; sl < p.split_k; ++sl) {
+                        const float4 x = ld_shared_v4(smem_base + (static_cast<uint32_t>(sl) * cap + li) * 16u);
+                        sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
                     }
                     uint2 o;
                     o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
@@ -604,9 +631,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                 }
             }
-            // nobody leaves while a peer may still read its shared memory
-            cluster_arrive();
-            cluster_wait();
+            if (threadIdx.x == 64) trace_stamp(p, 21);
         }
     }
 

@@ -172,6 +172,19 @@ __device__ __forceinline__ float4 ld_shared_cluster_v4(uint32_t cluster_addr)
     return v;
 }
 
+// 16-byte store into the shared memory of any CTA of the cluster (address from mapa).
+__device__ __forceinline__ void st_shared_cluster_v4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ void cluster_arrive()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -321,6 +334,28 @@ __device__ __forceinline__ void tma_load_2d_pair_if(uint32_t pred, uint32_t dst,
         "@e cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
         " [%1], [%2, {%3, %4}], [%5];\n\t}"
         ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+// 3-D forms (dimension 2 selects the 64-wide K sub-tile): one instruction fills a whole 128-wide stage.
+__device__ __forceinline__ void tma_load_3d_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, int32_t z,
+                                               uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+        "@e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%1], [%2, {%3, %4, %5}], [%6];\n\t}"
+        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d_pair_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y,
+                                                    int32_t z, uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+        "@e cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%1], [%2, {%3, %4, %5}], [%6];\n\t}"
+        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
 
