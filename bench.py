@@ -165,7 +165,7 @@ def run_reference(args) -> None:
 def run_ours(args) -> None:
     import torch
     from paper_2512_02551_b200 import build as hbuild
-    from paper_2512_02551_b200 import hgemm, inputs
+    from paper_2512_02551_b200 import hgemm, inputs, replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -182,8 +182,7 @@ def run_ours(args) -> None:
         dist.barrier()
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
+        replicas.barrier(dist)
         torch.cuda.synchronize()
 
     ctx = hgemm.Context(local)
@@ -233,11 +232,7 @@ def run_ours(args) -> None:
         barrier()
         torch.cuda.nvtx.range_pop()
         t1w = time.time()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = replicas.slowest_rank_ms(e0.elapsed_time(e1), dist, "cuda")
         return ms, t0w, t1w
 
     # ---- the timed region ---------------------------------------------------------------------
@@ -249,7 +244,7 @@ def run_ours(args) -> None:
     if st != hgemm.OK:
         raise SystemExit(f"device status {st} code {code:#x}")
     ms_per_step = ms_total / args.steps
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = replicas.job_throughput(step_flops, world, ms_per_step) / 1e12
     per_launch = {}
     for S, e0, e1 in events[-4 * args.steps:]:
         per_launch.setdefault(S, []).append(e0.elapsed_time(e1))
@@ -324,7 +319,7 @@ def run_ours(args) -> None:
             plan.run_host(hA, hB, hC, stream.cuda_stream)
     e2e_steps = max(3, min(args.steps, 10))
     e2e_ms, _, _ = timed(e2e_step, e2e_steps, 2, label="hgemm_e2e_region")
-    e2e_value = world * step_flops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_value = replicas.job_throughput(step_flops, world, e2e_ms / e2e_steps) / 1e12
     # the result that came back is the GEMM's (spot check against the device-resident run)
     if rank == 0:
         _, _, _, hC = host[0]

@@ -216,7 +216,8 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan
- * issue no TMA loads, bit 1 no MMAs (the pipeline still runs; C is garbage).
+ * issue no TMA loads, bit 1 no MMAs, bit 2 no TMA stores (the pipeline still runs;
+ * C is garbage).
  * 0 restores normal operation. */
 hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask);
 

@@ -521,7 +521,7 @@ hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf)
 
 hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask)
 {
-    if (!plan || mask > 3u) return HGEMM_ERR_INVALID_ARG;
+    if (!plan || mask > 7u) return HGEMM_ERR_INVALID_ARG;
     plan->debug_skip = mask;
     return HGEMM_OK;
 }

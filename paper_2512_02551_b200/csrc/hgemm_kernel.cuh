@@ -71,7 +71,7 @@ struct KernelParams {
     __half *C;
     long long wait_budget;        // clock cycles a wait may take before the kernel gives up
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
-    uint32_t debug_skip;          // instrumentation: bit 0 = issue no TMA loads, bit 1 = issue no MMAs (results are garbage)
+    uint32_t debug_skip;          // instrumentation: bit 0 = no TMA loads, bit 1 = no MMAs, bit 2 = no TMA stores (results are garbage)
 };
 
 __device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
@@ -421,7 +421,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     __syncwarp();
                     if (lane == 0) {
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                        if (box_row < p.M && col0 < p.N) tma_store_2d(&tmap_c, col0, box_row, buf);
+                        if (box_row < p.M && col0 < p.N && !(p.debug_skip & 4u)) tma_store_2d(&tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
                     ++store_count;
@@ -449,9 +449,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             };
 
+            // chunks of this tile that hold columns of C, and whether this warp's 32 rows hold rows of C:
+            // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
+            const int32_t live_chunks = min(chunks, (p.N - it.n0 + 31) / 32);
+            const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
             if (p.split_k == 1) {
                 // software pipeline: the load of the next chunk is in flight while this one is stored
                 uint32_t va[32], vb[32];
+                const int32_t chunks = live_rows ? live_chunks : 0;     // shadows the tile's chunk count
                 int32_t c = static_cast<int32_t>(first_chunk);
                 if (c < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, va);
                 while (c < chunks) {
@@ -594,7 +599,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const uint32_t row_in_tile = q * 32u + lane;
                 const uint32_t t_addr = tmem_base + ((q * 32u) << 16);      // the only work item used accumulator 0
                 tc_fence_after_sync();
-                for (int32_t c = static_cast<int32_t>(ew >> 2); c < chunks; c += 2) {
+                // rows and chunks outside C are neither pushed nor summed
+                const int32_t live_chunks = (it.m0 + static_cast<int32_t>(q) * 32 < p.M) ? min(chunks, (p.N - it.n0 + 31) / 32) : 0;
+                for (int32_t c = static_cast<int32_t>(ew >> 2); c < live_chunks; c += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
