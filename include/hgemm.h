@@ -20,9 +20,11 @@
  *     parameters are written only on HGEMM_OK.
  *   - Pointers passed to hgemm_run are DEVICE pointers on the context's device,
  *     16-byte aligned; the caller owns A, B, C; A and B must not overlap C.
- *   - Shapes: M, N, K >= 1, K % 8 == 0 and N % 8 == 0 (rows must be multiples of
- *     16 bytes); anything else makes hgemm_plan return HGEMM_ERR_UNSUPPORTED.
- *     There is no fallback path.
+ *   - Shapes: any M, N, K >= 1 (each at most 2^22).  The kernels address rows of
+ *     16-byte multiples; when K % 8 != 0 the plan owns zero-padded copies of A and B
+ *     that hgemm_run refreshes with a small copy kernel before the GEMM, and when
+ *     N % 8 != 0 the rows of C are stored element by element (both slower than the
+ *     aligned case, same results).  There is no CPU or library fallback path.
  *   - hgemm_run is asynchronous on the given stream.  It creates no stream,
  *     allocates nothing and never synchronises (the timing rules of paper
  *     section 2.4 "Avoiding Timing Measurement Hacking" forbid side streams);

@@ -32,7 +32,9 @@ struct hgemm_ctx_s {
 
 struct hgemm_plan_s {
     hgemm_ctx_s *ctx = nullptr;
-    int64_t M = 0, N = 0, K = 0;
+    int64_t M = 0, N = 0, K = 0;   // K is the padded K (multiple of 8) every kernel parameter is derived from
+    int64_t K_user = 0;            // the caller's K
+    void *pad_a = nullptr, *pad_b = nullptr;   // K-padded copies of A and B when K_user % 8 != 0
     hgemm_config_t cfg;
     KernelParams params;
     int grid = 0;
@@ -162,7 +164,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.stages = cfg.stages;
     p.raster_group = std::min(cfg.raster_group, p.tiles_m);
     p.tmem_cols = pow2_at_least(2 * cfg.block_n);
-    p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1) ? 1 : 0;
+    p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
+    p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;
     p.idesc = make_idesc(128 * cg, cfg.block_n);
     p.workspace = static_cast<float *>(pl->workspace);
     p.counters = pl->counters;
@@ -316,6 +319,8 @@ hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan)
     }
     if (plan->workspace) cudaFree(plan->workspace);
     if (plan->counters) cudaFree(plan->counters);
+    if (plan->pad_a) cudaFree(plan->pad_a);
+    if (plan->pad_b) cudaFree(plan->pad_b);
     if (plan->stage_a) cudaFree(plan->stage_a);
     if (plan->stage_b) cudaFree(plan->stage_b);
     if (plan->stage_c) cudaFree(plan->stage_c);
@@ -368,9 +373,10 @@ hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hge
     if (!ctx || !out) return HGEMM_ERR_INVALID_ARG;
     hgemm_status_t s = hgemm_host::validate_shape(M, N, K);
     if (s != HGEMM_OK) return s;
+    const int64_t Kp = hgemm_host::padded_k(K);
     hgemm_config_t cfg;
-    if (!hgemm_host::table_lookup(M, N, K, &cfg)) {
-        s = hgemm_host::heuristic(M, N, K, ctx->num_sms, &cfg);
+    if (!hgemm_host::table_lookup(M, N, Kp, &cfg)) {
+        s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);
         if (s != HGEMM_OK) return s;
     }
     hgemm_plan_s *pl = new (std::nothrow) hgemm_plan_s;
@@ -378,11 +384,25 @@ hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hge
     pl->ctx = ctx;
     pl->M = M;
     pl->N = N;
-    pl->K = K;
+    pl->K = Kp;
+    pl->K_user = K;
+    if (Kp != K) {
+        // rows of A and B are not multiples of 16 bytes: the kernels read zero-padded copies instead
+        cudaError_t e = cudaMalloc(&pl->pad_a, size_t(M) * size_t(Kp) * 2);
+        if (e == cudaSuccess) e = cudaMalloc(&pl->pad_b, size_t(N) * size_t(Kp) * 2);
+        if (e != cudaSuccess) {
+            if (pl->pad_a) cudaFree(pl->pad_a);
+            cuda_fail(ctx, e);
+            delete pl;
+            return HGEMM_ERR_ALLOC;
+        }
+    }
     s = apply_config(pl, cfg);
     if (s != HGEMM_OK) {
         if (pl->workspace) cudaFree(pl->workspace);
         if (pl->counters) cudaFree(pl->counters);
+        if (pl->pad_a) cudaFree(pl->pad_a);
+        if (pl->pad_b) cudaFree(pl->pad_b);
         delete pl;
         return s;
     }
@@ -422,6 +442,20 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     const hgemm_config_t &cfg = plan->cfg;
     const int cg = hgemm_host::cta_group_of(cfg);
 
+    if (plan->pad_a) {
+        // K is not a multiple of 8: copy A and B into the plan's zero-padded buffers first (same stream)
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        const int64_t ga = (plan->M * (plan->K / 8) + 255) / 256, gb = (plan->N * (plan->K / 8) + 255) / 256;
+        hgemm_dev::hgemm_pad_k_kernel<<<unsigned(std::min<int64_t>(ga, 65535)), 256, 0, st>>>(
+            static_cast<const __half *>(A), static_cast<__half *>(plan->pad_a), plan->M, plan->K_user, plan->K);
+        hgemm_dev::hgemm_pad_k_kernel<<<unsigned(std::min<int64_t>(gb, 65535)), 256, 0, st>>>(
+            static_cast<const __half *>(B), static_cast<__half *>(plan->pad_b), plan->N, plan->K_user, plan->K);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        A = plan->pad_a;
+        B = plan->pad_b;
+    }
+
     hgemm_plan_s::MapEntry *me = nullptr;
     for (int i = 0; i < plan->maps_used; ++i) {
         hgemm_plan_s::MapEntry &e = plan->maps[i];
@@ -443,7 +477,11 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
             if (!encode_2d(ctx, &e.tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
                 return HGEMM_ERR_CUDA;
         }
-        if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return HGEMM_ERR_CUDA;
+        if (plan->params.ragged_n) {
+            e.tmap_c = e.tmap_a;   // never used: a C with ragged rows is stored element by element
+        } else if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
+            return HGEMM_ERR_CUDA;
+        }
         e.a = A;
         e.b = B;
         e.c = C;
@@ -486,14 +524,16 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
 {
     if (!plan || !A_host || !B_host || !C_host) return HGEMM_ERR_INVALID_ARG;
     hgemm_ctx_s *ctx = plan->ctx;
-    const size_t a_bytes = size_t(plan->M) * size_t(plan->K) * 2, b_bytes = size_t(plan->N) * size_t(plan->K) * 2,
+    const size_t a_bytes = size_t(plan->M) * size_t(plan->K_user) * 2, b_bytes = size_t(plan->N) * size_t(plan->K_user) * 2,
                  c_bytes = size_t(plan->M) * size_t(plan->N) * 2;
     if (!plan->stage_a) {
         cudaError_t e = cudaMalloc(&plan->stage_a, a_bytes);
         if (e == cudaSuccess) e = cudaMalloc(&plan->stage_b, b_bytes);
         if (e == cudaSuccess) e = cudaMalloc(&plan->stage_c, c_bytes);
         if (e != cudaSuccess) {
-            if (plan->stage_a) cudaFree(plan->stage_a);
+            if (plan->pad_a) cudaFree(plan->pad_a);
+    if (plan->pad_b) cudaFree(plan->pad_b);
+    if (plan->stage_a) cudaFree(plan->stage_a);
             if (plan->stage_b) cudaFree(plan->stage_b);
             plan->stage_a = plan->stage_b = plan->stage_c = nullptr;
             cuda_fail(ctx, e);

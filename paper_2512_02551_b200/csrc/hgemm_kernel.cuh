@@ -62,6 +62,7 @@ struct KernelParams {
     int32_t raster_group;
     int32_t tmem_cols;            // power of two >= 2 * block_n
     int32_t epilogue_tma;         // 1: TMA-store epilogue (only when split_k == 1)
+    int32_t ragged_n;             // 1: N % 8 != 0: rows of C are not 16-byte multiples, store element by element
     int32_t tma_3d;               // 1: the A and B maps are 3-D {64, rows, K / 64}: one load per operand per stage
     int32_t cluster_split;        // 1: the split_k slices of a tile are one cluster and reduce through shared memory
     uint32_t idesc;               // tcgen05 instruction descriptor
@@ -134,6 +135,15 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_byte_addr
     d |= static_cast<uint64_t>(1) << 46;                                 // [46,48) descriptor version (sm_100)
     d |= static_cast<uint64_t>(2) << 61;                                 // [61,64) 128-byte swizzle
     return d;
+}
+
+// -------------------------------------------------------------------------------------
+// stores for a C whose rows are not multiples of 16 bytes (N % 8 != 0)
+
+__device__ __forceinline__ void store_ragged(__half *C, int64_t N, int32_t row, int32_t col, const float *vals, int count)
+{
+    for (int j = 0; j < count; ++j)
+        if (col + j < N) C[static_cast<size_t>(row) * N + col + j] = __float2half_rn(vals[j]);
 }
 
 // -------------------------------------------------------------------------------------
@@ -425,6 +435,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         bulk_commit_group();
                     }
                     ++store_count;
+                } else if (grow < p.M && p.ragged_n) {
+                    float f[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
+                    store_ragged(p.C, p.N, grow, col0, f, 32);
                 } else if (grow < p.M) {
                     __half *dst = p.C + static_cast<size_t>(grow) * p.N + col0;
 #pragma unroll
@@ -552,6 +567,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                 sum.x += x[j].x; sum.y += x[j].y; sum.z += x[j].z; sum.w += x[j].w;
                             }
                     }
+                    if (p.ragged_n) {
+                        const float f[4] = {sum.x, sum.y, sum.z, sum.w};
+                        store_ragged(p.C, p.N, orow, col, f, 4);
+                        continue;
+                    }
                     uint2 o;
                     o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
                     o.y = pack_half2_rn(__float_as_uint(sum.z), __float_as_uint(sum.w));
@@ -632,6 +652,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const float4 x = ld_shared_v4(smem_base + (static_cast<uint32_t>(sl) * cap + li) * 16u);
                         sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
                     }
+                    if (p.ragged_n) {
+                        const float f[4] = {sum.x, sum.y, sum.z, sum.w};
+                        store_ragged(p.C, p.N, orow, col, f, 4);
+                        continue;
+                    }
                     uint2 o;
                     o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
                     o.y = pack_half2_rn(__float_as_uint(sum.z), __float_as_uint(sum.w));
@@ -657,6 +682,24 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tc_fence_after_sync();
         tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
         if (lane == 0) trace_stamp(p, 7);
+    }
+}
+
+// Copies a rows x K fp16 matrix into a rows x K8 one (K8 = K rounded up to 8), zero-filling the new
+// columns: gives K-contiguous operands whose rows are multiples of 16 bytes, as TMA needs.  The
+// zero columns add nothing to any dot product.  One thread per 8 output columns.
+__global__ void hgemm_pad_k_kernel(const __half *src, __half *dst, int64_t rows, int64_t K, int64_t K8)
+{
+    grid_dependency_wait();
+    const int64_t groups = K8 / 8;
+    const int64_t total = rows * groups;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / groups, c0 = (i - r * groups) * 8;
+        __align__(16) __half out[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) out[j] = (c0 + j < K) ? src[r * K + c0 + j] : __float2half_rn(0.0f);
+        *reinterpret_cast<uint4 *>(dst + r * K8 + c0) = *reinterpret_cast<const uint4 *>(out);
     }
 }
 

@@ -59,6 +59,13 @@ hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K)
 {
     if (M < 1 || N < 1 || K < 1) return HGEMM_ERR_INVALID_ARG;
     if (M > kMaxDim || N > kMaxDim || K > kMaxDim) return HGEMM_ERR_UNSUPPORTED;
+    return HGEMM_OK;
+}
+
+hgemm_status_t validate_shape_aligned(int64_t M, int64_t N, int64_t K)
+{
+    const hgemm_status_t s = validate_shape(M, N, K);
+    if (s != HGEMM_OK) return s;
     if ((K % 8) != 0 || (N % 8) != 0) return HGEMM_ERR_UNSUPPORTED;   // rows must be multiples of 16 bytes
     return HGEMM_OK;
 }

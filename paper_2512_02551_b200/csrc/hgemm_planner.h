@@ -25,6 +25,10 @@ int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k);
 int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c);
 int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c);
 hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K);
+// The stricter rule of the kernels' own addressing: K % 8 == 0 and N % 8 == 0 (rows of 16-byte multiples).
+// hgemm_plan lifts it by padding K in a plan-owned copy and by storing ragged C rows element by element.
+hgemm_status_t validate_shape_aligned(int64_t M, int64_t N, int64_t K);
+inline int64_t padded_k(int64_t K) { return (K + 7) & ~int64_t(7); }
 hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c);
 hgemm_status_t heuristic(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
 

@@ -131,7 +131,9 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     cfg.stages = 1;
     if (block_n >= 32 && block_n <= 256 && block_n % 32 == 0)
         cfg.stages = std::max(1, std::min(6, hgemm_host::max_stages(cfg.family, block_n, cfg.block_k)));
-    hgemm_status_t st = hgemm_host::validate(M, N, K, cfg);
+    hgemm_status_t st = hgemm_host::validate_shape_aligned(M, N, K);   // no padded copies here: nothing may be allocated
+    if (st != HGEMM_OK) return st;
+    st = hgemm_host::validate(M, N, K, cfg);
     if (st != HGEMM_OK) return st;
 
     // the size check comes before anything touches the GPU

@@ -46,8 +46,7 @@ def test_argument_errors(ctx):
     assert L.hgemm_run(plan._h, a + 2, b, c, None) == hgemm.ERR_INVALID_ARG       # not 16-byte aligned
     assert L.hgemm_run(plan._h, a, b, c + 8, None) == hgemm.ERR_INVALID_ARG
     out = ctypes.c_void_p()
-    assert L.hgemm_plan(ctx._h, 64, 64, 60, ctypes.byref(out)) == hgemm.ERR_UNSUPPORTED and not out.value
-    assert L.hgemm_plan(ctx._h, 64, 60, 64, ctypes.byref(out)) == hgemm.ERR_UNSUPPORTED
+    assert L.hgemm_plan(ctx._h, 64, 64, 1 << 23, ctypes.byref(out)) == hgemm.ERR_UNSUPPORTED and not out.value
     assert L.hgemm_plan(ctx._h, 0, 64, 64, ctypes.byref(out)) == hgemm.ERR_INVALID_ARG
     assert L.hgemm_plan(None, 64, 64, 64, ctypes.byref(out)) == hgemm.ERR_INVALID_ARG
     assert L.hgemm_create(ctypes.byref(out), 99) == hgemm.ERR_INVALID_ARG
@@ -58,6 +57,36 @@ def test_argument_errors(ctx):
     plan.run(A, B, C)                                                              # still usable
     assert ctx.last_device_status() == (hgemm.OK, 0)
     plan.close()
+
+
+RAGGED = [(1, 1, 1), (64, 63, 8), (100, 135, 77), (257, 1000, 1003), (129, 9, 4099), (512, 520, 12), (33, 4100, 250)]
+
+
+@pytest.mark.parametrize("M,N,K", RAGGED)
+def test_ragged_k_and_n(ctx, gu, M, N, K):
+    """K % 8 != 0 runs on zero-padded copies of A and B, N % 8 != 0 stores C element by element: same
+    results as any other shape, for the library's own plan and for split-K in both modes."""
+    import oracle
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    ref_i = oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi))
+    cfgs = [None]
+    kp = (K + 7) // 8 * 8
+    if kp >= 128:
+        cfgs += [hgemm.Config.make(block_n=64, stages=4, split_k=2, raster_group=1, split_mode=m) for m in (0, 1)]
+        cfgs += [hgemm.Config.make(family=hgemm.FAMILY_UMMA_2CTA, block_n=96, stages=3, raster_group=2, epilogue=hgemm.EPILOGUE_TMA)]
+    for cfg in cfgs:
+        C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+        gu.assert_close_full(C, A, B, f"{(M, N, K)} {plan.config.as_dict()}")
+        Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+        gu.assert_exact(Ci, ref_i, f"{(M, N, K)} integers")
+        plan.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(16384, 256, 16384), (64, 16384, 4096), (16384, 16384, 1024), (512, 512, 16384)])
+def test_paper_grid_value_16384(ctx, gu, M, N, K):
+    """The paper's grid has a tenth value, 16384; untabulated shapes run on the planner's heuristic."""
+    gu.check_shape(ctx, M, N, K, "uniform")
 
 
 def test_plan_tracks_new_pointers(ctx, gu):
