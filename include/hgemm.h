@@ -104,6 +104,17 @@ hgemm_status_t hgemm_destroy(hgemm_ctx_t *ctx);
  * outside stream capture. */
 hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_plan_t **out);
 
+/* How B is stored (paper section 2.2 evaluates both): HGEMM_LAYOUT_TN is the default of
+ * hgemm_plan (B is N x K, K-contiguous: the K x N operand column-major); HGEMM_LAYOUT_NN
+ * takes B as the K x N operand ROW-major (N-contiguous, row stride N), so that
+ * C[i][j] = sum_k A[i][k] * B[k][j] with all three matrices row-major.  The NN layout
+ * needs K % 8 == 0 and N % 8 == 0 (HGEMM_ERR_UNSUPPORTED otherwise) and tile widths that
+ * are multiples of 64 (128 for the CTA-pair family); the planner rounds its choice up. */
+typedef enum { HGEMM_LAYOUT_TN = 0, HGEMM_LAYOUT_NN = 1 } hgemm_layout_t;
+
+hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_layout_t layout,
+                                 hgemm_plan_t **out);
+
 /* Launch C = A * B^T for the plan's shape on `stream` (a cudaStream_t, may be
  * NULL for the default stream).  A, B, C: device pointers as described above. */
 hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream);

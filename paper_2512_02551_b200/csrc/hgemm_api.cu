@@ -34,6 +34,7 @@ struct hgemm_plan_s {
     hgemm_ctx_s *ctx = nullptr;
     int64_t M = 0, N = 0, K = 0;   // K is the padded K (multiple of 8) every kernel parameter is derived from
     int64_t K_user = 0;            // the caller's K
+    int layout = HGEMM_LAYOUT_TN;  // how B is stored
     void *pad_a = nullptr, *pad_b = nullptr;   // K-padded copies of A and B when K_user % 8 != 0
     hgemm_config_t cfg;
     KernelParams params;
@@ -75,7 +76,7 @@ int32_t pow2_at_least(int32_t x)
     return p;
 }
 
-uint32_t make_idesc(int m, int n)
+uint32_t make_idesc(int m, int n, bool b_mn_major = false)
 {
     // tcgen05 instruction descriptor, kind::f16: D = fp32, A = B = fp16, both K-major, dense
     uint32_t d = 0;
@@ -83,7 +84,7 @@ uint32_t make_idesc(int m, int n)
     d |= 0u << 7;                      // [7,10)  A format: 0 = fp16
     d |= 0u << 10;                     // [10,13) B format: 0 = fp16
     d |= 0u << 15;                     // [15]    A major: 0 = K
-    d |= 0u << 16;                     // [16]    B major: 0 = K
+    d |= (b_mn_major ? 1u : 0u) << 16; // [16]    B major: 0 = K, 1 = N (B stored K x N row-major)
     d |= uint32_t(n >> 3) << 17;       // [17,23) N >> 3
     d |= uint32_t(m >> 4) << 24;       // [24,29) M >> 4
     return d;
@@ -96,6 +97,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     const int cg = hgemm_host::cta_group_of(cfg);
     // the slices of a tile wait for each other: each needs its own SM (or SM pair)
     if (cfg.split_k > 1 && cfg.split_k > ctx->num_sms / cg) return HGEMM_ERR_UNSUPPORTED;
+    if (pl->layout == HGEMM_LAYOUT_NN && (cfg.block_n % (64 * cg)) != 0) return HGEMM_ERR_UNSUPPORTED;
     const bool cluster_split = cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER;
     if (cluster_split) {
         // can the device place a cluster of split_k CTAs of this kernel at all?
@@ -166,12 +168,13 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.tmem_cols = pow2_at_least(2 * cfg.block_n);
     p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
     p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;
-    p.idesc = make_idesc(128 * cg, cfg.block_n);
+    p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN);
+    p.b_row_major = pl->layout == HGEMM_LAYOUT_NN ? 1 : 0;
     p.workspace = static_cast<float *>(pl->workspace);
     p.counters = pl->counters;
     p.status = ctx->d_status;
     p.cluster_split = cluster_split ? 1 : 0;
-    p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d) ? 1 : 0;
+    p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d && pl->layout == HGEMM_LAYOUT_TN) ? 1 : 0;
     p.C = nullptr;
     p.wait_budget = ctx->wait_budget;
     const int units = std::max(1, ctx->num_sms / cg);
@@ -370,8 +373,14 @@ int64_t hgemm_config_workspace_bytes(int64_t M, int64_t N, int64_t K, const hgem
 
 hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_plan_t **out)
 {
+    return hgemm_plan_layout(ctx, M, N, K, HGEMM_LAYOUT_TN, out);
+}
+
+hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_layout_t layout, hgemm_plan_t **out)
+{
     if (!ctx || !out) return HGEMM_ERR_INVALID_ARG;
-    hgemm_status_t s = hgemm_host::validate_shape(M, N, K);
+    if (layout != HGEMM_LAYOUT_TN && layout != HGEMM_LAYOUT_NN) return HGEMM_ERR_INVALID_ARG;
+    hgemm_status_t s = layout == HGEMM_LAYOUT_NN ? hgemm_host::validate_shape_aligned(M, N, K) : hgemm_host::validate_shape(M, N, K);
     if (s != HGEMM_OK) return s;
     const int64_t Kp = hgemm_host::padded_k(K);
     hgemm_config_t cfg;
@@ -379,8 +388,24 @@ hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hge
         s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);
         if (s != HGEMM_OK) return s;
     }
+    if (layout == HGEMM_LAYOUT_NN) {
+        // row-major B is staged in blocks of 64 columns: widen the tile to the next legal width and
+        // give back stages until it fits
+        const int unit = 64 * hgemm_host::cta_group_of(cfg);
+        cfg.block_n = std::min(256, (cfg.block_n + unit - 1) / unit * unit);
+        cfg.stages = std::min(cfg.stages, hgemm_host::max_stages(cfg.family, cfg.block_n, cfg.block_k));
+        if (cfg.stages < 1) {
+            cfg.block_k = 64;
+            cfg.stages = std::min(4, hgemm_host::max_stages(cfg.family, cfg.block_n, 64));
+        }
+        if (cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER &&
+            int64_t(cfg.stages) * hgemm_host::stage_bytes(cfg) < int64_t(128) * cfg.block_n * 4 + 16 * cfg.split_k)
+            cfg.split_mode = HGEMM_SPLIT_WORKSPACE;
+        if (hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK) return HGEMM_ERR_UNSUPPORTED;
+    }
     hgemm_plan_s *pl = new (std::nothrow) hgemm_plan_s;
     if (!pl) return HGEMM_ERR_ALLOC;
+    pl->layout = layout;
     pl->ctx = ctx;
     pl->M = M;
     pl->N = N;
@@ -472,6 +497,10 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
         if (plan->params.tma_3d) {
             if (!encode_3d_ksub(ctx, &e.tmap_a, A, K, M, 128)) return HGEMM_ERR_CUDA;
             if (!encode_3d_ksub(ctx, &e.tmap_b, B, K, N, uint32_t(cfg.block_n / cg))) return HGEMM_ERR_CUDA;
+        } else if (plan->layout == HGEMM_LAYOUT_NN) {
+            if (!encode_2d(ctx, &e.tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
+            // B is K rows of N: boxes of 64 columns x 64 k-rows
+            if (!encode_2d(ctx, &e.tmap_b, B, N, K, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
         } else {
             if (!encode_2d(ctx, &e.tmap_a, A, K, M, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
             if (!encode_2d(ctx, &e.tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))

@@ -62,6 +62,7 @@ struct KernelParams {
     int32_t raster_group;
     int32_t tmem_cols;            // power of two >= 2 * block_n
     int32_t epilogue_tma;         // 1: TMA-store epilogue (only when split_k == 1)
+    int32_t b_row_major;          // 1: B is the K x N row-major operand ("NN" layout): B tiles are N-major in shared memory
     int32_t ragged_n;             // 1: N % 8 != 0: rows of C are not 16-byte multiples, store element by element
     int32_t tma_3d;               // 1: the A and B maps are 3-D {64, rows, K / 64}: one load per operand per stage
     int32_t cluster_split;        // 1: the split_k slices of a tile are one cluster and reduce through shared memory
@@ -144,6 +145,21 @@ __device__ __forceinline__ void store_ragged(__half *C, int64_t N, int32_t row, 
 {
     for (int j = 0; j < count; ++j)
         if (col + j < N) C[static_cast<size_t>(row) * N + col + j] = __float2half_rn(vals[j]);
+}
+
+// The same for a tile that is contiguous along its M/N dimension (a row-major K x N operand): the tile
+// is stored as blocks of 64 columns, each block 64 k-rows of 128 bytes under the 128-byte swizzle.
+// Leading byte offset = distance between 64-column blocks, stride byte offset = distance between
+// groups of 8 k-rows (1024 bytes); one UMMA (K = 16) spans two such groups.
+__device__ __forceinline__ uint64_t make_smem_desc_sw128_mn_major(uint32_t smem_byte_addr, uint32_t block_bytes)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_byte_addr & 0x3ffffu) >> 4);
+    d |= static_cast<uint64_t>((block_bytes >> 4) & 0x3fffu) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
 }
 
 // -------------------------------------------------------------------------------------
@@ -288,6 +304,22 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (is_leader) mbar_arrive(bar_full + 8 * s);
                         else mbar_arrive_cluster(fb);
                     }
+                } else if (p.b_row_major) {
+                    // B is K x N row-major: per 64-wide K sub-tile, one {64 columns, 64 k-rows} box per 64-column block
+                    const int32_t b_col = it.n0 + static_cast<int32_t>(cta_rank) * b_rows;
+                    const int32_t blocks = b_rows / 64;
+                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                    else if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, stage_bytes);
+                    for (int32_t sub = 0; sub < subs; ++sub) {
+                        if constexpr (CTA_GROUP == 1) tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                        else tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                        for (int32_t nb = 0; nb < blocks; ++nb) {
+                            const uint32_t dst = b_dst + sub * b_sub_bytes + nb * (kSubK * 128);
+                            if constexpr (CTA_GROUP == 1) tma_load_2d_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
+                            else tma_load_2d_pair_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
+                        }
+                    }
                 } else if (p.tma_3d) {
                     // one instruction per operand: dimension 2 of the map counts 64-wide K sub-tiles
                     const int32_t ksub = k0 / kSubK;
@@ -333,7 +365,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t leader = (lane == 0) ? 1u : 0u; // the lane that issues every MMA and commit
             long long t_wait = 0, t_issue = 0, t_commit = 0, t_acc = 0, n_kb = 0;
             const uint64_t desc_a0 = make_smem_desc_sw128(smem_base);
-            const uint64_t desc_b0 = make_smem_desc_sw128(smem_base + a_stage_bytes);
+            // B tile: K-major (B stored N x K) or N-major in 64-column blocks of 64 k-rows (B stored K x N)
+            const uint64_t desc_b0 = p.b_row_major ? make_smem_desc_sw128_mn_major(smem_base + a_stage_bytes, kSubK * 128u)
+                                                   : make_smem_desc_sw128(smem_base + a_stage_bytes);
+            // advancing K by 16: +32 bytes inside a K-major swizzle row, +16 k-rows (2048 bytes) in an N-major tile
+            const uint32_t b_kstep = p.b_row_major ? (16u * 128u) >> 4 : 2u;
             const uint32_t desc_stage_step = stage_bytes >> 4;
             const bool issue_mma = !(p.debug_skip & 2u);
             bool ok = true;
@@ -365,7 +401,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                             for (int k = 0; k < kSubK / kUmmaK; ++k) {
                                 // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
-                                umma_f16_if<CTA_GROUP>(leader, d_tmem, a_sub + 2u * k, b_sub + 2u * k, p.idesc,
+                                umma_f16_if<CTA_GROUP>(leader, d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, p.idesc,
                                                        (kb | sub | k) != 0 ? 1u : 0u);
                             }
                         }

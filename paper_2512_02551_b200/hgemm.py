@@ -17,10 +17,11 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT
 FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA = 0, 1
 EPILOGUE_DIRECT, EPILOGUE_TMA = 0, 1
 SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
+LAYOUT_TN, LAYOUT_NN = 0, 1
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
-    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_run", "hgemm_run_host", "hgemm_run_splitk_static", "hgemm_plan_destroy",
+    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
@@ -77,6 +78,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_create": (i32, [ctypes.POINTER(p), ctypes.c_int]),
             "hgemm_destroy": (i32, [p]),
             "hgemm_plan": (i32, [p, i64, i64, i64, ctypes.POINTER(p)]),
+            "hgemm_plan_layout": (i32, [p, i64, i64, i64, i32, ctypes.POINTER(p)]),
             "hgemm_run": (i32, [p, p, p, p, p]),
             "hgemm_run_host": (i32, [p, p, p, p, p]),
             "hgemm_run_splitk_static": (i32, [i64, i64, i64, i32, i32, p, p, p, p]),
@@ -152,8 +154,8 @@ class Context:
         _check(lib().hgemm_create(ctypes.byref(self._h), int(device)), f"hgemm_create(device={device})")
         self.device = int(device)
 
-    def plan(self, M: int, N: int, K: int) -> "Plan":
-        return Plan(self, M, N, K)
+    def plan(self, M: int, N: int, K: int, layout: int = LAYOUT_TN) -> "Plan":
+        return Plan(self, M, N, K, layout)
 
     def set_wait_budget(self, cycles: int) -> None:
         _check(lib().hgemm_set_wait_budget(self._h, int(cycles)), "hgemm_set_wait_budget")
@@ -188,11 +190,13 @@ class Context:
 class Plan:
     """``hgemm_plan`` / ``hgemm_run`` / ``hgemm_plan_destroy``."""
 
-    def __init__(self, ctx: Context, M: int, N: int, K: int):
+    def __init__(self, ctx: Context, M: int, N: int, K: int, layout: int = LAYOUT_TN):
         self.ctx = ctx
         self.shape = (int(M), int(N), int(K))
+        self.layout = int(layout)
         self._h = ctypes.c_void_p()
-        _check(lib().hgemm_plan(ctx._h, int(M), int(N), int(K), ctypes.byref(self._h)), f"hgemm_plan({M},{N},{K})")
+        _check(lib().hgemm_plan_layout(ctx._h, int(M), int(N), int(K), int(layout), ctypes.byref(self._h)),
+               f"hgemm_plan_layout({M},{N},{K},layout={layout})")
         self._run = lib().hgemm_run
 
     @property
@@ -218,10 +222,12 @@ class Plan:
             raise HgemmError(st, f"hgemm_run{self.shape}")
 
     def run(self, A, B, C, stream=None) -> None:
-        """``hgemm_run`` on torch CUDA tensors: A (M,K), B (N,K), C (M,N), fp16, contiguous."""
+        """``hgemm_run`` on torch CUDA tensors: A (M,K), B (N,K) -- or (K,N) for an NN plan --, C (M,N),
+        fp16, contiguous."""
         import torch
         M, N, K = self.shape
-        for t, shp, name in ((A, (M, K), "A"), (B, (N, K), "B"), (C, (M, N), "C")):
+        b_shape = (K, N) if self.layout == LAYOUT_NN else (N, K)
+        for t, shp, name in ((A, (M, K), "A"), (B, b_shape, "B"), (C, (M, N), "C")):
             if t.dtype != torch.float16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shp:
                 raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
         s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)

@@ -221,6 +221,30 @@ def test_dependent_launch_keeps_stream_order(ctx, gu):
     p2.close()
 
 
+# ---- the NN layout: B given as the K x N operand, row-major ----------------------------------------------
+
+@pytest.mark.parametrize("M,N,K", [(128, 64, 64), (100, 136, 72), (300, 520, 200), (1024, 1024, 1024), (64, 64, 8192),
+                                    (512, 384, 640), (256, 4096, 4096), (2048, 2048, 2048)])
+def test_nn_layout(ctx, gu, M, N, K):
+    """All three matrices row-major (the paper's "NN" layout, section 2.2): same product, B indexed [k][j]."""
+    import oracle
+    for dist in ("uniform", "int5"):
+        A, B_nk = inputs.make_ab(M, N, K, dist, "cuda")
+        B_kn = B_nk.T.contiguous()                       # the same operand, stored K x N
+        plan = ctx.plan(M, N, K, hgemm.LAYOUT_NN)
+        buf, C = gu.alloc_c_with_guards(M, N)
+        plan.run(A, B_kn, C)
+        assert ctx.last_device_status() == (hgemm.OK, 0)
+        assert gu.guards_intact(buf, M, N)
+        if dist == "int5":
+            gu.assert_exact(C, oracle.hgemm_full(inputs.bits(A), inputs.bits(B_nk)), f"NN {M}x{N}x{K} integers")
+        else:
+            gu.assert_close_full(C, A, B_nk, f"NN {M}x{N}x{K} {plan.config.as_dict()}")
+        plan.close()
+    with pytest.raises(hgemm.HgemmError):
+        ctx.plan(64, 60, 64, hgemm.LAYOUT_NN)             # ragged rows of B cannot be fetched by TMA in this layout
+
+
 # ---- configuration 2: square sweep ---------------------------------------------------------------------
 
 @pytest.mark.parametrize("S", [1024, 2048, 4096, 8192])
