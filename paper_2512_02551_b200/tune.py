@@ -124,14 +124,29 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
             again[key(c)].append(batch_ms(run, n, stream))
     final = sorted(((statistics.median(again[key(c)]), e, c) for _, e, c in finalists),
                    key=lambda r: (round(r[0] * 1e3 / 0.25), r[1]))
+    if final[0][0] > 0.08:
+        # long kernels run under the power cap when called back to back: rank the finalists by a
+        # sustained run (about a quarter of a second each, shuffled order) instead of by short bursts
+        sustained = {}
+        order = list(final)
+        rng.shuffle(order)
+        for t, e, c in order:
+            plan.set_config(c)
+            n = max(5, int(250.0 / (t * 1e3 / 1e3) / 1e3))      # calls that fill about 0.25 s
+            n = max(5, min(2000, int(0.25 / (t * 1e-3))))
+            for _ in range(3):
+                run()
+            sustained[key(c)] = batch_ms(run, n, stream)
+        final = sorted(((sustained[key(c)], e, c) for _, e, c in final), key=lambda r: r[0])
     best_t, _, best = final[0]
     plan.set_config(best)
     C.zero_()
     run()
     ref = torch.matmul(A, B.T)
     ok = bool(torch.allclose(C.float(), ref.float(), rtol=4e-3, atol=4e-3 * K ** 0.5))
-    t_torch = statistics.median(batch_ms(lambda: torch.matmul(A, B.T, out=ref), max(3, min(100, int(0.6 / max(best_t, 1e-3)))), stream)
-                                for _ in range(3))
+    n_ref = max(5, min(2000, int(0.25 / (best_t * 1e-3)))) if best_t > 0.08 else max(3, min(100, int(0.6 / max(best_t, 1e-3))))
+    t_torch = statistics.median(batch_ms(lambda: torch.matmul(A, B.T, out=ref), n_ref, stream)
+                                for _ in range(1 if best_t > 0.08 else 3))
     default_t = next((t for t, _, c in results if key(c) == key(default)), None)
     plan.close()
     return {"M": M, "N": N, "K": K, "best": best.as_dict(), "us": best_t * 1e3, "default_us": None if default_t is None else default_t * 1e3,
