@@ -626,8 +626,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
         }
-        // shared memory must stay valid until the last TMA stores have read it
-        if (lane == 0) bulk_wait_group<0>();
+        // shared memory must stay valid until the last TMA stores have read it (their global writes are
+        // complete, like every other store of this grid, when the grid completes)
+        if (lane == 0) bulk_wait_group_read<0>();
         if (threadIdx.x == 64) trace_stamp(p, 6);
     }
 
