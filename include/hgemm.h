@@ -88,7 +88,11 @@ typedef struct {
     int32_t raster_group; /* m-tiles per raster group (>= 1): tile order for L2 reuse */
     int32_t epilogue;     /* HGEMM_EPILOGUE_* (split_k > 1 always finishes with direct stores) */
     int32_t split_mode;   /* HGEMM_SPLIT_* : how the K slices of a tile are summed (ignored when split_k == 1) */
-    int32_t reserved[7];  /* must be zero */
+    int32_t tail_split;   /* 0 or 1: off.  >= 2 (needs split_k == 1): when the tiles do not fill a whole number of
+                             waves of the persistent grid and the last wave is at most 1/tail_split full, its tiles
+                             are cut into tail_split K slices (summed in slice order through the workspace) so that
+                             every SM works until the end; otherwise ignored */
+    int32_t reserved[6];  /* must be zero */
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the

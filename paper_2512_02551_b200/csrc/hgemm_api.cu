@@ -121,8 +121,9 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         }
         if (clusters < 1) return HGEMM_ERR_UNSUPPORTED;
     }
-    const int64_t ws = hgemm_host::workspace_bytes(pl->M, pl->N, pl->K, cfg);
-    const int64_t cb = hgemm_host::counter_bytes(pl->M, pl->N, cfg);
+    const hgemm_host::SplitLayout layout = hgemm_host::split_layout(pl->M, pl->N, pl->K, ctx->num_sms, cfg);
+    const int64_t ws = hgemm_host::workspace_bytes(pl->M, pl->N, pl->K, cfg, ctx->num_sms);
+    const int64_t cb = hgemm_host::counter_bytes(pl->M, pl->N, cfg, ctx->num_sms, pl->K);
     if (ws > pl->workspace_bytes) {
         if (pl->workspace) cudaFree(pl->workspace);
         pl->workspace = nullptr;
@@ -158,8 +159,9 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.K = int32_t(pl->K);
     p.tiles_m = int32_t((pl->M + 128 * cg - 1) / (128 * cg));
     p.tiles_n = int32_t((pl->N + cfg.block_n - 1) / cfg.block_n);
-    p.split_k = cfg.split_k;
-    p.total_work = p.tiles_m * p.tiles_n * p.split_k;
+    p.split_k = int32_t(layout.slices);
+    p.first_split_tile = int32_t(layout.first_split_tile);
+    p.total_work = int32_t(layout.work_items);
     p.block_k = cfg.block_k;
     p.kblocks = int32_t((pl->K + cfg.block_k - 1) / cfg.block_k);
     p.block_n = cfg.block_n;
@@ -167,7 +169,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.raster_group = std::min(cfg.raster_group, p.tiles_m);
     p.tmem_cols = pow2_at_least(2 * cfg.block_n);
     p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
-    p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;
+    p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;   // whole tiles only
     p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN);
     p.b_row_major = pl->layout == HGEMM_LAYOUT_NN ? 1 : 0;
     p.workspace = static_cast<float *>(pl->workspace);

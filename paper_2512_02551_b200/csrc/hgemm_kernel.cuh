@@ -53,8 +53,10 @@ constexpr uint32_t kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3, kRoleProb
 struct KernelParams {
     int32_t M, N, K;
     int32_t tiles_m, tiles_n;     // tiles_m counts block_m-row tiles (256 rows for a pair)
-    int32_t total_work;           // tiles_m * tiles_n * split_k
-    int32_t split_k;
+    int32_t total_work;           // first_split_tile + (tiles - first_split_tile) * split_k
+    int32_t split_k;              // K slices per split tile
+    int32_t first_split_tile;     // tiles below this index are whole work items; tiles from it on are split into
+                                  // split_k slices (0: every tile is split; tiles_m * tiles_n with split_k == 1: none)
     int32_t kblocks;              // ceil(K / block_k)
     int32_t block_k;              // K extent of one pipeline stage: 64 or 128 (one or two 64-wide sub-tiles)
     int32_t block_n;
@@ -169,14 +171,28 @@ struct WorkItem {
     int32_t tile;       // linear tile index (tm, tn recovered by raster())
     int32_t m0, n0;     // first row / column of the (pair) tile
     int32_t slice;      // split-K slice
+    int32_t slices;     // number of slices of this tile (1: the tile is one work item)
+    int32_t split_index;   // index of this (tile, slice) among the split work items; split tiles are numbered from 0
     int32_t kb_begin, kb_count;
 };
 
 __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p, int32_t block_m_total)
 {
     WorkItem it;
-    it.tile = w / p.split_k;
-    it.slice = w - it.tile * p.split_k;
+    // Whole tiles first, then the split ones: with a persistent grid the split tiles form the last,
+    // partly filled wave, whose tiles are cut along K so that every SM has work until the end.
+    if (w < p.first_split_tile) {
+        it.tile = w;
+        it.slice = 0;
+        it.slices = 1;
+        it.split_index = 0;
+    } else {
+        it.split_index = w - p.first_split_tile;
+        const int32_t t = it.split_index / p.split_k;
+        it.tile = p.first_split_tile + t;
+        it.slice = it.split_index - t * p.split_k;
+        it.slices = p.split_k;
+    }
     // grouped raster: groups of raster_group m-tiles, swept along n inside a group
     const int32_t per_group = p.raster_group * p.tiles_n;
     const int32_t g = it.tile / per_group;
@@ -187,7 +203,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     const int32_t tm = first_m + (r - tn * gsize);
     it.m0 = tm * block_m_total;
     it.n0 = tn * p.block_n;
-    const int32_t base = p.kblocks / p.split_k, rem = p.kblocks - base * p.split_k;
+    const int32_t base = p.kblocks / it.slices, rem = p.kblocks - base * it.slices;
     it.kb_begin = it.slice * base + min(it.slice, rem);
     it.kb_count = base + (it.slice < rem ? 1 : 0);
     return it;
@@ -504,7 +520,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
             const int32_t live_chunks = min(chunks, (p.N - it.n0 + 31) / 32);
             const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
-            if (p.split_k == 1) {
+            if (it.slices == 1) {
                 // software pipeline: the load of the next chunk is in flight while this one is stored
                 uint32_t va[32], vb[32];
                 const int32_t chunks = live_rows ? live_chunks : 0;     // shadows the tile's chunk count
@@ -531,7 +547,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // ---- split-K through a global workspace ---------------------------------------------------
                 // 1. park this slice's fp32 partial in the workspace: slot layout [chunk][128 rows][32 cols]
                 const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
-                float *slot = p.workspace + (static_cast<size_t>(w) * CTA_GROUP + cta_rank) * slot_floats;
+                float *slot = p.workspace + (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank) * slot_floats;
                 for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
@@ -549,7 +565,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // 2. announce it, then wait (bounded) until every slice of this tile has done the same.
                 //    All slices of a tile are in flight together: the grid never exceeds the SM count, one
                 //    CTA per SM, and work items are handed out in tile order.
-                uint32_t *ctr = p.counters + (static_cast<size_t>(it.tile) * CTA_GROUP + cta_rank) * 2;
+                uint32_t *ctr = p.counters + (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2;
                 const uint32_t target = 8u * static_cast<uint32_t>(p.split_k);
                 __threadfence();
                 __syncwarp();
@@ -578,7 +594,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 //    row (one float4 per slice); slice s owns the contiguous unit range
                 //    [s U / S, (s + 1) U / S), so neighbouring threads read neighbouring addresses.  Each
                 //    unit is summed over the slices in slice order 0..S-1, up to 8 loads in flight.
-                const size_t first_slot = static_cast<size_t>(it.tile) * p.split_k;
+                const size_t first_slot = static_cast<size_t>(it.tile - p.first_split_tile) * p.split_k;
                 const size_t slice_stride = static_cast<size_t>(CTA_GROUP) * slot_floats;
                 const float *tile_ws = p.workspace + (first_slot * CTA_GROUP + cta_rank) * slot_floats;
                 const int64_t units = static_cast<int64_t>(chunks) * kBlockM * 8;

@@ -38,21 +38,42 @@ int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k)
     return int32_t(std::min<int64_t>(12, room / stage_bytes(c)));
 }
 
-int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c)
+SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c)
 {
-    (void)K;
-    if (c.split_k <= 1 || c.split_mode == HGEMM_SPLIT_CLUSTER) return 0;
     const int cg = cta_group_of(c);
-    const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
-    return tiles * c.split_k * cg * 128 * int64_t(c.block_n) * 4;
+    SplitLayout L;
+    L.tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
+    L.first_split_tile = L.tiles;
+    L.slices = 1;
+    if (c.split_k > 1) {
+        L.first_split_tile = 0;
+        L.slices = c.split_k;
+    } else if (c.tail_split >= 2) {
+        const int64_t units = std::max(1, num_sms / cg);
+        const int64_t tail = L.tiles % units;
+        if (L.tiles > units && tail > 0 && tail * c.tail_split <= units && c.tail_split <= ceil_div(K, c.block_k)) {
+            L.first_split_tile = L.tiles - tail;
+            L.slices = c.tail_split;
+        }
+    }
+    L.work_items = L.first_split_tile + (L.tiles - L.first_split_tile) * L.slices;
+    return L;
 }
 
-int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c)
+int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c, int32_t num_sms)
 {
-    if (c.split_k <= 1 || c.split_mode == HGEMM_SPLIT_CLUSTER) return 0;
-    const int cg = cta_group_of(c);
-    const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
-    return tiles * cg * 2 * 4;
+    if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) return 0;
+    const SplitLayout L = split_layout(M, N, K, num_sms, c);
+    if (L.slices <= 1) return 0;
+    return (L.tiles - L.first_split_tile) * L.slices * cta_group_of(c) * 128 * int64_t(c.block_n) * 4;
+}
+
+int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c, int32_t num_sms, int64_t K)
+{
+    if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) return 0;
+    const SplitLayout L = split_layout(M, N, K, num_sms, c);
+    if (L.slices <= 1) return 0;
+    return (L.tiles - L.first_split_tile) * cta_group_of(c) * 2 * 4;
 }
 
 hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K)
@@ -85,8 +106,9 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     if (c.split_k > kMaxSplitK) return HGEMM_ERR_UNSUPPORTED;
     if (c.raster_group < 1) return HGEMM_ERR_UNSUPPORTED;
     if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA) return HGEMM_ERR_UNSUPPORTED;
-    for (int i = 0; i < 7; ++i)
+    for (int i = 0; i < 6; ++i)
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (c.tail_split < 0 || c.tail_split > 16 || (c.tail_split >= 2 && c.split_k != 1)) return HGEMM_ERR_UNSUPPORTED;
     if (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) return HGEMM_ERR_UNSUPPORTED;
     if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) {
         if (cg != 1 || c.split_k > 16) return HGEMM_ERR_UNSUPPORTED;
@@ -114,9 +136,14 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     const int cg = cta_group_of(c);
     const int64_t bm = 128 * cg;
     const int64_t tiles = ceil_div(M, bm) * ceil_div(N, c.block_n);
-    const int64_t work = tiles * c.split_k;
     const int64_t units = std::max(1, num_sms / cg);
-    const int64_t waves = ceil_div(work, units);
+    const SplitLayout L = split_layout(M, N, K, num_sms, c);
+    const int64_t work = L.work_items;
+    // a split tail wave costs 1 / slices of a wave (plus the reduction, added below)
+    double wave_count;
+    if (c.split_k > 1) wave_count = double(ceil_div(work, units));
+    else if (L.slices > 1) wave_count = double(L.first_split_tile) / double(units) + 1.0 / double(L.slices);
+    else wave_count = double(ceil_div(L.tiles, units));
     const int64_t kb = ceil_div(K, c.block_k);
     const int64_t kb_per = ceil_div(kb, c.split_k);
     const double cta_bytes_kb = double(stage_bytes(c));
@@ -129,7 +156,8 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     const double l2_kb = concurrent_ctas * cta_bytes_kb / kL2BytesPerClk;
     const double t_kb = std::max(mma_kb, std::max(fill_kb, l2_kb));
     const double epilogue = 2.5 * c.block_n + 400.0;
-    double t = double(waves) * (double(kb_per) * t_kb + 0.25 * kFillLatency) + 0.75 * kFillLatency + epilogue;
+    double t = wave_count * (double(kb_per) * t_kb + 0.25 * kFillLatency) + 0.75 * kFillLatency + epilogue;
+    if (c.split_k == 1 && L.slices > 1) t += 128.0 * c.block_n * 4.0 / 48.0 + 9000.0;   // the tail's reduction
     double bytes = 2.0 * (double(M) * K + double(N) * K + double(M) * N);
     if (c.split_k > 1) {
         const double partial = 128.0 * c.block_n * 4.0;

@@ -22,8 +22,14 @@ inline int cta_group_of(const hgemm_config_t &c) { return c.family == HGEMM_FAMI
 int64_t stage_bytes(const hgemm_config_t &c);
 int64_t smem_bytes(const hgemm_config_t &c);
 int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k);
-int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c);
-int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c);
+// Which tiles are split: tiles [0, first_split_tile) are whole work items, the rest are cut into `slices`
+// K slices.  Uniform split-K: first = 0; tail split: first = tiles - (tiles mod units) when it applies.
+struct SplitLayout {
+    int64_t tiles, first_split_tile, slices, work_items;
+};
+SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c);
+int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c, int32_t num_sms = 148);
+int64_t counter_bytes(int64_t M, int64_t N, const hgemm_config_t &c, int32_t num_sms = 148, int64_t K = 1 << 20);
 hgemm_status_t validate_shape(int64_t M, int64_t N, int64_t K);
 // The stricter rule of the kernels' own addressing: K % 8 == 0 and N % 8 == 0 (rows of 16-byte multiples).
 // hgemm_plan lifts it by padding K in a plan-owned copy and by storing ragged C rows element by element.

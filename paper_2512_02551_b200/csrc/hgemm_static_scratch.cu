@@ -174,6 +174,7 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.tiles_m = int32_t((M + 127) / 128);
     p.tiles_n = int32_t((N + block_n - 1) / block_n);
     p.split_k = split_k;
+    p.first_split_tile = split_k > 1 ? 0 : int32_t(tiles);
     p.total_work = int32_t(tiles) * split_k;
     p.block_k = 64;
     p.kblocks = int32_t((K + 63) / 64);

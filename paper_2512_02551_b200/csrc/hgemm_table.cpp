@@ -9,11 +9,11 @@ namespace hgemm_host {
 namespace {
 struct Entry {
     int32_t M, N, K;
-    int32_t family, block_n, block_k, stages, split_k, split_mode, raster_group, epilogue;
+    int32_t family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue;
 };
 const Entry kTable[] = {
 #include "hgemm_table.inc"
-    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}   // sentinel
+    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}   // sentinel
 };
 } // namespace
 
@@ -32,6 +32,7 @@ bool table_lookup(int64_t M, int64_t N, int64_t K, hgemm_config_t *out)
             c.stages = e.stages;
             c.split_k = e.split_k;
             c.split_mode = e.split_mode;
+            c.tail_split = e.tail_split;
             c.raster_group = e.raster_group;
             c.epilogue = e.epilogue;
             if (validate(M, N, K, c) != HGEMM_OK) return false;

@@ -64,6 +64,14 @@ def candidates(M: int, N: int, K: int):
                                                   epilogue=epi, block_k=bk, split_mode=mode)
                             if hgemm.validate_config(M, N, K, c) == hgemm.OK:
                                 out.append(c)
+                            tail = tiles % units
+                            if split == 1 and tiles > units and 0 < tail <= units // 2:
+                                ts = min(units // tail, 8, -(-K // bk))
+                                if ts >= 2:
+                                    c2 = hgemm.Config.make(family=family, block_n=bn, stages=st, split_k=1, raster_group=rg,
+                                                           epilogue=epi, block_k=bk, split_mode=0, tail_split=ts)
+                                    if hgemm.validate_config(M, N, K, c2) == hgemm.OK:
+                                        out.append(c2)
     return out
 
 
@@ -79,7 +87,7 @@ def batch_ms(fn, n: int, stream) -> float:
 
 def key(c: hgemm.Config):
     d = c.as_dict()
-    return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "raster_group", "epilogue"))
+    return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "raster_group", "epilogue"))
 
 
 def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, stream) -> dict:
@@ -156,13 +164,13 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
 def write_table(rows, path):
     with open(path, "w") as f:
         f.write("// Tuned per-shape configurations for B200, written by tune.py on the GPU box.\n")
-        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, raster_group, epilogue}\n")
+        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue}\n")
         for r in rows:
             if not r["ok"]:
                 continue
             b = r["best"]
             f.write(f"{{{r['M']}, {r['N']}, {r['K']}, {b['family']}, {b['block_n']}, {b['block_k']}, {b['stages']}, "
-                    f"{b['split_k']}, {b['split_mode']}, {b['raster_group']}, {b['epilogue']}}},\n")
+                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}}},\n")
 
 
 def main():

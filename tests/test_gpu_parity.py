@@ -221,6 +221,24 @@ def test_dependent_launch_keeps_stream_order(ctx, gu):
     p2.close()
 
 
+# ---- tail split: only the tiles of the last, partly filled wave are cut along K ------------------------------
+
+@pytest.mark.parametrize("family,bn,bk,stages,tail", [(F2, 256, 64, 6, 2), (F1, 256, 64, 4, 2), (F1, 128, 128, 3, 2), (F2, 128, 128, 4, 3)])
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 512), (2000, 4104, 520), (12288, 4096, 256)])
+def test_tail_split(ctx, gu, family, bn, bk, stages, tail, M, N, K):
+    import oracle
+    cfg = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=9, epilogue=TMA, block_k=bk, tail_split=tail)
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    gu.assert_close_full(C, A, B, f"tail split {cfg.as_dict()}") if M * N * K <= gu.FULL_CHECK_VOLUME else \
+        gu.assert_close_sampled(C, A, B, "uniform", inputs.shape_seed(M, N, K), f"tail split {cfg.as_dict()}")
+    bits0 = C.view(torch.int16).clone()
+    for _ in range(3):                                   # the split tiles reproduce their bits
+        C2, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+        assert torch.equal(C2.view(torch.int16), bits0)
+    plan.close()
+
+
 # ---- the NN layout: B given as the K x N operand, row-major ----------------------------------------------
 
 @pytest.mark.parametrize("M,N,K", [(128, 64, 64), (100, 136, 72), (300, 520, 200), (1024, 1024, 1024), (64, 64, 8192),
