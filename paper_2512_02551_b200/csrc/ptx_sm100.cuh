@@ -267,14 +267,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
         asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// The same arrival delivered to the barrier at this shared-memory offset in every CTA of the
-// cluster named in cta_mask (used by a CTA pair to free a stage in both CTAs at once).
-__device__ __forceinline__ void umma_commit_pair_multicast(uint32_t bar, uint16_t cta_mask)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(cta_mask) : "memory");
-}
-
 // Whole warp: thread t reads 32 consecutive fp32 columns of tensor-memory lane (base lane + t).
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -377,19 +369,24 @@ __device__ __forceinline__ void umma_f16_if(uint32_t pred, uint32_t d_tmem, uint
             : "memory");
 }
 
+// For a CTA pair the arrival goes to the barrier at the same shared-memory offset in both CTAs of the
+// pair: two plain commits, one per CTA (addresses from mapa), both tracking the same MMAs.
 template <int CTA_GROUP>
 __device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar)
 {
-    if constexpr (CTA_GROUP == 1)
+    if constexpr (CTA_GROUP == 1) {
         asm volatile(
             "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
             "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
             ::"r"(pred), "r"(bar) : "memory");
-    else
+    } else {
         asm volatile(
-            "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
-            "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%1], %2;\n\t}"
-            ::"r"(pred), "r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+            "{\n\t.reg .pred e;\n\t.reg .b32 r0, r1;\n\telect.sync _|e, 0xffffffff;\n\t"
+            "mapa.shared::cluster.u32 r0, %1, 0;\n\tmapa.shared::cluster.u32 r1, %1, 1;\n\t"
+            "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [r0];\n\t"
+            "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [r1];\n\t}"
+            ::"r"(pred), "r"(bar) : "memory");
+    }
 }
 
 // ---- small helpers ------------------------------------------------------------------
