@@ -521,25 +521,17 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int32_t live_chunks = min(chunks, (p.N - it.n0 + 31) / 32);
             const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
             if (it.slices == 1) {
-                // software pipeline: the load of the next chunk is in flight while this one is stored
-                uint32_t va[32], vb[32];
+                // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second
+                // chunk in flight costs more in registers than it hides
+                uint32_t v[32];
                 const int32_t chunks = live_rows ? live_chunks : 0;     // shadows the tile's chunk count
-                int32_t c = static_cast<int32_t>(first_chunk);
-                if (c < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, va);
-                while (c < chunks) {
+                for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
+                    tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
-                    if (c + 2 < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c + 2) * 32u, vb);
-                    else release_accumulator();                    // every load of this warp has completed
-                    emit_chunk(va, c);
-                    c += 2;
-                    if (c >= chunks) break;
-                    tmem_ld_wait();
-                    if (c + 2 < chunks) tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c + 2) * 32u, va);
-                    else release_accumulator();
-                    emit_chunk(vb, c);
-                    c += 2;
+                    if (c + 2 >= chunks) release_accumulator();       // every load of this warp has completed
+                    emit_chunk(v, c);
                 }
-                if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load (block_n == 32)
+                if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load
             } else if (CTA_GROUP == 1 && p.cluster_split) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches
