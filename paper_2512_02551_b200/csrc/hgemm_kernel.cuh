@@ -716,7 +716,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     tc_fence_before_sync();
     __syncthreads();
     if constexpr (CTA_GROUP == 2) {   // no CTA of the pair leaves while the other may still signal it
-        cluster_arrive();
+        cluster_arrive_relaxed();
         cluster_wait();
     }
     if (warp == 1) {

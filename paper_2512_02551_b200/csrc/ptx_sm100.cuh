@@ -54,7 +54,10 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed(uint32_t c
 // Arrive on a barrier of another CTA of the cluster (address from mapa).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+    // default ordering (release at CTA scope): the barrier carries a "done" signal, no data.  A release at
+    // cluster scope here drains every earlier shared-memory and bulk-store operation of the thread first
+    // (measured ~1400 cycles in the epilogue).
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
@@ -188,6 +191,12 @@ __device__ __forceinline__ float4 ld_shared_v4(uint32_t addr)
 __device__ __forceinline__ void cluster_arrive()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+
+// Arrival without memory ordering: for barriers that only keep CTAs alive or in step.
+__device__ __forceinline__ void cluster_arrive_relaxed()
+{
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 }
 
 __device__ __forceinline__ void cluster_wait()
