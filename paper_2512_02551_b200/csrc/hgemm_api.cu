@@ -386,7 +386,7 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
     if (s != HGEMM_OK) return s;
     const int64_t Kp = hgemm_host::padded_k(K);
     hgemm_config_t cfg;
-    if (!hgemm_host::table_lookup(M, N, Kp, &cfg)) {
+    if (!hgemm_host::table_lookup(M, N, Kp, &cfg) || hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK) {
         s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);
         if (s != HGEMM_OK) return s;
     }
@@ -400,9 +400,8 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
             cfg.block_k = 64;
             cfg.stages = std::min(4, hgemm_host::max_stages(cfg.family, cfg.block_n, 64));
         }
-        if (cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER &&
-            int64_t(cfg.stages) * hgemm_host::stage_bytes(cfg) < int64_t(128) * cfg.block_n * 4 + 16 * cfg.split_k)
-            cfg.split_mode = HGEMM_SPLIT_WORKSPACE;
+        if (cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER && hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK)
+            cfg.split_mode = HGEMM_SPLIT_WORKSPACE;   // the wider tile's partial sums no longer fit in shared memory
         if (hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK) return HGEMM_ERR_UNSUPPORTED;
     }
     hgemm_plan_s *pl = new (std::nothrow) hgemm_plan_s;

@@ -230,13 +230,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t ctrl_base = staging_base + kStagingBytes;
     uint8_t *ctrl_gen = smem_gen + (ctrl_base - smem_base);
 
-    // control block: full[12] | empty[12] | tmem_full[2] | tmem_empty[2] | tmem base | abort
+    // control block: full[12] | empty[12] | tmem_full[2] | tmem_empty[2] | tmem base | abort | recv
     const uint32_t bar_full = ctrl_base;
     const uint32_t bar_empty = ctrl_base + 8 * kMaxStages;
     const uint32_t bar_tmem_full = ctrl_base + 16 * kMaxStages;
     const uint32_t bar_tmem_empty = bar_tmem_full + 16;
     volatile uint32_t *tmem_base_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 16 * kMaxStages + 32);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 16 * kMaxStages + 36);
+    const uint32_t bar_recv = ctrl_base + 16 * kMaxStages + 40;   // cluster split-K: bytes received from the other slices
 
     // the warp index through a shuffle: a value the compiler knows to be warp-uniform
     const uint32_t warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);
@@ -265,6 +266,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             mbar_init(bar_tmem_full + 8 * a, 1);              // one tcgen05.commit
             mbar_init(bar_tmem_empty + 8 * a, 8 * CTA_GROUP); // one arrive per epilogue warp (of both CTAs)
         }
+        mbar_init(bar_recv, 1);                               // one arrive.expect_tx
         fence_mbar_init();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
@@ -641,73 +643,110 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
 
     // ---- cluster split-K: sum the slices through distributed shared memory -----------------
-    // The S slices of a tile are the S CTAs of one cluster.  The tile's float4 units
-    // u = (chunk * 8 + column group) * 128 + row are dealt out in contiguous shares of `cap` units:
-    // CTA o owns [o cap, (o + 1) cap).  Every CTA pushes each unit of its fp32 partial into the owner's
-    // shared memory (slot = the pusher's slice index), and after a cluster barrier every owner adds
-    // the S slots of each of its units in slice order and stores fp16.  Both barriers are taken by
-    // every thread of every CTA of the cluster, also after an abort.
+    // The S slices of a tile are the S CTAs of one cluster.  Every CTA first lays its fp32 partial out in
+    // its own shared memory as float4 units: unit ((chunk * 128 + row) * 8 + g') holds columns
+    // 4 g .. 4 g + 3 of the chunk with g = g' ^ (row & 7) (the swizzle keeps the 16-byte stores of a
+    // quarter warp, whose rows are 128 bytes apart, on different banks).  The units are dealt out in
+    // contiguous shares of `cap`: CTA o owns [o cap, (o + 1) cap).  One thread per CTA then sends each
+    // other owner its share with one bulk copy through the cluster's shared-memory network, completing
+    // bytes on the owner's receive barrier; every owner adds, per unit, its own copy and the S - 1
+    // received ones in slice order and stores fp16.  Layout: [own tile | S - 1 receive slots of cap units].
+    // Both cluster barriers are taken by every thread of every CTA of the cluster, also after an abort.
     if constexpr (CTA_GROUP == 1) {
         if (p.cluster_split) {
-            // barrier 1: every CTA has finished its main loop (its epilogue warps arrive only after the last
-            // MMA has completed), so the stage rings are free to receive
-            cluster_arrive();
-            cluster_wait();
             const WorkItem it = decode_work(unit, p, kBlockMTotal);
+            const uint32_t S = static_cast<uint32_t>(p.split_k), me = static_cast<uint32_t>(it.slice);
             const int32_t chunks = p.block_n / 32;
             const uint32_t units = static_cast<uint32_t>(chunks) * 8u * kBlockM;
-            const uint32_t cap = (units + static_cast<uint32_t>(p.split_k) - 1u) / static_cast<uint32_t>(p.split_k);
-            const bool live = *abort_flag == 0u;
-            if (threadIdx.x == 64) trace_stamp(p, 19);
-            if (warp >= 2 && live) {
-                const uint32_t ew = warp - 2u, q = warp & 3u;
-                const uint32_t row_in_tile = q * 32u + lane;
-                const uint32_t t_addr = tmem_base + ((q * 32u) << 16);      // the only work item used accumulator 0
-                tc_fence_after_sync();
-                // rows and chunks outside C are neither pushed nor summed
-                const int32_t live_chunks = (it.m0 + static_cast<int32_t>(q) * 32 < p.M) ? min(chunks, (p.N - it.n0 + 31) / 32) : 0;
-                for (int32_t c = static_cast<int32_t>(ew >> 2); c < live_chunks; c += 2) {
-                    uint32_t v[32];
-                    tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (uint32_t g = 0; g < 8; ++g) {
-                        const uint32_t u = (static_cast<uint32_t>(c) * 8u + g) * kBlockM + row_in_tile;
-                        const uint32_t owner = u / cap, li = u - owner * cap;
-                        const uint32_t dst = smem_base + (static_cast<uint32_t>(it.slice) * cap + li) * 16u;
-                        st_shared_cluster_v4(mapa(dst, owner), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                    }
-                }
-            }
-            // barrier 2: every push has landed (release / acquire at cluster scope)
+            const uint32_t cap = (units + S - 1u) / S;
+            const uint32_t own_begin = me * cap;
+            const uint32_t own_count = own_begin >= units ? 0u : min(cap, units - own_begin);
+            const uint32_t recv_base = smem_base + units * 16u;
+            // the bytes this CTA is going to receive: S - 1 copies of its own share
+            if (threadIdx.x == 64) mbar_arrive_expect_tx(bar_recv, (S - 1u) * own_count * 16u);
+            // barrier 1: every CTA has finished its main loop (its epilogue warps arrive only after the last
+            // MMA has completed), so the stage rings are free to be overwritten, and has armed its barrier
             cluster_arrive();
             cluster_wait();
+            const bool live = *abort_flag == 0u;     // stable here: no thread of this CTA is in a wait
+            if (threadIdx.x == 64) trace_stamp(p, 19);
+            bool ok = live;
+            if (warp >= 2) {
+                const uint32_t ew = warp - 2u, q = warp & 3u;
+                const uint32_t row_in_tile = q * 32u + lane;
+                if (live) {
+                    const uint32_t t_addr = tmem_base + ((q * 32u) << 16);      // the only work item used accumulator 0
+                    tc_fence_after_sync();
+                    const uint32_t sw = row_in_tile & 7u;
+                    for (int32_t c = static_cast<int32_t>(ew >> 2); c < chunks; c += 2) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
+                        tmem_ld_wait();
+                        const uint32_t row_addr = smem_base + ((static_cast<uint32_t>(c) * kBlockM + row_in_tile) << 7);
+#pragma unroll
+                        for (uint32_t g = 0; g < 8; ++g)
+                            st_shared_v4(row_addr + ((g ^ sw) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    }
+                    fence_proxy_async_smem();        // the bulk copies below read these writes
+                }
+                named_barrier_sync(1, 8 * 32);       // the whole tile is in shared memory
+                if (live && threadIdx.x == 64) {
+                    for (uint32_t o = 0; o < S; ++o) {
+                        const uint32_t o_begin = o * cap;
+                        if (o == me || o_begin >= units) continue;
+                        const uint32_t slot = me < o ? me : me - 1u;              // receive slots skip the owner's own slice
+                        bulk_copy_to_cluster(mapa(recv_base + slot * cap * 16u, o), smem_base + o_begin * 16u,
+                                             min(cap, units - o_begin) * 16u, mapa(bar_recv, o));
+                    }
+                }
+                if (live) ok = mbar_wait(bar_recv, 0u, ctl, status_code(kRoleEpilogue, 4, 0));
+                ok = __all_sync(0xffffffffu, ok);
+            }
+            // barrier 2, arrival: this CTA has received everything (or given up).  Once every CTA of the cluster
+            // has arrived, no bulk copy is reading anyone's shared memory any more and all may leave.
+            cluster_arrive_relaxed();
             if (threadIdx.x == 64) trace_stamp(p, 20);
-            if (warp >= 2 && live) {
+            if (warp >= 2 && ok) {
                 const uint32_t ew = warp - 2u;
-                const uint32_t own_begin = static_cast<uint32_t>(it.slice) * cap;
-                const uint32_t own_count = own_begin >= units ? 0u : min(cap, units - own_begin);
-                for (uint32_t li = ew * 32u + lane; li < own_count; li += 256u) {
-                    const uint32_t u = own_begin + li;
-                    const int32_t c = static_cast<int32_t>(u >> 10), g = static_cast<int32_t>((u >> 7) & 7u), r = static_cast<int32_t>(u & 127u);
-                    const int32_t orow = it.m0 + r, col = it.n0 + c * 32 + g * 4;
-                    if (orow >= p.M || col >= p.N) continue;
-                    float4 sum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    for (int32_t sl = 0; sl < p.split_k; ++sl) {
-                        const float4 x = ld_shared_v4(smem_base + (static_cast<uint32_t>(sl) * cap + li) * 16u);
-                        sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+                const uint32_t own_addr = smem_base + own_begin * 16u;
+                // four units per thread and pass: four independent chains of loads and adds
+                for (uint32_t li0 = ew * 32u + lane; li0 < own_count; li0 += 4u * 256u) {
+                    float4 sum[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) sum[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    for (uint32_t sl = 0; sl < S; ++sl) {
+                        const uint32_t src = sl == me ? own_addr : recv_base + (sl < me ? sl : sl - 1u) * cap * 16u;
+#pragma unroll
+                        for (uint32_t j = 0; j < 4; ++j) {
+                            const uint32_t li = li0 + j * 256u;
+                            if (li < own_count) {
+                                const float4 x = ld_shared_v4(src + li * 16u);
+                                sum[j].x += x.x; sum[j].y += x.y; sum[j].z += x.z; sum[j].w += x.w;
+                            }
+                        }
                     }
-                    if (p.ragged_n) {
-                        const float f[4] = {sum.x, sum.y, sum.z, sum.w};
-                        store_ragged(p.C, p.N, orow, col, f, 4);
-                        continue;
+#pragma unroll
+                    for (uint32_t j = 0; j < 4; ++j) {
+                        const uint32_t li = li0 + j * 256u;
+                        if (li >= own_count) continue;
+                        const uint32_t u = own_begin + li;
+                        const uint32_t r = (u >> 3) & 127u;
+                        const int32_t c = static_cast<int32_t>(u >> 10), g = static_cast<int32_t>((u & 7u) ^ (r & 7u));
+                        const int32_t orow = it.m0 + static_cast<int32_t>(r), col = it.n0 + c * 32 + g * 4;
+                        if (orow >= p.M || col >= p.N) continue;
+                        if (p.ragged_n) {
+                            const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
+                            store_ragged(p.C, p.N, orow, col, f, 4);
+                            continue;
+                        }
+                        uint2 o;
+                        o.x = pack_half2_rn(__float_as_uint(sum[j].x), __float_as_uint(sum[j].y));
+                        o.y = pack_half2_rn(__float_as_uint(sum[j].z), __float_as_uint(sum[j].w));
+                        *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                     }
-                    uint2 o;
-                    o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
-                    o.y = pack_half2_rn(__float_as_uint(sum.z), __float_as_uint(sum.w));
-                    *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                 }
             }
+            cluster_wait();                          // barrier 2, wait
             if (threadIdx.x == 64) trace_stamp(p, 21);
         }
     }

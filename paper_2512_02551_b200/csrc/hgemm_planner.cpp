@@ -112,9 +112,11 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     if (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) return HGEMM_ERR_UNSUPPORTED;
     if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) {
         if (cg != 1 || c.split_k > 16) return HGEMM_ERR_UNSUPPORTED;
-        // the shared-memory ring receives the slices' fp32 partials (128 x block_n in all, plus rounding of
-        // the per-CTA shares) once the main loops are done
-        if (int64_t(c.stages) * stage_bytes(c) < int64_t(128) * c.block_n * 4 + 16 * c.split_k) return HGEMM_ERR_UNSUPPORTED;
+        // once the main loops are done, the stage ring and the store staging behind it hold this CTA's fp32
+        // partial (128 x block_n) and the S - 1 copies of its share that the other slices send
+        const int64_t units = int64_t(128) * c.block_n / 4;                    // float4 units of a tile
+        const int64_t cap = ceil_div(units, c.split_k);
+        if (int64_t(c.stages) * stage_bytes(c) + kStagingBytes < (units + (c.split_k - 1) * cap) * 16) return HGEMM_ERR_UNSUPPORTED;
     }
     const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
     if (tiles * c.split_k >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;

@@ -113,6 +113,22 @@ __device__ __forceinline__ void bulk_commit_group()
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the same cluster
+// (destination and barrier addresses from mapa); completes `bytes` on the destination's barrier.
+// Addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t mbar_cluster)
+{
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(src_cta), "r"(bytes), "r"(mbar_cluster)
+                 : "memory");
+}
+
+// Barrier among `threads` threads (a multiple of 32) of the CTA; id 0 is __syncthreads' own.
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // Wait until at most N of this thread's bulk groups still READ their shared-memory source.
 template <int N>
 __device__ __forceinline__ void bulk_wait_group_read()
