@@ -294,6 +294,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // wait results are voted), and only the single-thread instructions are predicated on lane 0:
     // TMA and tcgen05 instructions take their operands from uniform registers, so operands the
     // compiler can prove warp-uniform cost nothing to issue, while per-thread ones each need a move.
+    int32_t cs_m0 = 0, cs_n0 = 0, cs_slice = 0;   // cluster split-K: the epilogue warps' one work item, kept for the exchange
     if (warp == 0) {
         // ===== TMA producer =====
         int s = 0;
@@ -537,6 +538,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             } else if (CTA_GROUP == 1 && p.cluster_split) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches
+                cs_m0 = it.m0;
+                cs_n0 = it.n0;
+                cs_slice = it.slice;
             } else {
                 // ---- split-K through a global workspace ---------------------------------------------------
                 // 1. park this slice's fp32 partial in the workspace: slot layout [chunk][128 rows][32 cols]
@@ -644,7 +648,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     // ---- cluster split-K: sum the slices through distributed shared memory -----------------
     // The S slices of a tile are the S CTAs of one cluster.  Every CTA first lays its fp32 partial out in
-    // its own shared memory as float4 units: unit ((chunk * 128 + row) * 8 + g') holds columns
+    // its own shared memory as float4 units: unit ((chunk * rows + row) * 8 + g') holds columns
     // 4 g .. 4 g + 3 of the chunk with g = g' ^ (row & 7) (the swizzle keeps the 16-byte stores of a
     // quarter warp, whose rows are 128 bytes apart, on different banks).  The units are dealt out in
     // contiguous shares of `cap`: CTA o owns [o cap, (o + 1) cap).  One thread per CTA then sends each
@@ -654,41 +658,50 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // Both cluster barriers are taken by every thread of every CTA of the cluster, also after an abort.
     if constexpr (CTA_GROUP == 1) {
         if (p.cluster_split) {
-            const WorkItem it = decode_work(unit, p, kBlockMTotal);
-            const uint32_t S = static_cast<uint32_t>(p.split_k), me = static_cast<uint32_t>(it.slice);
-            const int32_t chunks = p.block_n / 32;
-            const uint32_t units = static_cast<uint32_t>(chunks) * 8u * kBlockM;
+            // (warps 0 and 1 only take part in the barriers; what they compute here from zeros is unused)
+            const uint32_t S = static_cast<uint32_t>(p.split_k), me = static_cast<uint32_t>(cs_slice);
+            // only the part of the tile that holds elements of C is exchanged: `rows` rows (a multiple of 32,
+            // the epilogue warps' granule) of `chunks` 32-column chunks
+            const int32_t chunks = min(p.block_n / 32, (p.N - cs_n0 + 31) / 32);
+            const uint32_t rows = static_cast<uint32_t>(min(kBlockM, (p.M - cs_m0 + 31) / 32 * 32));
+            const uint32_t units = static_cast<uint32_t>(chunks) * 8u * rows;
             const uint32_t cap = (units + S - 1u) / S;
             const uint32_t own_begin = me * cap;
             const uint32_t own_count = own_begin >= units ? 0u : min(cap, units - own_begin);
             const uint32_t recv_base = smem_base + units * 16u;
             // the bytes this CTA is going to receive: S - 1 copies of its own share
             if (threadIdx.x == 64) mbar_arrive_expect_tx(bar_recv, (S - 1u) * own_count * 16u);
-            // barrier 1: every CTA has finished its main loop (its epilogue warps arrive only after the last
-            // MMA has completed), so the stage rings are free to be overwritten, and has armed its barrier
+            // barrier 1, arrival: this CTA has finished its main loop (its epilogue warps get here only after the
+            // last MMA has completed), so its stage ring is free to be overwritten, and has armed its barrier
+            if (threadIdx.x == 64) trace_stamp(p, 16);
             cluster_arrive();
-            cluster_wait();
-            const bool live = *abort_flag == 0u;     // stable here: no thread of this CTA is in a wait
-            if (threadIdx.x == 64) trace_stamp(p, 19);
-            bool ok = live;
             if (warp >= 2) {
-                const uint32_t ew = warp - 2u, q = warp & 3u;
+                // while the other CTAs arrive, stage this CTA's partial in its own ring (after an abort the
+                // accumulator holds garbage, which then goes nowhere)
+                const uint32_t q = warp & 3u;
                 const uint32_t row_in_tile = q * 32u + lane;
-                if (live) {
+                if (row_in_tile < rows) {
                     const uint32_t t_addr = tmem_base + ((q * 32u) << 16);      // the only work item used accumulator 0
                     tc_fence_after_sync();
                     const uint32_t sw = row_in_tile & 7u;
-                    for (int32_t c = static_cast<int32_t>(ew >> 2); c < chunks; c += 2) {
+                    for (int32_t c = static_cast<int32_t>((warp - 2u) >> 2); c < chunks; c += 2) {
                         uint32_t v[32];
                         tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                         tmem_ld_wait();
-                        const uint32_t row_addr = smem_base + ((static_cast<uint32_t>(c) * kBlockM + row_in_tile) << 7);
+                        const uint32_t row_addr = smem_base + ((static_cast<uint32_t>(c) * rows + row_in_tile) << 7);
 #pragma unroll
                         for (uint32_t g = 0; g < 8; ++g)
                             st_shared_v4(row_addr + ((g ^ sw) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                     }
                     fence_proxy_async_smem();        // the bulk copies below read these writes
                 }
+            }
+            if (threadIdx.x == 64) trace_stamp(p, 17);
+            cluster_wait();                          // barrier 1, wait: every ring of the cluster is free
+            const bool live = *abort_flag == 0u;     // stable here: no thread of this CTA is in a wait
+            if (threadIdx.x == 64) trace_stamp(p, 19);
+            bool ok = live;
+            if (warp >= 2) {
                 named_barrier_sync(1, 8 * 32);       // the whole tile is in shared memory
                 if (live && threadIdx.x == 64) {
                     for (uint32_t o = 0; o < S; ++o) {
@@ -699,6 +712,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                              min(cap, units - o_begin) * 16u, mapa(bar_recv, o));
                     }
                 }
+                if (threadIdx.x == 64) trace_stamp(p, 18);
                 if (live) ok = mbar_wait(bar_recv, 0u, ctl, status_code(kRoleEpilogue, 4, 0));
                 ok = __all_sync(0xffffffffu, ok);
             }
@@ -709,6 +723,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             if (warp >= 2 && ok) {
                 const uint32_t ew = warp - 2u;
                 const uint32_t own_addr = smem_base + own_begin * 16u;
+                // chunk of a unit = (u / 8) / rows without a division: rows = 32 k, k = 1..4, and
+                // (t * mul) >> 17 = t / k for the few dozen 32-row groups t of a tile
+                const uint32_t kdiv = rows >> 5;
+                const uint32_t mul = kdiv == 3u ? 43691u : (1u << 17) >> (kdiv >> 1);
                 // four units per thread and pass: four independent chains of loads and adds
                 for (uint32_t li0 = ew * 32u + lane; li0 < own_count; li0 += 4u * 256u) {
                     float4 sum[4];
@@ -730,9 +748,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const uint32_t li = li0 + j * 256u;
                         if (li >= own_count) continue;
                         const uint32_t u = own_begin + li;
-                        const uint32_t r = (u >> 3) & 127u;
-                        const int32_t c = static_cast<int32_t>(u >> 10), g = static_cast<int32_t>((u & 7u) ^ (r & 7u));
-                        const int32_t orow = it.m0 + static_cast<int32_t>(r), col = it.n0 + c * 32 + g * 4;
+                        const uint32_t cr = u >> 3, cc = ((cr >> 5) * mul) >> 17, r = cr - cc * rows;
+                        const int32_t c = static_cast<int32_t>(cc), g = static_cast<int32_t>((u & 7u) ^ (r & 7u));
+                        const int32_t orow = cs_m0 + static_cast<int32_t>(r), col = cs_n0 + c * 32 + g * 4;
                         if (orow >= p.M || col >= p.N) continue;
                         if (p.ragged_n) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
@@ -746,6 +764,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
             }
+            if (threadIdx.x == 64) trace_stamp(p, 22);
             cluster_wait();                          // barrier 2, wait
             if (threadIdx.x == 64) trace_stamp(p, 21);
         }
