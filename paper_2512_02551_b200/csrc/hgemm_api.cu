@@ -47,6 +47,7 @@ struct hgemm_plan_s {
     int64_t workspace_bytes = 0;
     uint32_t *counters = nullptr;
     int64_t counter_bytes = 0;
+    uint32_t epoch = 0;            // launches that have used `counters` since they were last cleared
     // tensor maps depend on the pointers: a small cache keyed by (A, B, C), round-robin replacement
     struct MapEntry {
         const void *a = nullptr, *b = nullptr;
@@ -149,6 +150,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     if (pl->counters) {
         cudaError_t e = cudaMemset(pl->counters, 0, size_t(pl->counter_bytes));
         if (e != cudaSuccess) return cuda_fail(ctx, e);
+        pl->epoch = 0;
     }
 
     pl->cfg = cfg;
@@ -523,6 +525,7 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     plan->params.wait_budget = ctx->wait_budget;
     plan->params.trace = plan->trace;
     plan->params.debug_skip = plan->debug_skip;
+    if (plan->counters) plan->params.epoch = ++plan->epoch;   // the arrival counters count on from launch to launch
 
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof(lc));
@@ -607,6 +610,13 @@ hgemm_status_t hgemm_last_device_status(hgemm_ctx_t *ctx, uint32_t *code)
     if (v != 0) {
         e = cudaMemset(ctx->d_status, 0, 4);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
+        // a launch that gave up may have left split-K arrival counters part-way: start them again from zero
+        for (hgemm_plan_s *pl : ctx->plans) {
+            if (!pl->counters) continue;
+            e = cudaMemset(pl->counters, 0, size_t(pl->counter_bytes));
+            if (e != cudaSuccess) return cuda_fail(ctx, e);
+            pl->epoch = 0;
+        }
     }
     *code = v;
     return v ? HGEMM_ERR_TIMEOUT : HGEMM_OK;

@@ -76,6 +76,7 @@ struct KernelParams {
     long long wait_budget;        // clock cycles a wait may take before the kernel gives up
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
     uint32_t debug_skip;          // instrumentation: bit 0 = no TMA loads, bit 1 = no MMAs, bit 2 = no TMA stores (results are garbage)
+    uint32_t epoch;               // workspace split-K: number of this launch among the launches that used `counters` (from 1)
 };
 
 __device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
@@ -543,37 +544,54 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 cs_slice = it.slice;
             } else {
                 // ---- split-K through a global workspace ---------------------------------------------------
-                // 1. park this slice's fp32 partial in the workspace: slot layout [chunk][128 rows][32 cols]
+                // 1. park this slice's fp32 partial in the workspace.  A slot is a sequence of float4 units: unit
+                //    ((chunk * 128 + row) * 8 + g') holds columns 4 g .. 4 g + 3 of the chunk, g = g' ^ (row & 7)
+                //    (the swizzle keeps a quarter warp's 16-byte shared-memory stores, 128 bytes apart, on
+                //    different banks).  Each warp stages its 32 rows of a chunk (4 KB, contiguous in the slot) in
+                //    its store buffer and sends them with one bulk copy.
                 const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
                 float *slot = p.workspace + (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank) * slot_floats;
-                for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
+                const int32_t park_chunks = live_rows ? live_chunks : 0;
+                for (int32_t c = static_cast<int32_t>(first_chunk); c < park_chunks; c += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
+                    if (lane == 0) bulk_wait_group_read<0>();      // the buffer's last bulk copy has read it
                     tmem_ld_wait();
-                    if (grow < p.M && it.n0 + c * 32 < p.N) {
-                        float4 *dst = reinterpret_cast<float4 *>(slot + (static_cast<size_t>(c) * kBlockM + row_in_tile) * 32);
+                    __syncwarp();
+                    const uint32_t row_addr = staging + (lane << 7);
+                    const uint32_t sw = lane & 7u;                   // = row & 7: a warp's first row is a multiple of 32
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            __stcg(dst + j, make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                        __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3])));
+                    for (uint32_t g = 0; g < 8; ++g)
+                        st_shared_v4(row_addr + ((g ^ sw) << 4), v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        bulk_store_to_global(slot + (static_cast<size_t>(c) * kBlockM + q * 32u) * 32, staging, kStagingBytesPerWarp);
+                        bulk_commit_group();
                     }
                 }
                 release_accumulator();
+                if (lane == 0) {
+                    bulk_wait_group<0>();                            // this warp's part of the slot is written
+                    fence_proxy_async_all();                         // order those writes before the signal below
+                }
                 if (w == unit && threadIdx.x == 64) trace_stamp(p, 16);
                 // 2. announce it, then wait (bounded) until every slice of this tile has done the same.
                 //    All slices of a tile are in flight together: the grid never exceeds the SM count, one
                 //    CTA per SM, and work items are handed out in tile order.
                 uint32_t *ctr = p.counters + (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2;
-                const uint32_t target = 8u * static_cast<uint32_t>(p.split_k);
-                __threadfence();
+                //    The counter is never reset: every launch adds 8 S arrivals per tile (one per epilogue warp and
+                //    slice), so launch number e waits for e * 8 S, compared modulo 2^32.
+                const uint32_t target = p.epoch * 8u * static_cast<uint32_t>(it.slices);
                 __syncwarp();
                 if (lane == 0) {
+                    __threadfence();
                     atomicAdd(ctr, 1u);
                     const long long t0 = clock64();
                     while (true) {
                         uint32_t seen;
                         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(ctr) : "memory");
-                        if (seen >= target) break;
+                        if (static_cast<int32_t>(seen - target) >= 0) break;
                         if (*abort_flag) { ok = false; break; }
                         if (clock64() - t0 > p.wait_budget) {
                             *abort_flag = 1u;
@@ -588,56 +606,62 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!ok) break;
                 if (w == unit && threadIdx.x == 64) trace_stamp(p, 17);
                 __threadfence();
-                // 3. every slice reduces its share of the tile.  A unit is four consecutive columns of one
-                //    row (one float4 per slice); slice s owns the contiguous unit range
-                //    [s U / S, (s + 1) U / S), so neighbouring threads read neighbouring addresses.  Each
-                //    unit is summed over the slices in slice order 0..S-1, up to 8 loads in flight.
+                // 3. every slice reduces its share of the tile: slice s owns the contiguous unit range
+                //    [s U / S, (s + 1) U / S), so neighbouring threads read neighbouring addresses.  Each unit is
+                //    summed over the slices in slice order 0..S-1; a thread works on eight units at a time and
+                //    has the loads of two slices (sixteen float4) in flight.
                 const size_t first_slot = static_cast<size_t>(it.tile - p.first_split_tile) * p.split_k;
                 const size_t slice_stride = static_cast<size_t>(CTA_GROUP) * slot_floats;
-                const float *tile_ws = p.workspace + (first_slot * CTA_GROUP + cta_rank) * slot_floats;
+                const float4 *tile_ws = reinterpret_cast<const float4 *>(p.workspace + (first_slot * CTA_GROUP + cta_rank) * slot_floats);
                 const int64_t units = static_cast<int64_t>(chunks) * kBlockM * 8;
                 const int32_t u_begin = static_cast<int32_t>(units * it.slice / p.split_k);
                 const int32_t u_end = static_cast<int32_t>(units * (it.slice + 1) / p.split_k);
-                for (int32_t u = u_begin + static_cast<int32_t>(ew * 32u + lane); u < u_end; u += 256) {
-                    const int32_t c = u >> 10, r = (u >> 3) & 127, g = u & 7;   // chunk, row, column group
-                    const int32_t orow = row0 + r, col = it.n0 + c * 32 + g * 4;
-                    if (orow >= p.M || col >= p.N) continue;
-                    const float4 *src = reinterpret_cast<const float4 *>(tile_ws) + u;   // [chunk][row][8 float4]
-                    float4 sum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    for (int32_t sl0 = 0; sl0 < p.split_k; sl0 += 8) {
-                        float4 x[8];
+                constexpr int kUnitsPerPass = 8;
+                for (int32_t u0 = u_begin + static_cast<int32_t>(ew * 32u + lane); u0 < u_end; u0 += kUnitsPerPass * 256) {
+                    uint32_t on = 0;                                  // bit j: unit j of this pass holds elements of C
+                    float4 sum[kUnitsPerPass];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (sl0 + j < p.split_k)
-                                x[j] = __ldcg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(src) +
-                                                                               static_cast<size_t>(sl0 + j) * slice_stride));
+                    for (int j = 0; j < kUnitsPerPass; ++j) {
+                        const int32_t u = u0 + j * 256;
+                        const int32_t c = u >> 10, r = (u >> 3) & 127, g = (u & 7) ^ (r & 7);   // chunk, row, column group
+                        if (u < u_end && row0 + r < p.M && it.n0 + c * 32 + g * 4 < p.N) on |= 1u << j;
+                        sum[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    }
+                    for (int32_t sl0 = 0; sl0 < p.split_k; sl0 += 2) {
+                        float4 x[2][kUnitsPerPass];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            if (sl0 + j < p.split_k) {
-                                sum.x += x[j].x; sum.y += x[j].y; sum.z += x[j].z; sum.w += x[j].w;
-                            }
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int j = 0; j < kUnitsPerPass; ++j)
+                                if (((on >> j) & 1u) && sl0 + h < p.split_k)
+                                    x[h][j] = __ldcg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(tile_ws + u0 + j * 256) +
+                                                                                     static_cast<size_t>(sl0 + h) * slice_stride));
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int j = 0; j < kUnitsPerPass; ++j)
+                                if (((on >> j) & 1u) && sl0 + h < p.split_k) {
+                                    sum[j].x += x[h][j].x; sum[j].y += x[h][j].y; sum[j].z += x[h][j].z; sum[j].w += x[h][j].w;
+                                }
                     }
-                    if (p.ragged_n) {
-                        const float f[4] = {sum.x, sum.y, sum.z, sum.w};
-                        store_ragged(p.C, p.N, orow, col, f, 4);
-                        continue;
+#pragma unroll
+                    for (int j = 0; j < kUnitsPerPass; ++j) {
+                        if (!((on >> j) & 1u)) continue;
+                        const int32_t u = u0 + j * 256;
+                        const int32_t c = u >> 10, r = (u >> 3) & 127, g = (u & 7) ^ (r & 7);
+                        const int32_t orow = row0 + r, col = it.n0 + c * 32 + g * 4;
+                        if (p.ragged_n) {
+                            const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
+                            store_ragged(p.C, p.N, orow, col, f, 4);
+                            continue;
+                        }
+                        uint2 o;
+                        o.x = pack_half2_rn(__float_as_uint(sum[j].x), __float_as_uint(sum[j].y));
+                        o.y = pack_half2_rn(__float_as_uint(sum[j].z), __float_as_uint(sum[j].w));
+                        *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                     }
-                    uint2 o;
-                    o.x = pack_half2_rn(__float_as_uint(sum.x), __float_as_uint(sum.y));
-                    o.y = pack_half2_rn(__float_as_uint(sum.z), __float_as_uint(sum.w));
-                    *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                 }
-                // 4. the last warp of the last slice to finish re-arms the counters for the next launch
-                __syncwarp();
                 if (w == unit && threadIdx.x == 64) trace_stamp(p, 18);
-                if (lane == 0) {
-                    const uint32_t d = atomicAdd(ctr + 1, 1u);
-                    if (d == target - 1u) {
-                        ctr[0] = 0u;
-                        ctr[1] = 0u;
-                        __threadfence();
-                    }
-                }
             }
         }
         // shared memory must stay valid until the last TMA stores have read it (their global writes are

@@ -157,14 +157,18 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     const double concurrent_ctas = double(std::min(work, units)) * cg;
     const double l2_kb = concurrent_ctas * cta_bytes_kb / kL2BytesPerClk;
     const double t_kb = std::max(mma_kb, std::max(fill_kb, l2_kb));
-    const double epilogue = 2.5 * c.block_n + 400.0;
+    const double epilogue = 5.0 * c.block_n + 600.0;   // the last tile's drain: 32-column chunks, two warps per row quarter
     double t = wave_count * (double(kb_per) * t_kb + 0.25 * kFillLatency) + 0.75 * kFillLatency + epilogue;
     if (c.split_k == 1 && L.slices > 1) t += 128.0 * c.block_n * 4.0 / 48.0 + 9000.0;   // the tail's reduction
     double bytes = 2.0 * (double(M) * K + double(N) * K + double(M) * N);
     if (c.split_k > 1) {
         const double partial = 128.0 * c.block_n * 4.0;
         if (c.split_mode == HGEMM_SPLIT_CLUSTER) {
-            t += partial / 64.0 + partial / 96.0 + 2500.0;                      // stage in shared memory, two cluster barriers, pull
+            // stage in shared memory, send (S - 1) / S of it through the cluster network (about 18 bytes per
+            // clock per SM), ordered sum; only rows that exist in C take part
+            const double live = M < 128 ? double((M + 31) / 32 * 32) / 128.0 : 1.0;
+            const double p_live = partial * live;
+            t += p_live / 70.0 + p_live * double(c.split_k - 1) / double(c.split_k) / 18.0 + p_live / 45.0 + 800.0;
         } else {
             t += partial / 64.0 + partial / 48.0 + 9000.0;                      // park, signal, wait, pull through L2
             bytes += 2.0 * double(work) * cg * partial;

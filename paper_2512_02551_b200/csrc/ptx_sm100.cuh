@@ -123,6 +123,22 @@ __device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint3
                  : "memory");
 }
 
+// Bulk copy from this CTA's shared memory to global memory, as part of the thread's current bulk group.
+// Addresses and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_store_to_global(void *dst, uint32_t src_cta, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(reinterpret_cast<uint64_t>(dst)), "r"(src_cta), "r"(bytes)
+                 : "memory");
+}
+
+// Orders this thread's accesses made through the asynchronous-copy path with its ordinary ones, in every
+// memory space.
+__device__ __forceinline__ void fence_proxy_async_all()
+{
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+
 // Barrier among `threads` threads (a multiple of 32) of the CTA; id 0 is __syncthreads' own.
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads)
 {
