@@ -68,7 +68,10 @@ enum {
 enum {
     HGEMM_SPLIT_WORKSPACE = 0, /* partials parked in a global workspace; any family; split_k <= 64 */
     HGEMM_SPLIT_CLUSTER = 1    /* the slices of a tile form one thread-block cluster and are summed through
-                                  distributed shared memory; 1-CTA family only; split_k in [2, 16] */
+                                  distributed shared memory; 1-CTA family only; split_k in [2, 16]; the tile's
+                                  fp32 partial (512 * block_n bytes) plus split_k - 1 received shares of
+                                  ceil(1/split_k) of it must fit in the stage ring and store staging
+                                  (hgemm_validate_config answers) */
 };
 
 enum {
@@ -228,8 +231,10 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
  * 8/9/10 MMA thread waiting for data / issuing MMAs / committing, 11/12 producer
  * waiting for a free stage / issuing loads, 13 MMA thread waiting for a free
  * accumulator, 15 k-blocks processed; and for split-K stamps 16 partial parked,
- * 17 all slices arrived, 18 share reduced; for cluster split-K 19 cluster gathered,
- * 20 share reduced, 21 cluster released.  The caller owns the buffer. */
+ * 17 all slices arrived, 18 share reduced; for cluster split-K 16 arrived at the
+ * cluster's first barrier, 17 partial staged, 19 cluster gathered, 18 shares sent,
+ * 20 shares received, 22 share reduced, 21 cluster released.  The caller owns the
+ * buffer. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan
