@@ -126,6 +126,17 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
  * NULL for the default stream).  A, B, C: device pointers as described above. */
 hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream);
 
+/* The general form of the operation (paper section 2.1, "HGEMM"): C = alpha * A * B^T + beta * C,
+ * in place in C (DEVICE pointers and layouts as for hgemm_run; alpha and beta are fp32
+ * values passed by value).  The accumulator is fp32; each element is computed as
+ * fma(beta, C_old, alpha * acc) in fp32 and rounded to fp16 once.  With beta == 0 the old
+ * contents of C are never read (they may be uninitialised or NaN).  Every configuration the
+ * plan can hold supports it, split-K included (the scaling is applied where the slices are
+ * summed).  hgemm_run is the case alpha = 1, beta = 0, which the paper's experiments use.
+ * HGEMM_ERR_INVALID_ARG for a NaN factor. */
+hgemm_status_t hgemm_run_scaled(hgemm_plan_t *plan, float alpha, float beta, const void *A, const void *B, void *C,
+                                void *stream);
+
 /* The same operation on HOST buffers (paper section 2.3 builds its inputs on the
  * CPU): copies A and B to device staging owned by the plan, runs, copies C back,
  * all enqueued on `stream`.  A_host, B_host, C_host are HOST pointers with the

@@ -26,11 +26,17 @@ ABS_COEF = 1e-3
 FROBENIUS_LIMIT = 2.0 ** -11
 
 
-def contract_bound(c_ref: np.ndarray, k: int) -> np.ndarray:
-    return REL_TERM * np.abs(c_ref) + ABS_COEF * np.sqrt(float(k))
+def contract_bound(c_ref: np.ndarray, k: int, abs_scale: float = 1.0) -> np.ndarray:
+    """``abs_scale`` scales the absolute term: |alpha| for C = alpha A B^T + beta C, whose accumulation
+    error is alpha times that of A B^T (the beta C term is exact in fp32 and adds one rounding, which
+    the relative term covers).  For the scaled form 2^-24, half the spacing of fp16 subnormals, is added so
+    that alpha = 0 leaves a positive bound; the plain product keeps the contract's bound unchanged."""
+    if abs_scale == 1.0:
+        return REL_TERM * np.abs(c_ref) + ABS_COEF * np.sqrt(float(k))
+    return REL_TERM * np.abs(c_ref) + ABS_COEF * np.sqrt(float(k)) * abs(float(abs_scale)) + 2.0 ** -24
 
 
-def check_contract(c_gpu_f64: np.ndarray, c_ref: np.ndarray, k: int) -> dict:
+def check_contract(c_gpu_f64: np.ndarray, c_ref: np.ndarray, k: int, abs_scale: float = 1.0) -> dict:
     """Elementwise contract check. Returns a report; ``ok`` is the verdict."""
     c_gpu_f64 = np.asarray(c_gpu_f64, dtype=np.float64)
     c_ref = np.asarray(c_ref, dtype=np.float64)
@@ -38,7 +44,7 @@ def check_contract(c_gpu_f64: np.ndarray, c_ref: np.ndarray, k: int) -> dict:
         raise ValueError(f"shape mismatch {c_gpu_f64.shape} vs {c_ref.shape}")
     finite = np.isfinite(c_gpu_f64)
     err = np.abs(c_gpu_f64 - c_ref)
-    bound = contract_bound(c_ref, k)
+    bound = contract_bound(c_ref, k, abs_scale)
     bad = (~finite) | (err > bound)
     ratio = np.where(finite, err / bound, np.inf)
     return {

@@ -114,3 +114,21 @@ def hgemm_sampled(a_bits, b_bits, ii, jj) -> np.ndarray:
     _load().oracle_hgemm_sampled(a.shape[1], a.ctypes.data, a.shape[1], b.ctypes.data, b.shape[1],
                                  ii.size, ii.ctypes.data, jj.ctypes.data, out.ctypes.data)
     return out
+
+
+def hgemm_scaled_full(a_bits, b_bits, c_bits, alpha: float, beta: float) -> np.ndarray:
+    """alpha * A B^T + beta * C (fp64, M x N): the general form of the operation (paper section 2.1).
+
+    ``alpha`` and ``beta`` are taken as the fp32 values the library receives (both are exact in
+    fp64).  With ``beta == 0`` the old C does not enter the result at all, whatever it holds
+    (the BLAS convention the library follows).
+    """
+    ab = hgemm_full(a_bits, b_bits)
+    al = float(np.float32(alpha))
+    be = float(np.float32(beta))
+    if be == 0.0:
+        return al * ab
+    c = _bits(c_bits)
+    if c.shape != ab.shape:
+        raise ValueError(f"need C {ab.shape}, got {c.shape}")
+    return al * ab + be * f16_bits_to_f64(c)

@@ -461,7 +461,22 @@ int32_t hgemm_plan_launches_per_run(const hgemm_plan_t *plan)
     return plan ? 1 : 0;
 }
 
+static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool scaled, const void *A, const void *B, void *C,
+                               void *stream);
+
 hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream)
+{
+    return run_impl(plan, 1.0f, 0.0f, false, A, B, C, stream);
+}
+
+hgemm_status_t hgemm_run_scaled(hgemm_plan_t *plan, float alpha, float beta, const void *A, const void *B, void *C, void *stream)
+{
+    if (!(alpha == alpha) || !(beta == beta)) return HGEMM_ERR_INVALID_ARG;   // NaN factors
+    return run_impl(plan, alpha, beta, true, A, B, C, stream);
+}
+
+static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool scaled, const void *A, const void *B, void *C,
+                               void *stream)
 {
     if (!plan || !A || !B || !C) return HGEMM_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15u)
@@ -525,6 +540,9 @@ hgemm_status_t hgemm_run(hgemm_plan_t *plan, const void *A, const void *B, void 
     plan->params.wait_budget = ctx->wait_budget;
     plan->params.trace = plan->trace;
     plan->params.debug_skip = plan->debug_skip;
+    plan->params.scaled = scaled ? 1u : 0u;
+    plan->params.alpha = alpha;
+    plan->params.beta = beta;
     if (plan->counters) plan->params.epoch = ++plan->epoch;   // the arrival counters count on from launch to launch
 
     cudaLaunchConfig_t lc;

@@ -77,6 +77,8 @@ struct KernelParams {
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
     uint32_t debug_skip;          // instrumentation: bit 0 = no TMA loads, bit 1 = no MMAs, bit 2 = no TMA stores (results are garbage)
     uint32_t epoch;               // workspace split-K: number of this launch among the launches that used `counters` (from 1)
+    uint32_t scaled;              // 0: C = A B^T; 1: C = alpha A B^T + beta C (paper section 2.1)
+    float alpha, beta;
 };
 
 __device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
@@ -167,6 +169,66 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128_mn_major(uint32_t smem_
 
 // -------------------------------------------------------------------------------------
 // tile schedule
+
+// -------------------------------------------------------------------------------------
+// C = alpha A B^T + beta C (paper section 2.1, the general form of the operation): the scaling step of every
+// store path.  All in fp32 -- alpha * acc rounded once, then one fused multiply-add with the old element --
+// and the result is rounded to fp16 once by the caller.  With beta == 0 the old C is never read.
+
+__device__ __forceinline__ float scaled_value(float acc, float alpha, float beta, float old)
+{
+    return fmaf(beta, old, alpha * acc);
+}
+
+// v[0..7]: fp32 bit patterns of eight consecutive columns col .. col + 7 of row `row`.
+__device__ __forceinline__ void scale_group8(uint32_t *v, const KernelParams &p, int32_t row, int32_t col)
+{
+    float old[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) old[i] = 0.0f;
+    if (p.beta != 0.0f) {
+        const __half *src = p.C + static_cast<size_t>(row) * p.N + col;
+        if (!p.ragged_n && col + 8 <= p.N) {
+            const uint4 o = *reinterpret_cast<const uint4 *>(src);   // N % 8 == 0: 16-byte aligned
+            const __half2 *h = reinterpret_cast<const __half2 *>(&o);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h[i]);
+                old[2 * i] = f.x;
+                old[2 * i + 1] = f.y;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (col + i < p.N) old[i] = __half2float(src[i]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __float_as_uint(scaled_value(__uint_as_float(v[i]), p.alpha, p.beta, old[i]));
+}
+
+// s: four consecutive columns col .. col + 3 of row `row`.
+__device__ __forceinline__ void scale_unit4(float4 &s, const KernelParams &p, int32_t row, int32_t col)
+{
+    float old[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (p.beta != 0.0f) {
+        const __half *src = p.C + static_cast<size_t>(row) * p.N + col;
+        if (!p.ragged_n) {                                            // N % 8 == 0 and col % 4 == 0: 8-byte aligned, in bounds
+            const uint2 o = *reinterpret_cast<const uint2 *>(src);
+            const __half2 *h = reinterpret_cast<const __half2 *>(&o);
+            const float2 f0 = __half22float2(h[0]), f1 = __half22float2(h[1]);
+            old[0] = f0.x; old[1] = f0.y; old[2] = f1.x; old[3] = f1.y;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (col + i < p.N) old[i] = __half2float(src[i]);
+        }
+    }
+    s.x = scaled_value(s.x, p.alpha, p.beta, old[0]);
+    s.y = scaled_value(s.y, p.alpha, p.beta, old[1]);
+    s.z = scaled_value(s.z, p.alpha, p.beta, old[2]);
+    s.w = scaled_value(s.w, p.alpha, p.beta, old[3]);
+}
 
 struct WorkItem {
     int32_t tile;       // linear tile index (tm, tn recovered by raster())
@@ -533,6 +595,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
                     if (c + 2 >= chunks) release_accumulator();       // every load of this warp has completed
+                    if (p.scaled && grow < p.M) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (it.n0 + c * 32 + 8 * j < p.N) scale_group8(v + 8 * j, p, grow, it.n0 + c * 32 + 8 * j);
+                    }
                     emit_chunk(v, c);
                 }
                 if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load
@@ -650,6 +717,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const int32_t u = u0 + j * 256;
                         const int32_t c = u >> 10, r = (u >> 3) & 127, g = (u & 7) ^ (r & 7);
                         const int32_t orow = row0 + r, col = it.n0 + c * 32 + g * 4;
+                        if (p.scaled) scale_unit4(sum[j], p, orow, col);
                         if (p.ragged_n) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
                             store_ragged(p.C, p.N, orow, col, f, 4);
@@ -776,6 +844,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const int32_t c = static_cast<int32_t>(cc), g = static_cast<int32_t>((u & 7u) ^ (r & 7u));
                         const int32_t orow = cs_m0 + static_cast<int32_t>(r), col = cs_n0 + c * 32 + g * 4;
                         if (orow >= p.M || col >= p.N) continue;
+                        if (p.scaled) scale_unit4(sum[j], p, orow, col);
                         if (p.ragged_n) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
                             store_ragged(p.C, p.N, orow, col, f, 4);

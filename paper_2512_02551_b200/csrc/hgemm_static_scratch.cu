@@ -194,6 +194,9 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.wait_budget = 2000000000LL;
     p.trace = nullptr;
     p.debug_skip = 0;
+    p.scaled = 0;
+    p.alpha = 1.0f;
+    p.beta = 0.0f;
     p.epoch = 1;          // the control page was cleared just above: every call is the counters' first launch
 
     cudaLaunchConfig_t lc;

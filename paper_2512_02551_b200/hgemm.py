@@ -21,7 +21,7 @@ LAYOUT_TN, LAYOUT_NN = 0, 1
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
-    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_splitk_static", "hgemm_plan_destroy",
+    "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan_layout": (i32, [p, i64, i64, i64, i32, ctypes.POINTER(p)]),
             "hgemm_run": (i32, [p, p, p, p, p]),
             "hgemm_run_host": (i32, [p, p, p, p, p]),
+            "hgemm_run_scaled": (i32, [p, ctypes.c_float, ctypes.c_float, p, p, p, p]),
             "hgemm_run_splitk_static": (i32, [i64, i64, i64, i32, i32, p, p, p, p]),
             "hgemm_plan_destroy": (i32, [p]),
             "hgemm_plan_get_config": (i32, [p, cfgp]),
@@ -233,6 +234,19 @@ class Plan:
                 raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
         s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
         self.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+
+    def run_scaled(self, alpha: float, beta: float, A, B, C, stream=None) -> None:
+        """``hgemm_run_scaled``: C = alpha * A B^T + beta * C in place, on torch CUDA tensors as for ``run``."""
+        import torch
+        M, N, K = self.shape
+        b_shape = (K, N) if self.layout == LAYOUT_NN else (N, K)
+        for t, shp, name in ((A, (M, K), "A"), (B, b_shape, "B"), (C, (M, N), "C")):
+            if t.dtype != torch.float16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shp:
+                raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
+        s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
+        st = lib().hgemm_run_scaled(self._h, float(alpha), float(beta), A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+        if st != OK:
+            raise HgemmError(st, f"hgemm_run_scaled{self.shape}")
 
     def set_trace(self, device_ptr: int) -> None:
         _check(lib().hgemm_debug_set_trace(self._h, ctypes.c_void_p(device_ptr)), "hgemm_debug_set_trace")

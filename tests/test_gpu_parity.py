@@ -334,3 +334,62 @@ def test_generator_matches_across_devices():
         a = inputs.draw(77, inputs.TAG_A, 513, 264, dist, "cpu")
         b = inputs.draw(77, inputs.TAG_A, 513, 264, dist, "cuda")
         assert torch.equal(a, b.cpu()), dist
+
+
+# ---- the general form C = alpha A B^T + beta C (paper section 2.1) ------------------------------------------
+
+SCALED_CASES = [
+    # M, N, K, config (None: the planner's), why
+    (128, 128, 128, None, "one tile"),
+    (300, 264, 520, ("f1", 96, 4, 1, 64, WORKSPACE, TMA), "ragged tiles, TMA-store epilogue"),
+    (300, 264, 520, ("f1", 96, 4, 1, 64, WORKSPACE, DIRECT), "direct stores"),
+    (520, 392, 1024, ("f2", 128, 3, 1, 128, WORKSPACE, TMA), "CTA pairs"),
+    (77, 203, 333, None, "N and K not multiples of 8: element-wise reads of the old C"),
+    (256, 384, 4096, ("f1", 128, 4, 4, 64, WORKSPACE, DIRECT), "split-K through the workspace"),
+    (256, 384, 4096, ("f2", 128, 4, 3, 64, WORKSPACE, DIRECT), "split-K, CTA pairs"),
+    (64, 640, 2048, ("f1", 160, 2, 7, 128, CLUSTER, DIRECT), "split-K inside a cluster"),
+]
+
+
+@pytest.mark.parametrize("case", SCALED_CASES, ids=lambda c: f"{c[0]}x{c[1]}x{c[2]}-{c[4].split(':')[0].replace(' ', '_')}")
+def test_scaled_form_matches_oracle(ctx, gu, case):
+    import oracle
+    M, N, K, cfg_t, why = case
+    plan = ctx.plan(M, N, K)
+    if cfg_t is not None:
+        fam, bn, stages, split, bk, mode, epi = cfg_t
+        plan.set_config(_cfg(F1 if fam == "f1" else F2, bn, stages, split, 1, epi, bk, mode))
+    # exact case: 0/1 operands, small integers in C and factors that keep every fp32 intermediate exact
+    Ai, Bi = inputs.make_ab(M, N, K, "binary", "cuda")
+    C0 = inputs.draw(21, inputs.TAG_A, M, N, "int5", "cuda")
+    for alpha, beta in [(1.0, 1.0), (2.0, -3.0), (-1.0, 0.5), (0.0, 2.0), (0.5, 0.0)]:
+        buf, C = gu.alloc_c_with_guards(M, N)
+        C.copy_(C0)
+        plan.run_scaled(alpha, beta, Ai, Bi, C)
+        st, code = ctx.last_device_status()
+        assert st == hgemm.OK, f"device status {st} code {code:#x}"
+        assert gu.guards_intact(buf, M, N), f"{why}: the kernel wrote outside C"
+        ref = oracle.hgemm_scaled_full(inputs.bits(Ai), inputs.bits(Bi), inputs.bits(C0), alpha, beta)
+        assert np.abs(ref).max() < 2 ** 24          # every fp32 intermediate is exact: both sides round the same number once
+        gu.assert_exact(C, ref, f"{why}: alpha={alpha} beta={beta}")
+    # beta == 0 never reads the old C: NaN there must not reach the result
+    buf, C = gu.alloc_c_with_guards(M, N)               # pre-filled with a NaN pattern
+    plan.run_scaled(2.0, 0.0, Ai, Bi, C)
+    gu.assert_exact(C, oracle.hgemm_scaled_full(inputs.bits(Ai), inputs.bits(Bi), None, 2.0, 0.0), f"{why}: beta=0 over NaN")
+    # random inputs: the contract's bound with its absolute term scaled by |alpha|
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    Cu = inputs.draw(22, inputs.TAG_B, M, N, "uniform", "cuda")
+    for alpha, beta in [(0.75, -1.5), (-2.5, 0.3)]:
+        buf, C = gu.alloc_c_with_guards(M, N)
+        C.copy_(Cu)
+        plan.run_scaled(alpha, beta, A, B, C)
+        ref = oracle.hgemm_scaled_full(inputs.bits(A), inputs.bits(B), inputs.bits(Cu), alpha, beta)
+        rep = oracle.check_contract(gu.bits_to_f64(gu.c_bits(C)), ref, K, abs_scale=abs(alpha))
+        assert rep["ok"], f"{why}: alpha={alpha} beta={beta}: {rep}"
+    # hgemm_run is the case alpha = 1, beta = 0, bit for bit
+    C1, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+    buf, C2 = gu.alloc_c_with_guards(M, N)
+    plan.run_scaled(1.0, 0.0, A, B, C2)
+    assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
+    assert hgemm.lib().hgemm_run_scaled(plan._h, float("nan"), 0.0, A.data_ptr(), B.data_ptr(), C2.data_ptr(), 0) == hgemm.ERR_INVALID_ARG
+    plan.close()

@@ -152,3 +152,43 @@ def test_paper_style_binary_exact_match(oracle_lib):
     assert frac_checkable > 0.9
     r16 = _f16_exact(oracle_lib.f64_to_f16_bits(got.ravel())).reshape(M, N)
     assert np.array_equal(r16[want < 2048], want[want < 2048].astype(np.float64))
+
+
+# ---- the general form C = alpha A B^T + beta C (paper section 2.1) ------------------------------------------
+
+def test_scaled_form_exact_rationals(oracle_lib):
+    """Brute force on tiny shapes: alpha, beta and every element as exact rationals."""
+    for (M, N, K, alpha, beta) in [(2, 3, 5, 0.5, -2.0), (4, 7, 8, -1.25, 0.75), (3, 2, 9, 3.0, 1.0)]:
+        a, b = inputs.make_ab(M, N, K, dist="uniform", seed=7 + M + N + K)
+        c = inputs.draw(11, inputs.TAG_A, M, N, "uniform")
+        af = [[Fraction(float(x)) for x in row] for row in a.tolist()]
+        bf = [[Fraction(float(x)) for x in row] for row in b.tolist()]
+        cf = [[Fraction(float(x)) for x in row] for row in c.tolist()]
+        got = oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), inputs.bits(c), alpha, beta)
+        for i in range(M):
+            for j in range(N):
+                exact = Fraction(alpha) * sum(af[i][k] * bf[j][k] for k in range(K)) + Fraction(beta) * cf[i][j]
+                # a few dozen bits in all: every fp64 operation above is exact
+                assert Fraction(float(got[i, j])) == exact, (M, N, K, i, j)
+
+
+def test_scaled_form_special_cases(oracle_lib):
+    M, N, K = 33, 65, 96
+    a, b = inputs.make_ab(M, N, K, dist="int5")
+    c = inputs.draw(5, inputs.TAG_A, M, N, "int5")
+    ab = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    cb = inputs.bits(c)
+    # alpha = 1, beta = 0 is the plain product, whatever C holds (NaN included)
+    nan_c = np.full((M, N), 0x7E00, dtype=np.uint16)
+    assert np.array_equal(oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), nan_c, 1.0, 0.0), ab)
+    # alpha = 0 leaves beta C; integers keep everything exact
+    assert np.array_equal(oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), cb, 0.0, 3.0),
+                          3.0 * c.to(torch.float64).numpy())
+    # linear in (alpha, beta): int64 arithmetic decides
+    want = 2 * (a.to(torch.int64).numpy() @ b.to(torch.int64).numpy().T) - 3 * c.to(torch.int64).numpy()
+    assert np.array_equal(oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), cb, 2.0, -3.0), want.astype(np.float64))
+    # the factors are the fp32 values the library receives
+    third = oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), cb, 1.0 / 3.0, 0.0)
+    assert np.array_equal(third, float(np.float32(1.0 / 3.0)) * ab)
+    with pytest.raises(ValueError):
+        oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), cb[:, :-1], 1.0, 1.0)
