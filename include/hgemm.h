@@ -75,6 +75,11 @@ enum {
 };
 
 enum {
+    HGEMM_TAIL_K = 0,
+    HGEMM_TAIL_N = 1
+};
+
+enum {
     HGEMM_EPILOGUE_DIRECT = 0, /* registers -> 16-byte global stores */
     HGEMM_EPILOGUE_TMA = 1     /* registers -> swizzled shared memory -> TMA store */
 };
@@ -95,7 +100,10 @@ typedef struct {
                              waves of the persistent grid and the last wave is at most 1/tail_split full, its tiles
                              are cut into tail_split K slices (summed in slice order through the workspace) so that
                              every SM works until the end; otherwise ignored */
-    int32_t reserved[6];  /* must be zero */
+    int32_t tail_mode;    /* how tail_split cuts those tiles: HGEMM_TAIL_K (0) as above; HGEMM_TAIL_N (1): into
+                             tail_split (2 or 4) column pieces of block_n / tail_split columns (a multiple of 32),
+                             each an independent narrower tile -- no partial sums, no workspace */
+    int32_t reserved[5];  /* must be zero */
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the
@@ -250,7 +258,10 @@ hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan
  * issue no TMA loads, bit 1 no MMAs, bit 2 no TMA stores (the pipeline still runs;
- * C is garbage).
+ * C is garbage).  Bit 3 changes no arithmetic: with a trace buffer set, EVERY CTA
+ * also writes the stamps 0 (started) and 7 (finished) behind CTA 0's 24 slots, at
+ * entries 24 + 2 * blockIdx and 25 + 2 * blockIdx -- the buffer must then hold
+ * 24 + 2 * 148 uint64.
  * 0 restores normal operation. */
 hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask);
 

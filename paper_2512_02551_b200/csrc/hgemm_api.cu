@@ -53,6 +53,7 @@ struct hgemm_plan_s {
         const void *a = nullptr, *b = nullptr;
         void *c = nullptr;
         CUtensorMap tmap_a, tmap_b, tmap_c;
+        CUtensorMap tmap_bt;   // B for the column pieces of tail tiles (fewer rows per box)
     };
     static constexpr int kMapCache = 64;
     MapEntry maps[kMapCache];
@@ -99,6 +100,10 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     // the slices of a tile wait for each other: each needs its own SM (or SM pair)
     if (cfg.split_k > 1 && cfg.split_k > ctx->num_sms / cg) return HGEMM_ERR_UNSUPPORTED;
     if (pl->layout == HGEMM_LAYOUT_NN && (cfg.block_n % (64 * cg)) != 0) return HGEMM_ERR_UNSUPPORTED;
+    // row-major B is staged in blocks of 64 columns: column pieces of tail tiles must be whole blocks per CTA
+    if (pl->layout == HGEMM_LAYOUT_NN && cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 &&
+        ((cfg.block_n / cfg.tail_split) % (64 * cg)) != 0)
+        return HGEMM_ERR_UNSUPPORTED;
     const bool cluster_split = cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER;
     if (cluster_split) {
         // can the device place a cluster of split_k CTAs of this kernel at all?
@@ -164,6 +169,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.split_k = int32_t(layout.slices);
     p.first_split_tile = int32_t(layout.first_split_tile);
     p.total_work = int32_t(layout.work_items);
+    p.tail_pieces = int32_t(layout.pieces);
     p.block_k = cfg.block_k;
     p.kblocks = int32_t((pl->K + cfg.block_k - 1) / cfg.block_k);
     p.block_n = cfg.block_n;
@@ -402,6 +408,10 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
             cfg.block_k = 64;
             cfg.stages = std::min(4, hgemm_host::max_stages(cfg.family, cfg.block_n, 64));
         }
+        if (cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 && ((cfg.block_n / cfg.tail_split) % unit) != 0) {
+            cfg.tail_split = 0;
+            cfg.tail_mode = HGEMM_TAIL_K;
+        }
         if (cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER && hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK)
             cfg.split_mode = HGEMM_SPLIT_WORKSPACE;   // the wider tile's partial sums no longer fit in shared memory
         if (hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK) return HGEMM_ERR_UNSUPPORTED;
@@ -524,6 +534,10 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
             if (!encode_2d(ctx, &e.tmap_b, B, K, N, 64, uint32_t(cfg.block_n / cg), CU_TENSOR_MAP_SWIZZLE_128B))
                 return HGEMM_ERR_CUDA;
         }
+        e.tmap_bt = e.tmap_b;      // unused unless tail tiles are cut into column pieces
+        if (plan->params.tail_pieces > 1 && plan->layout != HGEMM_LAYOUT_NN &&
+            !encode_2d(ctx, &e.tmap_bt, B, K, N, 64, uint32_t(cfg.block_n / plan->params.tail_pieces / cg), CU_TENSOR_MAP_SWIZZLE_128B))
+            return HGEMM_ERR_CUDA;
         if (plan->params.ragged_n) {
             e.tmap_c = e.tmap_a;   // never used: a C with ragged rows is stored element by element
         } else if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
@@ -564,9 +578,9 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     lc.numAttrs = ctx->dependent_launch ? 2 : 1;
     cudaError_t e;
     if (cg == 1)
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, me->tmap_a, me->tmap_b, me->tmap_c, plan->params);
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
     else
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2>, me->tmap_a, me->tmap_b, me->tmap_c, plan->params);
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;
 }
@@ -612,7 +626,7 @@ hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf)
 
 hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask)
 {
-    if (!plan || mask > 7u) return HGEMM_ERR_INVALID_ARG;
+    if (!plan || mask > 15u) return HGEMM_ERR_INVALID_ARG;
     plan->debug_skip = mask;
     return HGEMM_OK;
 }

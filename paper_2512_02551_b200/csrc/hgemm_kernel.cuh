@@ -77,6 +77,7 @@ struct KernelParams {
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
     uint32_t debug_skip;          // instrumentation: bit 0 = no TMA loads, bit 1 = no MMAs, bit 2 = no TMA stores (results are garbage)
     uint32_t epoch;               // workspace split-K: number of this launch among the launches that used `counters` (from 1)
+    int32_t tail_pieces;          // > 1: work items from first_split_tile on are tiles cut into this many column pieces (no K split)
     uint32_t scaled;              // 0: C = A B^T; 1: C = alpha A B^T + beta C (paper section 2.1)
     float alpha, beta;
 };
@@ -87,6 +88,13 @@ __device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         p.trace[slot] = t;
+    }
+    // debug bit 3: every CTA also records when it started working (slot 0) and when it finished (slot 7)
+    // behind the 24 slots of CTA 0: entries 24 + 2 * blockIdx.x and + 1
+    if (p.trace != nullptr && (p.debug_skip & 8u) && (slot == 0 || slot == 7)) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[24 + 2 * blockIdx.x + (slot == 7 ? 1 : 0)] = t;
     }
 }
 
@@ -237,18 +245,31 @@ struct WorkItem {
     int32_t slices;     // number of slices of this tile (1: the tile is one work item)
     int32_t split_index;   // index of this (tile, slice) among the split work items; split tiles are numbered from 0
     int32_t kb_begin, kb_count;
+    int32_t bn;         // columns of this work item: block_n, or block_n / tail_pieces for a piece of a tail tile
 };
 
 __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p, int32_t block_m_total)
 {
     WorkItem it;
-    // Whole tiles first, then the split ones: with a persistent grid the split tiles form the last,
-    // partly filled wave, whose tiles are cut along K so that every SM has work until the end.
+    // Whole tiles first, then the cut ones: with a persistent grid the cut tiles form the last,
+    // partly filled wave, whose tiles are cut along K (slices, summed afterwards) or into column
+    // pieces (independent narrower tiles) so that every SM has work until the end.
+    int32_t n_off = 0;
+    it.bn = p.block_n;
     if (w < p.first_split_tile) {
         it.tile = w;
         it.slice = 0;
         it.slices = 1;
         it.split_index = 0;
+    } else if (p.tail_pieces > 1) {
+        const int32_t idx = w - p.first_split_tile;
+        const int32_t t = idx / p.tail_pieces;
+        it.tile = p.first_split_tile + t;
+        it.slice = 0;
+        it.slices = 1;
+        it.split_index = 0;
+        it.bn = p.block_n / p.tail_pieces;
+        n_off = (idx - t * p.tail_pieces) * it.bn;
     } else {
         it.split_index = w - p.first_split_tile;
         const int32_t t = it.split_index / p.split_k;
@@ -265,7 +286,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     const int32_t tn = r / gsize;
     const int32_t tm = first_m + (r - tn * gsize);
     it.m0 = tm * block_m_total;
-    it.n0 = tn * p.block_n;
+    it.n0 = tn * p.block_n + n_off;
     const int32_t base = p.kblocks / it.slices, rem = p.kblocks - base * it.slices;
     it.kb_begin = it.slice * base + min(it.slice, rem);
     it.kb_count = base + (it.slice < rem ? 1 : 0);
@@ -278,7 +299,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
 template <int CTA_GROUP>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                  const __grid_constant__ CUtensorMap tmap_c, const KernelParams p)
+                  const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_addr(smem_raw) + 1023u) & ~1023u;
@@ -333,6 +354,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         fence_mbar_init();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
+        if (p.tail_pieces > 1) prefetch_tensormap(&tmap_bt);
         prefetch_tensormap(&tmap_c);
     }
     if (warp == 1) {
@@ -370,7 +392,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
             const WorkItem it = decode_work(w, p, kBlockMTotal);
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
-            const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * b_rows;
+            // this CTA's rows of B: its share of the work item's columns
+            const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
             for (int32_t kb = 0; kb < it.kb_count; ++kb) {
                 const long long c0 = tr ? clock64() : 0;
                 ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, ctl, status_code(kRoleProducer, 0, s));
@@ -388,11 +411,12 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 } else if (p.b_row_major) {
                     // B is K x N row-major: per 64-wide K sub-tile, one {64 columns, 64 k-rows} box per 64-column block
-                    const int32_t b_col = it.n0 + static_cast<int32_t>(cta_rank) * b_rows;
-                    const int32_t blocks = b_rows / 64;
-                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
-                    else if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
-                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, stage_bytes);
+                    const int32_t b_col = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
+                    const int32_t blocks = (it.bn / CTA_GROUP) / 64;       // a column piece of a tail tile loads fewer blocks
+                    const uint32_t tx = a_stage_bytes + static_cast<uint32_t>(subs * blocks) * (kSubK * 128u);
+                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
+                    else if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
+                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, tx);
                     for (int32_t sub = 0; sub < subs; ++sub) {
                         if constexpr (CTA_GROUP == 1) tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
                         else tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
@@ -400,6 +424,26 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             const uint32_t dst = b_dst + sub * b_sub_bytes + nb * (kSubK * 128);
                             if constexpr (CTA_GROUP == 1) tma_load_2d_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
                             else tma_load_2d_pair_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
+                        }
+                    }
+                } else if (it.bn != p.block_n) {
+                    // a column piece of a tail tile: its rows of B come through the narrower map `tmap_bt`, one box per
+                    // 64-wide K sub-tile, each placed where the full-height box of that sub-tile would start
+                    const uint32_t tx = a_stage_bytes + static_cast<uint32_t>(subs * (it.bn / CTA_GROUP)) * (kSubK * 2u);
+                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
+                    else if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
+                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, tx);
+                    if (p.tma_3d) {
+                        if constexpr (CTA_GROUP == 1) tma_load_3d_if(leader, a_dst, &tmap_a, 0, a_row, k0 / kSubK, fb);
+                        else tma_load_3d_pair_if(leader, a_dst, &tmap_a, 0, a_row, k0 / kSubK, fb);
+                    }
+                    for (int32_t sub = 0; sub < subs; ++sub) {
+                        if constexpr (CTA_GROUP == 1) {
+                            if (!p.tma_3d) tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                            tma_load_2d_if(leader, b_dst + sub * b_sub_bytes, &tmap_bt, k0 + sub * kSubK, b_row, fb);
+                        } else {
+                            if (!p.tma_3d) tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                            tma_load_2d_pair_if(leader, b_dst + sub * b_sub_bytes, &tmap_bt, k0 + sub * kSubK, b_row, fb);
                         }
                     }
                 } else if (p.tma_3d) {
@@ -466,6 +510,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * static_cast<uint32_t>(p.block_n);
+                // the instruction descriptor's N field (bits 17..22, N / 8) follows the work item's width
+                const uint32_t idesc = (p.idesc & ~(0x3fu << 17)) | (static_cast<uint32_t>(it.bn >> 3) << 17);
                 for (int32_t kb = 0; kb < it.kb_count; ++kb) {
                     const long long c0 = tr ? clock64() : 0;
                     ok = mbar_wait(bar_full + 8 * s, ph, ctl, status_code(kRoleMma, 0, s));
@@ -483,7 +529,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                             for (int k = 0; k < kSubK / kUmmaK; ++k) {
                                 // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
-                                umma_f16_if<CTA_GROUP>(leader, d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, p.idesc,
+                                umma_f16_if<CTA_GROUP>(leader, d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, idesc,
                                                        (kb | sub | k) != 0 ? 1u : 0u);
                             }
                         }
@@ -584,7 +630,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
             // chunks of this tile that hold columns of C, and whether this warp's 32 rows hold rows of C:
             // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
-            const int32_t live_chunks = min(chunks, (p.N - it.n0 + 31) / 32);
+            const int32_t live_chunks = min(it.bn / 32, (p.N - it.n0 + 31) / 32);
             const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
             if (it.slices == 1) {
                 // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second

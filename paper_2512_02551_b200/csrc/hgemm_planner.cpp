@@ -45,18 +45,24 @@ SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const
     L.tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
     L.first_split_tile = L.tiles;
     L.slices = 1;
+    L.pieces = 1;
     if (c.split_k > 1) {
         L.first_split_tile = 0;
         L.slices = c.split_k;
     } else if (c.tail_split >= 2) {
         const int64_t units = std::max(1, num_sms / cg);
         const int64_t tail = L.tiles % units;
-        if (L.tiles > units && tail > 0 && tail * c.tail_split <= units && c.tail_split <= ceil_div(K, c.block_k)) {
-            L.first_split_tile = L.tiles - tail;
-            L.slices = c.tail_split;
+        if (L.tiles > units && tail > 0 && tail * c.tail_split <= units) {
+            if (c.tail_mode == HGEMM_TAIL_N) {
+                L.first_split_tile = L.tiles - tail;
+                L.pieces = c.tail_split;
+            } else if (c.tail_split <= ceil_div(K, c.block_k)) {
+                L.first_split_tile = L.tiles - tail;
+                L.slices = c.tail_split;
+            }
         }
     }
-    L.work_items = L.first_split_tile + (L.tiles - L.first_split_tile) * L.slices;
+    L.work_items = L.first_split_tile + (L.tiles - L.first_split_tile) * L.slices * L.pieces;
     return L;
 }
 
@@ -106,9 +112,14 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     if (c.split_k > kMaxSplitK) return HGEMM_ERR_UNSUPPORTED;
     if (c.raster_group < 1) return HGEMM_ERR_UNSUPPORTED;
     if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA) return HGEMM_ERR_UNSUPPORTED;
-    for (int i = 0; i < 6; ++i)
+    for (int i = 0; i < 5; ++i)
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
     if (c.tail_split < 0 || c.tail_split > 16 || (c.tail_split >= 2 && c.split_k != 1)) return HGEMM_ERR_UNSUPPORTED;
+    if (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N) return HGEMM_ERR_UNSUPPORTED;
+    if (c.tail_mode == HGEMM_TAIL_N && c.tail_split >= 2) {
+        // column pieces: whole 32-column chunks, and for a pair a whole number of 8-row groups of B per CTA
+        if ((c.tail_split != 2 && c.tail_split != 4) || (c.block_n % (32 * c.tail_split)) != 0) return HGEMM_ERR_UNSUPPORTED;
+    }
     if (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) return HGEMM_ERR_UNSUPPORTED;
     if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) {
         if (cg != 1 || c.split_k > 16) return HGEMM_ERR_UNSUPPORTED;
@@ -145,6 +156,7 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     double wave_count;
     if (c.split_k > 1) wave_count = double(ceil_div(work, units));
     else if (L.slices > 1) wave_count = double(L.first_split_tile) / double(units) + 1.0 / double(L.slices);
+    else if (L.pieces > 1) wave_count = double(L.first_split_tile) / double(units) + 1.1 / double(L.pieces);   // narrower tiles run a little below the wide ones' rate
     else wave_count = double(ceil_div(L.tiles, units));
     const int64_t kb = ceil_div(K, c.block_k);
     const int64_t kb_per = ceil_div(kb, c.split_k);

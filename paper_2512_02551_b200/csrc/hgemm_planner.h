@@ -26,6 +26,7 @@ int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k);
 // K slices.  Uniform split-K: first = 0; tail split: first = tiles - (tiles mod units) when it applies.
 struct SplitLayout {
     int64_t tiles, first_split_tile, slices, work_items;
+    int64_t pieces;   // > 1: the tiles from first_split_tile on are cut into this many column pieces (slices == 1)
 };
 SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c);
 int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c, int32_t num_sms = 148);

@@ -194,6 +194,7 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.wait_budget = 2000000000LL;
     p.trace = nullptr;
     p.debug_skip = 0;
+    p.tail_pieces = 1;
     p.scaled = 0;
     p.alpha = 1.0f;
     p.beta = 0.0f;
@@ -205,7 +206,7 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     lc.blockDim = dim3(hgemm_dev::kThreads, 1, 1);
     lc.dynamicSmemBytes = size_t(hgemm_host::kSmemOptInBytes);
     lc.stream = s;
-    cudaError_t e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, tmap_a, tmap_b, tmap_c, p);
+    cudaError_t e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, tmap_a, tmap_b, tmap_c, tmap_b, p);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return HGEMM_ERR_CUDA;

@@ -10,10 +10,11 @@ namespace {
 struct Entry {
     int32_t M, N, K;
     int32_t family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue;
+    int32_t tail_mode;   // last, so that rows written before it existed still read as 0
 };
 const Entry kTable[] = {
 #include "hgemm_table.inc"
-    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}   // sentinel
+    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}   // sentinel
 };
 } // namespace
 
@@ -33,6 +34,7 @@ bool table_lookup(int64_t M, int64_t N, int64_t K, hgemm_config_t *out)
             c.split_k = e.split_k;
             c.split_mode = e.split_mode;
             c.tail_split = e.tail_split;
+            c.tail_mode = e.tail_mode;
             c.raster_group = e.raster_group;
             c.epilogue = e.epilogue;
             if (validate(M, N, K, c) != HGEMM_OK) return false;

@@ -72,6 +72,15 @@ def candidates(M: int, N: int, K: int):
                                                            epilogue=epi, block_k=bk, split_mode=0, tail_split=ts)
                                     if hgemm.validate_config(M, N, K, c2) == hgemm.OK:
                                         out.append(c2)
+                            if split == 1 and tiles > units and 0 < tail <= units // 2:
+                                # the last wave's tiles as 2 or 4 independent column pieces
+                                for pieces in (2, 4):
+                                    if tail * pieces <= units and bn % (32 * pieces) == 0:
+                                        c3 = hgemm.Config.make(family=family, block_n=bn, stages=st, split_k=1, raster_group=rg,
+                                                               epilogue=epi, block_k=bk, split_mode=0, tail_split=pieces,
+                                                               tail_mode=hgemm.TAIL_N)
+                                        if hgemm.validate_config(M, N, K, c3) == hgemm.OK:
+                                            out.append(c3)
     return out
 
 
@@ -87,7 +96,7 @@ def batch_ms(fn, n: int, stream) -> float:
 
 def key(c: hgemm.Config):
     d = c.as_dict()
-    return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "raster_group", "epilogue"))
+    return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "tail_mode", "raster_group", "epilogue"))
 
 
 def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, stream) -> dict:
@@ -164,7 +173,7 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
 def write_table(rows, path):
     with open(path, "w") as f:
         f.write("// Tuned per-shape configurations for B200, written by tune.py on the GPU box.\n")
-        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue}\n")
+        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode}\n")
         for r in rows:
             if not r["ok"]:
                 continue

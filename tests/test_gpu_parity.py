@@ -241,6 +241,32 @@ def test_tail_split(ctx, gu, family, bn, bk, stages, tail, M, N, K):
     plan.close()
 
 
+# ---- tail split along N: the last wave's tiles as independent narrower tiles ---------------------------------
+
+@pytest.mark.parametrize("family,bn,bk,stages,pieces", [(F2, 256, 128, 3, 2), (F2, 256, 64, 6, 4), (F1, 256, 64, 4, 2), (F1, 128, 128, 3, 4),
+                                                        (F2, 192, 128, 3, 2), (F1, 64, 64, 8, 2)])
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 512), (2000, 4104, 520), (12288, 4096, 256), (2100, 3000, 300), (4096, 1280, 384)])
+def test_tail_split_along_n(ctx, gu, family, bn, bk, stages, pieces, M, N, K):
+    import oracle
+    for epi in (TMA, DIRECT):
+        cfg = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=9, epilogue=epi, block_k=bk,
+                                tail_split=pieces, tail_mode=hgemm.TAIL_N)
+        A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+        C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+        gu.assert_close_full(C, A, B, f"tail pieces {cfg.as_dict()}") if M * N * K <= gu.FULL_CHECK_VOLUME else \
+            gu.assert_close_sampled(C, A, B, "uniform", inputs.shape_seed(M, N, K), f"tail pieces {cfg.as_dict()}")
+        # the pieces compute the same dot products in the same order as whole tiles do: bit-identical results
+        plain = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=9, epilogue=epi, block_k=bk)
+        C_plain, _, _ = gu.run_gemm(ctx, A, B, plain, plan=plan)
+        assert torch.equal(C.view(torch.int16), C_plain.view(torch.int16))
+        Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+        if M * N * K <= gu.FULL_CHECK_VOLUME:
+            plan.set_config(cfg)
+            Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+            gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"tail pieces, integers {cfg.as_dict()}")
+        plan.close()
+
+
 # ---- the NN layout: B given as the K x N operand, row-major ----------------------------------------------
 
 @pytest.mark.parametrize("M,N,K", [(128, 64, 64), (100, 136, 72), (300, 520, 200), (1024, 1024, 1024), (64, 64, 8192),
