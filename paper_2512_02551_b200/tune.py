@@ -179,7 +179,7 @@ def write_table(rows, path):
                 continue
             b = r["best"]
             f.write(f"{{{r['M']}, {r['N']}, {r['K']}, {b['family']}, {b['block_n']}, {b['block_k']}, {b['stages']}, "
-                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}}},\n")
+                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}, {b.get('tail_mode', 0)}}},\n")
 
 
 def main():
