@@ -75,6 +75,11 @@ enum {
 };
 
 enum {
+    HGEMM_ACC_F32 = 0,
+    HGEMM_ACC_F16 = 1
+};
+
+enum {
     HGEMM_TAIL_K = 0,
     HGEMM_TAIL_N = 1
 };
@@ -103,7 +108,12 @@ typedef struct {
     int32_t tail_mode;    /* how tail_split cuts those tiles: HGEMM_TAIL_K (0) as above; HGEMM_TAIL_N (1): into
                              tail_split (2 or 4) column pieces of block_n / tail_split columns (a multiple of 32),
                              each an independent narrower tile -- no partial sums, no workspace */
-    int32_t reserved[5];  /* must be zero */
+    int32_t accumulate;   /* HGEMM_ACC_F32 (0): fp32 accumulators, the paper's main setting and this library's default;
+                             HGEMM_ACC_F16 (1): fp16 accumulators in tensor memory (the paper's other valid setting for
+                             fp16 inputs, section 1): every 16-wide K step rounds the running sums to fp16, so
+                             results carry the larger error of that arithmetic.  Needs split_k == 1 and no K tail
+                             split; never chosen by the planner or the tuned table */
+    int32_t reserved[4];  /* must be zero */
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the

@@ -9,6 +9,7 @@ from .hgemm_oracle import (  # noqa: F401
     f16_bits_to_f64,
     f64_to_f16_bits,
     hgemm_full,
+    hgemm_f16acc_full,
     hgemm_scaled_full,
     hgemm_sampled,
     max_threads,

@@ -132,3 +132,29 @@ def hgemm_scaled_full(a_bits, b_bits, c_bits, alpha: float, beta: float) -> np.n
     if c.shape != ab.shape:
         raise ValueError(f"need C {ab.shape}, got {c.shape}")
     return al * ab + be * f16_bits_to_f64(c)
+
+
+def hgemm_f16acc_full(a_bits, b_bits, k_step: int = 16) -> np.ndarray:
+    """C for fp16 ACCUMULATION, as fp16 bit patterns (M x N): the running sums are kept in fp16.
+
+    The paper names fp16 accumulators as the other valid setting for fp16 inputs (section 1) but
+    does not say where such a kernel rounds.  The reading taken here is the tensor core's unit of
+    work: the K dimension is consumed in steps of ``k_step`` = 16 (one MMA instruction); within a
+    step the 16 products and their sum are exact, and the running sum is rounded to fp16 (round
+    to nearest even) once per step:  D <- RN16(D + sum_{k in step} a_k b_k),  D_0 = 0.
+    Hardware whose inner sum is not exact can differ from this in the last bit of a step whose
+    exact value lies next to a rounding boundary; the comparison in the tests allows for that.
+    Parity unpinned: the paper fixes neither the rounding points nor the inner precision, so
+    beyond the exactly representable cases this function pins a reading, not the paper.
+    """
+    a, b = _bits(a_bits), _bits(b_bits)
+    if a.ndim != 2 or b.ndim != 2 or a.shape[1] != b.shape[1]:
+        raise ValueError(f"need A (M,K) and B (N,K); got {a.shape} and {b.shape}")
+    m, k = a.shape
+    n = b.shape[0]
+    d = np.zeros((m, n), dtype=np.float64)
+    for k0 in range(0, k, k_step):
+        # 16 products of 11-bit significands and their sum fit fp64 exactly: the plain routine's result is exact
+        part = hgemm_full(np.ascontiguousarray(a[:, k0:k0 + k_step]), np.ascontiguousarray(b[:, k0:k0 + k_step]))
+        d = f16_bits_to_f64(f64_to_f16_bits((d + part).ravel())).reshape(m, n)
+    return f64_to_f16_bits(d.ravel()).reshape(m, n)

@@ -78,11 +78,11 @@ int32_t pow2_at_least(int32_t x)
     return p;
 }
 
-uint32_t make_idesc(int m, int n, bool b_mn_major = false)
+uint32_t make_idesc(int m, int n, bool b_mn_major = false, bool d_f16 = false)
 {
-    // tcgen05 instruction descriptor, kind::f16: D = fp32, A = B = fp16, both K-major, dense
+    // tcgen05 instruction descriptor, kind::f16: D = fp32 (or fp16), A = B = fp16, both K-major, dense
     uint32_t d = 0;
-    d |= 1u << 4;                      // [4,6)   D format: 1 = fp32
+    d |= (d_f16 ? 0u : 1u) << 4;       // [4,6)   D format: 0 = fp16, 1 = fp32
     d |= 0u << 7;                      // [7,10)  A format: 0 = fp16
     d |= 0u << 10;                     // [10,13) B format: 0 = fp16
     d |= 0u << 15;                     // [15]    A major: 0 = K
@@ -178,7 +178,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.tmem_cols = pow2_at_least(2 * cfg.block_n);
     p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
     p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;   // whole tiles only
-    p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN);
+    p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN, cfg.accumulate == HGEMM_ACC_F16);
+    p.acc_f16 = cfg.accumulate == HGEMM_ACC_F16 ? 1 : 0;
     p.b_row_major = pl->layout == HGEMM_LAYOUT_NN ? 1 : 0;
     p.workspace = static_cast<float *>(pl->workspace);
     p.counters = pl->counters;

@@ -77,6 +77,7 @@ struct KernelParams {
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
     uint32_t debug_skip;          // instrumentation: bit 0 = no TMA loads, bit 1 = no MMAs, bit 2 = no TMA stores (results are garbage)
     uint32_t epoch;               // workspace split-K: number of this launch among the launches that used `counters` (from 1)
+    int32_t acc_f16;              // 1: fp16 accumulators (one result in the low half of each 32-bit tensor-memory column)
     int32_t tail_pieces;          // > 1: work items from first_split_tile on are tiles cut into this many column pieces (no K split)
     uint32_t scaled;              // 0: C = A B^T; 1: C = alpha A B^T + beta C (paper section 2.1)
     float alpha, beta;
@@ -640,6 +641,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
+                    if (p.acc_f16) {
+                        // fp16 accumulators (measured layout: one result per 32-bit column, in its low half):
+                        // widen them, exactly, so that the store paths below see what they see with fp32 ones
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
+                    }
                     if (c + 2 >= chunks) release_accumulator();       // every load of this warp has completed
                     if (p.scaled && grow < p.M) {
 #pragma unroll

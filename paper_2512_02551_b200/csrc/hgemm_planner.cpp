@@ -112,8 +112,11 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     if (c.split_k > kMaxSplitK) return HGEMM_ERR_UNSUPPORTED;
     if (c.raster_group < 1) return HGEMM_ERR_UNSUPPORTED;
     if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA) return HGEMM_ERR_UNSUPPORTED;
-    for (int i = 0; i < 5; ++i)
+    for (int i = 0; i < 4; ++i)
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (c.accumulate != HGEMM_ACC_F32 && c.accumulate != HGEMM_ACC_F16) return HGEMM_ERR_UNSUPPORTED;
+    // fp16 accumulators: no fp16 partial sums are exchanged, so no split along K
+    if (c.accumulate == HGEMM_ACC_F16 && (c.split_k != 1 || (c.tail_split >= 2 && c.tail_mode == HGEMM_TAIL_K))) return HGEMM_ERR_UNSUPPORTED;
     if (c.tail_split < 0 || c.tail_split > 16 || (c.tail_split >= 2 && c.split_k != 1)) return HGEMM_ERR_UNSUPPORTED;
     if (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N) return HGEMM_ERR_UNSUPPORTED;
     if (c.tail_mode == HGEMM_TAIL_N && c.tail_split >= 2) {

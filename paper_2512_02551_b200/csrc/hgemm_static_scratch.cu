@@ -195,6 +195,7 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.trace = nullptr;
     p.debug_skip = 0;
     p.tail_pieces = 1;
+    p.acc_f16 = 0;
     p.scaled = 0;
     p.alpha = 1.0f;
     p.beta = 0.0f;

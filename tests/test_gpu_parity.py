@@ -419,3 +419,66 @@ def test_scaled_form_matches_oracle(ctx, gu, case):
     assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
     assert hgemm.lib().hgemm_run_scaled(plan._h, float("nan"), 0.0, A.data_ptr(), B.data_ptr(), C2.data_ptr(), 0) == hgemm.ERR_INVALID_ARG
     plan.close()
+
+
+# ---- fp16 accumulators (the paper's other setting for fp16 inputs, section 1) ----------------------------------
+
+def _ulp16(x):
+    """Spacing of fp16 at |x| (2^-24 below the smallest normal)."""
+    ax = np.maximum(np.abs(x), 2.0 ** -14)
+    return 2.0 ** (np.floor(np.log2(ax)) - 10)
+
+
+F16ACC_CASES = [
+    # family, bn, bk, stages, epilogue, tail pieces, M, N, K
+    (F1, 128, 64, 4, TMA, 0, 128, 128, 128),
+    (F1, 64, 128, 4, DIRECT, 0, 200, 136, 520),
+    (F2, 256, 64, 4, TMA, 0, 512, 520, 1024),
+    (F2, 128, 128, 4, DIRECT, 0, 300, 264, 2048),
+    (F1, 96, 64, 4, TMA, 0, 77, 203, 333),              # ragged N and K
+    (F2, 256, 64, 6, TMA, 2, 2100, 3000, 300),          # with the last wave cut into column pieces
+    (F1, 256, 64, 4, TMA, 0, 256, 256, 4096),
+]
+
+
+@pytest.mark.parametrize("case", F16ACC_CASES, ids=lambda c: f"f{c[0]}bn{c[1]}bk{c[2]}e{c[4]}t{c[5]}-{c[6]}x{c[7]}x{c[8]}")
+def test_fp16_accumulation(ctx, gu, case):
+    import oracle
+    family, bn, bk, stages, epi, pieces, M, N, K = case
+    cfg = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=epi, block_k=bk,
+                            tail_split=pieces, tail_mode=hgemm.TAIL_N if pieces else hgemm.TAIL_K, accumulate=hgemm.ACC_F16)
+    # exact case: every partial sum, in any order, is an integer of magnitude <= 2048
+    Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
+    bound = float((Ab.float() @ Bb.float().T).max())
+    assert bound <= 2048
+    C, _, plan = gu.run_gemm(ctx, Ab, Bb, cfg)
+    gu.assert_exact(C, oracle.hgemm_full(inputs.bits(Ab), inputs.bits(Bb)), f"fp16 accumulation, 0/1 operands {cfg.as_dict()}")
+    # random inputs against the model that rounds the running sum once per 16-wide K step: bit-identical
+    # except where the hardware's inexact inner sum lands on the other side of a rounding boundary
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+    model = oracle.f16_bits_to_f64(oracle.hgemm_f16acc_full(inputs.bits(A), inputs.bits(B)).ravel()).reshape(M, N)
+    got = gu.bits_to_f64(gu.c_bits(C))
+    same = float(np.mean(got == model))
+    # a flipped rounding happens at the magnitude the running sum had at that step, which can be far above the
+    # final value's: measure deviations in units of the fp16 spacing at the largest magnitudes of the matrix
+    dev = np.abs(got - model) / _ulp16(2.0 * np.abs(model).max())
+    assert same >= 0.99, f"only {same:.4f} of the entries equal the model"
+    assert dev.max() <= 2.0, f"largest deviation from the model: {dev.max()} spacings of the largest magnitudes"
+    # and it is a different arithmetic from fp32 accumulation: the same plan with fp32 accumulators
+    # meets the contract, whose bound fp16 accumulation exceeds once K is large
+    exact = oracle.hgemm_full(inputs.bits(A), inputs.bits(B))
+    if K >= 1024:
+        assert np.abs(got - exact).max() > np.abs(model - exact).max() * 0.25
+    cfg32 = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=epi, block_k=bk,
+                              tail_split=pieces, tail_mode=hgemm.TAIL_N if pieces else hgemm.TAIL_K)
+    C32, _, _ = gu.run_gemm(ctx, A, B, cfg32, plan=plan)
+    assert oracle.check_contract(gu.bits_to_f64(gu.c_bits(C32)), exact, K)["ok"]
+    plan.close()
+
+
+def test_fp16_accumulation_rejects_splits_along_k(ctx):
+    bad = hgemm.Config.make(block_n=128, stages=4, split_k=2, accumulate=hgemm.ACC_F16)
+    assert hgemm.validate_config(256, 256, 4096, bad) == hgemm.ERR_UNSUPPORTED
+    bad = hgemm.Config.make(block_n=128, stages=4, tail_split=2, accumulate=hgemm.ACC_F16)
+    assert hgemm.validate_config(256, 256, 4096, bad) == hgemm.ERR_UNSUPPORTED

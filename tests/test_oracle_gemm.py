@@ -192,3 +192,57 @@ def test_scaled_form_special_cases(oracle_lib):
     assert np.array_equal(third, float(np.float32(1.0 / 3.0)) * ab)
     with pytest.raises(ValueError):
         oracle_lib.hgemm_scaled_full(inputs.bits(a), inputs.bits(b), cb[:, :-1], 1.0, 1.0)
+
+
+# ---- fp16 accumulation: the running sum is rounded once per 16-wide K step -------------------------------------
+
+def test_f16_accumulation_rounding_points(oracle_lib):
+    """Hand-made rows that show where the model rounds: 2048 + 1 + 1 in three K steps stays 2048
+    (each +1 is a tie that goes to the even neighbour), while the exact sum is 2050; the same
+    numbers inside ONE step are added exactly and give 2050."""
+    one = np.float16(1.0).view(np.uint16)
+    def row(vals, K):
+        r = np.zeros(K, dtype=np.float16); r[:len(vals)] = vals; return r.view(np.uint16)
+    K = 48
+    a = np.zeros((1, K), dtype=np.float16); b = np.zeros((1, K), dtype=np.float16)
+    a[0, :16] = 32.0; b[0, :16] = 4.0          # first step: 16 * 128 = 2048
+    a[0, 16] = 1.0; b[0, 16] = 1.0             # second step: +1
+    a[0, 32] = 1.0; b[0, 32] = 1.0             # third step: +1
+    got = oracle_lib.hgemm_f16acc_full(a.view(np.uint16), b.view(np.uint16))
+    assert oracle_lib.f16_bits_to_f64(got.ravel())[0] == 2048.0
+    assert oracle_lib.hgemm_full(a.view(np.uint16), b.view(np.uint16))[0, 0] == 2050.0
+    # the same three contributions inside one 16-wide step: exact inner sum, one rounding
+    a2 = np.zeros((1, 16), dtype=np.float16); b2 = np.zeros((1, 16), dtype=np.float16)
+    a2[0, :14] = 32.0; b2[0, :14] = 4.0; a2[0, 14] = 16.0; b2[0, 14] = 16.0   # 14 * 128 + 256 = 2048
+    a2[0, 15] = 2.0; b2[0, 15] = 1.0                                          # + 2
+    got2 = oracle_lib.hgemm_f16acc_full(a2.view(np.uint16), b2.view(np.uint16))
+    assert oracle_lib.f16_bits_to_f64(got2.ravel())[0] == 2050.0
+    # a step size of the whole K is one rounding of the exact product
+    a3, b3 = inputs.make_ab(9, 11, 64, dist="uniform")
+    whole = oracle_lib.hgemm_f16acc_full(inputs.bits(a3), inputs.bits(b3), k_step=64)
+    assert np.array_equal(whole, oracle_lib.f64_to_f16_bits(oracle_lib.hgemm_full(inputs.bits(a3), inputs.bits(b3)).ravel()).reshape(9, 11))
+
+
+def test_f16_accumulation_exact_when_sums_are_representable(oracle_lib):
+    """Integer operands whose absolute products sum to at most 2048 per element: every partial sum,
+    in any order, is an integer fp16 holds exactly, so the model must return the exact product."""
+    M, N, K = 40, 56, 640
+    a, b = inputs.make_ab(M, N, K, dist="int5")
+    bound = np.abs(a.to(torch.int64).numpy()) @ np.abs(b.to(torch.int64).numpy()).T
+    assert bound.max() <= 2048
+    want = (a.to(torch.int64).numpy() @ b.to(torch.int64).numpy().T).astype(np.float64)
+    got = oracle_lib.f16_bits_to_f64(oracle_lib.hgemm_f16acc_full(inputs.bits(a), inputs.bits(b)).ravel()).reshape(M, N)
+    assert np.array_equal(got, want)
+
+
+def test_f16_accumulation_error_grows_with_k(oracle_lib):
+    """On random inputs the model differs from the exact product by roughly sqrt(K / 16) roundings of the
+    running magnitude -- more than fp32 accumulation would, less than the worst case."""
+    M, N, K = 32, 48, 2048
+    a, b = inputs.make_ab(M, N, K, dist="uniform")
+    exact = oracle_lib.hgemm_full(inputs.bits(a), inputs.bits(b))
+    got = oracle_lib.f16_bits_to_f64(oracle_lib.hgemm_f16acc_full(inputs.bits(a), inputs.bits(b)).ravel()).reshape(M, N)
+    err = np.abs(got - exact)
+    half_ulp = 2.0 ** -7                       # half the fp16 spacing at the largest running magnitudes (32..64)
+    assert err.max() > 2.0 ** -11 * np.abs(exact).max()          # worse than one final rounding
+    assert err.max() < (K / 16) * half_ulp                       # far inside the worst case
