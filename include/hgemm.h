@@ -68,7 +68,8 @@ enum {
 enum {
     HGEMM_SPLIT_WORKSPACE = 0, /* partials parked in a global workspace; any family; split_k <= 64 */
     HGEMM_SPLIT_CLUSTER = 1    /* the slices of a tile form one thread-block cluster and are summed through
-                                  distributed shared memory; 1-CTA family only; split_k in [2, 16]; the tile's
+                                  distributed shared memory; split_k CTAs (1-CTA family) or CTA pairs (2-CTA family)
+                                  per cluster, at most 16 CTAs: split_k in [2, 16] or [2, 8]; the tile's
                                   fp32 partial (512 * block_n bytes) plus split_k - 1 received shares of
                                   ceil(1/split_k) of it must fit in the stage ring and store staging
                                   (hgemm_validate_config answers) */

@@ -109,18 +109,19 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         // can the device place a cluster of split_k CTAs of this kernel at all?
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof(lc));
-        lc.gridDim = dim3(unsigned(cfg.split_k), 1, 1);
+        lc.gridDim = dim3(unsigned(cfg.split_k * cg), 1, 1);
         lc.blockDim = dim3(hgemm_dev::kThreads, 1, 1);
         lc.dynamicSmemBytes = size_t(hgemm_host::kSmemOptInBytes);
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = unsigned(cfg.split_k);
+        attr[0].val.clusterDim.x = unsigned(cfg.split_k * cg);      // the slices' CTAs (CTA pairs) form one cluster
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
         lc.attrs = attr;
         lc.numAttrs = 1;
         int clusters = 0;
-        cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1>, &lc);
+        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2>, &lc)
+                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1>, &lc);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return HGEMM_ERR_UNSUPPORTED;
@@ -190,8 +191,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.wait_budget = ctx->wait_budget;
     const int units = std::max(1, ctx->num_sms / cg);
     // cluster split-K is not persistent: one CTA per (tile, slice), the hardware schedules the clusters
-    pl->grid = cluster_split ? p.total_work : cg * std::min(p.total_work, units);
-    pl->cluster_dim = cluster_split ? cfg.split_k : cg;
+    pl->grid = cluster_split ? cg * p.total_work : cg * std::min(p.total_work, units);
+    pl->cluster_dim = cluster_split ? cg * cfg.split_k : cg;
     // Always ask for the whole opt-in shared memory: it keeps a second CTA off the SM, so two
     // CTAs can never wait on each other's tensor-memory allocation.
     pl->smem = int(hgemm_host::kSmemOptInBytes);
@@ -302,6 +303,11 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             break;
         }
         e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) {
+            st = cuda_fail(ctx, e);
+            break;
+        }
+        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) {
             st = cuda_fail(ctx, e);
             break;

@@ -327,7 +327,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // the warp index through a shuffle: a value the compiler knows to be warp-uniform
     const uint32_t warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);
     const uint32_t lane = lane_id();
-    const uint32_t cta_rank = (CTA_GROUP == 2) ? cluster_ctarank() : 0u;
+    // A pair is two CTAs whose ranks in the cluster differ in the last bit (cluster split-K puts several pairs
+    // in one cluster); cta_rank is the CTA's place in its pair, leader_rank the cluster rank of the pair's leader.
+    const uint32_t cluster_rank = (CTA_GROUP == 2) ? cluster_ctarank() : 0u;
+    const uint32_t cta_rank = cluster_rank & 1u;
+    const uint32_t leader_rank = cluster_rank & ~1u;
     const bool is_leader = (cta_rank == 0);
     const int32_t unit = (CTA_GROUP == 2) ? static_cast<int32_t>(blockIdx.x >> 1) : static_cast<int32_t>(blockIdx.x);
     const int32_t num_units = (CTA_GROUP == 2) ? static_cast<int32_t>(gridDim.x >> 1) : static_cast<int32_t>(gridDim.x);
@@ -385,7 +389,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // ===== TMA producer =====
         int s = 0;
         uint32_t ph = 0;
-        const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, 0) : bar_full;
+        const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, leader_rank) : bar_full;
         const bool tr = p.trace != nullptr && blockIdx.x == 0;
         const uint32_t leader = (lane == 0) ? 1u : 0u;     // the lane that issues the loads
         long long t_wait = 0, t_work = 0;
@@ -537,13 +541,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     const long long c2 = tr ? clock64() : 0;
                     // free the stage (in both CTAs of a pair) once these MMAs have read it
-                    umma_commit_if<CTA_GROUP>(leader, bar_empty + 8 * s);
+                    umma_commit_if<CTA_GROUP>(leader, bar_empty + 8 * s, leader_rank);
                     if (tr) { t_wait += c1 - c0; t_issue += c2 - c1; t_commit += clock64() - c2; ++n_kb; }
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
                 if (w == unit && lane == 0) trace_stamp(p, 4);
-                umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc);
+                umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc, leader_rank);
             }
             if (tr && lane == 0) { p.trace[8] = t_wait; p.trace[9] = t_issue; p.trace[10] = t_commit; p.trace[13] = t_acc; p.trace[15] = n_kb; }
         }
@@ -556,7 +560,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const uint32_t first_chunk = ew >> 2;                       // chunks first_chunk, first_chunk + 2, ...
         const uint32_t row_in_tile = q * 32u + lane;                // accumulator row = tensor-memory lane
         const uint32_t staging = staging_base + ew * kStagingBytesPerWarp;
-        const uint32_t tmem_empty_leader = (CTA_GROUP == 2) ? mapa(bar_tmem_empty, 0) : bar_tmem_empty;
+        const uint32_t tmem_empty_leader = (CTA_GROUP == 2) ? mapa(bar_tmem_empty, leader_rank) : bar_tmem_empty;
         const int32_t chunks = p.block_n / 32;
         uint32_t local_tile = 0;
         uint32_t store_count = 0;
@@ -657,10 +661,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     emit_chunk(v, c);
                 }
                 if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load
-            } else if (CTA_GROUP == 1 && p.cluster_split) {
+            } else if (p.cluster_split) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches
-                cs_m0 = it.m0;
+                cs_m0 = row0;
                 cs_n0 = it.n0;
                 cs_slice = it.slice;
             } else {
@@ -802,14 +806,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // bytes on the owner's receive barrier; every owner adds, per unit, its own copy and the S - 1
     // received ones in slice order and stores fp16.  Layout: [own tile | S - 1 receive slots of cap units].
     // Both cluster barriers are taken by every thread of every CTA of the cluster, also after an abort.
-    if constexpr (CTA_GROUP == 1) {
+    {
         if (p.cluster_split) {
             // (warps 0 and 1 only take part in the barriers; what they compute here from zeros is unused)
             const uint32_t S = static_cast<uint32_t>(p.split_k), me = static_cast<uint32_t>(cs_slice);
             // only the part of the tile that holds elements of C is exchanged: `rows` rows (a multiple of 32,
             // the epilogue warps' granule) of `chunks` 32-column chunks
             const int32_t chunks = min(p.block_n / 32, (p.N - cs_n0 + 31) / 32);
-            const uint32_t rows = static_cast<uint32_t>(min(kBlockM, (p.M - cs_m0 + 31) / 32 * 32));
+            const uint32_t rows = static_cast<uint32_t>(max(0, min(kBlockM, (p.M - cs_m0 + 31) / 32 * 32)));
             const uint32_t units = static_cast<uint32_t>(chunks) * 8u * rows;
             const uint32_t cap = (units + S - 1u) / S;
             const uint32_t own_begin = me * cap;
@@ -854,8 +858,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const uint32_t o_begin = o * cap;
                         if (o == me || o_begin >= units) continue;
                         const uint32_t slot = me < o ? me : me - 1u;              // receive slots skip the owner's own slice
-                        bulk_copy_to_cluster(mapa(recv_base + slot * cap * 16u, o), smem_base + o_begin * 16u,
-                                             min(cap, units - o_begin) * 16u, mapa(bar_recv, o));
+                        // slice o of this tile is the CTA (of a pair: the CTA with this one's place in its pair) o pairs on
+                        const uint32_t o_rank = (CTA_GROUP == 2) ? 2u * o + cta_rank : o;
+                        bulk_copy_to_cluster(mapa(recv_base + slot * cap * 16u, o_rank), smem_base + o_begin * 16u,
+                                             min(cap, units - o_begin) * 16u, mapa(bar_recv, o_rank));
                     }
                 }
                 if (threadIdx.x == 64) trace_stamp(p, 18);

@@ -125,7 +125,7 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     }
     if (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) return HGEMM_ERR_UNSUPPORTED;
     if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_CLUSTER) {
-        if (cg != 1 || c.split_k > 16) return HGEMM_ERR_UNSUPPORTED;
+        if (cg * c.split_k > 16) return HGEMM_ERR_UNSUPPORTED;   // the largest cluster holds 16 CTAs
         // once the main loops are done, the stage ring and the store staging behind it hold this CTA's fp32
         // partial (128 x block_n) and the S - 1 copies of its share that the other slices send
         const int64_t units = int64_t(128) * c.block_n / 4;                    // float4 units of a tile
@@ -210,7 +210,7 @@ hgemm_status_t heuristic(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm
             for (int32_t split : kSplits) {
                 if (split > kb) break;
                 for (int mode = 0; mode < 2; ++mode) {
-                if (mode == 1 && (split == 1 || split > 16 || family != HGEMM_FAMILY_UMMA_1CTA)) continue;
+                if (mode == 1 && (split == 1 || split * cg > 16)) continue;
                 hgemm_config_t c;
                 std::memset(&c, 0, sizeof(c));
                 c.split_mode = mode;

@@ -413,7 +413,7 @@ __device__ __forceinline__ void umma_f16_if(uint32_t pred, uint32_t d_tmem, uint
 // For a CTA pair the arrival goes to the barrier at the same shared-memory offset in both CTAs of the
 // pair: two plain commits, one per CTA (addresses from mapa), both tracking the same MMAs.
 template <int CTA_GROUP>
-__device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar)
+__device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar, uint32_t leader_rank)
 {
     if constexpr (CTA_GROUP == 1) {
         asm volatile(
@@ -421,12 +421,14 @@ __device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar)
             "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
             ::"r"(pred), "r"(bar) : "memory");
     } else {
+        // the pair's CTAs have the cluster ranks leader_rank and leader_rank + 1
         asm volatile(
-            "{\n\t.reg .pred e;\n\t.reg .b32 r0, r1;\n\telect.sync _|e, 0xffffffff;\n\t"
-            "mapa.shared::cluster.u32 r0, %1, 0;\n\tmapa.shared::cluster.u32 r1, %1, 1;\n\t"
+            "{\n\t.reg .pred e;\n\t.reg .b32 r0, r1, k1;\n\telect.sync _|e, 0xffffffff;\n\t"
+            "add.u32 k1, %2, 1;\n\t"
+            "mapa.shared::cluster.u32 r0, %1, %2;\n\tmapa.shared::cluster.u32 r1, %1, k1;\n\t"
             "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [r0];\n\t"
             "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [r1];\n\t}"
-            ::"r"(pred), "r"(bar) : "memory");
+            ::"r"(pred), "r"(bar), "r"(leader_rank) : "memory");
     }
 }
 

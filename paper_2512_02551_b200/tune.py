@@ -57,7 +57,7 @@ def candidates(M: int, N: int, K: int):
                     if split > 1 and tiles * split > 2 * units:
                         continue
                     rg = max(1, min(-(-M // (128 * cg)), round((units * bn / (128.0 * cg)) ** 0.5)))
-                    modes = (0,) if split == 1 else ((0, 1) if (family == 0 and split <= 16) else (0,))
+                    modes = (0,) if split == 1 else ((0, 1) if split * cg <= 16 else (0,))
                     for mode in modes:
                         for epi in ((hgemm.EPILOGUE_TMA, hgemm.EPILOGUE_DIRECT) if split == 1 else (hgemm.EPILOGUE_DIRECT,)):
                             c = hgemm.Config.make(family=family, block_n=bn, stages=st, split_k=split, raster_group=rg,

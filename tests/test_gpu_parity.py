@@ -184,8 +184,10 @@ def test_unit_shapes(ctx, gu, family, case):
 def test_unit_shapes_wide_stages_and_cluster_split(ctx, gu, case):
     import oracle
     M, N, K, bn, stages, split, raster, bk, mode = case
-    for family in ((F1,) if mode == CLUSTER else (F1, F2)):
+    for family in (F1, F2):
         cfg = _cfg(family, bn, stages, split, raster, TMA if split == 1 else DIRECT, bk, mode)
+        if hgemm.validate_config(M, N, K, cfg) == hgemm.ERR_UNSUPPORTED and family == F2 and mode == CLUSTER:
+            continue                      # more than 8 pairs per cluster, or a stage count only the 1-CTA family fits
         A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
         C, _, plan = gu.run_gemm(ctx, A, B, cfg)
         gu.assert_close_full(C, A, B, f"{case} family={family}")
@@ -324,15 +326,15 @@ def test_config4_small_mn_large_k(ctx, gu, MN, K):
     gu.check_shape(ctx, MN, MN, K, "uniform")
 
 
-@pytest.mark.parametrize("family,mode", [(F1, WORKSPACE), (F2, WORKSPACE), (F1, CLUSTER)])
+@pytest.mark.parametrize("family,mode", [(F1, WORKSPACE), (F2, WORKSPACE), (F1, CLUSTER), (F2, CLUSTER)])
 @pytest.mark.parametrize("MN,K,bn,split", [(64, 8192, 64, 8), (64, 12288, 32, 48), (256, 12288, 128, 12),
                                             (512, 8192, 128, 6), (512, 12288, 256, 16), (512, 12288, 256, 4),
                                             (512, 12288, 192, 16)])
 def test_split_k_is_deterministic(ctx, gu, family, mode, MN, K, bn, split):
     """Every split-K configuration reproduces its own bits run after run, with other work in flight
     to perturb the order in which slices finish."""
-    if mode == CLUSTER and split > 16:
-        pytest.skip("a cluster holds at most 16 slices")
+    if mode == CLUSTER and split * (2 if family == F2 else 1) > 16:
+        pytest.skip("a cluster holds at most 16 CTAs")
     cfg = _cfg(family, bn, 4, split, 1, DIRECT, 64, mode)
     if mode == CLUSTER and hgemm.validate_config(MN, MN, K, cfg) == hgemm.ERR_UNSUPPORTED:
         pytest.skip("this tile's partial sums and received shares do not fit in shared memory")
@@ -374,6 +376,7 @@ SCALED_CASES = [
     (256, 384, 4096, ("f1", 128, 4, 4, 64, WORKSPACE, DIRECT), "split-K through the workspace"),
     (256, 384, 4096, ("f2", 128, 4, 3, 64, WORKSPACE, DIRECT), "split-K, CTA pairs"),
     (64, 640, 2048, ("f1", 160, 2, 7, 128, CLUSTER, DIRECT), "split-K inside a cluster"),
+    (300, 520, 4096, ("f2", 128, 4, 4, 64, CLUSTER, DIRECT), "split-K inside a cluster of CTA pairs"),
 ]
 
 

@@ -74,9 +74,10 @@ def test_validate_rejects_illegal_configs(lib):
     c = hgemm.Config.make(block_n=128, stages=4)
     c.reserved[3] = 1
     assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
-    # cluster split-K: 1-CTA family only, at most 16 slices, the ring must hold the fp32 partial
+    # cluster split-K: at most 16 CTAs per cluster (16 slices, 8 for CTA pairs), the ring must hold the fp32 partial
     assert hgemm.validate_config(M, N, 4096, hgemm.Config.make(block_n=128, stages=4, split_k=8, split_mode=1)) == hgemm.OK
-    for kw in [dict(family=1, split_k=4), dict(split_k=32), dict(block_n=256, stages=2, split_k=4)]:
+    assert hgemm.validate_config(M, N, 4096, hgemm.Config.make(family=1, block_n=128, stages=4, split_k=8, split_mode=1)) == hgemm.OK
+    for kw in [dict(family=1, split_k=12), dict(split_k=32), dict(block_n=256, stages=2, split_k=4)]:
         c = hgemm.Config.make(**{**dict(block_n=128, stages=4, split_mode=1), **kw})
         assert hgemm.validate_config(M, N, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
     pair = hgemm.Config.make(family=hgemm.FAMILY_UMMA_2CTA, block_n=256, stages=6)
