@@ -215,6 +215,12 @@ hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *c
  * needed): configuration for (M, N, K) on a device with `num_sms` SMs. */
 hgemm_status_t hgemm_heuristic_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
 
+/* The configuration hgemm_plan starts from, as a pure host function: the tuned table's
+ * entry for a tabulated shape; for any other shape the best, by the cost model calibrated
+ * on the measured times of the tabulated shapes around it, of the heuristic's choice and
+ * those neighbours' configurations re-fitted to the shape. */
+hgemm_status_t hgemm_planned_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
+
 /* Check a configuration against a shape without a GPU: HGEMM_OK if legal. */
 hgemm_status_t hgemm_validate_config(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg);
 

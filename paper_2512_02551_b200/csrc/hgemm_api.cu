@@ -357,6 +357,17 @@ hgemm_status_t hgemm_destroy(hgemm_ctx_t *ctx)
     return HGEMM_OK;
 }
 
+hgemm_status_t hgemm_planned_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out)
+{
+    if (!out) return HGEMM_ERR_INVALID_ARG;
+    hgemm_status_t s = hgemm_host::validate_shape(M, N, K);
+    if (s != HGEMM_OK) return s;
+    hgemm_config_t c;
+    s = hgemm_host::plan_config(M, N, hgemm_host::padded_k(K), num_sms, &c);
+    if (s == HGEMM_OK) *out = c;
+    return s;
+}
+
 hgemm_status_t hgemm_heuristic_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out)
 {
     if (!out) return HGEMM_ERR_INVALID_ARG;
@@ -401,10 +412,8 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
     if (s != HGEMM_OK) return s;
     const int64_t Kp = hgemm_host::padded_k(K);
     hgemm_config_t cfg;
-    if (!hgemm_host::table_lookup(M, N, Kp, &cfg) || hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK) {
-        s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);
-        if (s != HGEMM_OK) return s;
-    }
+    s = hgemm_host::plan_config(M, N, Kp, ctx->num_sms, &cfg);   // the table, else the neighbours' configurations re-fitted
+    if (s != HGEMM_OK) return s;
     if (layout == HGEMM_LAYOUT_NN) {
         // row-major B is staged in blocks of 64 columns: widen the tile to the next legal width and
         // give back stages until it fits

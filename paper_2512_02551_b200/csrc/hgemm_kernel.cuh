@@ -604,11 +604,31 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         bulk_commit_group();
                     }
                     ++store_count;
-                } else if (grow < p.M && p.ragged_n) {
-                    float f[32];
+                } else if (p.ragged_n) {
+                    // rows of C are not multiples of 16 bytes: neither TMA nor vector stores apply.  The chunk is
+                    // transposed through the warp's staging buffer (same 64-byte swizzle as above) so that each
+                    // store instruction writes 32 consecutive elements of one row instead of one element of 32 rows.
+                    const uint32_t row_addr = staging + lane * 64u;
+                    const uint32_t sw = (lane >> 1) & 3u;
+                    __syncwarp();                                   // the previous chunk's reads of the buffer are done
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
-                    store_ragged(p.C, p.N, grow, col0, f, 32);
+                    for (uint32_t j = 0; j < 4; ++j) {
+                        st_shared_v4(row_addr + ((j ^ sw) << 4),
+                                     pack_half2_rn(v[8 * j + 0], v[8 * j + 1]), pack_half2_rn(v[8 * j + 2], v[8 * j + 3]),
+                                     pack_half2_rn(v[8 * j + 4], v[8 * j + 5]), pack_half2_rn(v[8 * j + 6], v[8 * j + 7]));
+                    }
+                    __syncwarp();
+                    const int32_t col = col0 + static_cast<int32_t>(lane);
+                    const int32_t first_row = row0 + static_cast<int32_t>(q) * 32;
+                    const int32_t rows_here = min(32, p.M - first_row);
+                    if (col < p.N) {
+                        unsigned short *dst = reinterpret_cast<unsigned short *>(p.C) + static_cast<size_t>(first_row) * p.N + col;
+                        for (int32_t r = 0; r < rows_here; ++r) {
+                            const uint32_t src = staging + static_cast<uint32_t>(r) * 64u +
+                                                 (((lane >> 3) ^ ((static_cast<uint32_t>(r) >> 1) & 3u)) << 4) + (lane & 7u) * 2u;
+                            dst[static_cast<size_t>(r) * p.N] = ld_shared_u16(src);
+                        }
+                    }
                 } else if (grow < p.M) {
                     __half *dst = p.C + static_cast<size_t>(grow) * p.N + col0;
 #pragma unroll

@@ -46,4 +46,19 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
 // Tuned table (generated on the box by the tuner; may be empty).  Returns true on a hit.
 bool table_lookup(int64_t M, int64_t N, int64_t K, hgemm_config_t *out);
 
+// The tuned shapes around an untabulated one: the (up to 8) tabulated shapes nearest to it in log space,
+// nearest first, each with the time the tuner measured.
+struct TableNeighbour {
+    int64_t M, N, K;
+    hgemm_config_t cfg;
+    double us;          // measured time of cfg on (M, N, K); 0 if the table does not record it
+};
+int table_neighbours(int64_t M, int64_t N, int64_t K, TableNeighbour *out, int max_out);
+
+// The configuration hgemm_plan uses: the table's entry for a tabulated shape; otherwise the candidate with
+// the lowest calibrated estimate among the cost model's own choice and the neighbouring tuned shapes'
+// configurations re-fitted to this shape (split factor clamped and also scaled with K, raster group and tail
+// split recomputed), where a neighbour's candidates are scaled by (measured time / estimate) at that neighbour.
+hgemm_status_t plan_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
+
 } // namespace hgemm_host

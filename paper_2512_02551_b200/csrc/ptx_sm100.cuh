@@ -220,6 +220,13 @@ __device__ __forceinline__ float4 ld_shared_v4(uint32_t addr)
     return v;
 }
 
+__device__ __forceinline__ unsigned short ld_shared_u16(uint32_t addr)
+{
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ void cluster_arrive()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");

@@ -24,7 +24,7 @@ LAYOUT_TN, LAYOUT_NN = 0, 1
 # every symbol include/hgemm.h declares
 EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
-    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_validate_config", "hgemm_estimate_config",
+    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
@@ -92,6 +92,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan_get_config": (i32, [p, cfgp]),
             "hgemm_plan_set_config": (i32, [p, cfgp]),
             "hgemm_heuristic_config": (i32, [i64, i64, i64, i32, cfgp]),
+            "hgemm_planned_config": (i32, [i64, i64, i64, i32, cfgp]),
             "hgemm_validate_config": (i32, [i64, i64, i64, cfgp]),
             "hgemm_estimate_config": (ctypes.c_double, [i64, i64, i64, i32, cfgp]),
             "hgemm_config_smem_bytes": (i64, [cfgp]),
@@ -126,6 +127,12 @@ def _check(status: int, what: str) -> None:
 def heuristic_config(M: int, N: int, K: int, num_sms: int = 148) -> Config:
     c = Config()
     _check(lib().hgemm_heuristic_config(M, N, K, num_sms, ctypes.byref(c)), f"hgemm_heuristic_config({M},{N},{K})")
+    return c
+
+
+def planned_config(M: int, N: int, K: int, num_sms: int = 148) -> Config:
+    c = Config()
+    _check(lib().hgemm_planned_config(M, N, K, num_sms, ctypes.byref(c)), f"hgemm_planned_config({M},{N},{K})")
     return c
 
 

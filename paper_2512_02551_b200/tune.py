@@ -99,7 +99,7 @@ def key(c: hgemm.Config):
     return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "tail_mode", "raster_group", "epilogue"))
 
 
-def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, stream) -> dict:
+def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, stream, explore: int = 0) -> dict:
     A = A_all.view(-1)[:M * K].view(M, K)
     B = B_all.view(-1)[:N * K].view(N, K)
     C = C_all[:M * N].view(M, N)
@@ -108,7 +108,8 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     cands = candidates(M, N, K)
     cands.sort(key=lambda c: hgemm.estimate_config(M, N, K, c))
     chosen, seen = [], set()
-    for c in [default] + cands[:top]:
+    extra = rng.sample(cands[top:], min(explore, max(0, len(cands) - top))) if explore > 0 else []   # for refitting the cost model
+    for c in [default] + cands[:top] + extra:
         if key(c) not in seen:
             seen.add(key(c))
             chosen.append(c)
@@ -167,19 +168,20 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     default_t = next((t for t, _, c in results if key(c) == key(default)), None)
     plan.close()
     return {"M": M, "N": N, "K": K, "best": best.as_dict(), "us": best_t * 1e3, "default_us": None if default_t is None else default_t * 1e3,
-            "torch_us": t_torch * 1e3, "ok": ok, "tried": len(results)}
+            "torch_us": t_torch * 1e3, "ok": ok, "tried": len(results),
+            "all": [list(key(c)) + [round(t * 1e3, 3)] for t, _, c in results]}   # every first-pass timing: key fields, us
 
 
 def write_table(rows, path):
     with open(path, "w") as f:
         f.write("// Tuned per-shape configurations for B200, written by tune.py on the GPU box.\n")
-        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode}\n")
+        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode, measured us}\n")
         for r in rows:
             if not r["ok"]:
                 continue
             b = r["best"]
             f.write(f"{{{r['M']}, {r['N']}, {r['K']}, {b['family']}, {b['block_n']}, {b['block_k']}, {b['stages']}, "
-                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}, {b.get('tail_mode', 0)}}},\n")
+                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}, {b.get('tail_mode', 0)}, {r['us']:.2f}f}},\n")
 
 
 def main():
@@ -188,6 +190,7 @@ def main():
     ap.add_argument("--shapes", nargs="*")
     ap.add_argument("--top", type=int, default=20)
     ap.add_argument("--resume", action="store_true")
+    ap.add_argument("--explore", type=int, default=0, help="also time this many randomly drawn candidates per shape")
     args = ap.parse_args()
     os.makedirs(args.out, exist_ok=True)
     shapes = ([tuple(int(v) for v in s.lower().split("x")) for s in args.shapes] if args.shapes
@@ -210,7 +213,7 @@ def main():
         for (M, N, K) in shapes:
             r = done.get((M, N, K))
             if r is None:
-                r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream)
+                r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream, args.explore)
                 log.write(json.dumps(r) + "\n")
                 log.flush()
             rows.append(r)
