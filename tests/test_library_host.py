@@ -97,3 +97,25 @@ def test_no_gpu_create_fails_loudly(lib):
         pytest.skip("a GPU is present")
     with pytest.raises(hgemm.HgemmError):
         hgemm.Context(0)
+
+
+def test_planned_config_for_tabulated_and_other_shapes(lib):
+    """hgemm_planned_config: the table's entry on a tabulated shape; elsewhere a legal configuration that the
+    cost model does not rank behind the pure heuristic's choice by more than the neighbours' calibration allows."""
+    c = hgemm.planned_config(4096, 4096, 4096)
+    assert hgemm.validate_config(4096, 4096, 4096, c) == hgemm.OK
+    assert (c.family, c.block_n) == (hgemm.FAMILY_UMMA_2CTA, 256)          # the tuned entry of the flagship square
+    shapes = [(1, 1, 1), (7, 9, 11), (1536, 1536, 1536), (96, 11008, 4096), (3000, 5000, 7000), (200, 200, 20000),
+              (16384, 16384, 16384), (4194304, 64, 64), (64, 64, 4194304), (77, 203, 333)]
+    for (M, N, K) in shapes:
+        c = hgemm.planned_config(M, N, K)
+        Kp = (K + 7) // 8 * 8                                               # plans run on K padded to a multiple of 8
+        assert hgemm.validate_config(M, N, Kp, c) == hgemm.OK, (M, N, K, c.as_dict())
+        assert 1 <= c.split_k <= -(-Kp // c.block_k)
+        assert c.accumulate == hgemm.ACC_F32                                # fp16 accumulators are never chosen
+        h = hgemm.heuristic_config(M, N, Kp)
+        # a re-fitted neighbour only replaces the heuristic's choice when the model, scaled by what was measured
+        # around the shape, prefers it; the raw estimates therefore stay within the spread of those scales
+        assert hgemm.estimate_config(M, N, Kp, c) <= 3.0 * hgemm.estimate_config(M, N, Kp, h)
+    with pytest.raises(hgemm.HgemmError):
+        hgemm.planned_config(0, 64, 64)
