@@ -176,6 +176,16 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.block_n = cfg.block_n;
     p.stages = cfg.stages;
     p.raster_group = std::min(cfg.raster_group, p.tiles_m);
+    {
+        // divisors of the work decode as multiply-and-shift constants
+        const int32_t rg = std::max(1, std::min(p.raster_group, p.tiles_m));
+        const int32_t last = p.tiles_m - ((p.tiles_m - 1) / rg) * rg;       // m-tiles of the last raster group
+        p.fd_per_group = hgemm_dev::make_fast_div(uint32_t(rg) * uint32_t(p.tiles_n));
+        p.fd_raster = hgemm_dev::make_fast_div(uint32_t(rg));
+        p.fd_last_group = hgemm_dev::make_fast_div(uint32_t(last));
+        p.fd_split = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.split_k)));
+        p.fd_pieces = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.tail_pieces)));
+    }
     p.tmem_cols = pow2_at_least(2 * cfg.block_n);
     p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
     p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;   // whole tiles only

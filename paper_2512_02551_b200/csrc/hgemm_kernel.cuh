@@ -50,6 +50,33 @@ constexpr int kCtrlBytes = 512;       // barriers, tensor-memory base, abort fla
 // Status-word roles
 constexpr uint32_t kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3, kRoleProbe = 4;
 
+// x / d for x < 2^31 without a division instruction: q = umulhi(x, mul) >> shr (d == 1: q = x).
+// mul = ceil(2^(31 + ceil(log2 d)) / d), shr = ceil(log2 d) - 1.
+struct FastDiv {
+    uint32_t mul, shr, d;
+};
+
+__host__ __device__ inline FastDiv make_fast_div(uint32_t d)
+{
+    FastDiv f;
+    f.d = d < 1u ? 1u : d;
+    f.mul = 0u;
+    f.shr = 0u;
+    if (f.d > 1u) {
+        uint32_t lg = 0;
+        while ((1ull << lg) < f.d) ++lg;                                 // ceil(log2 d) >= 1
+        const unsigned long long pw = 1ull << (31u + lg);
+        f.mul = static_cast<uint32_t>((pw + f.d - 1u) / f.d);
+        f.shr = lg - 1u;
+    }
+    return f;
+}
+
+__device__ __forceinline__ int32_t fast_div(int32_t x, const FastDiv &f)
+{
+    return f.d == 1u ? x : static_cast<int32_t>(__umulhi(static_cast<uint32_t>(x), f.mul) >> f.shr);
+}
+
 struct KernelParams {
     int32_t M, N, K;
     int32_t tiles_m, tiles_n;     // tiles_m counts block_m-row tiles (256 rows for a pair)
@@ -77,6 +104,8 @@ struct KernelParams {
     unsigned long long *trace;    // optional: CTA 0 writes %globaltimer stamps of its pipeline events (8 slots)
     uint32_t debug_skip;          // instrumentation: bit 0 = no TMA loads, bit 1 = no MMAs, bit 2 = no TMA stores (results are garbage)
     uint32_t epoch;               // workspace split-K: number of this launch among the launches that used `counters` (from 1)
+    // division by run-time constants of the work decode as multiply-high and shift (set by the host)
+    FastDiv fd_per_group, fd_raster, fd_last_group, fd_split, fd_pieces;
     int32_t acc_f16;              // 1: fp16 accumulators (one result in the low half of each 32-bit tensor-memory column)
     int32_t tail_pieces;          // > 1: work items from first_split_tile on are tiles cut into this many column pieces (no K split)
     uint32_t scaled;              // 0: C = A B^T; 1: C = alpha A B^T + beta C (paper section 2.1)
@@ -264,7 +293,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
         it.split_index = 0;
     } else if (p.tail_pieces > 1) {
         const int32_t idx = w - p.first_split_tile;
-        const int32_t t = idx / p.tail_pieces;
+        const int32_t t = fast_div(idx, p.fd_pieces);
         it.tile = p.first_split_tile + t;
         it.slice = 0;
         it.slices = 1;
@@ -273,24 +302,29 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
         n_off = (idx - t * p.tail_pieces) * it.bn;
     } else {
         it.split_index = w - p.first_split_tile;
-        const int32_t t = it.split_index / p.split_k;
+        const int32_t t = fast_div(it.split_index, p.fd_split);
         it.tile = p.first_split_tile + t;
         it.slice = it.split_index - t * p.split_k;
         it.slices = p.split_k;
     }
     // grouped raster: groups of raster_group m-tiles, swept along n inside a group
     const int32_t per_group = p.raster_group * p.tiles_n;
-    const int32_t g = it.tile / per_group;
+    const int32_t g = fast_div(it.tile, p.fd_per_group);
     const int32_t first_m = g * p.raster_group;
-    const int32_t gsize = min(p.raster_group, p.tiles_m - first_m);
+    const int32_t gsize = min(p.raster_group, p.tiles_m - first_m);   // the last group may hold fewer m-tiles
     const int32_t r = it.tile - g * per_group;
-    const int32_t tn = r / gsize;
+    const int32_t tn = gsize == p.raster_group ? fast_div(r, p.fd_raster) : fast_div(r, p.fd_last_group);
     const int32_t tm = first_m + (r - tn * gsize);
     it.m0 = tm * block_m_total;
     it.n0 = tn * p.block_n + n_off;
-    const int32_t base = p.kblocks / it.slices, rem = p.kblocks - base * it.slices;
-    it.kb_begin = it.slice * base + min(it.slice, rem);
-    it.kb_count = base + (it.slice < rem ? 1 : 0);
+    if (it.slices == 1) {
+        it.kb_begin = 0;
+        it.kb_count = p.kblocks;
+    } else {
+        const int32_t base = fast_div(p.kblocks, p.fd_split), rem = p.kblocks - base * it.slices;   // slices == split_k here
+        it.kb_begin = it.slice * base + min(it.slice, rem);
+        it.kb_count = base + (it.slice < rem ? 1 : 0);
+    }
     return it;
 }
 

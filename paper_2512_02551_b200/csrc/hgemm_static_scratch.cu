@@ -181,6 +181,11 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.block_n = block_n;
     p.stages = cfg.stages;
     p.raster_group = 1;
+    p.fd_per_group = hgemm_dev::make_fast_div(uint32_t(p.tiles_n));
+    p.fd_raster = hgemm_dev::make_fast_div(1u);
+    p.fd_last_group = hgemm_dev::make_fast_div(1u);
+    p.fd_split = hgemm_dev::make_fast_div(uint32_t(std::max(1, split_k)));
+    p.fd_pieces = hgemm_dev::make_fast_div(1u);
     int32_t cols = 32;
     while (cols < 2 * block_n) cols <<= 1;
     p.tmem_cols = cols;
