@@ -154,6 +154,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtl &ctl, uint32_t code)
 {
+    if (mbar_test_wait(bar, parity)) return true;      // already complete: the cheap query answers
 #pragma unroll 1
     for (int i = 0; i < 16; ++i)
         if (mbar_try_wait(bar, parity)) return true;
