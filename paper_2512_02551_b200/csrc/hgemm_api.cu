@@ -191,6 +191,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;   // whole tiles only
     p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN, cfg.accumulate == HGEMM_ACC_F16);
     p.acc_f16 = cfg.accumulate == HGEMM_ACC_F16 ? 1 : 0;
+    p.idesc_tail = make_idesc(128 * cg, cfg.block_n / int(std::max<int64_t>(1, layout.pieces)), pl->layout == HGEMM_LAYOUT_NN,
+                              cfg.accumulate == HGEMM_ACC_F16);
     p.b_row_major = pl->layout == HGEMM_LAYOUT_NN ? 1 : 0;
     p.workspace = static_cast<float *>(pl->workspace);
     p.counters = pl->counters;

@@ -96,6 +96,7 @@ struct KernelParams {
     int32_t tma_3d;               // 1: the A and B maps are 3-D {64, rows, K / 64}: one load per operand per stage
     int32_t cluster_split;        // 1: the split_k slices of a tile are one cluster and reduce through shared memory
     uint32_t idesc;               // tcgen05 instruction descriptor
+    uint32_t idesc_tail;          // the same with N = block_n / tail_pieces (column pieces of tail tiles)
     float *workspace;             // split-K partials: [work item][cta of pair][chunk][128 rows][32 cols]
     uint32_t *counters;           // split-K counters: [tile][cta of pair][arrived, finished]
     uint32_t *status;             // device status word (0 = fine)
@@ -329,6 +330,24 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     return it;
 }
 
+// The same work item with every field passed through a shuffle from lane 0: all lanes already hold the same
+// values, but only after the shuffle does the compiler know it, and TMA and tcgen05 instructions take their
+// operands from uniform registers -- values it cannot prove uniform cost a move per instruction.
+__device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
+{
+    WorkItem u;
+    u.tile = __shfl_sync(0xffffffffu, it.tile, 0);
+    u.m0 = __shfl_sync(0xffffffffu, it.m0, 0);
+    u.n0 = __shfl_sync(0xffffffffu, it.n0, 0);
+    u.slice = __shfl_sync(0xffffffffu, it.slice, 0);
+    u.slices = __shfl_sync(0xffffffffu, it.slices, 0);
+    u.split_index = __shfl_sync(0xffffffffu, it.split_index, 0);
+    u.kb_begin = __shfl_sync(0xffffffffu, it.kb_begin, 0);
+    u.kb_count = __shfl_sync(0xffffffffu, it.kb_count, 0);
+    u.bn = __shfl_sync(0xffffffffu, it.bn, 0);
+    return u;
+}
+
 // -------------------------------------------------------------------------------------
 // the kernel
 
@@ -430,7 +449,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         long long t_wait = 0, t_work = 0;
         bool ok = true;
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
-            const WorkItem it = decode_work(w, p, kBlockMTotal);
+            const WorkItem it = warp_uniform(decode_work(w, p, kBlockMTotal));
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
             // this CTA's rows of B: its share of the work item's columns
             const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
@@ -540,7 +559,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const bool issue_mma = !(p.debug_skip & 2u);
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-                const WorkItem it = decode_work(w, p, kBlockMTotal);
+                const WorkItem it = warp_uniform(decode_work(w, p, kBlockMTotal));
                 const uint32_t acc = local_tile & 1u;
                 const uint32_t acc_ph = (local_tile >> 1) & 1u;
                 const long long ca = tr ? clock64() : 0;
@@ -550,8 +569,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * static_cast<uint32_t>(p.block_n);
-                // the instruction descriptor's N field (bits 17..22, N / 8) follows the work item's width
-                const uint32_t idesc = (p.idesc & ~(0x3fu << 17)) | (static_cast<uint32_t>(it.bn >> 3) << 17);
+                // The instruction descriptor's N field follows the work item's width: p.idesc for whole tiles,
+                // p.idesc_tail for the column pieces of tail tiles.  Both are kernel parameters on purpose: a
+                // descriptor computed at run time cost every MMA about 25 more cycles to issue than one that the
+                // instruction takes straight from the parameter bank, so the k-block loop exists once per descriptor.
+                auto run_k_blocks = [&](const uint32_t idesc) {
                 for (int32_t kb = 0; kb < it.kb_count; ++kb) {
                     const long long c0 = tr ? clock64() : 0;
                     ok = mbar_wait(bar_full + 8 * s, ph, ctl, status_code(kRoleMma, 0, s));
@@ -580,6 +602,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (tr) { t_wait += c1 - c0; t_issue += c2 - c1; t_commit += clock64() - c2; ++n_kb; }
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
+                };
+                if (it.bn == p.block_n) run_k_blocks(p.idesc);
+                else run_k_blocks(p.idesc_tail);
                 if (!ok) break;
                 if (w == unit && lane == 0) trace_stamp(p, 4);
                 umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc, leader_rank);

@@ -192,6 +192,7 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.epilogue_tma = 0;
     p.cluster_split = 0;
     p.idesc = (1u << 4) | (uint32_t(block_n >> 3) << 17) | (uint32_t(128 >> 4) << 24);   // fp32 accumulate, fp16 A/B, K-major
+    p.idesc_tail = p.idesc;
     p.workspace = reinterpret_cast<float *>(d->scratch + kControlBytes);
     p.counters = reinterpret_cast<uint32_t *>(d->scratch);
     p.status = reinterpret_cast<uint32_t *>(d->scratch + kStatusOffset);
