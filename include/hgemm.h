@@ -23,7 +23,8 @@
  *   - Shapes: any M, N, K >= 1 (each at most 2^22).  The kernels address rows of
  *     16-byte multiples; when K % 8 != 0 the plan owns zero-padded copies of A and B
  *     that hgemm_run refreshes with a small copy kernel before the GEMM, and when
- *     N % 8 != 0 the rows of C are stored element by element (both slower than the
+ *     N % 8 != 0 the rows of C are stored with 2-byte stores, 32 consecutive elements of
+ *     a row per instruction (both slower than the
  *     aligned case, same results).  There is no CPU or library fallback path.
  *   - hgemm_run is asynchronous on the given stream.  It creates no stream,
  *     allocates nothing and never synchronises (the timing rules of paper

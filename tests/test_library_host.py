@@ -119,3 +119,18 @@ def test_planned_config_for_tabulated_and_other_shapes(lib):
         assert hgemm.estimate_config(M, N, Kp, c) <= 3.0 * hgemm.estimate_config(M, N, Kp, h)
     with pytest.raises(hgemm.HgemmError):
         hgemm.planned_config(0, 64, 64)
+
+
+def test_every_grid_shape_plans_to_a_legal_configuration(lib):
+    """The tuned table covers the 9 x 9 x 9 grid: every entry must validate against its own shape (a stale
+    entry would silently fall back to the neighbours' configurations)."""
+    grid = [64, 128, 256, 512, 1024, 2048, 4096, 8192, 12288]
+    families = set()
+    for M in grid:
+        for N in grid:
+            for K in grid:
+                c = hgemm.planned_config(M, N, K)
+                assert hgemm.validate_config(M, N, K, c) == hgemm.OK, (M, N, K, c.as_dict())
+                assert hgemm.config_smem_bytes(c) <= 232448
+                families.add(c.family)
+    assert families == {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA}
