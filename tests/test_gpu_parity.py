@@ -293,6 +293,51 @@ def test_nn_layout(ctx, gu, M, N, K):
         ctx.plan(64, 60, 64, hgemm.LAYOUT_NN)             # ragged rows of B cannot be fetched by TMA in this layout
 
 
+NN_FEATURE_CASES = [
+    # M, N, K, configuration keywords, what it combines with the NN layout
+    (4096, 1280, 384, dict(family=F2, block_n=256, stages=6, block_k=64, epilogue=TMA, tail_split=2, tail_mode=hgemm.TAIL_N), "tail tiles cut into column pieces"),
+    (4096, 2560, 512, dict(family=F1, block_n=256, stages=4, block_k=64, epilogue=DIRECT, tail_split=2, tail_mode=hgemm.TAIL_N), "column pieces, 1-CTA family"),
+    (300, 520, 4096, dict(family=F2, block_n=128, stages=4, block_k=64, epilogue=DIRECT, split_k=4, split_mode=CLUSTER), "cluster split-K of CTA pairs"),
+    (256, 384, 4096, dict(family=F1, block_n=128, stages=4, block_k=64, epilogue=DIRECT, split_k=3, split_mode=WORKSPACE), "workspace split-K"),
+    (520, 392, 1024, dict(family=F1, block_n=128, stages=3, block_k=128, epilogue=TMA, accumulate=hgemm.ACC_F16), "fp16 accumulators"),
+]
+
+
+@pytest.mark.parametrize("case", NN_FEATURE_CASES, ids=lambda c: f"{c[0]}x{c[1]}x{c[2]}-{c[4].replace(' ', '_').replace(',', '')}")
+def test_nn_layout_with_other_features(ctx, gu, case):
+    """The row-major-B layout combined with the tail pieces, both split-K exchanges, the scaled form and fp16
+    accumulators: the same results as the TN layout gives for the same operands, bit for bit."""
+    import oracle
+    M, N, K, kw, what = case
+    cfg = hgemm.Config.make(raster_group=4, **kw)
+    A, B_nk = inputs.make_ab(M, N, K, "binary", "cuda")      # 0/1 operands: every sum exact in either accumulator
+    B_kn = B_nk.T.contiguous()
+    plan_nn = ctx.plan(M, N, K, hgemm.LAYOUT_NN)
+    plan_nn.set_config(cfg)
+    plan_tn = ctx.plan(M, N, K)
+    plan_tn.set_config(cfg)
+    buf, C_nn = gu.alloc_c_with_guards(M, N)
+    plan_nn.run(A, B_kn, C_nn)
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    assert gu.guards_intact(buf, M, N)
+    gu.assert_exact(C_nn, oracle.hgemm_full(inputs.bits(A), inputs.bits(B_nk)), f"NN with {what}")
+    Au, Bu_nk = inputs.make_ab(M, N, K, "uniform", "cuda")
+    Bu_kn = Bu_nk.T.contiguous()
+    C0 = inputs.draw(31, inputs.TAG_A, M, N, "uniform", "cuda")
+    C_nn = C0.clone()
+    C_tn = C0.clone()
+    plan_nn.run_scaled(1.5, -0.5, Au, Bu_kn, C_nn)
+    plan_tn.run_scaled(1.5, -0.5, Au, Bu_nk, C_tn)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    assert torch.equal(C_nn.view(torch.int16), C_tn.view(torch.int16)), f"NN and TN differ with {what}"
+    if kw.get("accumulate", 0) == 0:
+        ref = oracle.hgemm_scaled_full(inputs.bits(Au), inputs.bits(Bu_nk), inputs.bits(C0), 1.5, -0.5)
+        assert oracle.check_contract(gu.bits_to_f64(gu.c_bits(C_nn)), ref, K, abs_scale=1.5)["ok"]
+    plan_nn.close()
+    plan_tn.close()
+
+
 # ---- configuration 2: square sweep ---------------------------------------------------------------------
 
 @pytest.mark.parametrize("S", [1024, 2048, 4096, 8192])
