@@ -396,8 +396,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // ---- set-up -----------------------------------------------------------------------
     // Programmatic dependent launch: the next kernel in the stream may become resident (on SMs this
     // grid does not occupy, or as its CTAs retire) and run its own set-up while this grid works.
-    // Nothing below touches global memory until grid_dependency_wait() has returned, so a dependent
-    // launch never sees or disturbs the data of the kernel before it.
+    // No thread touches global memory before its own grid_dependency_wait() has returned, so a dependent
+    // launch never sees or disturbs the data of the kernel before it: the producer waits just before its
+    // first load (its first work item is decoded and its first stage claimed by then), the epilogue warps
+    // before their loop, the MMA warp -- which reads and writes only shared and tensor memory -- only when
+    // it has trace stamps to write.
     grid_launch_dependents();
     if (threadIdx.x == 0) {
         *abort_flag = 0u;
@@ -427,11 +430,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         cluster_wait();
     }
     tc_fence_after_sync();
-    grid_dependency_wait();          // from here on global memory may be read and written
-    if (threadIdx.x == 0) trace_stamp(p, 0);
     // broadcast through a shuffle so that the compiler knows the address is warp-uniform
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_base_slot, 0);
-    if (threadIdx.x == 0) trace_stamp(p, 1);
 
     // ---- roles ------------------------------------------------------------------------
     // Producer and MMA loops are executed by their whole warp with warp-uniform control flow (the
@@ -448,6 +448,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const uint32_t leader = (lane == 0) ? 1u : 0u;     // the lane that issues the loads
         long long t_wait = 0, t_work = 0;
         bool ok = true;
+        bool dependencies_met = false;
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
             const WorkItem it = warp_uniform(decode_work(w, p, kBlockMTotal));
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
@@ -463,6 +464,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const uint32_t b_dst = a_dst + a_stage_bytes;
                 const int32_t k0 = (it.kb_begin + kb) * p.block_k;
                 const uint32_t fb = full_leader + 8 * s;      // the (leader's) full barrier of this stage
+                if (!dependencies_met) {
+                    grid_dependency_wait();                   // the kernels before this one are complete: global memory may be read
+                    dependencies_met = true;
+                    if (threadIdx.x == 0) {
+                        trace_stamp(p, 0);
+                        trace_stamp(p, 1);
+                    }
+                }
                 if (p.debug_skip & 1u) {
                     if (lane == 0) {
                         if (is_leader) mbar_arrive(bar_full + 8 * s);
@@ -541,6 +550,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         if (tr && lane == 0) { p.trace[11] = t_wait; p.trace[12] = t_work; }
     } else if (warp == 1) {
+        if (p.trace != nullptr) grid_dependency_wait();   // this warp's only global accesses are trace stamps
         if (is_leader) {
             // ===== MMA issuer =====
             int s = 0;
@@ -625,6 +635,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         uint32_t local_tile = 0;
         uint32_t store_count = 0;
         bool ok = true;
+        grid_dependency_wait();                            // before the first store to C, workspace or counters
         for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
             const WorkItem it = decode_work(w, p, kBlockMTotal);
             const uint32_t acc = local_tile & 1u;
