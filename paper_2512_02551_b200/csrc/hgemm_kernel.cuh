@@ -438,6 +438,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // wait results are voted), and only the single-thread instructions are predicated on lane 0:
     // TMA and tcgen05 instructions take their operands from uniform registers, so operands the
     // compiler can prove warp-uniform cost nothing to issue, while per-thread ones each need a move.
+    bool tmem_freed = false;                       // warp 1: tensor memory was freed before the teardown
     int32_t cs_m0 = 0, cs_n0 = 0, cs_slice = 0;   // cluster split-K: the epilogue warps' one work item, kept for the exchange
     if (warp == 0) {
         // ===== TMA producer =====
@@ -620,6 +621,27 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc, leader_rank);
             }
             if (tr && lane == 0) { p.trace[8] = t_wait; p.trace[9] = t_issue; p.trace[10] = t_commit; p.trace[13] = t_acc; p.trace[15] = n_kb; }
+            if constexpr (CTA_GROUP == 1) {
+                // Free tensor memory as soon as the epilogue has read the last of it -- each accumulator's last
+                // use has been released -- instead of after the CTA-wide barrier of the teardown: the epilogue's
+                // final stores then overlap the deallocation.  (Not for cluster split-K, which reads tensor
+                // memory after the role loops, and not after an abort.)
+                if (ok && !p.cluster_split) {
+                    for (uint32_t a = 0; ok && a < 2u; ++a) {
+                        const uint32_t uses = (local_tile + 1u - a) / 2u;      // work items that used accumulator a (local_tile items in all)
+                        if (local_tile > a && uses > 0u) {
+                            ok = mbar_wait(bar_tmem_empty + 8 * a, (uses - 1u) & 1u, ctl, status_code(kRoleMma, 2, a));
+                            ok = __all_sync(0xffffffffu, ok);
+                        }
+                    }
+                    if (ok) {
+                        tc_fence_after_sync();
+                        tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+                        tmem_freed = true;
+                        if (lane == 0) trace_stamp(p, 7);
+                    }
+                }
+            }
         }
     } else {
         // ===== epilogue (warps 2..9) =====
@@ -1021,7 +1043,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         cluster_arrive_relaxed();
         cluster_wait();
     }
-    if (warp == 1) {
+    if (warp == 1 && !tmem_freed) {
         if (*abort_flag) {
             // give loads and MMAs that were in flight when a wait ran out time to land
             for (int i = 0; i < 200; ++i) __nanosleep(1000);
