@@ -262,7 +262,8 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
 
 /* Instrumentation: when `device_buf` (DEVICE pointer to 24 uint64, or NULL to switch
  * it off) is set, CTA 0 of every later launch of this plan writes nanosecond
- * %globaltimer stamps of its pipeline events: 0 dependencies met, 1 set-up done,
+ * %globaltimer stamps of its pipeline events: 0 and 1 the producer's dependency wait
+ * has returned (set-up done, first work item decoded, first stage claimed),
  * 2 first TMA load issued, 3 first k-block landed, 4 last MMA issued, 5 first
  * accumulator ready, 6 epilogue done, 7 tensor memory freed; and SM-clock totals:
  * 8/9/10 MMA thread waiting for data / issuing MMAs / committing, 11/12 producer
