@@ -67,7 +67,12 @@ enum {
 /* Where the fp32 partial sums of a split-K tile meet.  Both sum the slices in slice
  * order 0..S-1, so a configuration reproduces its own bits run after run. */
 enum {
-    HGEMM_SPLIT_WORKSPACE = 0, /* partials parked in a global workspace; any family; split_k <= 64 */
+    HGEMM_SPLIT_WORKSPACE = 0, /* partials parked in a global workspace; any family; split_k <= 64.  The slices of a
+                                  tile wait for one another on the GPU, which is safe because the grid never exceeds
+                                  the SM count and holds one CTA per SM: all of them are resident at once WHEN THE
+                                  GPU IS THEIRS.  If another long-running kernel holds SMs at the same time, slices
+                                  may wait for CTAs that cannot start; the wait is bounded (hgemm_set_wait_budget),
+                                  the launch then gives up and hgemm_last_device_status reports HGEMM_ERR_TIMEOUT */
     HGEMM_SPLIT_CLUSTER = 1    /* the slices of a tile form one thread-block cluster and are summed through
                                   distributed shared memory; split_k CTAs (1-CTA family) or CTA pairs (2-CTA family)
                                   per cluster, at most 16 CTAs: split_k in [2, 16] or [2, 8]; the tile's
