@@ -530,3 +530,38 @@ def test_fp16_accumulation_rejects_splits_along_k(ctx):
     assert hgemm.validate_config(256, 256, 4096, bad) == hgemm.ERR_UNSUPPORTED
     bad = hgemm.Config.make(block_n=128, stages=4, tail_split=2, accumulate=hgemm.ACC_F16)
     assert hgemm.validate_config(256, 256, 4096, bad) == hgemm.ERR_UNSUPPORTED
+
+
+# ---- special values: infinities, NaN, overflow of the fp16 result -------------------------------------------
+
+def test_infinities_nan_and_overflow(ctx, gu):
+    """IEEE behaviour the paper does not discuss but a drop-in GEMM must have: inf and NaN operands propagate
+    as the exact arithmetic of the oracle says, and sums beyond 65504 round to infinity."""
+    import oracle
+    M, N, K = 128, 96, 128
+    A, B = inputs.make_ab(M, N, K, "int5", "cuda")
+    A = A.clone(); B = B.clone()
+    A[23, :] = 60000.0; B[5, :] = 1.0; B[6, :] = -1.0             # overflow: about +-7.7e6 -> +-inf after rounding to fp16
+    A[3, 5] = float("inf"); B[:, 5] = B[:, 5].abs() + 1           # row 3: +inf times positive values -> +inf everywhere
+    A[7, 9] = float("-inf"); B[0:48, 9] = 2.0; B[48:, 9] = -2.0   # row 7: -inf and +inf halves
+    A[11, 20] = float("inf"); B[17, 20] = 0.0                     # inf * 0 -> NaN in one element (row 11, column 17)
+    A[19, 33] = float("nan")                                      # row 19: NaN everywhere
+    C, _, plan = gu.run_gemm(ctx, A, B, _cfg(F1, 96, 4, 1, 1, TMA))
+    ref = oracle.hgemm_full(inputs.bits(A), inputs.bits(B))       # fp64 arithmetic: inf, NaN as IEEE defines them
+    want = oracle.f64_to_f16_bits(ref.ravel()).reshape(M, N)
+    got = gu.c_bits(C)
+    want_nan = np.isnan(ref)
+    got_nan = np.isnan(gu.bits_to_f64(got))
+    assert np.array_equal(got_nan, want_nan), "NaN pattern differs"
+    assert want_nan[19].all() and want_nan[11, 17] and not want_nan[3].any()
+    ok = ~want_nan
+    assert np.array_equal(oracle.canonical_bits(got)[ok], oracle.canonical_bits(want)[ok])
+    assert np.isposinf(ref[3]).all() and np.isneginf(ref[7, :48]).all() and np.isposinf(ref[7, 48:]).all()
+    assert gu.bits_to_f64(got)[23, 5] == np.inf and gu.bits_to_f64(got)[23, 6] == -np.inf       # 7.68e6 does not fit fp16
+    # the same through the CTA-pair kernel and a split-K reduction (partial sums carry inf / NaN through fp32)
+    for cfg in (_cfg(F2, 96, 4, 1, 1, DIRECT), _cfg(F1, 96, 4, 2, 1, DIRECT, 64, CLUSTER), _cfg(F1, 96, 4, 2, 1, DIRECT, 64, WORKSPACE)):
+        C2, _, _ = gu.run_gemm(ctx, A, B, cfg, plan=plan)
+        g2 = gu.c_bits(C2)
+        assert np.array_equal(np.isnan(gu.bits_to_f64(g2)), want_nan), cfg.as_dict()
+        assert np.array_equal(oracle.canonical_bits(g2)[ok], oracle.canonical_bits(want)[ok]), cfg.as_dict()
+    plan.close()
