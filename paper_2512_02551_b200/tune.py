@@ -150,8 +150,7 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
         rng.shuffle(order)
         for t, e, c in order:
             plan.set_config(c)
-            n = max(5, int(250.0 / (t * 1e3 / 1e3) / 1e3))      # calls that fill about 0.25 s
-            n = max(5, min(2000, int(0.25 / (t * 1e-3))))
+            n = max(5, min(2000, int(0.25 / (t * 1e-3))))      # calls that fill about 0.25 s
             for _ in range(3):
                 run()
             sustained[key(c)] = batch_ms(run, n, stream)
