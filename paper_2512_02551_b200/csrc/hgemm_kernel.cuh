@@ -677,7 +677,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (p.epilogue_tma) {
                     const uint32_t buf = staging + (store_count & 1u) * (kStagingBytesPerWarp / 2);
                     // the buffer written two stores ago must have been read by its TMA store
-                    if (lane == 0) bulk_wait_group_read<1>();
+                    bulk_wait_group_read<1>();                      // lanes other than 0 own no groups
                     __syncwarp();
                     // row `lane` of the 32 x 32 box is 64 bytes; 64-byte swizzle: 16-byte chunk j of
                     // row r lives at chunk j ^ ((r >> 1) & 3)
@@ -691,9 +691,12 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) {
+                    {
+                        // warp-uniform code: the store is predicated inside its asm block, the commit is executed
+                        // by every lane (an empty group for all but lane 0)
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                        if (box_row < p.M && col0 < p.N && !(p.debug_skip & 4u)) tma_store_2d(&tmap_c, col0, box_row, buf);
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !(p.debug_skip & 4u);
+                        tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
                     ++store_count;
