@@ -92,8 +92,14 @@ enum {
 };
 
 enum {
-    HGEMM_EPILOGUE_DIRECT = 0, /* registers -> 16-byte global stores */
-    HGEMM_EPILOGUE_TMA = 1     /* registers -> swizzled shared memory -> TMA store */
+    HGEMM_EPILOGUE_DIRECT = 0,  /* registers -> 16-byte global stores */
+    HGEMM_EPILOGUE_TMA = 1,     /* registers -> swizzled shared memory -> TMA store, 32 x 32 boxes */
+    HGEMM_EPILOGUE_TMA_WIDE = 2 /* the same with 32-row x 64-column boxes: half as many fences, stores and
+                                   commits per tile, for 32 KB more shared memory (fewer stages fit).  Needs
+                                   split_k == 1 and block_n -- and the column pieces of HGEMM_TAIL_N -- a
+                                   multiple of 64; with tail_split cutting along K, or a C whose rows are not
+                                   multiples of 16 bytes, the cut tiles / the whole problem finish as with
+                                   HGEMM_EPILOGUE_TMA resp. with element stores */
 };
 
 /* One point of the per-shape configuration space (the paper's BM/BN/BK, stage

@@ -120,8 +120,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         lc.attrs = attr;
         lc.numAttrs = 1;
         int clusters = 0;
-        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2>, &lc)
-                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1>, &lc);
+        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false>, &lc)
+                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false>, &lc);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return HGEMM_ERR_UNSUPPORTED;
@@ -188,7 +188,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     }
     p.tmem_cols = pow2_at_least(2 * cfg.block_n);
     p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
-    p.epilogue_tma = (cfg.epilogue == HGEMM_EPILOGUE_TMA && cfg.split_k == 1 && !p.ragged_n) ? 1 : 0;   // whole tiles only
+    p.epilogue_tma = (cfg.epilogue != HGEMM_EPILOGUE_DIRECT && cfg.split_k == 1 && !p.ragged_n)             // whole tiles only
+                         ? (cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? 2 : 1) : 0;
     p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN, cfg.accumulate == HGEMM_ACC_F16);
     p.acc_f16 = cfg.accumulate == HGEMM_ACC_F16 ? 1 : 0;
     p.idesc_tail = make_idesc(128 * cg, cfg.block_n / int(std::max<int64_t>(1, layout.pieces)), pl->layout == HGEMM_LAYOUT_NN,
@@ -308,24 +309,15 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             st = cuda_fail(ctx, e);
             break;
         }
-        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 int(hgemm_host::kSmemOptInBytes));
-        if (e != cudaSuccess) {
-            st = cuda_fail(ctx, e);
-            break;
+        // the four instantiations: 1-CTA / CTA-pair, narrow / wide store boxes
+        const void *kernels[4] = {reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<1, false>),
+                                  reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<2, false>),
+                                  reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<1, true>),
+                                  reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<2, true>)};
+        for (int k = 0; k < 4 && e == cudaSuccess; ++k) {
+            e = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
-        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) {
-            st = cuda_fail(ctx, e);
-            break;
-        }
-        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) {
-            st = cuda_fail(ctx, e);
-            break;
-        }
-        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 int(hgemm_host::kSmemOptInBytes));
         if (e != cudaSuccess) {
             st = cuda_fail(ctx, e);
             break;
@@ -568,6 +560,9 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
             return HGEMM_ERR_CUDA;
         if (plan->params.ragged_n) {
             e.tmap_c = e.tmap_a;   // never used: a C with ragged rows is stored element by element
+        } else if (plan->params.epilogue_tma == 2) {
+            // wide epilogue: 32-row x 64-column store boxes (128-byte rows)
+            if (!encode_2d(ctx, &e.tmap_c, C, N, M, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
         } else if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
             return HGEMM_ERR_CUDA;
         }
@@ -605,10 +600,17 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     lc.attrs = attr;
     lc.numAttrs = ctx->dependent_launch ? 2 : 1;
     cudaError_t e;
-    if (cg == 1)
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
+    // the wide instantiation lays its store staging out differently, so it runs whenever the configuration asks for
+    // it, also when a C with ragged rows makes it fall back to element stores
+    const bool wide = plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE;
+    if (cg == 1 && !wide)
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1, false>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
+    else if (cg == 1)
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1, true>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
+    else if (!wide)
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2, false>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
     else
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
+        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2, true>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;
 }

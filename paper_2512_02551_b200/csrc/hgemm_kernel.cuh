@@ -45,6 +45,7 @@ constexpr int kATileBytes = kBlockM * kSubK * 2;             // 16 KB: one 128 x
 constexpr int kStoreBoxRows = 32, kStoreBoxCols = 32;        // TMA-store box: one warp's 32 x 32 chunk
 constexpr int kStagingBytesPerWarp = 2 * kStoreBoxRows * kStoreBoxCols * 2;  // two 2 KB buffers
 constexpr int kStagingBytes = 8 * kStagingBytesPerWarp;      // 32 KB
+constexpr int kWideBoxBytes = kStoreBoxRows * 64 * 2;        // wide TMA epilogue: 32 rows x 64 columns, two per warp (64 KB in all)
 constexpr int kCtrlBytes = 512;       // barriers, tensor-memory base, abort flag
 
 // Status-word roles
@@ -90,7 +91,7 @@ struct KernelParams {
     int32_t stages;
     int32_t raster_group;
     int32_t tmem_cols;            // power of two >= 2 * block_n
-    int32_t epilogue_tma;         // 1: TMA-store epilogue (only when split_k == 1)
+    int32_t epilogue_tma;         // 1: TMA-store epilogue, 32 x 32 boxes; 2: 32 x 64 boxes (only when split_k == 1)
     int32_t b_row_major;          // 1: B is the K x N row-major operand ("NN" layout): B tiles are N-major in shared memory
     int32_t ragged_n;             // 1: N % 8 != 0: rows of C are not 16-byte multiples, store element by element
     int32_t tma_3d;               // 1: the A and B maps are 3-D {64, rows, K / 64}: one load per operand per stage
@@ -351,7 +352,9 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // -------------------------------------------------------------------------------------
 // the kernel
 
-template <int CTA_GROUP>
+// WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
+// store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
+template <int CTA_GROUP, bool WIDE_STORE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -366,7 +369,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t a_stage_bytes = static_cast<uint32_t>(subs) * kATileBytes;
     const uint32_t stage_bytes = a_stage_bytes + static_cast<uint32_t>(subs) * b_sub_bytes;   // [A sub-tiles | B sub-tiles]
     const uint32_t staging_base = smem_base + static_cast<uint32_t>(p.stages) * stage_bytes;
-    const uint32_t ctrl_base = staging_base + kStagingBytes;
+    constexpr uint32_t staging_per_warp = WIDE_STORE ? 2u * kWideBoxBytes : static_cast<uint32_t>(kStagingBytesPerWarp);
+    const uint32_t ctrl_base = staging_base + 8u * staging_per_warp;
     uint8_t *ctrl_gen = smem_gen + (ctrl_base - smem_base);
 
     // control block: full[12] | empty[12] | tmem_full[2] | tmem_empty[2] | tmem base | abort | recv
@@ -651,7 +655,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const uint32_t q = warp & 3u;                               // tensor-memory lane quarter of this warp
         const uint32_t first_chunk = ew >> 2;                       // chunks first_chunk, first_chunk + 2, ...
         const uint32_t row_in_tile = q * 32u + lane;                // accumulator row = tensor-memory lane
-        const uint32_t staging = staging_base + ew * kStagingBytesPerWarp;
+        const uint32_t staging = staging_base + ew * staging_per_warp;
         const uint32_t tmem_empty_leader = (CTA_GROUP == 2) ? mapa(bar_tmem_empty, leader_rank) : bar_tmem_empty;
         const int32_t chunks = p.block_n / 32;
         uint32_t local_tile = 0;
@@ -674,7 +678,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // One 32-column chunk of this thread's row, converted and sent to C.
             auto emit_chunk = [&](const uint32_t (&v)[32], int32_t c) {
                 const int32_t col0 = it.n0 + c * 32;
-                if (p.epilogue_tma) {
+                if (!WIDE_STORE && p.epilogue_tma) {
                     const uint32_t buf = staging + (store_count & 1u) * (kStagingBytesPerWarp / 2);
                     // the buffer written two stores ago must have been read by its TMA store
                     bulk_wait_group_read<1>();                      // lanes other than 0 own no groups
@@ -753,7 +757,58 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
             const int32_t live_chunks = min(it.bn / 32, (p.N - it.n0 + 31) / 32);
             const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
-            if (it.slices == 1) {
+            if (WIDE_STORE && it.slices == 1 && p.epilogue_tma == 2) {
+                // Wide TMA stores: two 32-column chunks are staged side by side as one 32-row x 64-column box
+                // (128-byte rows, 128-byte swizzle: 16-byte chunk j of row r lives at chunk j ^ (r & 7)) and leave
+                // with one fence, one store and one commit.  The two warps of a lane quarter take alternate boxes.
+                // A box whose second half lies beyond N is staged half empty: the store is clipped there.
+                uint32_t v[32];
+                const int32_t chunks = live_rows ? live_chunks : 0;     // shadows the tile's chunk count
+                const int32_t boxes = (chunks + 1) >> 1;
+                for (int32_t b = static_cast<int32_t>(first_chunk); b < boxes; b += 2) {
+                    const uint32_t buf = staging + (store_count & 1u) * kWideBoxBytes;
+                    bulk_wait_group_read<1>();                      // the box written two stores ago has been read
+                    __syncwarp();
+                    const uint32_t row_addr = buf + lane * 128u;
+                    const uint32_t sw = lane & 7u;
+#pragma unroll
+                    for (int32_t half = 0; half < 2; ++half) {
+                        const int32_t c = 2 * b + half;
+                        if (c < chunks) {
+                            tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
+                            tmem_ld_wait();
+                            if (p.acc_f16) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
+                            }
+                            if (b + 2 >= boxes && c + 1 >= min(chunks, 2 * b + 2)) release_accumulator();   // this warp's last load
+                            if (p.scaled && grow < p.M) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    if (it.n0 + c * 32 + 8 * j < p.N) scale_group8(v + 8 * j, p, grow, it.n0 + c * 32 + 8 * j);
+                            }
+#pragma unroll
+                            for (uint32_t j = 0; j < 4; ++j) {
+                                st_shared_v4(row_addr + (((4u * static_cast<uint32_t>(half) + j) ^ sw) << 4),
+                                             pack_half2_rn(v[8 * j + 0], v[8 * j + 1]), pack_half2_rn(v[8 * j + 2], v[8 * j + 3]),
+                                             pack_half2_rn(v[8 * j + 4], v[8 * j + 5]), pack_half2_rn(v[8 * j + 6], v[8 * j + 7]));
+                            }
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    {
+                        const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
+                        const int32_t col0 = it.n0 + b * 64;
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !(p.debug_skip & 4u);
+                        tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
+                        bulk_commit_group();
+                    }
+                    ++store_count;
+                }
+                if (static_cast<int32_t>(first_chunk) >= boxes) release_accumulator();    // nothing to load
+            } else if (it.slices == 1) {
                 // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second
                 // chunk in flight costs more in registers than it hides
                 uint32_t v[32];

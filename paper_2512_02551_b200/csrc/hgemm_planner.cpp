@@ -22,9 +22,15 @@ int64_t stage_bytes(const hgemm_config_t &c)
     return subs * (kATileBytes + int64_t(c.block_n / cta_group_of(c)) * 64 * 2);
 }
 
+// Store staging of the eight epilogue warps: two 2 KB boxes each, or two 4 KB ones for the wide TMA epilogue.
+int64_t staging_bytes(const hgemm_config_t &c)
+{
+    return c.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? 2 * kStagingBytes : kStagingBytes;
+}
+
 int64_t smem_bytes(const hgemm_config_t &c)
 {
-    return kAlignSlack + int64_t(c.stages) * stage_bytes(c) + kStagingBytes + kCtrlBytes;
+    return kAlignSlack + int64_t(c.stages) * stage_bytes(c) + staging_bytes(c) + kCtrlBytes;
 }
 
 int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k)
@@ -35,6 +41,12 @@ int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k)
     c.block_n = block_n;
     c.block_k = block_k;
     const int64_t room = kSmemOptInBytes - kAlignSlack - kStagingBytes - kCtrlBytes;
+    return int32_t(std::min<int64_t>(12, room / stage_bytes(c)));
+}
+
+int32_t max_stages_of(const hgemm_config_t &c)
+{
+    const int64_t room = kSmemOptInBytes - kAlignSlack - staging_bytes(c) - kCtrlBytes;
     return int32_t(std::min<int64_t>(12, room / stage_bytes(c)));
 }
 
@@ -111,7 +123,13 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     // the slices of one tile wait for each other, so they must all be resident at once
     if (c.split_k > kMaxSplitK) return HGEMM_ERR_UNSUPPORTED;
     if (c.raster_group < 1) return HGEMM_ERR_UNSUPPORTED;
-    if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA) return HGEMM_ERR_UNSUPPORTED;
+    if (c.epilogue != HGEMM_EPILOGUE_DIRECT && c.epilogue != HGEMM_EPILOGUE_TMA && c.epilogue != HGEMM_EPILOGUE_TMA_WIDE)
+        return HGEMM_ERR_UNSUPPORTED;
+    if (c.epilogue == HGEMM_EPILOGUE_TMA_WIDE) {
+        // 64-column store boxes: whole boxes per tile and per column piece, and no partial sums to exchange
+        if (c.split_k != 1 || (c.block_n % 64) != 0) return HGEMM_ERR_UNSUPPORTED;
+        if (c.tail_split >= 2 && c.tail_mode == HGEMM_TAIL_N && (c.block_n % (64 * c.tail_split)) != 0) return HGEMM_ERR_UNSUPPORTED;
+    }
     for (int i = 0; i < 4; ++i)
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
     if (c.accumulate != HGEMM_ACC_F32 && c.accumulate != HGEMM_ACC_F16) return HGEMM_ERR_UNSUPPORTED;
@@ -157,6 +175,7 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     const double kLatencyWarm = 1942.8, kLatencyCold = 3130.1;   // what the stage ring has to hide: operands in L2 / in HBM
     const double kPairExtra = 496.8;          // set-up and teardown of a CTA pair
     const double kDirectStores = 1.65;         // drain with direct stores relative to TMA stores
+    const double kWideStores = 0.8;            // ... with 64-column boxes (measured on the chunk loop, not fitted)
 
     const int cg = cta_group_of(c);
     const int64_t units = std::max(1, num_sms / cg);
@@ -180,7 +199,8 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     const bool cold = 2.0 * (double(M) * K + double(N) * K) > 100e6;          // the operands do not stay in L2
     const double latency_kb = (cold ? kLatencyCold : kLatencyWarm) / double(c.stages);
     const double t_kb = std::max(std::max(mma_kb, fill_kb), std::max(l2_kb, latency_kb));
-    const double epilogue = (12.73 * c.block_n + 75.0) * (c.epilogue == HGEMM_EPILOGUE_DIRECT ? kDirectStores : 1.0);
+    const double epilogue = (12.73 * c.block_n + 75.0) *
+                            (c.epilogue == HGEMM_EPILOGUE_DIRECT ? kDirectStores : c.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? kWideStores : 1.0);
     double t = wave_count * (double(kb_per) * t_kb + 0.25 * kFillLatency) + 0.75 * kFillLatency + epilogue + (cg - 1) * kPairExtra;
     const double partial = 128.0 * c.block_n * 4.0;
     if (c.split_k == 1 && L.slices > 1) t += partial / 26.4 + 10069.4;   // the tail's reduction
@@ -305,7 +325,7 @@ hgemm_status_t plan_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hge
         c.raster_group = raster_group_for(M, num_sms, c);
         c.tail_split = 0;
         c.tail_mode = HGEMM_TAIL_K;
-        c.stages = std::min(c.stages, max_stages(c.family, c.block_n, c.block_k));
+        c.stages = std::min(c.stages, max_stages_of(c));
         if (c.stages < 1) continue;
         const int cg = cta_group_of(c);
         const int64_t kb_here = ceil_div(K, c.block_k), kb_there = ceil_div(nb[i].K, c.block_k);

@@ -21,7 +21,9 @@ inline int cta_group_of(const hgemm_config_t &c) { return c.family == HGEMM_FAMI
 
 int64_t stage_bytes(const hgemm_config_t &c);
 int64_t smem_bytes(const hgemm_config_t &c);
-int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k);
+int64_t staging_bytes(const hgemm_config_t &c);   // store staging of the epilogue warps (32 KB, 64 KB for the wide epilogue)
+int32_t max_stages(int32_t family, int32_t block_n, int32_t block_k);   // with 32 KB of store staging
+int32_t max_stages_of(const hgemm_config_t &c);                         // with this configuration's staging
 // Which tiles are split: tiles [0, first_split_tile) are whole work items, the rest are cut into `slices`
 // K slices.  Uniform split-K: first = 0; tail split: first = tiles - (tiles mod units) when it applies.
 struct SplitLayout {

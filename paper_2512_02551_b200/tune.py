@@ -13,6 +13,7 @@ Listing 8): warm-up, then timed rounds in shuffled order, median per candidate.
 from __future__ import annotations
 
 import argparse
+import functools
 import json
 import os
 import random
@@ -27,10 +28,11 @@ SPLITS = [1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64]
 NUM_SMS = 148
 
 
-def max_stages(family: int, bn: int, bk: int) -> int:
+@functools.lru_cache(maxsize=None)
+def max_stages(family: int, bn: int, bk: int, epilogue: int = hgemm.EPILOGUE_TMA) -> int:
     best = 0
     for st in range(1, 13):
-        c = hgemm.Config.make(family=family, block_n=bn, stages=st, block_k=bk)
+        c = hgemm.Config.make(family=family, block_n=bn, stages=st, block_k=bk, epilogue=epilogue)
         if hgemm.config_smem_bytes(c) <= 232448:
             best = st
     return best
@@ -59,7 +61,13 @@ def candidates(M: int, N: int, K: int):
                     rg = max(1, min(-(-M // (128 * cg)), round((units * bn / (128.0 * cg)) ** 0.5)))
                     modes = (0,) if split == 1 else ((0, 1) if split * cg <= 16 else (0,))
                     for mode in modes:
-                        for epi in ((hgemm.EPILOGUE_TMA, hgemm.EPILOGUE_DIRECT) if split == 1 else (hgemm.EPILOGUE_DIRECT,)):
+                        epis = (hgemm.EPILOGUE_DIRECT,)
+                        if split == 1:
+                            epis = (hgemm.EPILOGUE_TMA, hgemm.EPILOGUE_DIRECT) + ((hgemm.EPILOGUE_TMA_WIDE,) if bn % 64 == 0 else ())
+                        for epi in epis:
+                            st = min(max_stages(family, bn, bk, epi), 8)      # the wide epilogue's staging leaves fewer stages
+                            if st < 1:
+                                continue
                             c = hgemm.Config.make(family=family, block_n=bn, stages=st, split_k=split, raster_group=rg,
                                                   epilogue=epi, block_k=bk, split_mode=mode)
                             if hgemm.validate_config(M, N, K, c) == hgemm.OK:
@@ -107,9 +115,12 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     default = plan.config
     cands = candidates(M, N, K)
     cands.sort(key=lambda c: hgemm.estimate_config(M, N, K, c))
+    # the wide-store candidates are ranked on their own (8 of them), so that they take no place among the `top`
+    wide = [c for c in cands if c.epilogue == hgemm.EPILOGUE_TMA_WIDE][:8]
+    cands = [c for c in cands if c.epilogue != hgemm.EPILOGUE_TMA_WIDE]
     chosen, seen = [], set()
     extra = rng.sample(cands[top:], min(explore, max(0, len(cands) - top))) if explore > 0 else []   # for refitting the cost model
-    for c in [default] + cands[:top] + extra:
+    for c in [default] + cands[:top] + wide + extra:
         if key(c) not in seen:
             seen.add(key(c))
             chosen.append(c)

@@ -15,6 +15,7 @@ from paper_2512_02551_b200 import hgemm, inputs  # noqa: E402
 
 F1, F2 = hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA
 DIRECT, TMA = hgemm.EPILOGUE_DIRECT, hgemm.EPILOGUE_TMA
+WIDE = hgemm.EPILOGUE_TMA_WIDE
 
 
 @pytest.fixture(scope="module")
@@ -267,6 +268,58 @@ def test_tail_split_along_n(ctx, gu, family, bn, bk, stages, pieces, M, N, K):
             Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
             gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"tail pieces, integers {cfg.as_dict()}")
         plan.close()
+
+
+# ---- wide TMA-store epilogue: 32-row x 64-column boxes --------------------------------------------------------
+
+WIDE_CASES = [
+    # family, bn, bk, stages, tail_split, tail_mode, M, N, K
+    (F1, 64, 64, 4, 0, 0, 128, 64, 64),                 # one box per warp pair
+    (F1, 128, 64, 4, 0, 0, 100, 136, 72),               # ragged M, N and K; the last box of a row is clipped inside its first half
+    (F1, 256, 64, 3, 0, 0, 130, 264, 200),              # one row / one column group past a tile edge
+    (F2, 256, 128, 2, 0, 0, 520, 552, 1024),            # CTA pairs, 128-wide stages; N leaves a 40-column edge (second half box empty)
+    (F1, 192, 128, 1, 0, 0, 384, 416, 192),             # three boxes per tile: the warps of a quarter get two and one
+    (F2, 64, 64, 8, 0, 0, 1024, 2048, 128),             # several tiles per CTA: accumulators and store buffers alternate
+    (F1, 256, 64, 3, 0, 0, 4096, 4096, 64),             # epilogue-bound: one k-block per tile
+    (F2, 256, 64, 5, 2, 0, 4096, 4096, 512),            # last wave cut along K: whole tiles leave through wide boxes, cut ones through the workspace
+    (F2, 256, 64, 5, 2, 1, 2100, 3000, 300),            # last wave cut into two 128-column pieces
+    (F1, 256, 64, 3, 4, 1, 4096, 1280, 384),            # ... into four 64-column pieces
+    (F1, 128, 64, 4, 0, 0, 77, 204, 333),               # N % 8 != 0: falls back to element stores
+]
+
+
+@pytest.mark.parametrize("case", WIDE_CASES, ids=lambda c: f"f{c[0]}bn{c[1]}bk{c[2]}s{c[3]}t{c[4]}m{c[5]}-{c[6]}x{c[7]}x{c[8]}")
+def test_wide_store_epilogue(ctx, gu, case):
+    import oracle
+    family, bn, bk, stages, tail, tmode, M, N, K = case
+    wide = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=WIDE, block_k=bk,
+                             tail_split=tail, tail_mode=tmode)
+    narrow = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=TMA, block_k=bk,
+                               tail_split=tail, tail_mode=tmode)
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, wide)
+    gu.assert_close_full(C, A, B, f"wide {wide.as_dict()}") if M * N * K <= gu.FULL_CHECK_VOLUME else \
+        gu.assert_close_sampled(C, A, B, "uniform", inputs.shape_seed(M, N, K), f"wide {wide.as_dict()}")
+    # the box width changes nothing in the arithmetic: the same bits as through 32-column boxes
+    C_narrow, _, _ = gu.run_gemm(ctx, A, B, narrow, plan=plan)
+    assert torch.equal(C.view(torch.int16), C_narrow.view(torch.int16))
+    if M * N * K <= gu.FULL_CHECK_VOLUME:
+        Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+        plan.set_config(wide)
+        Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+        gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"wide, integers {wide.as_dict()}")
+    plan.close()
+
+
+def test_wide_store_epilogue_limits(ctx):
+    ok = hgemm.Config.make(family=F1, block_n=128, stages=2, epilogue=WIDE, block_k=64)
+    assert hgemm.validate_config(512, 512, 512, ok) == hgemm.OK
+    for bad in (dict(block_n=96), dict(split_k=2), dict(block_n=128, tail_split=4, tail_mode=hgemm.TAIL_N), dict(block_n=256, stages=4)):
+        kw = dict(family=F1, block_n=128, stages=2, epilogue=WIDE, block_k=64)
+        kw.update(bad)
+        assert hgemm.validate_config(512, 512, 512, hgemm.Config.make(**kw)) == hgemm.ERR_UNSUPPORTED, bad
+    # 32 KB more staging: one stage fewer fits than with 32-column boxes
+    assert hgemm.validate_config(512, 512, 512, hgemm.Config.make(family=F1, block_n=256, stages=4, epilogue=TMA, block_k=64)) == hgemm.OK
 
 
 # ---- the NN layout: B given as the K x N operand, row-major ----------------------------------------------

@@ -65,7 +65,7 @@ def test_validate_rejects_illegal_configs(lib):
     assert hgemm.validate_config(M, N, K, ok) == hgemm.OK
     for kw in [dict(block_n=48), dict(block_n=288), dict(block_n=0), dict(stages=0), dict(stages=13),
                dict(block_n=256, stages=5), dict(split_k=0), dict(split_k=17), dict(block_k=32), dict(block_k=256), dict(raster_group=0),
-               dict(epilogue=2), dict(family=2)]:
+               dict(epilogue=3), dict(family=2)]:
         c = hgemm.Config.make(**{**dict(block_n=128, stages=4), **kw})
         assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED, kw
     c = hgemm.Config.make(block_n=128, stages=4)
@@ -80,6 +80,16 @@ def test_validate_rejects_illegal_configs(lib):
     for kw in [dict(family=1, split_k=12), dict(split_k=32), dict(block_n=256, stages=2, split_k=4)]:
         c = hgemm.Config.make(**{**dict(block_n=128, stages=4, split_mode=1), **kw})
         assert hgemm.validate_config(M, N, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
+    # wide TMA-store epilogue: 64-column boxes need block_n (and column pieces) in multiples of 64, no split along K,
+    # and 32 KB more store staging
+    wide = hgemm.Config.make(block_n=128, stages=4, epilogue=hgemm.EPILOGUE_TMA_WIDE)
+    assert hgemm.validate_config(M, N, K, wide) == hgemm.OK
+    assert hgemm.config_smem_bytes(wide) == hgemm.config_smem_bytes(ok) + 32768
+    for kw in [dict(block_n=96), dict(block_n=160), dict(split_k=2), dict(block_n=256, stages=4), dict(tail_split=4, tail_mode=hgemm.TAIL_N)]:
+        c = hgemm.Config.make(**{**dict(block_n=128, stages=4, epilogue=hgemm.EPILOGUE_TMA_WIDE), **kw})
+        assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED, kw
+    assert hgemm.validate_config(M, N, K, hgemm.Config.make(block_n=256, stages=3, epilogue=hgemm.EPILOGUE_TMA_WIDE,
+                                                            tail_split=4, tail_mode=hgemm.TAIL_N)) == hgemm.OK
     pair = hgemm.Config.make(family=hgemm.FAMILY_UMMA_2CTA, block_n=256, stages=6)
     assert hgemm.validate_config(M, N, K, pair) == hgemm.OK
     assert hgemm.config_smem_bytes(pair) == 1024 + 6 * (16384 + 128 * 128) + 32768 + 512
