@@ -120,8 +120,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         lc.attrs = attr;
         lc.numAttrs = 1;
         int clusters = 0;
-        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false>, &lc)
-                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false>, &lc);
+        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, true>, &lc)
+                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, true>, &lc);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return HGEMM_ERR_UNSUPPORTED;
@@ -211,6 +211,22 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     pl->smem = int(hgemm_host::kSmemOptInBytes);
     pl->maps_used = pl->maps_next = 0;   // the B box depends on the configuration
     return HGEMM_OK;
+}
+
+// The kernel instantiation for a CTA group size, store-box width and presence of K slices.
+const void *kernel_for(int cg, bool wide, bool split)
+{
+    using namespace hgemm_dev;
+    if (cg == 1) {
+        if (!wide) return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<1, false, true>)
+                                : reinterpret_cast<const void *>(hgemm_umma_kernel<1, false, false>);
+        return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<1, true, true>)
+                     : reinterpret_cast<const void *>(hgemm_umma_kernel<1, true, false>);
+    }
+    if (!wide) return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, true>)
+                            : reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, false>);
+    return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<2, true, true>)
+                 : reinterpret_cast<const void *>(hgemm_umma_kernel<2, true, false>);
 }
 
 bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_inner,
@@ -309,14 +325,11 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             st = cuda_fail(ctx, e);
             break;
         }
-        // the four instantiations: 1-CTA / CTA-pair, narrow / wide store boxes
-        const void *kernels[4] = {reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<1, false>),
-                                  reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<2, false>),
-                                  reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<1, true>),
-                                  reinterpret_cast<const void *>(hgemm_dev::hgemm_umma_kernel<2, true>)};
-        for (int k = 0; k < 4 && e == cudaSuccess; ++k) {
-            e = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, without / with K slices
+        for (int k = 0; k < 8 && e == cudaSuccess; ++k) {
+            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k & 4) != 0);
+            e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
         if (e != cudaSuccess) {
             st = cuda_fail(ctx, e);
@@ -600,17 +613,12 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     lc.attrs = attr;
     lc.numAttrs = ctx->dependent_launch ? 2 : 1;
     cudaError_t e;
-    // the wide instantiation lays its store staging out differently, so it runs whenever the configuration asks for
-    // it, also when a C with ragged rows makes it fall back to element stores
-    const bool wide = plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE;
-    if (cg == 1 && !wide)
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1, false>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
-    else if (cg == 1)
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1, true>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
-    else if (!wide)
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2, false>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
-    else
-        e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<2, true>, me->tmap_a, me->tmap_b, me->tmap_c, me->tmap_bt, plan->params);
+    // The wide instantiation lays its store staging out differently, so it runs whenever the configuration asks for
+    // it, also when a C with ragged rows makes it fall back to element stores; the instantiation without the
+    // split-K reductions runs whenever no work item is a K slice.
+    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, plan->params.split_k > 1);
+    void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
+    e = cudaLaunchKernelExC(&lc, fn, args);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;
 }

@@ -281,6 +281,8 @@ struct WorkItem {
     int32_t bn;         // columns of this work item: block_n, or block_n / tail_pieces for a piece of a tail tile
 };
 
+// SPLIT = false: the caller knows that no work item is a K slice (split_k == 1 and no tail cut along K).
+template <bool SPLIT = true>
 __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p, int32_t block_m_total)
 {
     WorkItem it;
@@ -303,6 +305,11 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
         it.split_index = 0;
         it.bn = p.block_n / p.tail_pieces;
         n_off = (idx - t * p.tail_pieces) * it.bn;
+    } else if (!SPLIT) {
+        it.tile = w;                     // not reached: without K slices every item is a whole tile or a column piece
+        it.slice = 0;
+        it.slices = 1;
+        it.split_index = 0;
     } else {
         it.split_index = w - p.first_split_tile;
         const int32_t t = fast_div(it.split_index, p.fd_split);
@@ -320,7 +327,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     const int32_t tm = first_m + (r - tn * gsize);
     it.m0 = tm * block_m_total;
     it.n0 = tn * p.block_n + n_off;
-    if (it.slices == 1) {
+    if (!SPLIT || it.slices == 1) {
         it.kb_begin = 0;
         it.kb_count = p.kblocks;
     } else {
@@ -352,9 +359,11 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // -------------------------------------------------------------------------------------
 // the kernel
 
+// SPLIT = false: the instantiation for configurations without K slices (split_k == 1, no tail cut along K): the
+// workspace and cluster reductions are compiled out, which shortens the start-up of every such call.
 // WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
 // store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
-template <int CTA_GROUP, bool WIDE_STORE = false>
+template <int CTA_GROUP, bool WIDE_STORE = false, bool SPLIT = true>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -455,7 +464,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         bool ok = true;
         bool dependencies_met = false;
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
-            const WorkItem it = warp_uniform(decode_work(w, p, kBlockMTotal));
+            const WorkItem it = warp_uniform(decode_work<SPLIT>(w, p, kBlockMTotal));
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
             // this CTA's rows of B: its share of the work item's columns
             const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
@@ -574,7 +583,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const bool issue_mma = !(p.debug_skip & 2u);
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-                const WorkItem it = warp_uniform(decode_work(w, p, kBlockMTotal));
+                const WorkItem it = warp_uniform(decode_work<SPLIT>(w, p, kBlockMTotal));
                 const uint32_t acc = local_tile & 1u;
                 const uint32_t acc_ph = (local_tile >> 1) & 1u;
                 const long long ca = tr ? clock64() : 0;
@@ -630,7 +639,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // use has been released -- instead of after the CTA-wide barrier of the teardown: the epilogue's
                 // final stores then overlap the deallocation.  (Not for cluster split-K, which reads tensor
                 // memory after the role loops, and not after an abort.)
-                if (ok && !p.cluster_split) {
+                if (ok && !(SPLIT && p.cluster_split)) {
                     for (uint32_t a = 0; ok && a < 2u; ++a) {
                         const uint32_t uses = (local_tile + 1u - a) / 2u;      // work items that used accumulator a (local_tile items in all)
                         if (local_tile > a && uses > 0u) {
@@ -663,7 +672,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         bool ok = true;
         grid_dependency_wait();                            // before the first store to C, workspace or counters
         for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-            const WorkItem it = decode_work(w, p, kBlockMTotal);
+            const WorkItem it = decode_work<SPLIT>(w, p, kBlockMTotal);
             const uint32_t acc = local_tile & 1u;
             const uint32_t acc_ph = (local_tile >> 1) & 1u;
             ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
@@ -757,7 +766,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
             const int32_t live_chunks = min(it.bn / 32, (p.N - it.n0 + 31) / 32);
             const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
-            if (WIDE_STORE && it.slices == 1 && p.epilogue_tma == 2) {
+            if (WIDE_STORE && (!SPLIT || it.slices == 1) && p.epilogue_tma == 2) {
                 // Wide TMA stores: two 32-column chunks are staged side by side as one 32-row x 64-column box
                 // (128-byte rows, 128-byte swizzle: 16-byte chunk j of row r lives at chunk j ^ (r & 7)) and leave
                 // with one fence, one store and one commit.  The two warps of a lane quarter take alternate boxes.
@@ -808,7 +817,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     ++store_count;
                 }
                 if (static_cast<int32_t>(first_chunk) >= boxes) release_accumulator();    // nothing to load
-            } else if (it.slices == 1) {
+            } else if (!SPLIT || it.slices == 1) {
                 // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second
                 // chunk in flight costs more in registers than it hides
                 uint32_t v[32];
@@ -832,7 +841,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     emit_chunk(v, c);
                 }
                 if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load
-            } else if (p.cluster_split) {
+            } else if (SPLIT && p.cluster_split) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches
                 cs_m0 = row0;
@@ -977,7 +986,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // bytes on the owner's receive barrier; every owner adds, per unit, its own copy and the S - 1
     // received ones in slice order and stores fp16.  Layout: [own tile | S - 1 receive slots of cap units].
     // Both cluster barriers are taken by every thread of every CTA of the cluster, also after an abort.
-    {
+    if constexpr (SPLIT) {
         if (p.cluster_split) {
             // (warps 0 and 1 only take part in the barriers; what they compute here from zeros is unused)
             const uint32_t S = static_cast<uint32_t>(p.split_k), me = static_cast<uint32_t>(cs_slice);
