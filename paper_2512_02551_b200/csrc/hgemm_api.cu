@@ -120,8 +120,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         lc.attrs = attr;
         lc.numAttrs = 1;
         int clusters = 0;
-        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, true>, &lc)
-                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, true>, &lc);
+        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, 2>, &lc)
+                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, 2>, &lc);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return HGEMM_ERR_UNSUPPORTED;
@@ -213,20 +213,19 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     return HGEMM_OK;
 }
 
-// The kernel instantiation for a CTA group size, store-box width and presence of K slices.
-const void *kernel_for(int cg, bool wide, bool split)
+// The kernel instantiation for a CTA group size, store-box width and kind of split-K reduction
+// (0: no K slices, 1: through the workspace -- also a tail cut along K --, 2: inside a cluster).
+const void *kernel_for(int cg, bool wide, int split)
 {
     using namespace hgemm_dev;
+#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S>)
     if (cg == 1) {
-        if (!wide) return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<1, false, true>)
-                                : reinterpret_cast<const void *>(hgemm_umma_kernel<1, false, false>);
-        return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<1, true, true>)
-                     : reinterpret_cast<const void *>(hgemm_umma_kernel<1, true, false>);
+        if (wide) return split == 0 ? HGEMM_K(1, true, 0) : HGEMM_K(1, true, 1);      // no split_k > 1 with wide boxes
+        return split == 0 ? HGEMM_K(1, false, 0) : split == 1 ? HGEMM_K(1, false, 1) : HGEMM_K(1, false, 2);
     }
-    if (!wide) return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, true>)
-                            : reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, false>);
-    return split ? reinterpret_cast<const void *>(hgemm_umma_kernel<2, true, true>)
-                 : reinterpret_cast<const void *>(hgemm_umma_kernel<2, true, false>);
+    if (wide) return split == 0 ? HGEMM_K(2, true, 0) : HGEMM_K(2, true, 1);
+    return split == 0 ? HGEMM_K(2, false, 0) : split == 1 ? HGEMM_K(2, false, 1) : HGEMM_K(2, false, 2);
+#undef HGEMM_K
 }
 
 bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_inner,
@@ -325,9 +324,9 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             st = cuda_fail(ctx, e);
             break;
         }
-        // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, without / with K slices
-        for (int k = 0; k < 8 && e == cudaSuccess; ++k) {
-            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k & 4) != 0);
+        // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, no K slices / workspace / cluster reduction
+        for (int k = 0; k < 12 && e == cudaSuccess; ++k) {
+            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, k >> 2);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
@@ -616,7 +615,8 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     // The wide instantiation lays its store staging out differently, so it runs whenever the configuration asks for
     // it, also when a C with ragged rows makes it fall back to element stores; the instantiation without the
     // split-K reductions runs whenever no work item is a K slice.
-    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, plan->params.split_k > 1);
+    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE,
+                                plan->params.split_k > 1 ? (plan->params.cluster_split ? 2 : 1) : 0);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
     e = cudaLaunchKernelExC(&lc, fn, args);
     if (e != cudaSuccess) return cuda_fail(ctx, e);

@@ -359,11 +359,12 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // -------------------------------------------------------------------------------------
 // the kernel
 
-// SPLIT = false: the instantiation for configurations without K slices (split_k == 1, no tail cut along K): the
-// workspace and cluster reductions are compiled out, which shortens the start-up of every such call.
+// SPLIT: 0 for configurations without K slices (split_k == 1, no tail cut along K), 1 for slices summed through the
+// global workspace, 2 for slices summed inside a cluster; each instantiation carries only its own reduction, which
+// saves registers and shortens the start-up of every call.
 // WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
 // store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
-template <int CTA_GROUP, bool WIDE_STORE = false, bool SPLIT = true>
+template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -464,7 +465,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         bool ok = true;
         bool dependencies_met = false;
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
-            const WorkItem it = warp_uniform(decode_work<SPLIT>(w, p, kBlockMTotal));
+            const WorkItem it = warp_uniform(decode_work<SPLIT != 0>(w, p, kBlockMTotal));
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
             // this CTA's rows of B: its share of the work item's columns
             const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
@@ -583,7 +584,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const bool issue_mma = !(p.debug_skip & 2u);
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-                const WorkItem it = warp_uniform(decode_work<SPLIT>(w, p, kBlockMTotal));
+                const WorkItem it = warp_uniform(decode_work<SPLIT != 0>(w, p, kBlockMTotal));
                 const uint32_t acc = local_tile & 1u;
                 const uint32_t acc_ph = (local_tile >> 1) & 1u;
                 const long long ca = tr ? clock64() : 0;
@@ -639,7 +640,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // use has been released -- instead of after the CTA-wide barrier of the teardown: the epilogue's
                 // final stores then overlap the deallocation.  (Not for cluster split-K, which reads tensor
                 // memory after the role loops, and not after an abort.)
-                if (ok && !(SPLIT && p.cluster_split)) {
+                if (ok && SPLIT != 2) {
                     for (uint32_t a = 0; ok && a < 2u; ++a) {
                         const uint32_t uses = (local_tile + 1u - a) / 2u;      // work items that used accumulator a (local_tile items in all)
                         if (local_tile > a && uses > 0u) {
@@ -672,7 +673,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         bool ok = true;
         grid_dependency_wait();                            // before the first store to C, workspace or counters
         for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-            const WorkItem it = decode_work<SPLIT>(w, p, kBlockMTotal);
+            const WorkItem it = decode_work<SPLIT != 0>(w, p, kBlockMTotal);
             const uint32_t acc = local_tile & 1u;
             const uint32_t acc_ph = (local_tile >> 1) & 1u;
             ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
@@ -766,7 +767,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
             const int32_t live_chunks = min(it.bn / 32, (p.N - it.n0 + 31) / 32);
             const bool live_rows = row0 + static_cast<int32_t>(q) * 32 < p.M;
-            if (WIDE_STORE && (!SPLIT || it.slices == 1) && p.epilogue_tma == 2) {
+            if (WIDE_STORE && (SPLIT == 0 || it.slices == 1) && p.epilogue_tma == 2) {
                 // Wide TMA stores: two 32-column chunks are staged side by side as one 32-row x 64-column box
                 // (128-byte rows, 128-byte swizzle: 16-byte chunk j of row r lives at chunk j ^ (r & 7)) and leave
                 // with one fence, one store and one commit.  The two warps of a lane quarter take alternate boxes.
@@ -817,7 +818,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     ++store_count;
                 }
                 if (static_cast<int32_t>(first_chunk) >= boxes) release_accumulator();    // nothing to load
-            } else if (!SPLIT || it.slices == 1) {
+            } else if (SPLIT == 0 || it.slices == 1) {
                 // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second
                 // chunk in flight costs more in registers than it hides
                 uint32_t v[32];
@@ -841,7 +842,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     emit_chunk(v, c);
                 }
                 if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load
-            } else if (SPLIT && p.cluster_split) {
+            } else if (SPLIT == 2) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches
                 cs_m0 = row0;
@@ -986,7 +987,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // bytes on the owner's receive barrier; every owner adds, per unit, its own copy and the S - 1
     // received ones in slice order and stores fp16.  Layout: [own tile | S - 1 receive slots of cap units].
     // Both cluster barriers are taken by every thread of every CTA of the cluster, also after an abort.
-    if constexpr (SPLIT) {
+    if constexpr (SPLIT == 2) {
         if (p.cluster_split) {
             // (warps 0 and 1 only take part in the barriers; what they compute here from zeros is unused)
             const uint32_t S = static_cast<uint32_t>(p.split_k), me = static_cast<uint32_t>(cs_slice);
