@@ -207,7 +207,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     pl->grid = cluster_split ? cg * p.total_work : cg * std::min(p.total_work, units);
     pl->cluster_dim = cluster_split ? cg * cfg.split_k : cg;
     // Always ask for the whole opt-in shared memory: it keeps a second CTA off the SM, so two
-    // CTAs can never wait on each other's tensor-memory allocation.
+    // CTAs can never wait on each other's tensor-memory allocation.  (Letting small configurations ask for what
+    // they use, so that the next call's CTAs become resident beside this call's, made those calls slower.)
     pl->smem = int(hgemm_host::kSmemOptInBytes);
     pl->maps_used = pl->maps_next = 0;   // the B box depends on the configuration
     return HGEMM_OK;
@@ -634,9 +635,7 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
         if (e == cudaSuccess) e = cudaMalloc(&plan->stage_b, b_bytes);
         if (e == cudaSuccess) e = cudaMalloc(&plan->stage_c, c_bytes);
         if (e != cudaSuccess) {
-            if (plan->pad_a) cudaFree(plan->pad_a);
-    if (plan->pad_b) cudaFree(plan->pad_b);
-    if (plan->stage_a) cudaFree(plan->stage_a);
+            if (plan->stage_a) cudaFree(plan->stage_a);
             if (plan->stage_b) cudaFree(plan->stage_b);
             plan->stage_a = plan->stage_b = plan->stage_c = nullptr;
             cuda_fail(ctx, e);
