@@ -114,8 +114,10 @@ struct KernelParams {
     float alpha, beta;
 };
 
+template <bool OFF = false>
 __device__ __forceinline__ void trace_stamp(const KernelParams &p, int slot)
 {
+    if constexpr (OFF) return;
     if (p.trace != nullptr && blockIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -282,7 +284,7 @@ struct WorkItem {
 };
 
 // SPLIT = false: the caller knows that no work item is a K slice (split_k == 1 and no tail cut along K).
-template <bool SPLIT = true>
+template <bool SPLIT = true, bool PLAIN = false>
 __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p, int32_t block_m_total)
 {
     WorkItem it;
@@ -296,7 +298,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
         it.slice = 0;
         it.slices = 1;
         it.split_index = 0;
-    } else if (p.tail_pieces > 1) {
+    } else if (!PLAIN && p.tail_pieces > 1) {
         const int32_t idx = w - p.first_split_tile;
         const int32_t t = fast_div(idx, p.fd_pieces);
         it.tile = p.first_split_tile + t;
@@ -362,9 +364,11 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // SPLIT: 0 for configurations without K slices (split_k == 1, no tail cut along K), 1 for slices summed through the
 // global workspace, 2 for slices summed inside a cluster; each instantiation carries only its own reduction, which
 // saves registers and shortens the start-up of every call.
+// PLAIN: the instantiation for the plain call -- C = A B^T with fp32 accumulators, K-contiguous B, rows of C that are
+// multiples of 16 bytes, whole-width tail tiles, no instrumentation: all of those branches are compiled out.
 // WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
 // store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
-template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1>
+template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -430,7 +434,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         fence_mbar_init();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
-        if (p.tail_pieces > 1) prefetch_tensormap(&tmap_bt);
+        if ((!PLAIN && p.tail_pieces > 1)) prefetch_tensormap(&tmap_bt);
         prefetch_tensormap(&tmap_c);
     }
     if (warp == 1) {
@@ -459,13 +463,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         int s = 0;
         uint32_t ph = 0;
         const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, leader_rank) : bar_full;
-        const bool tr = p.trace != nullptr && blockIdx.x == 0;
+        const bool tr = (!PLAIN && p.trace != nullptr) && blockIdx.x == 0;
         const uint32_t leader = (lane == 0) ? 1u : 0u;     // the lane that issues the loads
         long long t_wait = 0, t_work = 0;
         bool ok = true;
         bool dependencies_met = false;
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
-            const WorkItem it = warp_uniform(decode_work<SPLIT != 0>(w, p, kBlockMTotal));
+            const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
             // this CTA's rows of B: its share of the work item's columns
             const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
@@ -483,16 +487,16 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     grid_dependency_wait();                   // the kernels before this one are complete: global memory may be read
                     dependencies_met = true;
                     if (threadIdx.x == 0) {
-                        trace_stamp(p, 0);
-                        trace_stamp(p, 1);
+                        trace_stamp<PLAIN>(p, 0);
+                        trace_stamp<PLAIN>(p, 1);
                     }
                 }
-                if (p.debug_skip & 1u) {
+                if ((PLAIN ? 0u : p.debug_skip) & 1u) {
                     if (lane == 0) {
                         if (is_leader) mbar_arrive(bar_full + 8 * s);
                         else mbar_arrive_cluster(fb);
                     }
-                } else if (p.b_row_major) {
+                } else if ((!PLAIN && p.b_row_major)) {
                     // B is K x N row-major: per 64-wide K sub-tile, one {64 columns, 64 k-rows} box per 64-column block
                     const int32_t b_col = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
                     const int32_t blocks = (it.bn / CTA_GROUP) / 64;       // a column piece of a tail tile loads fewer blocks
@@ -509,7 +513,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             else tma_load_2d_pair_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
                         }
                     }
-                } else if (it.bn != p.block_n) {
+                } else if ((!PLAIN && it.bn != p.block_n)) {
                     // a column piece of a tail tile: its rows of B come through the narrower map `tmap_bt`, one box per
                     // 64-wide K sub-tile, each placed where the full-height box of that sub-tile would start
                     const uint32_t tx = a_stage_bytes + static_cast<uint32_t>(subs * (it.bn / CTA_GROUP)) * (kSubK * 2u);
@@ -558,33 +562,33 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         tma_load_2d_pair_if(leader, b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, fb);
                     }
                 }
-                if (w == unit && kb == 0 && lane == 0) trace_stamp(p, 2);
+                if (w == unit && kb == 0 && lane == 0) trace_stamp<PLAIN>(p, 2);
                 if (tr) { t_wait += c1 - c0; t_work += clock64() - c1; }
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
         if (tr && lane == 0) { p.trace[11] = t_wait; p.trace[12] = t_work; }
     } else if (warp == 1) {
-        if (p.trace != nullptr) grid_dependency_wait();   // this warp's only global accesses are trace stamps
+        if ((!PLAIN && p.trace != nullptr)) grid_dependency_wait();   // this warp's only global accesses are trace stamps
         if (is_leader) {
             // ===== MMA issuer =====
             int s = 0;
             uint32_t ph = 0;
             uint32_t local_tile = 0;
-            const bool tr = p.trace != nullptr && blockIdx.x == 0;
+            const bool tr = (!PLAIN && p.trace != nullptr) && blockIdx.x == 0;
             const uint32_t leader = (lane == 0) ? 1u : 0u; // the lane that issues every MMA and commit
             long long t_wait = 0, t_issue = 0, t_commit = 0, t_acc = 0, n_kb = 0;
             const uint64_t desc_a0 = make_smem_desc_sw128(smem_base);
             // B tile: K-major (B stored N x K) or N-major in 64-column blocks of 64 k-rows (B stored K x N)
-            const uint64_t desc_b0 = p.b_row_major ? make_smem_desc_sw128_mn_major(smem_base + a_stage_bytes, kSubK * 128u)
+            const uint64_t desc_b0 = (!PLAIN && p.b_row_major) ? make_smem_desc_sw128_mn_major(smem_base + a_stage_bytes, kSubK * 128u)
                                                    : make_smem_desc_sw128(smem_base + a_stage_bytes);
             // advancing K by 16: +32 bytes inside a K-major swizzle row, +16 k-rows (2048 bytes) in an N-major tile
-            const uint32_t b_kstep = p.b_row_major ? (16u * 128u) >> 4 : 2u;
+            const uint32_t b_kstep = (!PLAIN && p.b_row_major) ? (16u * 128u) >> 4 : 2u;
             const uint32_t desc_stage_step = stage_bytes >> 4;
-            const bool issue_mma = !(p.debug_skip & 2u);
+            const bool issue_mma = !((PLAIN ? 0u : p.debug_skip) & 2u);
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-                const WorkItem it = warp_uniform(decode_work<SPLIT != 0>(w, p, kBlockMTotal));
+                const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
                 const uint32_t acc = local_tile & 1u;
                 const uint32_t acc_ph = (local_tile >> 1) & 1u;
                 const long long ca = tr ? clock64() : 0;
@@ -608,7 +612,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     tc_fence_after_sync();
                     const uint64_t a_desc = desc_a0 + static_cast<uint64_t>(static_cast<uint32_t>(s) * desc_stage_step);
                     const uint64_t b_desc = desc_b0 + static_cast<uint64_t>(static_cast<uint32_t>(s) * desc_stage_step);
-                    if (w == unit && kb == 0 && lane == 0) trace_stamp(p, 3);
+                    if (w == unit && kb == 0 && lane == 0) trace_stamp<PLAIN>(p, 3);
                     if (issue_mma) {
                         for (int32_t sub = 0; sub < subs; ++sub) {
                             const uint64_t a_sub = a_desc + static_cast<uint64_t>(static_cast<uint32_t>(sub) * (kATileBytes >> 4));
@@ -631,7 +635,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (it.bn == p.block_n) run_k_blocks(p.idesc);
                 else run_k_blocks(p.idesc_tail);
                 if (!ok) break;
-                if (w == unit && lane == 0) trace_stamp(p, 4);
+                if (w == unit && lane == 0) trace_stamp<PLAIN>(p, 4);
                 umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc, leader_rank);
             }
             if (tr && lane == 0) { p.trace[8] = t_wait; p.trace[9] = t_issue; p.trace[10] = t_commit; p.trace[13] = t_acc; p.trace[15] = n_kb; }
@@ -652,7 +656,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         tc_fence_after_sync();
                         tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
                         tmem_freed = true;
-                        if (lane == 0) trace_stamp(p, 7);
+                        if (lane == 0) trace_stamp<PLAIN>(p, 7);
                     }
                 }
             }
@@ -673,13 +677,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         bool ok = true;
         grid_dependency_wait();                            // before the first store to C, workspace or counters
         for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
-            const WorkItem it = decode_work<SPLIT != 0>(w, p, kBlockMTotal);
+            const WorkItem it = decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal);
             const uint32_t acc = local_tile & 1u;
             const uint32_t acc_ph = (local_tile >> 1) & 1u;
             ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
             ok = __all_sync(0xffffffffu, ok);   // the warp-wide tensor-memory loads below need the whole warp
             if (!ok) break;
-            if (w == unit && threadIdx.x == 64) trace_stamp(p, 5);
+            if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 5);
             tc_fence_after_sync();
             const int32_t row0 = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;  // first row of this CTA's 128
             const int32_t grow = row0 + static_cast<int32_t>(row_in_tile);          // this thread's global row
@@ -709,12 +713,12 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         // warp-uniform code: the store is predicated inside its asm block, the commit is executed
                         // by every lane (an empty group for all but lane 0)
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !(p.debug_skip & 4u);
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((PLAIN ? 0u : p.debug_skip) & 4u);
                         tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
                     ++store_count;
-                } else if (p.ragged_n) {
+                } else if ((!PLAIN && p.ragged_n)) {
                     // rows of C are not multiples of 16 bytes: neither TMA nor vector stores apply.  The chunk is
                     // transposed through the warp's staging buffer (same 64-byte swizzle as above) so that each
                     // store instruction writes 32 consecutive elements of one row instead of one element of 32 rows.
@@ -787,13 +791,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (c < chunks) {
                             tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                             tmem_ld_wait();
-                            if (p.acc_f16) {
+                            if ((!PLAIN && p.acc_f16)) {
 #pragma unroll
                                 for (int j = 0; j < 32; ++j)
                                     v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
                             }
                             if (b + 2 >= boxes && c + 1 >= min(chunks, 2 * b + 2)) release_accumulator();   // this warp's last load
-                            if (p.scaled && grow < p.M) {
+                            if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                                 for (int j = 0; j < 4; ++j)
                                     if (it.n0 + c * 32 + 8 * j < p.N) scale_group8(v + 8 * j, p, grow, it.n0 + c * 32 + 8 * j);
@@ -811,7 +815,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     {
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
                         const int32_t col0 = it.n0 + b * 64;
-                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !(p.debug_skip & 4u);
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((PLAIN ? 0u : p.debug_skip) & 4u);
                         tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
@@ -826,7 +830,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
-                    if (p.acc_f16) {
+                    if ((!PLAIN && p.acc_f16)) {
                         // fp16 accumulators (measured layout: one result per 32-bit column, in its low half):
                         // widen them, exactly, so that the store paths below see what they see with fp32 ones
 #pragma unroll
@@ -834,7 +838,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
                     }
                     if (c + 2 >= chunks) release_accumulator();       // every load of this warp has completed
-                    if (p.scaled && grow < p.M) {
+                    if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             if (it.n0 + c * 32 + 8 * j < p.N) scale_group8(v + 8 * j, p, grow, it.n0 + c * 32 + 8 * j);
@@ -881,7 +885,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     bulk_wait_group<0>();                            // this warp's part of the slot is written
                     fence_proxy_async_all();                         // order those writes before the signal below
                 }
-                if (w == unit && threadIdx.x == 64) trace_stamp(p, 16);
+                if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 16);
                 // 2. announce it, then wait (bounded) until every slice of this tile has done the same.
                 //    All slices of a tile are in flight together: the grid never exceeds the SM count, one
                 //    CTA per SM, and work items are handed out in tile order.
@@ -910,7 +914,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (w == unit && threadIdx.x == 64) trace_stamp(p, 17);
+                if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 17);
                 __threadfence();
                 // 3. every slice reduces its share of the tile: slice s owns the contiguous unit range
                 //    [s U / S, (s + 1) U / S), so neighbouring threads read neighbouring addresses.  Each unit is
@@ -956,8 +960,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const int32_t u = u0 + j * 256;
                         const int32_t c = u >> 10, r = (u >> 3) & 127, g = (u & 7) ^ (r & 7);
                         const int32_t orow = row0 + r, col = it.n0 + c * 32 + g * 4;
-                        if (p.scaled) scale_unit4(sum[j], p, orow, col);
-                        if (p.ragged_n) {
+                        if ((!PLAIN && p.scaled)) scale_unit4(sum[j], p, orow, col);
+                        if ((!PLAIN && p.ragged_n)) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
                             store_ragged(p.C, p.N, orow, col, f, 4);
                             continue;
@@ -968,13 +972,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                     }
                 }
-                if (w == unit && threadIdx.x == 64) trace_stamp(p, 18);
+                if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 18);
             }
         }
         // shared memory must stay valid until the last TMA stores have read it (their global writes are
         // complete, like every other store of this grid, when the grid completes)
         if (lane == 0) bulk_wait_group_read<0>();
-        if (threadIdx.x == 64) trace_stamp(p, 6);
+        if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 6);
     }
 
     // ---- cluster split-K: sum the slices through distributed shared memory -----------------
@@ -1004,7 +1008,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             if (threadIdx.x == 64) mbar_arrive_expect_tx(bar_recv, (S - 1u) * own_count * 16u);
             // barrier 1, arrival: this CTA has finished its main loop (its epilogue warps get here only after the
             // last MMA has completed), so its stage ring is free to be overwritten, and has armed its barrier
-            if (threadIdx.x == 64) trace_stamp(p, 16);
+            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 16);
             cluster_arrive();
             if (warp >= 2) {
                 // while the other CTAs arrive, stage this CTA's partial in its own ring (after an abort the
@@ -1027,10 +1031,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     fence_proxy_async_smem();        // the bulk copies below read these writes
                 }
             }
-            if (threadIdx.x == 64) trace_stamp(p, 17);
+            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 17);
             cluster_wait();                          // barrier 1, wait: every ring of the cluster is free
             const bool live = *abort_flag == 0u;     // stable here: no thread of this CTA is in a wait
-            if (threadIdx.x == 64) trace_stamp(p, 19);
+            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 19);
             bool ok = live;
             if (warp >= 2) {
                 named_barrier_sync(1, 8 * 32);       // the whole tile is in shared memory
@@ -1045,14 +1049,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                              min(cap, units - o_begin) * 16u, mapa(bar_recv, o_rank));
                     }
                 }
-                if (threadIdx.x == 64) trace_stamp(p, 18);
+                if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 18);
                 if (live) ok = mbar_wait(bar_recv, 0u, ctl, status_code(kRoleEpilogue, 4, 0));
                 ok = __all_sync(0xffffffffu, ok);
             }
             // barrier 2, arrival: this CTA has received everything (or given up).  Once every CTA of the cluster
             // has arrived, no bulk copy is reading anyone's shared memory any more and all may leave.
             cluster_arrive_relaxed();
-            if (threadIdx.x == 64) trace_stamp(p, 20);
+            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 20);
             if (warp >= 2 && ok) {
                 const uint32_t ew = warp - 2u;
                 const uint32_t own_addr = smem_base + own_begin * 16u;
@@ -1085,8 +1089,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const int32_t c = static_cast<int32_t>(cc), g = static_cast<int32_t>((u & 7u) ^ (r & 7u));
                         const int32_t orow = cs_m0 + static_cast<int32_t>(r), col = cs_n0 + c * 32 + g * 4;
                         if (orow >= p.M || col >= p.N) continue;
-                        if (p.scaled) scale_unit4(sum[j], p, orow, col);
-                        if (p.ragged_n) {
+                        if ((!PLAIN && p.scaled)) scale_unit4(sum[j], p, orow, col);
+                        if ((!PLAIN && p.ragged_n)) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
                             store_ragged(p.C, p.N, orow, col, f, 4);
                             continue;
@@ -1098,9 +1102,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
             }
-            if (threadIdx.x == 64) trace_stamp(p, 22);
+            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 22);
             cluster_wait();                          // barrier 2, wait
-            if (threadIdx.x == 64) trace_stamp(p, 21);
+            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 21);
         }
     }
 
@@ -1118,7 +1122,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         tc_fence_after_sync();
         tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
-        if (lane == 0) trace_stamp(p, 7);
+        if (lane == 0) trace_stamp<PLAIN>(p, 7);
     }
 }
 
