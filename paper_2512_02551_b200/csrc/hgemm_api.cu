@@ -120,8 +120,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         lc.attrs = attr;
         lc.numAttrs = 1;
         int clusters = 0;
-        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, 2, false>, &lc)
-                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, 2, false>, &lc);
+        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, 2, true, false>, &lc)
+                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, 2, true, false>, &lc);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return HGEMM_ERR_UNSUPPORTED;
@@ -216,12 +216,12 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
 
 // The kernel instantiation for a CTA group size, store-box width and kind of split-K reduction
 // (0: no K slices, 1: through the workspace -- also a tail cut along K --, 2: inside a cluster); `plain` selects
-// the instantiation without the optional features.
-template <bool PLAIN>
+// the instantiation without the optional features, `trace` the one with the instrumentation (never plain).
+template <bool PLAIN, bool TRACE>
 const void *kernel_of(int cg, bool wide, int split)
 {
     using namespace hgemm_dev;
-#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S, PLAIN>)
+#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S, PLAIN, TRACE>)
     if (cg == 1) {
         if (wide) return split == 0 ? HGEMM_K(1, true, 0) : HGEMM_K(1, true, 1);      // no split_k > 1 with wide boxes
         return split == 0 ? HGEMM_K(1, false, 0) : split == 1 ? HGEMM_K(1, false, 1) : HGEMM_K(1, false, 2);
@@ -231,9 +231,10 @@ const void *kernel_of(int cg, bool wide, int split)
 #undef HGEMM_K
 }
 
-const void *kernel_for(int cg, bool wide, int split, bool plain)
+const void *kernel_for(int cg, bool wide, int split, bool plain, bool trace)
 {
-    return plain ? kernel_of<true>(cg, wide, split) : kernel_of<false>(cg, wide, split);
+    if (trace) return kernel_of<false, true>(cg, wide, split);
+    return plain ? kernel_of<true, false>(cg, wide, split) : kernel_of<false, false>(cg, wide, split);
 }
 
 bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_inner,
@@ -333,8 +334,8 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             break;
         }
         // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, no K slices / workspace / cluster reduction
-        for (int k = 0; k < 24 && e == cudaSuccess; ++k) {
-            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k >= 12);
+        for (int k = 0; k < 36 && e == cudaSuccess; ++k) {
+            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k / 12 == 1, k / 12 == 2);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
@@ -624,9 +625,10 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     // it, also when a C with ragged rows makes it fall back to element stores; the instantiation without the
     // split-K reductions runs whenever no work item is a K slice.
     const KernelParams &kp = plan->params;
-    const bool plain = !kp.scaled && !kp.acc_f16 && !kp.ragged_n && !kp.b_row_major && kp.tail_pieces <= 1 && kp.trace == nullptr &&
-                       kp.debug_skip == 0;
-    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain);
+    const bool trace = kp.trace != nullptr || kp.debug_skip != 0;
+    const bool plain = !kp.scaled && !kp.acc_f16 && !kp.ragged_n && !kp.b_row_major && kp.tail_pieces <= 1;
+    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
+                                trace);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
     e = cudaLaunchKernelExC(&lc, fn, args);
     if (e != cudaSuccess) return cuda_fail(ctx, e);

@@ -365,10 +365,12 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // global workspace, 2 for slices summed inside a cluster; each instantiation carries only its own reduction, which
 // saves registers and shortens the start-up of every call.
 // PLAIN: the instantiation for the plain call -- C = A B^T with fp32 accumulators, K-contiguous B, rows of C that are
-// multiples of 16 bytes, whole-width tail tiles, no instrumentation: all of those branches are compiled out.
+// multiples of 16 bytes, whole-width tail tiles: all of those branches are compiled out.
+// TRACE: the instantiation that carries the instrumentation (trace stamps, per-role cycle counters, the skip mask);
+// compiled in but switched off it cost 10-15 % on small and mid-size shapes, so it only runs when one of them is set.
 // WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
 // store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
-template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false>
+template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false, bool TRACE = !PLAIN>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -463,7 +465,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         int s = 0;
         uint32_t ph = 0;
         const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, leader_rank) : bar_full;
-        const bool tr = (!PLAIN && p.trace != nullptr) && blockIdx.x == 0;
+        const bool tr = (TRACE && p.trace != nullptr) && blockIdx.x == 0;
         const uint32_t leader = (lane == 0) ? 1u : 0u;     // the lane that issues the loads
         long long t_wait = 0, t_work = 0;
         bool ok = true;
@@ -487,11 +489,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     grid_dependency_wait();                   // the kernels before this one are complete: global memory may be read
                     dependencies_met = true;
                     if (threadIdx.x == 0) {
-                        trace_stamp<PLAIN>(p, 0);
-                        trace_stamp<PLAIN>(p, 1);
+                        trace_stamp<!TRACE>(p, 0);
+                        trace_stamp<!TRACE>(p, 1);
                     }
                 }
-                if ((PLAIN ? 0u : p.debug_skip) & 1u) {
+                if ((TRACE ? p.debug_skip : 0u) & 1u) {
                     if (lane == 0) {
                         if (is_leader) mbar_arrive(bar_full + 8 * s);
                         else mbar_arrive_cluster(fb);
@@ -562,20 +564,20 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         tma_load_2d_pair_if(leader, b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, fb);
                     }
                 }
-                if (w == unit && kb == 0 && lane == 0) trace_stamp<PLAIN>(p, 2);
+                if (w == unit && kb == 0 && lane == 0) trace_stamp<!TRACE>(p, 2);
                 if (tr) { t_wait += c1 - c0; t_work += clock64() - c1; }
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
         if (tr && lane == 0) { p.trace[11] = t_wait; p.trace[12] = t_work; }
     } else if (warp == 1) {
-        if ((!PLAIN && p.trace != nullptr)) grid_dependency_wait();   // this warp's only global accesses are trace stamps
+        if ((TRACE && p.trace != nullptr)) grid_dependency_wait();   // this warp's only global accesses are trace stamps
         if (is_leader) {
             // ===== MMA issuer =====
             int s = 0;
             uint32_t ph = 0;
             uint32_t local_tile = 0;
-            const bool tr = (!PLAIN && p.trace != nullptr) && blockIdx.x == 0;
+            const bool tr = (TRACE && p.trace != nullptr) && blockIdx.x == 0;
             const uint32_t leader = (lane == 0) ? 1u : 0u; // the lane that issues every MMA and commit
             long long t_wait = 0, t_issue = 0, t_commit = 0, t_acc = 0, n_kb = 0;
             const uint64_t desc_a0 = make_smem_desc_sw128(smem_base);
@@ -585,7 +587,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             // advancing K by 16: +32 bytes inside a K-major swizzle row, +16 k-rows (2048 bytes) in an N-major tile
             const uint32_t b_kstep = (!PLAIN && p.b_row_major) ? (16u * 128u) >> 4 : 2u;
             const uint32_t desc_stage_step = stage_bytes >> 4;
-            const bool issue_mma = !((PLAIN ? 0u : p.debug_skip) & 2u);
+            const bool issue_mma = !((TRACE ? p.debug_skip : 0u) & 2u);
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
                 const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
@@ -612,7 +614,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     tc_fence_after_sync();
                     const uint64_t a_desc = desc_a0 + static_cast<uint64_t>(static_cast<uint32_t>(s) * desc_stage_step);
                     const uint64_t b_desc = desc_b0 + static_cast<uint64_t>(static_cast<uint32_t>(s) * desc_stage_step);
-                    if (w == unit && kb == 0 && lane == 0) trace_stamp<PLAIN>(p, 3);
+                    if (w == unit && kb == 0 && lane == 0) trace_stamp<!TRACE>(p, 3);
                     if (issue_mma) {
                         for (int32_t sub = 0; sub < subs; ++sub) {
                             const uint64_t a_sub = a_desc + static_cast<uint64_t>(static_cast<uint32_t>(sub) * (kATileBytes >> 4));
@@ -635,7 +637,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (it.bn == p.block_n) run_k_blocks(p.idesc);
                 else run_k_blocks(p.idesc_tail);
                 if (!ok) break;
-                if (w == unit && lane == 0) trace_stamp<PLAIN>(p, 4);
+                if (w == unit && lane == 0) trace_stamp<!TRACE>(p, 4);
                 umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc, leader_rank);
             }
             if (tr && lane == 0) { p.trace[8] = t_wait; p.trace[9] = t_issue; p.trace[10] = t_commit; p.trace[13] = t_acc; p.trace[15] = n_kb; }
@@ -656,7 +658,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         tc_fence_after_sync();
                         tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
                         tmem_freed = true;
-                        if (lane == 0) trace_stamp<PLAIN>(p, 7);
+                        if (lane == 0) trace_stamp<!TRACE>(p, 7);
                     }
                 }
             }
@@ -683,7 +685,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
             ok = __all_sync(0xffffffffu, ok);   // the warp-wide tensor-memory loads below need the whole warp
             if (!ok) break;
-            if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 5);
+            if (w == unit && threadIdx.x == 64) trace_stamp<!TRACE>(p, 5);
             tc_fence_after_sync();
             const int32_t row0 = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;  // first row of this CTA's 128
             const int32_t grow = row0 + static_cast<int32_t>(row_in_tile);          // this thread's global row
@@ -713,7 +715,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         // warp-uniform code: the store is predicated inside its asm block, the commit is executed
                         // by every lane (an empty group for all but lane 0)
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((PLAIN ? 0u : p.debug_skip) & 4u);
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((TRACE ? p.debug_skip : 0u) & 4u);
                         tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
@@ -815,7 +817,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     {
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
                         const int32_t col0 = it.n0 + b * 64;
-                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((PLAIN ? 0u : p.debug_skip) & 4u);
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((TRACE ? p.debug_skip : 0u) & 4u);
                         tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
@@ -885,7 +887,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     bulk_wait_group<0>();                            // this warp's part of the slot is written
                     fence_proxy_async_all();                         // order those writes before the signal below
                 }
-                if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 16);
+                if (w == unit && threadIdx.x == 64) trace_stamp<!TRACE>(p, 16);
                 // 2. announce it, then wait (bounded) until every slice of this tile has done the same.
                 //    All slices of a tile are in flight together: the grid never exceeds the SM count, one
                 //    CTA per SM, and work items are handed out in tile order.
@@ -914,7 +916,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 17);
+                if (w == unit && threadIdx.x == 64) trace_stamp<!TRACE>(p, 17);
                 __threadfence();
                 // 3. every slice reduces its share of the tile: slice s owns the contiguous unit range
                 //    [s U / S, (s + 1) U / S), so neighbouring threads read neighbouring addresses.  Each unit is
@@ -972,13 +974,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                     }
                 }
-                if (w == unit && threadIdx.x == 64) trace_stamp<PLAIN>(p, 18);
+                if (w == unit && threadIdx.x == 64) trace_stamp<!TRACE>(p, 18);
             }
         }
         // shared memory must stay valid until the last TMA stores have read it (their global writes are
         // complete, like every other store of this grid, when the grid completes)
         if (lane == 0) bulk_wait_group_read<0>();
-        if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 6);
+        if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 6);
     }
 
     // ---- cluster split-K: sum the slices through distributed shared memory -----------------
@@ -1008,7 +1010,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             if (threadIdx.x == 64) mbar_arrive_expect_tx(bar_recv, (S - 1u) * own_count * 16u);
             // barrier 1, arrival: this CTA has finished its main loop (its epilogue warps get here only after the
             // last MMA has completed), so its stage ring is free to be overwritten, and has armed its barrier
-            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 16);
+            if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 16);
             cluster_arrive();
             if (warp >= 2) {
                 // while the other CTAs arrive, stage this CTA's partial in its own ring (after an abort the
@@ -1031,10 +1033,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     fence_proxy_async_smem();        // the bulk copies below read these writes
                 }
             }
-            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 17);
+            if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 17);
             cluster_wait();                          // barrier 1, wait: every ring of the cluster is free
             const bool live = *abort_flag == 0u;     // stable here: no thread of this CTA is in a wait
-            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 19);
+            if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 19);
             bool ok = live;
             if (warp >= 2) {
                 named_barrier_sync(1, 8 * 32);       // the whole tile is in shared memory
@@ -1049,14 +1051,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                              min(cap, units - o_begin) * 16u, mapa(bar_recv, o_rank));
                     }
                 }
-                if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 18);
+                if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 18);
                 if (live) ok = mbar_wait(bar_recv, 0u, ctl, status_code(kRoleEpilogue, 4, 0));
                 ok = __all_sync(0xffffffffu, ok);
             }
             // barrier 2, arrival: this CTA has received everything (or given up).  Once every CTA of the cluster
             // has arrived, no bulk copy is reading anyone's shared memory any more and all may leave.
             cluster_arrive_relaxed();
-            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 20);
+            if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 20);
             if (warp >= 2 && ok) {
                 const uint32_t ew = warp - 2u;
                 const uint32_t own_addr = smem_base + own_begin * 16u;
@@ -1102,9 +1104,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
             }
-            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 22);
+            if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 22);
             cluster_wait();                          // barrier 2, wait
-            if (threadIdx.x == 64) trace_stamp<PLAIN>(p, 21);
+            if (threadIdx.x == 64) trace_stamp<!TRACE>(p, 21);
         }
     }
 
@@ -1122,7 +1124,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         tc_fence_after_sync();
         tmem_dealloc<CTA_GROUP>(tmem_base, static_cast<uint32_t>(p.tmem_cols));
-        if (lane == 0) trace_stamp<PLAIN>(p, 7);
+        if (lane == 0) trace_stamp<!TRACE>(p, 7);
     }
 }
 

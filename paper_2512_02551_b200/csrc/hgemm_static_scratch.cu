@@ -82,7 +82,7 @@ hgemm_status_t setup_device(int device, DeviceState **out)
             (void)cudaGetLastError();
             return HGEMM_ERR_CUDA;
         }
-        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(hgemm_dev::hgemm_umma_kernel<1, false, 1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  int(hgemm_host::kSmemOptInBytes));
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
@@ -213,7 +213,7 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     lc.blockDim = dim3(hgemm_dev::kThreads, 1, 1);
     lc.dynamicSmemBytes = size_t(hgemm_host::kSmemOptInBytes);
     lc.stream = s;
-    cudaError_t e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1>, tmap_a, tmap_b, tmap_c, tmap_b, p);
+    cudaError_t e = cudaLaunchKernelEx(&lc, hgemm_dev::hgemm_umma_kernel<1, false, 1, false, false>, tmap_a, tmap_b, tmap_c, tmap_b, p);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return HGEMM_ERR_CUDA;
