@@ -634,7 +634,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 };
-                if (it.bn == p.block_n) run_k_blocks(p.idesc);
+                if (PLAIN || it.bn == p.block_n) run_k_blocks(p.idesc);      // no column pieces in the plain instantiations
                 else run_k_blocks(p.idesc_tail);
                 if (!ok) break;
                 if (w == unit && lane == 0) trace_stamp<!TRACE>(p, 4);
