@@ -283,7 +283,10 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
  * 17 all slices arrived, 18 share reduced; for cluster split-K 16 arrived at the
  * cluster's first barrier, 17 partial staged, 19 cluster gathered, 18 shares sent,
  * 20 shares received, 22 share reduced, 21 cluster released.  The caller owns the
- * buffer. */
+ * buffer.  While a trace buffer or a skip mask (below) is set, launches run the
+ * instrumented instantiation of the kernel, which is 10-15 % slower on small and
+ * mid-size shapes than the one that runs otherwise: the stamps describe the
+ * pipeline's structure and proportions, not the production kernel's absolute times. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan
