@@ -223,6 +223,29 @@ hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan);
 hgemm_status_t hgemm_plan_get_config(const hgemm_plan_t *plan, hgemm_config_t *out);
 hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *cfg);
 
+/* Run-time tuning of one plan (the library auto-tuning baseline of the paper's
+ * section 6.1, for shapes the tuned table does not hold): times the plan's current
+ * configuration and up to `max_candidates` others -- the legal configurations of
+ * the shape, ranked by the planner's cost model -- with the caller's buffers on
+ * `stream` (two untimed calls, then 3-64 back-to-back calls between CUDA events,
+ * each candidate), installs the fastest, and runs it once more, so that on return
+ * C (DEVICE, M x N) holds A B^T computed by the installed configuration.  A, B:
+ * DEVICE pointers laid out as for hgemm_run; C is overwritten (no alpha / beta).
+ * *best_us (HOST, may be NULL) receives the installed configuration's time per
+ * call in microseconds.  Synchronous: it waits for the stream, many times, and may
+ * reallocate the workspace.  It reads and clears the context's device status; if a
+ * bounded wait ran out during the search the plan keeps the configuration it had
+ * and HGEMM_ERR_TIMEOUT is returned.  Candidates the plan's layout does not
+ * support are skipped.  Costs about (max_candidates + 1) x 0.3-1 ms. */
+hgemm_status_t hgemm_plan_autotune(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream,
+                                   int32_t max_candidates, float *best_us);
+
+/* The candidates hgemm_plan_autotune draws from, as a pure host function: the legal
+ * configurations of (M, N, K) on a device with `num_sms` SMs, ranked by the cost
+ * model, best first; writes at most `max` of them to `out` (HOST array) and returns
+ * how many (0 for an illegal shape or arguments). */
+int32_t hgemm_candidate_configs(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out, int32_t max);
+
 /* The heuristic the planner falls back to, as a pure host function (no GPU
  * needed): configuration for (M, N, K) on a device with `num_sms` SMs. */
 hgemm_status_t hgemm_heuristic_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);

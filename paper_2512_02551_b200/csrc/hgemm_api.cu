@@ -507,6 +507,83 @@ hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *c
     return apply_config(plan, *cfg);
 }
 
+int32_t hgemm_candidate_configs(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out, int32_t max)
+{
+    if (!out || max < 1) return 0;
+    if (hgemm_host::validate_shape(M, N, K) != HGEMM_OK) return 0;
+    return hgemm_host::ranked_candidates(M, N, hgemm_host::padded_k(K), num_sms, out, max);
+}
+
+hgemm_status_t hgemm_plan_autotune(hgemm_plan_t *plan, const void *A, const void *B, void *C, void *stream, int32_t max_candidates,
+                                   float *best_us)
+{
+    if (!plan || !A || !B || !C || max_candidates < 1) return HGEMM_ERR_INVALID_ARG;
+    hgemm_ctx_s *ctx = plan->ctx;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const hgemm_config_t start = plan->cfg;
+    std::vector<hgemm_config_t> cands(size_t(std::min<int32_t>(max_candidates, 256)) + 1);
+    cands[0] = start;                                            // the planner's own choice is always timed
+    const int32_t n = 1 + hgemm_host::ranked_candidates(plan->M, plan->N, plan->K, ctx->num_sms, cands.data() + 1,
+                                                        int32_t(cands.size()) - 1);
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    if (e != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        return cuda_fail(ctx, e);
+    }
+    hgemm_status_t result = HGEMM_OK;
+    hgemm_config_t best = start;
+    float best_ms = -1.0f;
+    for (int32_t i = 0; i < n && result == HGEMM_OK; ++i) {
+        if (i > 0 && std::memcmp(&cands[size_t(i)], &start, sizeof(start)) == 0) continue;
+        if (hgemm_plan_set_config(plan, &cands[size_t(i)]) != HGEMM_OK) continue;      // e.g. a layout's extra rules
+        // two untimed calls, then enough back-to-back calls to fill about a quarter of a millisecond
+        hgemm_status_t s = hgemm_run(plan, A, B, C, stream);
+        if (s == HGEMM_OK) s = hgemm_run(plan, A, B, C, stream);
+        float probe_ms = 0.0f;
+        if (s == HGEMM_OK) {
+            cudaEventRecord(e0, st);
+            s = hgemm_run(plan, A, B, C, stream);
+            cudaEventRecord(e1, st);
+            e = cudaEventSynchronize(e1);
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&probe_ms, e0, e1);
+            if (e != cudaSuccess) result = cuda_fail(ctx, e);
+        }
+        if (s != HGEMM_OK || result != HGEMM_OK) continue;
+        const int reps = std::max(3, std::min(64, int(0.25f / std::max(probe_ms, 1e-3f))));
+        cudaEventRecord(e0, st);
+        for (int r = 0; r < reps && s == HGEMM_OK; ++r) s = hgemm_run(plan, A, B, C, stream);
+        cudaEventRecord(e1, st);
+        float ms = 0.0f;
+        e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+        if (e != cudaSuccess) {
+            result = cuda_fail(ctx, e);
+            break;
+        }
+        if (s != HGEMM_OK) continue;
+        ms /= float(reps);
+        if (best_ms < 0.0f || ms < best_ms) {
+            best_ms = ms;
+            best = cands[size_t(i)];
+        }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    // a wait that ran out during the search disqualifies the search, not the plan: back to where it started
+    uint32_t code = 0;
+    if (result == HGEMM_OK && hgemm_last_device_status(ctx, &code) != HGEMM_OK) {
+        (void)hgemm_plan_set_config(plan, &start);
+        return HGEMM_ERR_TIMEOUT;
+    }
+    const hgemm_status_t s = hgemm_plan_set_config(plan, result == HGEMM_OK ? &best : &start);
+    if (result != HGEMM_OK) return result;
+    if (s != HGEMM_OK) return s;
+    if (best_us) *best_us = best_ms * 1e3f;
+    return hgemm_run(plan, A, B, C, stream);                     // C holds the product computed by the installed configuration
+}
+
 int32_t hgemm_plan_launches_per_run(const hgemm_plan_t *plan)
 {
     return plan ? 1 : 0;

@@ -4,6 +4,8 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <utility>
+#include <vector>
 
 namespace hgemm_host {
 
@@ -281,6 +283,75 @@ int32_t raster_group_for(int64_t M, int32_t num_sms, const hgemm_config_t &c)
 }
 
 } // namespace
+
+int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out, int32_t max)
+{
+    if (!out || max < 1 || validate_shape(M, N, K) != HGEMM_OK) return 0;
+    if (num_sms < 2) num_sms = 148;
+    static const int32_t kSplits[] = {1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64};
+    std::vector<std::pair<double, hgemm_config_t>> all;
+    auto add = [&](const hgemm_config_t &c) {
+        if (validate(M, N, K, c) == HGEMM_OK) all.emplace_back(estimate_cycles(M, N, K, num_sms, c), c);
+    };
+    for (int family = 0; family < 2; ++family) {
+        const int cg = family == HGEMM_FAMILY_UMMA_2CTA ? 2 : 1;
+        const int64_t units = std::max(1, num_sms / cg);
+        for (int32_t bn = 32; bn <= 256; bn += 32) {
+            if (bn > 32 && bn - 32 >= N) break;                       // a wider tile would only add padding
+            const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, bn);
+            const int64_t tail = tiles % units;
+            for (int32_t bk = 64; bk <= 128; bk += 64) {
+                if (bk == 128 && K < 128) continue;
+                const int64_t kb = ceil_div(K, bk);
+                for (int32_t split : kSplits) {
+                    if (split > kb) break;
+                    if (split > 1 && tiles * split > 2 * units) continue;   // split-K only to fill an under-full machine
+                    for (int mode = 0; mode < 2; ++mode) {
+                        if (mode == 1 && (split == 1 || split * cg > 16)) continue;
+                        for (int epi = 0; epi < 3; ++epi) {
+                            if (split > 1 && epi != HGEMM_EPILOGUE_DIRECT) continue;
+                            if (epi == HGEMM_EPILOGUE_TMA_WIDE && (bn % 64) != 0) continue;
+                            hgemm_config_t c;
+                            std::memset(&c, 0, sizeof(c));
+                            c.family = family;
+                            c.block_m = 128 * cg;
+                            c.block_n = bn;
+                            c.block_k = bk;
+                            c.split_k = split;
+                            c.split_mode = mode;
+                            c.epilogue = epi;
+                            c.stages = std::min<int32_t>(max_stages_of(c), 8);
+                            if (c.stages < 1) continue;
+                            c.raster_group = raster_group_for(M, num_sms, c);
+                            add(c);
+                            if (split == 1 && tiles > units && tail > 0 && tail <= units / 2) {
+                                const int32_t ts = int32_t(std::min<int64_t>(std::min<int64_t>(units / tail, 8), kb));
+                                if (ts >= 2) {
+                                    hgemm_config_t t = c;
+                                    t.tail_split = ts;
+                                    t.tail_mode = HGEMM_TAIL_K;
+                                    add(t);
+                                }
+                                for (int32_t pieces = 2; pieces <= 4; pieces *= 2) {
+                                    if (tail * pieces > units || (bn % (32 * pieces)) != 0) continue;
+                                    hgemm_config_t t = c;
+                                    t.tail_split = pieces;
+                                    t.tail_mode = HGEMM_TAIL_N;
+                                    add(t);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    std::stable_sort(all.begin(), all.end(), [](const auto &a, const auto &b) { return a.first < b.first; });
+    const int32_t n = int32_t(std::min<size_t>(all.size(), size_t(max)));
+    for (int32_t i = 0; i < n; ++i) out[i] = all[size_t(i)].second;
+    return n;
+}
+
 
 hgemm_status_t plan_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out)
 {

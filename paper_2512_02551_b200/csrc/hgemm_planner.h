@@ -61,6 +61,10 @@ int table_neighbours(int64_t M, int64_t N, int64_t K, TableNeighbour *out, int m
 // the lowest calibrated estimate among the cost model's own choice and the neighbouring tuned shapes'
 // configurations re-fitted to this shape (split factor clamped and also scaled with K, raster group and tail
 // split recomputed), where a neighbour's candidates are scaled by (measured time / estimate) at that neighbour.
+// The legal configurations of a shape, ranked by estimate_cycles (best first), at most `max` of them: both
+// families, every tile width, both stage widths, the split factors that fill an under-full machine in both
+// split modes, the three epilogues, and the tail cuts where the last wave is at most half full.  Returns the count.
+int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out, int32_t max);
 hgemm_status_t plan_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgemm_config_t *out);
 
 } // namespace hgemm_host

@@ -24,7 +24,7 @@ LAYOUT_TN, LAYOUT_NN = 0, 1
 # every symbol include/hgemm.h declares
 EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
-    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
+    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_plan_autotune", "hgemm_candidate_configs", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
@@ -91,7 +91,9 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan_destroy": (i32, [p]),
             "hgemm_plan_get_config": (i32, [p, cfgp]),
             "hgemm_plan_set_config": (i32, [p, cfgp]),
+            "hgemm_plan_autotune": (i32, [p, p, p, p, p, i32, ctypes.POINTER(ctypes.c_float)]),
             "hgemm_heuristic_config": (i32, [i64, i64, i64, i32, cfgp]),
+            "hgemm_candidate_configs": (i32, [i64, i64, i64, i32, cfgp, i32]),
             "hgemm_planned_config": (i32, [i64, i64, i64, i32, cfgp]),
             "hgemm_validate_config": (i32, [i64, i64, i64, cfgp]),
             "hgemm_estimate_config": (ctypes.c_double, [i64, i64, i64, i32, cfgp]),
@@ -134,6 +136,18 @@ def planned_config(M: int, N: int, K: int, num_sms: int = 148) -> Config:
     c = Config()
     _check(lib().hgemm_planned_config(M, N, K, num_sms, ctypes.byref(c)), f"hgemm_planned_config({M},{N},{K})")
     return c
+
+
+def candidate_configs(M: int, N: int, K: int, max_count: int = 64, num_sms: int = 148) -> list:
+    """The configurations ``Plan.autotune`` draws from, best estimate first."""
+    arr = (Config * max_count)()
+    n = int(lib().hgemm_candidate_configs(M, N, K, num_sms, arr, max_count))
+    out = []
+    for i in range(n):
+        c = Config()
+        ctypes.memmove(ctypes.byref(c), ctypes.byref(arr[i]), ctypes.sizeof(Config))
+        out.append(c)
+    return out
 
 
 def validate_config(M: int, N: int, K: int, cfg: Config) -> int:
@@ -245,6 +259,21 @@ class Plan:
                 raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
         s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
         self.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s)
+
+    def autotune(self, A, B, C, max_candidates: int = 24, stream=None) -> float:
+        """``hgemm_plan_autotune``: times the plan's configuration and up to ``max_candidates`` others on these
+        tensors, installs the fastest (C then holds A B^T) and returns its time per call in microseconds."""
+        import torch
+        M, N, K = self.shape
+        b_shape = (K, N) if self.layout == LAYOUT_NN else (N, K)
+        for t, shp, name in ((A, (M, K), "A"), (B, b_shape, "B"), (C, (M, N), "C")):
+            if t.dtype != torch.float16 or not t.is_cuda or not t.is_contiguous() or tuple(t.shape) != shp:
+                raise ValueError(f"{name} must be a contiguous CUDA fp16 tensor of shape {shp}")
+        s = torch.cuda.current_stream().cuda_stream if stream is None else int(stream)
+        us = ctypes.c_float(0.0)
+        _check(lib().hgemm_plan_autotune(self._h, A.data_ptr(), B.data_ptr(), C.data_ptr(), s, int(max_candidates), ctypes.byref(us)),
+               f"hgemm_plan_autotune{self.shape}")
+        return float(us.value)
 
     def run_scaled(self, alpha: float, beta: float, A, B, C, stream=None) -> None:
         """``hgemm_run_scaled``: C = alpha * A B^T + beta * C in place, on torch CUDA tensors as for ``run``."""

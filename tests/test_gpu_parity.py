@@ -618,3 +618,55 @@ def test_infinities_nan_and_overflow(ctx, gu):
         assert np.array_equal(np.isnan(gu.bits_to_f64(g2)), want_nan), cfg.as_dict()
         assert np.array_equal(oracle.canonical_bits(g2)[ok], oracle.canonical_bits(want)[ok]), cfg.as_dict()
     plan.close()
+
+
+# ---- run-time tuning of a plan --------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("M,N,K", [(3584, 896, 1024), (320, 5000, 512), (100, 136, 77), (64, 640, 4096)])
+def test_plan_autotune(ctx, gu, M, N, K):
+    """hgemm_plan_autotune leaves a legal configuration that is at least as fast as the one it started from,
+    C holding the product, and the plan usable as before."""
+    import oracle
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C = torch.zeros(M, N, dtype=torch.float16, device="cuda")
+    plan = ctx.plan(M, N, K)
+    before = plan.config
+
+    def per_call_us(n=50):
+        for _ in range(5):
+            plan.run(A, B, C)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            plan.run(A, B, C)
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) / n * 1e3
+
+    t_before = min(per_call_us() for _ in range(3))
+    C.zero_()
+    us = plan.autotune(A, B, C, max_candidates=24)
+    assert us > 0.0
+    after = plan.config
+    assert hgemm.validate_config(M, N, (K + 7) // 8 * 8, after) == hgemm.OK
+    gu.assert_close_full(C, A, B, f"autotuned {after.as_dict()}")          # C is the product on return
+    t_after = min(per_call_us() for _ in range(3))
+    # (margin for timing noise: the small shapes are bound by the host's launch rate)
+    assert t_after <= 1.25 * t_before + 1.0, (t_before, t_after, before.as_dict(), after.as_dict())
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), "autotuned plan, integers")
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    plan.close()
+
+
+def test_plan_autotune_on_nn_layout_skips_unsupported_candidates(ctx, gu):
+    M, N, K = 520, 392, 1024
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    Bt = B.T.contiguous()                                                  # the K x N operand
+    C = torch.empty(M, N, dtype=torch.float16, device="cuda")
+    plan = ctx.plan(M, N, K, hgemm.LAYOUT_NN)
+    us = plan.autotune(A, Bt, C, max_candidates=16)
+    assert us > 0.0
+    gu.assert_close_full(C, A, B, f"autotuned NN {plan.config.as_dict()}")
+    plan.close()

@@ -144,3 +144,21 @@ def test_every_grid_shape_plans_to_a_legal_configuration(lib):
                 assert hgemm.config_smem_bytes(c) <= 232448
                 families.add(c.family)
     assert families == {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA}
+
+
+def test_candidate_configs_are_legal_ranked_and_distinct(lib):
+    for (M, N, K) in [(64, 64, 64), (8, 8, 8), (3584, 896, 1024), (13824, 512, 16384), (4096, 4096, 4096), (100, 136, 77)]:
+        Kp = (K + 7) // 8 * 8                                        # the library pads K to a multiple of 8
+        cands = hgemm.candidate_configs(M, N, K, max_count=48)
+        assert 1 <= len(cands) <= 48
+        est = [hgemm.estimate_config(M, N, Kp, c) for c in cands]
+        assert est == sorted(est)                                    # best estimate first
+        assert all(hgemm.validate_config(M, N, Kp, c) == hgemm.OK for c in cands)
+        keys = {tuple(sorted(c.as_dict().items())) for c in cands}
+        assert len(keys) == len(cands)
+    # both families, both stage widths, split-K and the wide epilogue all occur among the candidates of a shape that admits them
+    pool = hgemm.candidate_configs(512, 512, 4096, max_count=256)
+    assert {c.family for c in pool} == {0, 1} and {c.block_k for c in pool} == {64, 128}
+    assert any(c.split_k > 1 and c.split_mode == 1 for c in pool) and any(c.split_k > 1 and c.split_mode == 0 for c in pool)
+    assert any(c.epilogue == hgemm.EPILOGUE_TMA_WIDE for c in pool)
+    assert hgemm.candidate_configs(0, 64, 64) == [] and hgemm.candidate_configs(64, 64, 1 << 30) == []
