@@ -120,8 +120,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         lc.attrs = attr;
         lc.numAttrs = 1;
         int clusters = 0;
-        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, 2, true, false>, &lc)
-                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, 2, true, false>, &lc);
+        cudaError_t e = cg == 2 ? cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<2, false, 2, true, false, 1>, &lc)
+                                : cudaOccupancyMaxActiveClusters(&clusters, hgemm_dev::hgemm_umma_kernel<1, false, 2, true, false, 1>, &lc);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             return HGEMM_ERR_UNSUPPORTED;
@@ -217,11 +217,11 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
 // The kernel instantiation for a CTA group size, store-box width and kind of split-K reduction
 // (0: no K slices, 1: through the workspace -- also a tail cut along K --, 2: inside a cluster); `plain` selects
 // the instantiation without the optional features, `trace` the one with the instrumentation (never plain).
-template <bool PLAIN, bool TRACE>
+template <bool PLAIN, bool TRACE, int SUBS>
 const void *kernel_of(int cg, bool wide, int split)
 {
     using namespace hgemm_dev;
-#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S, PLAIN, TRACE>)
+#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S, PLAIN, TRACE, SUBS>)
     if (cg == 1) {
         if (wide) return split == 0 ? HGEMM_K(1, true, 0) : HGEMM_K(1, true, 1);      // no split_k > 1 with wide boxes
         return split == 0 ? HGEMM_K(1, false, 0) : split == 1 ? HGEMM_K(1, false, 1) : HGEMM_K(1, false, 2);
@@ -231,10 +231,12 @@ const void *kernel_of(int cg, bool wide, int split)
 #undef HGEMM_K
 }
 
-const void *kernel_for(int cg, bool wide, int split, bool plain, bool trace)
+// `subs`: 64-wide sub-tiles per stage (block_k / 64); the plain instantiations are compiled for each value.
+const void *kernel_for(int cg, bool wide, int split, bool plain, bool trace, int subs)
 {
-    if (trace) return kernel_of<false, true>(cg, wide, split);
-    return plain ? kernel_of<true, false>(cg, wide, split) : kernel_of<false, false>(cg, wide, split);
+    if (trace) return kernel_of<false, true, 0>(cg, wide, split);
+    if (!plain) return kernel_of<false, false, 0>(cg, wide, split);
+    return subs == 2 ? kernel_of<true, false, 2>(cg, wide, split) : kernel_of<true, false, 1>(cg, wide, split);
 }
 
 bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_inner,
@@ -334,8 +336,8 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             break;
         }
         // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, no K slices / workspace / cluster reduction
-        for (int k = 0; k < 36 && e == cudaSuccess; ++k) {
-            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k / 12 == 1, k / 12 == 2);
+        for (int k = 0; k < 48 && e == cudaSuccess; ++k) {
+            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k / 12 >= 2, k / 12 == 1, k / 12 == 3 ? 2 : 1);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
@@ -705,7 +707,7 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     const bool trace = kp.trace != nullptr || kp.debug_skip != 0;
     const bool plain = !kp.scaled && !kp.acc_f16 && !kp.ragged_n && !kp.b_row_major && kp.tail_pieces <= 1;
     const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
-                                trace);
+                                trace, kp.block_k / 64);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
     e = cudaLaunchKernelExC(&lc, fn, args);
     if (e != cudaSuccess) return cuda_fail(ctx, e);

@@ -366,11 +366,14 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // saves registers and shortens the start-up of every call.
 // PLAIN: the instantiation for the plain call -- C = A B^T with fp32 accumulators, K-contiguous B, rows of C that are
 // multiples of 16 bytes, whole-width tail tiles: all of those branches are compiled out.
+// SUBS: 1 or 2 fixes the stage width (64 or 128 columns of K) at compile time, so that the producer's and the MMA
+// issuer's loops over the 64-wide sub-tiles of a stage unroll (1-4 % on small and mid-size shapes); 0 reads it from the
+// parameters.  The plain instantiations exist for both widths, the others use 0.
 // TRACE: the instantiation that carries the instrumentation (trace stamps, per-role cycle counters, the skip mask);
 // compiled in but switched off it cost 10-15 % on small and mid-size shapes, so it only runs when one of them is set.
 // WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
 // store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
-template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false, bool TRACE = !PLAIN>
+template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false, bool TRACE = !PLAIN, int SUBS = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -380,7 +383,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     uint8_t *smem_gen = smem_raw + (smem_base - smem_addr(smem_raw));
 
     const int32_t b_rows = p.block_n / CTA_GROUP;            // B rows this CTA stages per k-block
-    const int32_t subs = p.block_k / kSubK;                  // 64-wide sub-tiles per stage (1 or 2)
+    const int32_t subs = SUBS != 0 ? SUBS : p.block_k / kSubK;   // 64-wide sub-tiles per stage (1 or 2)
     const uint32_t b_sub_bytes = static_cast<uint32_t>(b_rows) * kSubK * 2;
     const uint32_t a_stage_bytes = static_cast<uint32_t>(subs) * kATileBytes;
     const uint32_t stage_bytes = a_stage_bytes + static_cast<uint32_t>(subs) * b_sub_bytes;   // [A sub-tiles | B sub-tiles]
