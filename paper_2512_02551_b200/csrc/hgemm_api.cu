@@ -446,10 +446,14 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
         // give back stages until it fits
         const int unit = 64 * hgemm_host::cta_group_of(cfg);
         cfg.block_n = std::min(256, (cfg.block_n + unit - 1) / unit * unit);
-        cfg.stages = std::min(cfg.stages, hgemm_host::max_stages(cfg.family, cfg.block_n, cfg.block_k));
+        cfg.stages = std::min(cfg.stages, hgemm_host::max_stages_of(cfg));       // with this epilogue's store staging
         if (cfg.stages < 1) {
             cfg.block_k = 64;
-            cfg.stages = std::min(4, hgemm_host::max_stages(cfg.family, cfg.block_n, 64));
+            cfg.stages = std::min(4, hgemm_host::max_stages_of(cfg));
+        }
+        if (cfg.stages < 1) {                                                     // the wide epilogue's staging is what does not fit
+            cfg.epilogue = HGEMM_EPILOGUE_TMA;
+            cfg.stages = std::min(4, hgemm_host::max_stages_of(cfg));
         }
         if (cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 && ((cfg.block_n / cfg.tail_split) % unit) != 0) {
             cfg.tail_split = 0;

@@ -670,3 +670,19 @@ def test_plan_autotune_on_nn_layout_skips_unsupported_candidates(ctx, gu):
     assert us > 0.0
     gu.assert_close_full(C, A, B, f"autotuned NN {plan.config.as_dict()}")
     plan.close()
+
+
+def test_every_grid_shape_plans_in_both_layouts(ctx):
+    """hgemm_plan / hgemm_plan_layout accept all 729 grid shapes: the NN layout adapts the tabulated configuration
+    (whole 64-column blocks per CTA, fewer stages with the planned epilogue's staging) and must end up legal."""
+    grid = [64, 128, 256, 512, 1024, 2048, 4096, 8192, 12288]
+    for M in grid:
+        for N in grid:
+            for K in grid:
+                for layout in (hgemm.LAYOUT_TN, hgemm.LAYOUT_NN):
+                    plan = ctx.plan(M, N, K, layout)
+                    c = plan.config
+                    assert hgemm.validate_config(M, N, K, c) == hgemm.OK, (M, N, K, layout, c.as_dict())
+                    if layout == hgemm.LAYOUT_NN:
+                        assert c.block_n % (64 * (c.family + 1)) == 0
+                    plan.close()

@@ -162,3 +162,4 @@ def test_candidate_configs_are_legal_ranked_and_distinct(lib):
     assert any(c.split_k > 1 and c.split_mode == 1 for c in pool) and any(c.split_k > 1 and c.split_mode == 0 for c in pool)
     assert any(c.epilogue == hgemm.EPILOGUE_TMA_WIDE for c in pool)
     assert hgemm.candidate_configs(0, 64, 64) == [] and hgemm.candidate_configs(64, 64, 1 << 30) == []
+
