@@ -130,7 +130,8 @@ typedef struct {
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the
- * device has compute capability 10.0.  Allocates a 4-byte device status word. */
+ * device has compute capability 10.0.  Allocates 16 KB of device status words
+ * (one for the context, one per live plan: at most 4095 plans at a time). */
 hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device);
 
 /* Free the context, every plan it still owns and their workspaces. */
@@ -187,29 +188,37 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
  * and calls no cudaMalloc, cudaFree or any other allocating routine.  The split-K
  * partial sums, the arrival counters and the status word live in one static device
  * array inside the library: 8 MiB of partial sums plus a 4 KiB control page, held by
- * every GPU that loads the library until the process exits.
+ * every GPU that loads the library until the process exits.  That array receives its
+ * memory when the CUDA runtime loads the library's module on the device: under
+ * CUDA's default lazy loading that is this function's FIRST call on the device,
+ * under CUDA_MODULE_LOADING=EAGER it is context creation.  Make that first call (or
+ * load eagerly) before memory is frozen; every later call leaves the amount of free
+ * device memory as it found it.
  *
  * Same operation and layouts as hgemm_run (A: M x K, B: N x K, C: M x N, fp16, DEVICE
  * pointers, 16-byte aligned, caller-owned) on the calling thread's CURRENT device,
  * with the 1-CTA kernel family, tile width `block_n` (multiple of 32 in [32, 256]),
  * 64-wide K stages and `split_k` K slices summed in slice order through that array
- * (split_k == 1 is allowed and uses no scratch).  Asynchronous on `stream`.
+ * (split_k == 1 is allowed; it neither reads nor writes the array).  Asynchronous on
+ * `stream`.
  *
  * Limits and errors, checked before anything is launched:
  *   - ceil(M/128) * ceil(N/block_n) * split_k * 128 * block_n * 4 bytes of partial sums
  *     must fit in 8 MiB and the tile count in the control page (at most 480 tiles),
  *     else HGEMM_ERR_SCRATCH_LIMIT;
- *   - split_k <= min(64, ceil(K/64), SM count); shape rules as for hgemm_plan, else
- *     HGEMM_ERR_UNSUPPORTED / HGEMM_ERR_INVALID_ARG; HGEMM_ERR_ARCH off sm_100.
+ *   - split_k <= min(64, ceil(K/64), SM count); K % 8 == 0 and N % 8 == 0 (no padded
+ *     copies can be made here); otherwise as for hgemm_plan: HGEMM_ERR_UNSUPPORTED /
+ *     HGEMM_ERR_INVALID_ARG; HGEMM_ERR_ARCH off sm_100.
  *
- * The first call on each device looks up the array's device address
- * (cudaGetSymbolAddress) and sets the kernel's shared-memory limit; make that first
- * call before any stream capture begins.  Every call shares the one array, which
- * keeps the previous call's contents: the function clears the control page on
- * `stream` before each launch (the partial sums need no clearing), and two calls that
- * overlap on the GPU -- different streams, or different threads -- race on it.
- * Serialise them.  A bounded wait that runs out leaves C undefined; this variant has
- * no status read-back. */
+ * The first call on each device also looks up the array's device address
+ * (cudaGetSymbolAddress) and sets the kernel's shared-memory limit; make it before any
+ * stream capture begins.  That set-up is serialised inside the library, so first calls
+ * from several threads are safe as far as the set-up goes.  Every call with
+ * split_k > 1 shares the one array, which keeps the previous call's contents: the
+ * function clears the control page on `stream` before each such launch (the partial
+ * sums need no clearing), and two such calls that overlap on the GPU -- different
+ * streams, or different threads -- race on it.  Serialise them.  A bounded wait that
+ * runs out leaves C undefined; this variant has no status read-back. */
 hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t K, int32_t block_n, int32_t split_k,
                                        const void *A, const void *B, void *C, void *stream);
 
@@ -219,7 +228,8 @@ hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan);
 /* Read / override the plan's configuration (tuner, tests).  set_config returns
  * HGEMM_ERR_UNSUPPORTED, leaving the plan unchanged, if the configuration is
  * illegal for the shape or does not fit shared/tensor memory; it may reallocate
- * the workspace (synchronising). */
+ * the workspace (synchronising).  If that allocation fails it returns
+ * HGEMM_ERR_ALLOC and the plan keeps its configuration and buffers and still runs. */
 hgemm_status_t hgemm_plan_get_config(const hgemm_plan_t *plan, hgemm_config_t *out);
 hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *cfg);
 
@@ -233,7 +243,7 @@ hgemm_status_t hgemm_plan_set_config(hgemm_plan_t *plan, const hgemm_config_t *c
  * DEVICE pointers laid out as for hgemm_run; C is overwritten (no alpha / beta).
  * *best_us (HOST, may be NULL) receives the installed configuration's time per
  * call in microseconds.  Synchronous: it waits for the stream, many times, and may
- * reallocate the workspace.  It reads and clears the context's device status; if a
+ * reallocate the workspace.  It reads and clears the plan's device status; if a
  * bounded wait ran out during the search the plan keeps the configuration it had
  * and HGEMM_ERR_TIMEOUT is returned.  Candidates the plan's layout does not
  * support are skipped.  Costs about (max_candidates + 1) x 0.3-1 ms. */
@@ -270,11 +280,22 @@ int64_t hgemm_config_workspace_bytes(int64_t M, int64_t N, int64_t K, const hgem
 /* Number of kernels the last hgemm_run of this plan launched (1). */
 int32_t hgemm_plan_launches_per_run(const hgemm_plan_t *plan);
 
-/* Every device-side wait is bounded; when one runs out the kernel records
- * (role << 24 | barrier index << 8 | stage) in the context's status word, drains
- * and returns.  This call synchronises the device, reads the word into *code
- * (0 = no event), clears it, and returns HGEMM_ERR_TIMEOUT if it was non-zero. */
-hgemm_status_t hgemm_last_device_status(hgemm_ctx_t *ctx, uint32_t *code);
+/* Every device-side wait is bounded (the timing rules of paper section 2.4 presuppose calls that
+ * return); when one runs out the kernel records (role << 24 | barrier index << 8 | stage) in the
+ * status word of the plan whose launch it was, drains and returns.  Each plan has its own word, so
+ * two plans running on two streams can tell whose wait ran out.
+ *
+ * hgemm_last_device_status(plan, code): synchronises the device, reads the plan's word into *code
+ * (HOST pointer; 0 = no event), clears it, and returns HGEMM_ERR_TIMEOUT if it was non-zero; in that
+ * case the plan's split-K arrival counters (no other plan's) are started again from zero, so the
+ * plan is usable afterwards.
+ *
+ * hgemm_ctx_last_device_status(ctx, code): the same over the whole context -- its own word (written
+ * by hgemm_debug_timeout_probe) and the word of every live plan; *code receives the first non-zero
+ * one (the context's, then plans in creation order), all are cleared, and every plan whose word was
+ * set has its counters restarted. */
+hgemm_status_t hgemm_last_device_status(hgemm_plan_t *plan, uint32_t *code);
+hgemm_status_t hgemm_ctx_last_device_status(hgemm_ctx_t *ctx, uint32_t *code);
 
 /* Wait budget of the bounded waits, in SM clock cycles (default 2e9, about a
  * second).  Affects plans created afterwards and later hgemm_run calls. */
@@ -290,7 +311,7 @@ hgemm_status_t hgemm_set_dependent_launch(hgemm_ctx_t *ctx, int32_t enabled);
 
 /* Test hook for the timeout path: launches one small kernel on `stream` whose
  * only wait is on a barrier that nothing signals, with the context's wait
- * budget.  The kernel returns by itself; hgemm_last_device_status then reports
+ * budget.  The kernel returns by itself; hgemm_ctx_last_device_status then reports
  * HGEMM_ERR_TIMEOUT.  Nothing faults or hangs. */
 hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
 
@@ -320,6 +341,13 @@ hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
  * 24 + 2 * 148 uint64.
  * 0 restores normal operation. */
 hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask);
+
+/* Test hook for the allocation-failure paths (an injected error code, no memory pressure on the
+ * GPU): of the device allocations the library makes through this context from now on -- split-K
+ * workspace and counters, padded operand copies, host-call staging -- the first `after` go
+ * through, the next `count` report failure without calling cudaMalloc, so the caller sees
+ * HGEMM_ERR_ALLOC.  count = 0 switches it off. */
+hgemm_status_t hgemm_debug_fail_allocs(hgemm_ctx_t *ctx, int32_t after, int32_t count);
 
 /* cudaError_t (as int) of the last failing CUDA call made through this context. */
 int32_t hgemm_last_cuda_error(const hgemm_ctx_t *ctx);

@@ -10,6 +10,8 @@ from .hgemm_oracle import (  # noqa: F401
     f64_to_f16_bits,
     hgemm_full,
     hgemm_f16acc_full,
+    f16acc_envelope,
+    f16_spacing,
     hgemm_scaled_full,
     hgemm_sampled,
     max_threads,

@@ -18,10 +18,16 @@ typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32
                                     const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Device status words: one array per context.  Slot 0 belongs to the context itself (the timeout probe), every
+// plan owns one of the others, so that a wait that ran out names the plan whose launch it was.
+constexpr int kStatusSlots = 4096;
+
 struct hgemm_ctx_s {
     int device = 0;
     int num_sms = 0;
-    uint32_t *d_status = nullptr;
+    uint32_t *d_status = nullptr;          // kStatusSlots words
+    std::vector<int> free_status_slots;    // slots no plan owns (never holds 0)
+    int pass_allocs = 0, fail_allocs = 0;  // test hook: after pass_allocs more device allocations, fail_allocs of them report failure
     long long wait_budget = 2000000000LL;
     encode_tiled_fn encode = nullptr;
     int last_cuda_error = 0;
@@ -48,6 +54,7 @@ struct hgemm_plan_s {
     uint32_t *counters = nullptr;
     int64_t counter_bytes = 0;
     uint32_t epoch = 0;            // launches that have used `counters` since they were last cleared
+    int status_slot = 0;           // this plan's word in the context's status array
     // tensor maps depend on the pointers: a small cache keyed by (A, B, C), round-robin replacement
     struct MapEntry {
         const void *a = nullptr, *b = nullptr;
@@ -69,6 +76,21 @@ hgemm_status_t cuda_fail(hgemm_ctx_s *ctx, cudaError_t e)
     if (ctx) ctx->last_cuda_error = int(e);
     (void)cudaGetLastError();
     return HGEMM_ERR_CUDA;
+}
+
+// Every device allocation of the library goes through here (hgemm_debug_fail_allocs can make it fail).
+cudaError_t ctx_malloc(hgemm_ctx_s *ctx, void **out, size_t bytes)
+{
+    if (ctx && ctx->fail_allocs > 0) {
+        if (ctx->pass_allocs > 0) {
+            --ctx->pass_allocs;
+        } else {
+            --ctx->fail_allocs;
+            *out = nullptr;
+            return cudaErrorMemoryAllocation;
+        }
+    }
+    return cudaMalloc(out, bytes);
 }
 
 int32_t pow2_at_least(int32_t x)
@@ -131,32 +153,49 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     const hgemm_host::SplitLayout layout = hgemm_host::split_layout(pl->M, pl->N, pl->K, ctx->num_sms, cfg);
     const int64_t ws = hgemm_host::workspace_bytes(pl->M, pl->N, pl->K, cfg, ctx->num_sms);
     const int64_t cb = hgemm_host::counter_bytes(pl->M, pl->N, cfg, ctx->num_sms, pl->K);
+    // Nothing of the plan changes until every step that can fail has succeeded: larger buffers are allocated
+    // beside the old ones and swapped in only then, so a failed call leaves a plan that still runs as before.
+    void *new_ws = nullptr;
+    uint32_t *new_ctr = nullptr;
     if (ws > pl->workspace_bytes) {
-        if (pl->workspace) cudaFree(pl->workspace);
-        pl->workspace = nullptr;
-        pl->workspace_bytes = 0;
-        cudaError_t e = cudaMalloc(&pl->workspace, size_t(ws));
+        cudaError_t e = ctx_malloc(ctx, &new_ws, size_t(ws));
         if (e != cudaSuccess) {
             cuda_fail(ctx, e);
             return HGEMM_ERR_ALLOC;
         }
-        pl->workspace_bytes = ws;
     }
     if (cb > pl->counter_bytes) {
-        if (pl->counters) cudaFree(pl->counters);
-        pl->counters = nullptr;
-        pl->counter_bytes = 0;
-        cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&pl->counters), size_t(cb));
+        cudaError_t e = ctx_malloc(ctx, reinterpret_cast<void **>(&new_ctr), size_t(cb));
         if (e != cudaSuccess) {
+            if (new_ws) cudaFree(new_ws);
             cuda_fail(ctx, e);
             return HGEMM_ERR_ALLOC;
         }
-        pl->counter_bytes = cb;
     }
-    if (pl->counters) {
-        cudaError_t e = cudaMemset(pl->counters, 0, size_t(pl->counter_bytes));
-        if (e != cudaSuccess) return cuda_fail(ctx, e);
-        pl->epoch = 0;
+    {
+        // arrival counters start from zero under a new configuration (harmless for the old one, whose next
+        // launch then counts from epoch 1 again)
+        uint32_t *ctr = new_ctr ? new_ctr : pl->counters;
+        const int64_t ctr_bytes = new_ctr ? cb : pl->counter_bytes;
+        if (ctr) {
+            cudaError_t e = cudaMemset(ctr, 0, size_t(ctr_bytes));
+            if (e != cudaSuccess) {
+                if (new_ws) cudaFree(new_ws);
+                if (new_ctr) cudaFree(new_ctr);
+                return cuda_fail(ctx, e);
+            }
+            pl->epoch = 0;
+        }
+    }
+    if (new_ws) {
+        if (pl->workspace) cudaFree(pl->workspace);
+        pl->workspace = new_ws;
+        pl->workspace_bytes = ws;
+    }
+    if (new_ctr) {
+        if (pl->counters) cudaFree(pl->counters);
+        pl->counters = new_ctr;
+        pl->counter_bytes = cb;
     }
 
     pl->cfg = cfg;
@@ -197,7 +236,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.b_row_major = pl->layout == HGEMM_LAYOUT_NN ? 1 : 0;
     p.workspace = static_cast<float *>(pl->workspace);
     p.counters = pl->counters;
-    p.status = ctx->d_status;
+    p.status = ctx->d_status + pl->status_slot;
     p.cluster_split = cluster_split ? 1 : 0;
     p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d && pl->layout == HGEMM_LAYOUT_TN) ? 1 : 0;
     p.C = nullptr;
@@ -324,17 +363,19 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             break;
         }
         ctx->encode = reinterpret_cast<encode_tiled_fn>(fn);
-        e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 256);
+        e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), kStatusSlots * sizeof(uint32_t));
         if (e != cudaSuccess) {
             cuda_fail(ctx, e);
             st = HGEMM_ERR_ALLOC;
             break;
         }
-        e = cudaMemset(ctx->d_status, 0, 256);
+        e = cudaMemset(ctx->d_status, 0, kStatusSlots * sizeof(uint32_t));
         if (e != cudaSuccess) {
             st = cuda_fail(ctx, e);
             break;
         }
+        ctx->free_status_slots.reserve(kStatusSlots);
+        for (int slot = kStatusSlots - 1; slot >= 1; --slot) ctx->free_status_slots.push_back(slot);
         // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, no K slices / workspace / cluster reduction
         for (int k = 0; k < 48 && e == cudaSuccess; ++k) {
             const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k / 12 >= 2, k / 12 == 1, k / 12 == 3 ? 2 : 1);
@@ -363,6 +404,7 @@ hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan)
     if (ctx) {
         auto it = std::find(ctx->plans.begin(), ctx->plans.end(), plan);
         if (it != ctx->plans.end()) ctx->plans.erase(it);
+        if (plan->status_slot > 0) ctx->free_status_slots.push_back(plan->status_slot);
     }
     if (plan->workspace) cudaFree(plan->workspace);
     if (plan->counters) cudaFree(plan->counters);
@@ -463,18 +505,20 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
             cfg.split_mode = HGEMM_SPLIT_WORKSPACE;   // the wider tile's partial sums no longer fit in shared memory
         if (hgemm_host::validate(M, N, Kp, cfg) != HGEMM_OK) return HGEMM_ERR_UNSUPPORTED;
     }
+    if (ctx->free_status_slots.empty()) return HGEMM_ERR_ALLOC;   // more live plans than status words
     hgemm_plan_s *pl = new (std::nothrow) hgemm_plan_s;
     if (!pl) return HGEMM_ERR_ALLOC;
     pl->layout = layout;
     pl->ctx = ctx;
+    pl->status_slot = ctx->free_status_slots.back();             // taken for good only when the plan is handed out
     pl->M = M;
     pl->N = N;
     pl->K = Kp;
     pl->K_user = K;
     if (Kp != K) {
         // rows of A and B are not multiples of 16 bytes: the kernels read zero-padded copies instead
-        cudaError_t e = cudaMalloc(&pl->pad_a, size_t(M) * size_t(Kp) * 2);
-        if (e == cudaSuccess) e = cudaMalloc(&pl->pad_b, size_t(N) * size_t(Kp) * 2);
+        cudaError_t e = ctx_malloc(ctx, &pl->pad_a, size_t(M) * size_t(Kp) * 2);
+        if (e == cudaSuccess) e = ctx_malloc(ctx, &pl->pad_b, size_t(N) * size_t(Kp) * 2);
         if (e != cudaSuccess) {
             if (pl->pad_a) cudaFree(pl->pad_a);
             cuda_fail(ctx, e);
@@ -491,6 +535,7 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
         delete pl;
         return s;
     }
+    ctx->free_status_slots.pop_back();
     ctx->plans.push_back(pl);
     *out = pl;
     return HGEMM_OK;
@@ -579,11 +624,12 @@ hgemm_status_t hgemm_plan_autotune(hgemm_plan_t *plan, const void *A, const void
     cudaEventDestroy(e1);
     // a wait that ran out during the search disqualifies the search, not the plan: back to where it started
     uint32_t code = 0;
-    if (result == HGEMM_OK && hgemm_last_device_status(ctx, &code) != HGEMM_OK) {
-        (void)hgemm_plan_set_config(plan, &start);
-        return HGEMM_ERR_TIMEOUT;
+    if (result == HGEMM_OK && hgemm_last_device_status(plan, &code) != HGEMM_OK) {
+        const hgemm_status_t back = hgemm_plan_set_config(plan, &start);
+        return back != HGEMM_OK ? back : HGEMM_ERR_TIMEOUT;
     }
-    const hgemm_status_t s = hgemm_plan_set_config(plan, result == HGEMM_OK ? &best : &start);
+    hgemm_status_t s = hgemm_plan_set_config(plan, result == HGEMM_OK ? &best : &start);
+    if (s != HGEMM_OK && result == HGEMM_OK) s = hgemm_plan_set_config(plan, &start);   // the plan never shrinks its buffers: this fits
     if (result != HGEMM_OK) return result;
     if (s != HGEMM_OK) return s;
     if (best_us) *best_us = best_ms * 1e3f;
@@ -725,9 +771,9 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
     const size_t a_bytes = size_t(plan->M) * size_t(plan->K_user) * 2, b_bytes = size_t(plan->N) * size_t(plan->K_user) * 2,
                  c_bytes = size_t(plan->M) * size_t(plan->N) * 2;
     if (!plan->stage_a) {
-        cudaError_t e = cudaMalloc(&plan->stage_a, a_bytes);
-        if (e == cudaSuccess) e = cudaMalloc(&plan->stage_b, b_bytes);
-        if (e == cudaSuccess) e = cudaMalloc(&plan->stage_c, c_bytes);
+        cudaError_t e = ctx_malloc(ctx, &plan->stage_a, a_bytes);
+        if (e == cudaSuccess) e = ctx_malloc(ctx, &plan->stage_b, b_bytes);
+        if (e == cudaSuccess) e = ctx_malloc(ctx, &plan->stage_c, c_bytes);
         if (e != cudaSuccess) {
             if (plan->stage_a) cudaFree(plan->stage_a);
             if (plan->stage_b) cudaFree(plan->stage_b);
@@ -762,27 +808,68 @@ hgemm_status_t hgemm_debug_set_skip(hgemm_plan_t *plan, uint32_t mask)
     return HGEMM_OK;
 }
 
-hgemm_status_t hgemm_last_device_status(hgemm_ctx_t *ctx, uint32_t *code)
+// A launch that gave up may have left the plan's split-K arrival counters part-way: start them again from zero.
+static hgemm_status_t reset_counters(hgemm_plan_s *pl)
+{
+    if (!pl->counters) return HGEMM_OK;
+    cudaError_t e = cudaMemset(pl->counters, 0, size_t(pl->counter_bytes));
+    if (e != cudaSuccess) return cuda_fail(pl->ctx, e);
+    pl->epoch = 0;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_last_device_status(hgemm_plan_t *plan, uint32_t *code)
+{
+    if (!plan || !code) return HGEMM_ERR_INVALID_ARG;
+    hgemm_ctx_s *ctx = plan->ctx;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    uint32_t v = 0;
+    uint32_t *word = ctx->d_status + plan->status_slot;
+    e = cudaMemcpy(&v, word, 4, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (v != 0) {
+        e = cudaMemset(word, 0, 4);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        const hgemm_status_t s = reset_counters(plan);
+        if (s != HGEMM_OK) return s;
+    }
+    *code = v;
+    return v ? HGEMM_ERR_TIMEOUT : HGEMM_OK;
+}
+
+hgemm_status_t hgemm_ctx_last_device_status(hgemm_ctx_t *ctx, uint32_t *code)
 {
     if (!ctx || !code) return HGEMM_ERR_INVALID_ARG;
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    uint32_t v = 0;
-    e = cudaMemcpy(&v, ctx->d_status, 4, cudaMemcpyDeviceToHost);
+    std::vector<uint32_t> words(size_t(kStatusSlots), 0u);
+    e = cudaMemcpy(words.data(), ctx->d_status, words.size() * sizeof(uint32_t), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    if (v != 0) {
-        e = cudaMemset(ctx->d_status, 0, 4);
+    uint32_t v = words[0];                                   // the context's own word first, then the plans' in creation order
+    bool any = v != 0;
+    for (hgemm_plan_s *pl : ctx->plans) {
+        const uint32_t w = words[size_t(pl->status_slot)];
+        if (w == 0) continue;
+        any = true;
+        if (v == 0) v = w;
+        const hgemm_status_t s = reset_counters(pl);
+        if (s != HGEMM_OK) return s;
+    }
+    if (any) {
+        e = cudaMemset(ctx->d_status, 0, words.size() * sizeof(uint32_t));
         if (e != cudaSuccess) return cuda_fail(ctx, e);
-        // a launch that gave up may have left split-K arrival counters part-way: start them again from zero
-        for (hgemm_plan_s *pl : ctx->plans) {
-            if (!pl->counters) continue;
-            e = cudaMemset(pl->counters, 0, size_t(pl->counter_bytes));
-            if (e != cudaSuccess) return cuda_fail(ctx, e);
-            pl->epoch = 0;
-        }
     }
     *code = v;
     return v ? HGEMM_ERR_TIMEOUT : HGEMM_OK;
+}
+
+hgemm_status_t hgemm_debug_fail_allocs(hgemm_ctx_t *ctx, int32_t after, int32_t count)
+{
+    if (!ctx || after < 0 || count < 0) return HGEMM_ERR_INVALID_ARG;
+    ctx->pass_allocs = after;
+    ctx->fail_allocs = count;
+    return HGEMM_OK;
 }
 
 hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles)
@@ -802,7 +889,7 @@ hgemm_status_t hgemm_set_dependent_launch(hgemm_ctx_t *ctx, int32_t enabled)
 hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream)
 {
     if (!ctx) return HGEMM_ERR_INVALID_ARG;
-    hgemm_dev::hgemm_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, ctx->wait_budget);
+    hgemm_dev::hgemm_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, ctx->wait_budget);   // slot 0
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;

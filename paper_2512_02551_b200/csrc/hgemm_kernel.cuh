@@ -458,7 +458,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     // ---- roles ------------------------------------------------------------------------
     // Producer and MMA loops are executed by their whole warp with warp-uniform control flow (the
-    // wait results are voted), and only the single-thread instructions are predicated on lane 0:
+    // wait results are voted), and the single-thread instructions elect their lane inside the asm block:
     // TMA and tcgen05 instructions take their operands from uniform registers, so operands the
     // compiler can prove warp-uniform cost nothing to issue, while per-thread ones each need a move.
     bool tmem_freed = false;                       // warp 1: tensor memory was freed before the teardown
@@ -469,7 +469,6 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         uint32_t ph = 0;
         const uint32_t full_leader = (CTA_GROUP == 2) ? mapa(bar_full, leader_rank) : bar_full;
         const bool tr = (TRACE && p.trace != nullptr) && blockIdx.x == 0;
-        const uint32_t leader = (lane == 0) ? 1u : 0u;     // the lane that issues the loads
         long long t_wait = 0, t_work = 0;
         bool ok = true;
         bool dependencies_met = false;
@@ -506,65 +505,65 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const int32_t b_col = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
                     const int32_t blocks = (it.bn / CTA_GROUP) / 64;       // a column piece of a tail tile loads fewer blocks
                     const uint32_t tx = a_stage_bytes + static_cast<uint32_t>(subs * blocks) * (kSubK * 128u);
-                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
-                    else if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
-                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, tx);
+                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_elect(bar_full + 8 * s, tx);
+                    else if (is_leader) mbar_arrive_expect_tx_elect(bar_full + 8 * s, tx);
+                    else mbar_arrive_expect_tx_cluster_relaxed_elect(fb, tx);
                     for (int32_t sub = 0; sub < subs; ++sub) {
-                        if constexpr (CTA_GROUP == 1) tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
-                        else tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                        if constexpr (CTA_GROUP == 1) tma_load_2d_elect(a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                        else tma_load_2d_pair_elect(a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
                         for (int32_t nb = 0; nb < blocks; ++nb) {
                             const uint32_t dst = b_dst + sub * b_sub_bytes + nb * (kSubK * 128);
-                            if constexpr (CTA_GROUP == 1) tma_load_2d_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
-                            else tma_load_2d_pair_if(leader, dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
+                            if constexpr (CTA_GROUP == 1) tma_load_2d_elect(dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
+                            else tma_load_2d_pair_elect(dst, &tmap_b, b_col + nb * 64, k0 + sub * kSubK, fb);
                         }
                     }
                 } else if ((!PLAIN && it.bn != p.block_n)) {
                     // a column piece of a tail tile: its rows of B come through the narrower map `tmap_bt`, one box per
                     // 64-wide K sub-tile, each placed where the full-height box of that sub-tile would start
                     const uint32_t tx = a_stage_bytes + static_cast<uint32_t>(subs * (it.bn / CTA_GROUP)) * (kSubK * 2u);
-                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
-                    else if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, tx);
-                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, tx);
+                    if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_elect(bar_full + 8 * s, tx);
+                    else if (is_leader) mbar_arrive_expect_tx_elect(bar_full + 8 * s, tx);
+                    else mbar_arrive_expect_tx_cluster_relaxed_elect(fb, tx);
                     if (p.tma_3d) {
-                        if constexpr (CTA_GROUP == 1) tma_load_3d_if(leader, a_dst, &tmap_a, 0, a_row, k0 / kSubK, fb);
-                        else tma_load_3d_pair_if(leader, a_dst, &tmap_a, 0, a_row, k0 / kSubK, fb);
+                        if constexpr (CTA_GROUP == 1) tma_load_3d_elect(a_dst, &tmap_a, 0, a_row, k0 / kSubK, fb);
+                        else tma_load_3d_pair_elect(a_dst, &tmap_a, 0, a_row, k0 / kSubK, fb);
                     }
                     for (int32_t sub = 0; sub < subs; ++sub) {
                         if constexpr (CTA_GROUP == 1) {
-                            if (!p.tma_3d) tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
-                            tma_load_2d_if(leader, b_dst + sub * b_sub_bytes, &tmap_bt, k0 + sub * kSubK, b_row, fb);
+                            if (!p.tma_3d) tma_load_2d_elect(a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                            tma_load_2d_elect(b_dst + sub * b_sub_bytes, &tmap_bt, k0 + sub * kSubK, b_row, fb);
                         } else {
-                            if (!p.tma_3d) tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
-                            tma_load_2d_pair_if(leader, b_dst + sub * b_sub_bytes, &tmap_bt, k0 + sub * kSubK, b_row, fb);
+                            if (!p.tma_3d) tma_load_2d_pair_elect(a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                            tma_load_2d_pair_elect(b_dst + sub * b_sub_bytes, &tmap_bt, k0 + sub * kSubK, b_row, fb);
                         }
                     }
                 } else if (p.tma_3d) {
                     // one instruction per operand: dimension 2 of the map counts 64-wide K sub-tiles
                     const int32_t ksub = k0 / kSubK;
                     if constexpr (CTA_GROUP == 1) {
-                        mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
-                        tma_load_3d_if(leader, a_dst, &tmap_a, 0, a_row, ksub, bar_full + 8 * s);
-                        tma_load_3d_if(leader, b_dst, &tmap_b, 0, b_row, ksub, bar_full + 8 * s);
+                        mbar_arrive_expect_tx_elect(bar_full + 8 * s, stage_bytes);
+                        tma_load_3d_elect(a_dst, &tmap_a, 0, a_row, ksub, bar_full + 8 * s);
+                        tma_load_3d_elect(b_dst, &tmap_b, 0, b_row, ksub, bar_full + 8 * s);
                     } else {
-                        if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
-                        else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, stage_bytes);
-                        tma_load_3d_pair_if(leader, a_dst, &tmap_a, 0, a_row, ksub, fb);
-                        tma_load_3d_pair_if(leader, b_dst, &tmap_b, 0, b_row, ksub, fb);
+                        if (is_leader) mbar_arrive_expect_tx_elect(bar_full + 8 * s, stage_bytes);
+                        else mbar_arrive_expect_tx_cluster_relaxed_elect(fb, stage_bytes);
+                        tma_load_3d_pair_elect(a_dst, &tmap_a, 0, a_row, ksub, fb);
+                        tma_load_3d_pair_elect(b_dst, &tmap_b, 0, b_row, ksub, fb);
                     }
                 } else if constexpr (CTA_GROUP == 1) {
-                    mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
+                    mbar_arrive_expect_tx_elect(bar_full + 8 * s, stage_bytes);
                     for (int32_t sub = 0; sub < subs; ++sub) {
-                        tma_load_2d_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, bar_full + 8 * s);
-                        tma_load_2d_if(leader, b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, bar_full + 8 * s);
+                        tma_load_2d_elect(a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, bar_full + 8 * s);
+                        tma_load_2d_elect(b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, bar_full + 8 * s);
                     }
                 } else {
                     // both CTAs of the pair announce their bytes on the leader's barrier; the peer's
                     // remote arrive is relaxed (it orders nothing: the data arrives through TMA)
-                    if (is_leader) mbar_arrive_expect_tx_if(leader, bar_full + 8 * s, stage_bytes);
-                    else mbar_arrive_expect_tx_cluster_relaxed_if(leader, fb, stage_bytes);
+                    if (is_leader) mbar_arrive_expect_tx_elect(bar_full + 8 * s, stage_bytes);
+                    else mbar_arrive_expect_tx_cluster_relaxed_elect(fb, stage_bytes);
                     for (int32_t sub = 0; sub < subs; ++sub) {
-                        tma_load_2d_pair_if(leader, a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
-                        tma_load_2d_pair_if(leader, b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, fb);
+                        tma_load_2d_pair_elect(a_dst + sub * kATileBytes, &tmap_a, k0 + sub * kSubK, a_row, fb);
+                        tma_load_2d_pair_elect(b_dst + sub * b_sub_bytes, &tmap_b, k0 + sub * kSubK, b_row, fb);
                     }
                 }
                 if (w == unit && kb == 0 && lane == 0) trace_stamp<!TRACE>(p, 2);
@@ -581,7 +580,6 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             uint32_t ph = 0;
             uint32_t local_tile = 0;
             const bool tr = (TRACE && p.trace != nullptr) && blockIdx.x == 0;
-            const uint32_t leader = (lane == 0) ? 1u : 0u; // the lane that issues every MMA and commit
             long long t_wait = 0, t_issue = 0, t_commit = 0, t_acc = 0, n_kb = 0;
             const uint64_t desc_a0 = make_smem_desc_sw128(smem_base);
             // B tile: K-major (B stored N x K) or N-major in 64-column blocks of 64 k-rows (B stored K x N)
@@ -625,14 +623,14 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                             for (int k = 0; k < kSubK / kUmmaK; ++k) {
                                 // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
-                                umma_f16_if<CTA_GROUP>(leader, d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, idesc,
+                                umma_f16_elect<CTA_GROUP>(d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, idesc,
                                                        (kb | sub | k) != 0 ? 1u : 0u);
                             }
                         }
                     }
                     const long long c2 = tr ? clock64() : 0;
                     // free the stage (in both CTAs of a pair) once these MMAs have read it
-                    umma_commit_if<CTA_GROUP>(leader, bar_empty + 8 * s, leader_rank);
+                    umma_commit_elect<CTA_GROUP>(bar_empty + 8 * s, leader_rank);
                     if (tr) { t_wait += c1 - c0; t_issue += c2 - c1; t_commit += clock64() - c2; ++n_kb; }
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
@@ -641,7 +639,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 else run_k_blocks(p.idesc_tail);
                 if (!ok) break;
                 if (w == unit && lane == 0) trace_stamp<!TRACE>(p, 4);
-                umma_commit_if<CTA_GROUP>(leader, bar_tmem_full + 8 * acc, leader_rank);
+                umma_commit_elect<CTA_GROUP>(bar_tmem_full + 8 * acc, leader_rank);
             }
             if (tr && lane == 0) { p.trace[8] = t_wait; p.trace[9] = t_issue; p.trace[10] = t_commit; p.trace[13] = t_acc; p.trace[15] = n_kb; }
             if constexpr (CTA_GROUP == 1) {

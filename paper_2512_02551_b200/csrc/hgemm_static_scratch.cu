@@ -5,11 +5,19 @@
 // fixed-footprint policy where every byte of HBM was handed out at start-up.  hgemm_plan needs
 // cudaMalloc for the split-K workspace, so those callers could never use split-K.  This entry point
 // gives them the same kernel with the workspace, the arrival counters and the status word placed in
-// one file-scope __device__ array: no context, no plan, no allocation of any kind.
+// one file-scope __device__ array: no context, no plan, and no call to cudaMalloc, cudaFree or any
+// other allocating routine.  The array itself gets its memory when the CUDA runtime loads this
+// file's module on a device -- with lazy module loading (CUDA's default) that is the first call of
+// this entry point on that device, with CUDA_MODULE_LOADING=EAGER it is context creation.  A process
+// whose memory is frozen later should therefore make one call per device (or load eagerly) before
+// the freeze; every later call leaves the amount of free device memory unchanged.
 //
 // Cost and limits: every GPU that loads the library holds the array (kScratchBytes + one control
 // page) until the process exits; a call whose partial sums need more than that is refused; all
 // calls share the one array, so two calls that overlap on the GPU would corrupt each other.
+// Every system header that hgemm_kernel.cuh and ptx_sm100.cuh include is included here first, at
+// global scope: the kernel header is pulled in inside an anonymous namespace below, and a system
+// header first seen there would declare its names (std:: among them) inside that namespace.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -17,12 +25,18 @@
 
 #include <algorithm>
 #include <cstring>
+#include <mutex>
+#include <type_traits>
 
 #include "../../include/hgemm.h"
 #include "hgemm_planner.h"
 
-// This translation unit gets its own, internal-linkage copy of the kernel (the other copy lives in
-// hgemm_api.cu): the array below has to be in the same file as the code that resolves its address.
+// This translation unit compiles its own, internal-linkage copy of the one kernel instantiation it
+// launches (the library's other copy lives in hgemm_api.cu).  The kernel does not need it -- it
+// receives the scratch address through its parameters like any workspace -- but it keeps this entry
+// point self-contained: the array, the code that resolves its device address and the launch that
+// uses it sit in one file, and nothing in the plan-based code path changed when it was added.  The
+// price is a second compile of that instantiation and a duplicate of it in the binary.
 namespace {
 #include "hgemm_kernel.cuh"
 } // namespace
@@ -49,6 +63,7 @@ struct DeviceState {
     encode_tiled_fn encode = nullptr;
 };
 DeviceState g_devices[kMaxDevices];     // fixed table: no heap allocation on any path
+std::mutex g_setup_mutex;               // first calls from several threads fill the table one at a time
 
 // Once per device, with that device current: resolve the array's device address, read the SM
 // count, fetch the tensor-map encoder, raise the kernel's shared-memory limit.  None of these
@@ -57,6 +72,7 @@ hgemm_status_t setup_device(int device, DeviceState **out)
 {
     if (device < 0 || device >= kMaxDevices) return HGEMM_ERR_INVALID_ARG;
     DeviceState &d = g_devices[device];
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!d.ready) {
         int major = 0, minor = 0;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
@@ -159,9 +175,10 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
         return HGEMM_ERR_CUDA;
 
     // The array keeps whatever the last call left.  The partial sums need no clearing (every slot
-    // that is read is written first); the counters and the status word must start at zero.
+    // that is read is written first); the counters and the status word must start at zero.  Without
+    // K slices the kernel touches neither, and the array is left alone.
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(d->scratch, 0, kControlBytes, s) != cudaSuccess) {
+    if (split_k > 1 && cudaMemsetAsync(d->scratch, 0, kControlBytes, s) != cudaSuccess) {
         (void)cudaGetLastError();
         return HGEMM_ERR_CUDA;
     }

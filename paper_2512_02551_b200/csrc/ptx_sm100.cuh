@@ -353,107 +353,105 @@ __device__ __forceinline__ void tmem_ld_wait()
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// ---- predicated single-thread forms ------------------------------------------------------
-// The same instructions, executed by the whole warp in convergent code with a per-thread
-// predicate (true in one lane).  Predicating inside the asm block instead of branching in C++
-// keeps the surrounding code warp-uniform, so the compiler can hold the operands (descriptors,
-// barrier and shared-memory addresses, coordinates) in uniform registers, where TMA and tcgen05
-// instructions read them, instead of moving them there before every instruction.
+// ---- elected single-thread forms -----------------------------------------------------------
+// The same instructions, executed by the whole (converged) warp: `elect.sync` picks one lane inside
+// the asm block and only that lane issues.  Electing inside the block instead of branching on a
+// lane index in C++ keeps the surrounding code warp-uniform, so the compiler can hold the operands
+// (descriptors, barrier and shared-memory addresses, coordinates) in uniform registers, where TMA
+// and tcgen05 instructions read them, instead of moving them there before every instruction.
+// All 32 lanes must call these together.
 
-__device__ __forceinline__ void mbar_arrive_expect_tx_if(uint32_t pred, uint32_t bar, uint32_t bytes)
+__device__ __forceinline__ void mbar_arrive_expect_tx_elect(uint32_t bar, uint32_t bytes)
 {
     asm volatile(
         "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
-        "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t}"
-        ::"r"(pred), "r"(bar), "r"(bytes) : "memory");
+        "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}"
+        ::"r"(bar), "r"(bytes) : "memory");
 }
 
-__device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed_if(uint32_t pred, uint32_t cluster_bar, uint32_t bytes)
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster_relaxed_elect(uint32_t cluster_bar, uint32_t bytes)
 {
     asm volatile(
         "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
-        "@e mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%1], %2;\n\t}"
-        ::"r"(pred), "r"(cluster_bar), "r"(bytes) : "memory");
+        "@e mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;\n\t}"
+        ::"r"(cluster_bar), "r"(bytes) : "memory");
 }
 
-__device__ __forceinline__ void tma_load_2d_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
+__device__ __forceinline__ void tma_load_2d_elect(uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
 {
     asm volatile(
         "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
-        "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%1], [%2, {%3, %4}], [%5];\n\t}"
-        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+        "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n\t}"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
 
-__device__ __forceinline__ void tma_load_2d_pair_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
+__device__ __forceinline__ void tma_load_2d_pair_elect(uint32_t dst, const void *tmap, int32_t x, int32_t y, uint32_t bar)
 {
     asm volatile(
         "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
         "@e cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-        " [%1], [%2, {%3, %4}], [%5];\n\t}"
-        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
+        " [%0], [%1, {%2, %3}], [%4];\n\t}"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
 
 // 3-D forms (dimension 2 selects the 64-wide K sub-tile): one instruction fills a whole 128-wide stage.
-__device__ __forceinline__ void tma_load_3d_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y, int32_t z,
-                                               uint32_t bar)
+__device__ __forceinline__ void tma_load_3d_elect(uint32_t dst, const void *tmap, int32_t x, int32_t y, int32_t z, uint32_t bar)
 {
     asm volatile(
         "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
-        "@e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%1], [%2, {%3, %4, %5}], [%6];\n\t}"
-        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
+        "@e cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];\n\t}"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
 
-__device__ __forceinline__ void tma_load_3d_pair_if(uint32_t pred, uint32_t dst, const void *tmap, int32_t x, int32_t y,
-                                                    int32_t z, uint32_t bar)
+__device__ __forceinline__ void tma_load_3d_pair_elect(uint32_t dst, const void *tmap, int32_t x, int32_t y, int32_t z, uint32_t bar)
 {
     asm volatile(
         "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
         "@e cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-        " [%1], [%2, {%3, %4, %5}], [%6];\n\t}"
-        ::"r"(pred), "r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
+        " [%0], [%1, {%2, %3, %4}], [%5];\n\t}"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
 
 template <int CTA_GROUP>
-__device__ __forceinline__ void umma_f16_if(uint32_t pred, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate)
+__device__ __forceinline__ void umma_f16_elect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
     if constexpr (CTA_GROUP == 1)
         asm volatile(
-            "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-            "@e tcgen05.mma.cta_group::1.kind::f16 [%1], %2, %3, %4, p;\n\t}"
-            ::"r"(pred), "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
     else
         asm volatile(
-            "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-            "@e tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %4, p;\n\t}"
-            ::"r"(pred), "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            "{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "@e tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
             : "memory");
 }
 
 // For a CTA pair the arrival goes to the barrier at the same shared-memory offset in both CTAs of the
 // pair: two plain commits, one per CTA (addresses from mapa), both tracking the same MMAs.
 template <int CTA_GROUP>
-__device__ __forceinline__ void umma_commit_if(uint32_t pred, uint32_t bar, uint32_t leader_rank)
+__device__ __forceinline__ void umma_commit_elect(uint32_t bar, uint32_t leader_rank)
 {
     if constexpr (CTA_GROUP == 1) {
         asm volatile(
             "{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
-            "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%1];\n\t}"
-            ::"r"(pred), "r"(bar) : "memory");
+            "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+            ::"r"(bar) : "memory");
     } else {
         // the pair's CTAs have the cluster ranks leader_rank and leader_rank + 1
         asm volatile(
             "{\n\t.reg .pred e;\n\t.reg .b32 r0, r1, k1;\n\telect.sync _|e, 0xffffffff;\n\t"
-            "add.u32 k1, %2, 1;\n\t"
-            "mapa.shared::cluster.u32 r0, %1, %2;\n\tmapa.shared::cluster.u32 r1, %1, k1;\n\t"
+            "add.u32 k1, %1, 1;\n\t"
+            "mapa.shared::cluster.u32 r0, %0, %1;\n\tmapa.shared::cluster.u32 r1, %0, k1;\n\t"
             "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [r0];\n\t"
             "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [r1];\n\t}"
-            ::"r"(pred), "r"(bar), "r"(leader_rank) : "memory");
+            ::"r"(bar), "r"(leader_rank) : "memory");
     }
 }
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_plan_autotune", "hgemm_candidate_configs", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
-    "hgemm_last_device_status", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
+    "hgemm_last_device_status", "hgemm_ctx_last_device_status", "hgemm_debug_fail_allocs", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
 ]
 
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
             "hgemm_config_workspace_bytes": (i64, [i64, i64, i64, cfgp]),
             "hgemm_plan_launches_per_run": (i32, [p]),
             "hgemm_last_device_status": (i32, [p, ctypes.POINTER(ctypes.c_uint32)]),
+            "hgemm_ctx_last_device_status": (i32, [p, ctypes.POINTER(ctypes.c_uint32)]),
+            "hgemm_debug_fail_allocs": (i32, [p, i32, i32]),
             "hgemm_set_wait_budget": (i32, [p, i64]),
             "hgemm_set_dependent_launch": (i32, [p, i32]),
             "hgemm_debug_timeout_probe": (i32, [p, p]),
@@ -191,10 +193,14 @@ class Context:
         _check(lib().hgemm_set_dependent_launch(self._h, 1 if enabled else 0), "hgemm_set_dependent_launch")
 
     def last_device_status(self) -> tuple[int, int]:
-        """(status, code); synchronises the device."""
+        """``hgemm_ctx_last_device_status``: (status, code) over the context's own status word and those of
+        all its live plans; synchronises the device."""
         code = ctypes.c_uint32(0)
-        st = lib().hgemm_last_device_status(self._h, ctypes.byref(code))
+        st = lib().hgemm_ctx_last_device_status(self._h, ctypes.byref(code))
         return int(st), int(code.value)
+
+    def debug_fail_allocs(self, after: int, count: int) -> None:
+        _check(lib().hgemm_debug_fail_allocs(self._h, int(after), int(count)), "hgemm_debug_fail_allocs")
 
     def debug_timeout_probe(self, stream: int = 0) -> None:
         _check(lib().hgemm_debug_timeout_probe(self._h, ctypes.c_void_p(stream)), "hgemm_debug_timeout_probe")
@@ -237,6 +243,12 @@ class Plan:
 
     def try_set_config(self, cfg: Config) -> int:
         return int(lib().hgemm_plan_set_config(self._h, ctypes.byref(cfg)))
+
+    def last_device_status(self) -> tuple[int, int]:
+        """``hgemm_last_device_status``: (status, code) of this plan's own status word; synchronises the device."""
+        code = ctypes.c_uint32(0)
+        st = lib().hgemm_last_device_status(self._h, ctypes.byref(code))
+        return int(st), int(code.value)
 
     @property
     def launches_per_run(self) -> int:

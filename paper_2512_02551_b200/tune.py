@@ -170,8 +170,18 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     plan.set_config(best)
     C.zero_()
     run()
-    ref = torch.matmul(A, B.T)
-    ok = bool(torch.allclose(C.float(), ref.float(), rtol=4e-3, atol=4e-3 * K ** 0.5))
+    # the winner must meet the library's own acceptance formula, |C - C_ref| <= 2^-10 |C_ref| + 1e-3 sqrt(K), here
+    # against an fp32 product of the same operands (the tuner is product code and may not use the test oracle)
+    ref32 = torch.matmul(A.float(), B.float().T) if M * N <= (1 << 26) else None
+    if ref32 is not None:
+        ok = bool(((C.float() - ref32).abs() <= 2.0 ** -10 * ref32.abs() + 1e-3 * K ** 0.5).all())
+    else:                                                   # large outputs: the first and last 2048 rows
+        ok = True
+        rows = max(1, min(M, (1 << 26) // N))
+        for r0 in (0, M - rows):
+            r32 = torch.matmul(A[r0:r0 + rows].float(), B.float().T)
+            ok = ok and bool(((C[r0:r0 + rows].float() - r32).abs() <= 2.0 ** -10 * r32.abs() + 1e-3 * K ** 0.5).all())
+    ref = torch.empty_like(C)
     n_ref = max(5, min(2000, int(0.25 / (best_t * 1e-3)))) if best_t > 0.08 else max(3, min(100, int(0.6 / max(best_t, 1e-3))))
     t_torch = statistics.median(batch_ms(lambda: torch.matmul(A, B.T, out=ref), n_ref, stream)
                                 for _ in range(1 if best_t > 0.08 else 3))
@@ -196,7 +206,7 @@ def write_table(rows, path):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--out", default="gpurun_out")
+    ap.add_argument("--out", default="tune_out", help="directory for tune.jsonl and hgemm_table.inc")
     ap.add_argument("--shapes", nargs="*")
     ap.add_argument("--top", type=int, default=20)
     ap.add_argument("--resume", action="store_true")

@@ -128,6 +128,58 @@ def test_bounded_wait_reports_timeout_and_context_survives(ctx, gu):
     gu.check_shape(ctx, 256, 256, 256, "uniform")
 
 
+def test_status_words_are_per_plan(ctx, gu):
+    """Each plan has its own status word: an event recorded in the context's word (the probe kernel's) is not
+    reported by a plan's query, and the context-wide query finds and clears it."""
+    p1, p2 = ctx.plan(256, 256, 256), ctx.plan(512, 256, 1024)
+    ctx.set_wait_budget(2_000_000)
+    ctx.debug_timeout_probe()
+    assert p1.last_device_status() == (hgemm.OK, 0)
+    assert p2.last_device_status() == (hgemm.OK, 0)
+    st, code = ctx.last_device_status()
+    assert st == hgemm.ERR_TIMEOUT and (code >> 24) == 4
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    ctx.set_wait_budget(2_000_000_000)
+    L = hgemm.lib()
+    code = ctypes.c_uint32(7)
+    assert L.hgemm_last_device_status(None, ctypes.byref(code)) == hgemm.ERR_INVALID_ARG and code.value == 7
+    assert L.hgemm_last_device_status(p1._h, None) == hgemm.ERR_INVALID_ARG
+    p1.close()
+    p2.close()
+
+
+def test_failed_allocation_leaves_the_plan_as_it_was(ctx, gu):
+    """hgemm_plan_set_config that cannot get its larger workspace (the failure is injected: an error code from
+    a stand-in for cudaMalloc) returns HGEMM_ERR_ALLOC and the plan keeps its configuration, its buffers and its
+    results."""
+    import oracle
+    M, N, K = 512, 512, 4096
+    A, B = inputs.make_ab(M, N, K, "int5", "cuda")
+    want = oracle.hgemm_full(inputs.bits(A), inputs.bits(B))
+    small = hgemm.Config.make(block_n=128, stages=4, split_k=2, raster_group=1, split_mode=hgemm.SPLIT_WORKSPACE)
+    # more tiles and more slices: both the workspace and the arrival counters have to grow
+    large = hgemm.Config.make(block_n=64, stages=4, split_k=8, raster_group=1, split_mode=hgemm.SPLIT_WORKSPACE)
+    C, _, plan = gu.run_gemm(ctx, A, B, small)
+    gu.assert_exact(C, want, "before the failed call")
+    before = plan.config.as_dict()
+    for after in (0, 1):                                # the workspace allocation fails; then the counters' one
+        ctx.debug_fail_allocs(after, 1)
+        assert plan.try_set_config(large) == hgemm.ERR_ALLOC
+        ctx.debug_fail_allocs(0, 0)
+        assert plan.config.as_dict() == before
+        C2, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+        gu.assert_exact(C2, want, "after the failed call")
+    plan.set_config(large)                              # and without the injected failure the larger one goes in
+    C3, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+    gu.assert_exact(C3, want, "larger configuration")
+    # a plan that cannot get its buffers at creation is not created
+    ctx.debug_fail_allocs(0, 1)
+    out = ctypes.c_void_p()
+    assert hgemm.lib().hgemm_plan(ctx._h, 200, 136, 77, ctypes.byref(out)) == hgemm.ERR_ALLOC and not out.value   # K % 8 != 0: padded copies
+    ctx.debug_fail_allocs(0, 0)
+    plan.close()
+
+
 def test_full_grid_default_plans(ctx, gu):
     """All 729 grid shapes with the plan the library picks: full-output oracle check up to 2048^3
     by volume, 4096 samples + one row + one column above."""

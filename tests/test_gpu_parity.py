@@ -524,12 +524,6 @@ def test_scaled_form_matches_oracle(ctx, gu, case):
 
 # ---- fp16 accumulators (the paper's other setting for fp16 inputs, section 1) ----------------------------------
 
-def _ulp16(x):
-    """Spacing of fp16 at |x| (2^-24 below the smallest normal)."""
-    ax = np.maximum(np.abs(x), 2.0 ** -14)
-    return 2.0 ** (np.floor(np.log2(ax)) - 10)
-
-
 F16ACC_CASES = [
     # family, bn, bk, stages, epilogue, tail pieces, M, N, K
     (F1, 128, 64, 4, TMA, 0, 128, 128, 128),
@@ -554,23 +548,25 @@ def test_fp16_accumulation(ctx, gu, case):
     assert bound <= 2048
     C, _, plan = gu.run_gemm(ctx, Ab, Bb, cfg)
     gu.assert_exact(C, oracle.hgemm_full(inputs.bits(Ab), inputs.bits(Bb)), f"fp16 accumulation, 0/1 operands {cfg.as_dict()}")
-    # random inputs against the model that rounds the running sum once per 16-wide K step: bit-identical
-    # except where the hardware's inexact inner sum lands on the other side of a rounding boundary
+    # Random inputs.  What is asserted is what holds for every schedule that rounds the running sum at most once
+    # per 16-wide K step (one MMA instruction) to one of its two fp16 neighbours: the envelope computed from the
+    # fp64 oracle's prefix sums.  No hardware-fitted model takes part in the verdict.
     A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
     C, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
-    model = oracle.f16_bits_to_f64(oracle.hgemm_f16acc_full(inputs.bits(A), inputs.bits(B)).ravel()).reshape(M, N)
+    exact, bound = oracle.f16acc_envelope(inputs.bits(A), inputs.bits(B))
     got = gu.bits_to_f64(gu.c_bits(C))
-    same = float(np.mean(got == model))
-    # a flipped rounding happens at the magnitude the running sum had at that step, which can be far above the
-    # final value's: measure deviations in units of the fp16 spacing at the largest magnitudes of the matrix
-    dev = np.abs(got - model) / _ulp16(2.0 * np.abs(model).max())
-    assert same >= 0.99, f"only {same:.4f} of the entries equal the model"
-    assert dev.max() <= 2.0, f"largest deviation from the model: {dev.max()} spacings of the largest magnitudes"
-    # and it is a different arithmetic from fp32 accumulation: the same plan with fp32 accumulators
-    # meets the contract, whose bound fp16 accumulation exceeds once K is large
-    exact = oracle.hgemm_full(inputs.bits(A), inputs.bits(B))
+    err = np.abs(got - exact)
+    assert np.isfinite(got).all()
+    assert (err <= bound).all(), f"outside the fp16-accumulation envelope: worst {float((err / bound).max()):.3f} of it"
+    # Reported, never asserted: how much of the result equals the schedule "one round-to-nearest per MMA step"
+    model = oracle.f16_bits_to_f64(oracle.hgemm_f16acc_full(inputs.bits(A), inputs.bits(B)).ravel()).reshape(M, N)
+    print(f"fp16 accumulation {M}x{N}x{K}: {float(np.mean(got == model)):.4f} of the entries equal the per-step "
+          f"round-to-nearest model; worst error {float((err / bound).max()):.3f} of the envelope")
+    # and it is a different arithmetic from fp32 accumulation: once K is large its relative Frobenius error is
+    # above the 2^-11 that fp32 accumulators must stay under (they leave one final rounding, about 2^-12.2; K / 16
+    # roundings of the running sum leave about 2^-9 at K = 1024); the same plan with fp32 accumulators meets the contract
     if K >= 1024:
-        assert np.abs(got - exact).max() > np.abs(model - exact).max() * 0.25
+        assert np.sqrt((err ** 2).sum() / (exact ** 2).sum()) > 2.0 ** -11
     cfg32 = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=epi, block_k=bk,
                               tail_split=pieces, tail_mode=hgemm.TAIL_N if pieces else hgemm.TAIL_K)
     C32, _, _ = gu.run_gemm(ctx, A, B, cfg32, plan=plan)

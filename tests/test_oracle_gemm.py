@@ -246,3 +246,116 @@ def test_f16_accumulation_error_grows_with_k(oracle_lib):
     half_ulp = 2.0 ** -7                       # half the fp16 spacing at the largest running magnitudes (32..64)
     assert err.max() > 2.0 ** -11 * np.abs(exact).max()          # worse than one final rounding
     assert err.max() < (K / 16) * half_ulp                       # far inside the worst case
+
+
+# ---- the envelope that fp16 accumulation is held to: valid for every faithful rounding schedule -----------------
+
+def test_f16_spacing_is_the_ieee_spacing(oracle_lib):
+    """Against numpy's own float16 spacing on every finite non-negative fp16 value."""
+    bits = np.arange(0, 0x7C00, dtype=np.uint16)
+    vals = bits.view(np.float16)
+    with np.errstate(over="ignore"):
+        want = np.spacing(vals).astype(np.float64)
+    # np.spacing at the largest finite value overflows to inf in float16: the spacing there is 32
+    want[-1] = 32.0
+    assert np.array_equal(oracle_lib.f16_spacing(vals.astype(np.float64)), want)
+
+
+def _neighbours16(x):
+    """The two fp16 values that enclose the real number x (equal when x is representable)."""
+    h = np.float16(x)
+    if float(h) == x:
+        return float(h), float(h)
+    other = np.nextafter(h, np.float16(np.inf) if float(h) < x else np.float16(-np.inf))
+    lo, hi = sorted((float(h), float(other)))
+    assert lo < x < hi
+    return lo, hi
+
+
+@pytest.mark.parametrize("dist,K", [("uniform", 64), ("uniform", 512), ("int5", 2048), ("normal", 256)])
+def test_f16acc_envelope_holds_for_every_faithful_schedule(oracle_lib, dist, K):
+    """Brute force on small problems: run the accumulation in python floats under adversarial roundings --
+    always up, always down, away from the exact prefix, to nearest, random -- and with rounding every 16, 32
+    or 64 columns or once at the end; every result must lie inside the envelope computed for steps of 16."""
+    M, N = 3, 4
+    a, b = inputs.make_ab(M, N, K, dist=dist)
+    af, bf = _f16_exact(inputs.bits(a)), _f16_exact(inputs.bits(b))
+    exact, bound = oracle_lib.f16acc_envelope(inputs.bits(a), inputs.bits(b))
+    assert np.allclose(exact, af @ bf.T, rtol=1e-13, atol=0)
+    rng = np.random.default_rng(7)
+    worst = 0.0
+    for every in (16, 32, 64, K):
+        for policy in ("up", "down", "away", "nearest", "random"):
+            for i in range(M):
+                for j in range(N):
+                    d, prefix = 0.0, 0.0
+                    for k0 in range(0, K, every):
+                        s = float(np.dot(af[i, k0:k0 + every], bf[j, k0:k0 + every]))   # exact: few short products
+                        prefix += s
+                        lo, hi = _neighbours16(d + s)
+                        if policy == "up":
+                            d = hi
+                        elif policy == "down":
+                            d = lo
+                        elif policy == "away":
+                            d = hi if hi - prefix >= prefix - lo else lo
+                        elif policy == "nearest":
+                            d = float(np.float16(d + s))
+                        else:
+                            d = hi if rng.random() < 0.5 else lo
+                    e = abs(d - exact[i, j])
+                    assert e <= bound[i, j], (every, policy, i, j, e, bound[i, j])
+                    worst = max(worst, e / bound[i, j])
+    if dist == "int5":
+        assert worst == 0.0      # every partial sum is a small integer: nothing is ever rounded
+    else:
+        assert worst > 0.05      # the envelope is not vacuous: adversarial schedules come within sight of it
+
+
+def test_f16acc_envelope_on_the_hand_made_row(oracle_lib):
+    """2048 + 1 + 1 over three steps: round-to-nearest-even loses both ones (error 2), rounding up gains
+    two (2052); the envelope must admit both and is a handful of spacings wide, not more."""
+    K = 48
+    a = np.zeros((1, K), dtype=np.float16); b = np.zeros((1, K), dtype=np.float16)
+    a[0, :16] = 32.0; b[0, :16] = 4.0
+    a[0, 16] = 1.0; b[0, 16] = 1.0
+    a[0, 32] = 1.0; b[0, 32] = 1.0
+    exact, bound = oracle_lib.f16acc_envelope(a.view(np.uint16), b.view(np.uint16))
+    assert exact[0, 0] == 2050.0
+    assert 2.0 <= bound[0, 0] <= 6.0          # spacing 1 below 2048 once, then spacing 2 twice: 1 + 2 + 2 = 5
+
+
+# ---- IEEE special values through the loop ------------------------------------------------------------------------
+
+def test_infinities_and_nan_propagate_as_ieee_says(oracle_lib):
+    """Three hand-written rows of A against three of B (K = 4); the expected values are IEEE 754's own:
+    inf * finite = inf with the product's sign, inf * 0 = NaN, inf - inf = NaN, NaN absorbs everything,
+    and finite sums beyond 65504 + 16 round to infinity only in the fp16 encoding, not in the fp64 result."""
+    inf, nan = np.inf, np.nan
+    A = np.array([[inf, 1.0, 2.0, 0.0],
+                  [-inf, 0.0, 0.0, 3.0],
+                  [nan, 1.0, 1.0, 1.0]], dtype=np.float16)
+    B = np.array([[1.0, 1.0, 1.0, 1.0],        # row 0: +inf, row 1: -inf, row 2: NaN
+                  [0.0, 5.0, 5.0, 5.0],        # inf * 0 = NaN for rows 0 and 1, NaN for row 2
+                  [-2.0, 60000.0, 60000.0, 0.0]],  # row 0: -inf + finite = -inf; row 1: +inf; row 2: NaN
+                 dtype=np.float16)
+    got = oracle_lib.hgemm_full(A.view(np.uint16), B.view(np.uint16))
+    want = np.array([[inf, nan, -inf],
+                     [-inf, nan, inf],
+                     [nan, nan, nan]])
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok], want[ok])
+    # inf - inf inside one dot product
+    A2 = np.array([[inf, -inf, 1.0, 1.0], [inf, inf, 1.0, 1.0]], dtype=np.float16)
+    B2 = np.array([[1.0, 1.0, 1.0, 1.0]], dtype=np.float16)
+    got2 = oracle_lib.hgemm_full(A2.view(np.uint16), B2.view(np.uint16))
+    assert np.isnan(got2[0, 0]) and got2[1, 0] == inf
+    # overflow belongs to the fp16 encoding: the fp64 sum is finite, its fp16 image is infinite
+    A3 = np.array([[60000.0, 60000.0, 0.0, 0.0]], dtype=np.float16)
+    B3 = np.array([[1.0, 1.0, 0.0, 0.0], [-1.0, -1.0, 0.0, 0.0], [1.0, 0.09, 0.0, 0.0]], dtype=np.float16)
+    got3 = oracle_lib.hgemm_full(A3.view(np.uint16), B3.view(np.uint16))
+    assert got3[0, 0] == 2.0 * float(np.float16(60000.0)) and np.isfinite(got3).all()
+    enc = oracle_lib.f64_to_f16_bits(got3.ravel())
+    assert enc[0] == 0x7C00 and enc[1] == 0xFC00                  # +inf, -inf
+    assert enc[2] == np.float16(got3[0, 2]).view(np.uint16) and enc[2] < 0x7C00   # about 65400: still finite
