@@ -1,16 +1,22 @@
 #!/usr/bin/env python
 """HGEMM benchmark: prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-grid]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-grid] [--grid-csv PATH]
 
 A "step" is one pass of the hot path over the square HGEMM sweep (M = N = K in
 {1024, 2048, 4096, 8192}: one plan/launch per shape, fp16 operands uniform in [-1, 1]
 seeded per shape, fp32 accumulation, fp16 result).  `value` is the whole-job TFLOP/s
 (flops of the sweep / device time, max over ranks) with inputs resident in HBM; `e2e` is the
 same metric through the host-buffer entry point with the copies inside the timed region.
-Extra keys: per-shape TFLOP/s beside torch.matmul on the same box, the 729-shape grid
-geomean against torch.matmul (single GPU only), the roofline of the dominant kernel, the CPU
-oracle timed on the machine's cores, and SM clocks sampled during the timed region.
+Extra keys: per-shape TFLOP/s beside torch.matmul on the same box; a sustained comparison (phases
+of about a second, ours and torch.matmul alternating, SM clock per phase); the 729-shape grid against
+torch.matmul (single GPU only) in four regimes -- warm back-to-back calls, cold L2 (buffer sets
+rotate), single calls after idle gaps, and the GPU-side duration of one call of each arm as the
+profiler records it, which leaves the host path out --; the memory-bound projection shapes against
+the HBM roofline; one line each for the row-major-B layout, the alpha/beta form and fp16
+accumulators; the roofline of the dominant kernel; the CPU oracle timed on the machine's cores; SM clocks
+sampled during the timed region.  The long per-shape arrays come first in the JSON line and the
+scalars last.
 
 Timing follows the paper's listing (section 2.4): synchronise, record an event, launch, record
 an event, synchronise; no side streams.  With N > 1 every rank runs the same sweep on its own
@@ -188,6 +194,11 @@ def run_ours(args) -> None:
     ctx = hgemm.Context(local)
     stream = torch.cuda.current_stream()
 
+    def check_status(where: str):
+        st, code = ctx.last_device_status()
+        if st != hgemm.OK:
+            raise SystemExit(f"device status {st} code {code:#x} after {where}")
+
     # ---- buffers: enough distinct (A, B, C) sets per shape that the footprint exceeds 2x L2 ----
     work = []
     for S in SWEEP:
@@ -213,6 +224,18 @@ def run_ours(args) -> None:
                 events.append((w["S"], e0, e1))
             else:
                 w["plan"].run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), stream.cuda_stream)
+
+    def torch_step(i, events=None):
+        for w in work:
+            A, B, C = w["bufs"][i % len(w["bufs"])]
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                torch.matmul(A, B.T, out=C)
+                e1.record(stream)
+                events.append((w["S"], e0, e1))
+            else:
+                torch.matmul(A, B.T, out=C)
 
     def timed(fn, steps, warmup, sampler=None, label="hgemm_timed_region"):
         for i in range(warmup):
@@ -240,9 +263,7 @@ def run_ours(args) -> None:
     events = []
     ms_total, t0w, t1w = timed(lambda i: one_step(i, events), args.steps, args.warmup, sampler)
     clocks = sampler.stop(t0w, t1w) if sampler else None
-    st, code = ctx.last_device_status()
-    if st != hgemm.OK:
-        raise SystemExit(f"device status {st} code {code:#x}")
+    check_status("the timed region")
     ms_per_step = ms_total / args.steps
     value = replicas.job_throughput(step_flops, world, ms_per_step) / 1e12
     per_launch = {}
@@ -254,7 +275,7 @@ def run_ours(args) -> None:
         per_shape[str(S)] = {"us": ms * 1e3, "tflops": flops(S, S, S) / (ms * 1e-3) / 1e12,
                              "config": work[SWEEP.index(S)]["plan"].config.as_dict()}
 
-    line = None
+    roofline = None
     if rank == 0:
         peaks = measured_peaks()
         dom = per_shape[str(SWEEP[-1])]
@@ -263,34 +284,23 @@ def run_ours(args) -> None:
         roofline = {"bound": "tensor", "kernel": "hgemm_umma_kernel, 8192^3 launch", "achieved": dom["tflops"], "peak": peak,
                     "unit": "TFLOP/s", "frac": dom["tflops"] / peak,
                     "peak_source": f"{peaks['source']} cuBLAS bf16 {'sustained' if timed_s > 1.0 else 'burst'} (fp16 dense = bf16 dense)",
-                    "traffic": DOMINANT_KERNEL_DRAM_BYTES, "algorithmic_flops_per_launch": flops(8192, 8192, 8192),
+                    "traffic": DOMINANT_KERNEL_DRAM_BYTES,
+                    "traffic_source": "one ncu capture of this launch, profiles/hgemm_umma_kernel_pair_8192x8192x8192.md; not measured in this run",
+                    "algorithmic_flops_per_launch": flops(8192, 8192, 8192),
                     "compulsory_bytes_per_launch": compulsory_bytes(8192, 8192, 8192),
                     "frac_of_spec_peak": dom["tflops"] / SPEC_TFLOPS}
 
     # ---- torch.matmul on the same buffers, same protocol (comparison point, single rank) --------
     torch_cmp = None
     if rank == 0:
-        def torch_step(i):
-            for w in work:
-                A, B, C = w["bufs"][i % len(w["bufs"])]
-                torch.matmul(A, B.T, out=C)
         tev = []
-
-        def torch_step_ev(i):
-            for w in work:
-                A, B, C = w["bufs"][i % len(w["bufs"])]
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
-                torch.matmul(A, B.T, out=C)
-                e1.record(stream)
-                tev.append((w["S"], e0, e1))
         for i in range(args.warmup):
             torch_step(i)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for i in range(args.steps):
-            torch_step_ev(args.warmup + i)
+            torch_step(args.warmup + i, tev)
         e1.record(stream)
         torch.cuda.synchronize()
         tms = e0.elapsed_time(e1) / args.steps
@@ -299,6 +309,12 @@ def run_ours(args) -> None:
             tps.setdefault(S, []).append(a.elapsed_time(b))
         torch_cmp = {"value": step_flops / (tms * 1e-3) / 1e12, "unit": "TFLOP/s",
                      "per_shape_tflops": {str(S): flops(S, S, S) / (statistics.mean(v) * 1e-3) / 1e12 for S, v in tps.items()}}
+
+    # ---- sustained comparison: phases of about a second under the power cap, arms alternating ----------
+    sustained = None
+    if rank == 0 and world == 1 and not args.no_grid:
+        sustained = sustained_report(torch, one_step, torch_step, step_flops, ms_per_step, local, stream)
+        check_status("the sustained phases")
 
     # ---- end to end: host buffers, copies inside the timed region --------------------------------
     host = []
@@ -329,14 +345,25 @@ def run_ours(args) -> None:
         assert torch.equal(hC, C.cpu()), "host-buffer path returned a different result"
     del host
 
+    variants = None
+    if rank == 0 and world == 1 and not args.no_grid:
+        variants = variant_lines(ctx, torch, hgemm, inputs, stream)
+        check_status("the variant lines")
+    for w in work:
+        w["plan"].close()
+    del work
+    torch.cuda.empty_cache()
+
     # ---- the 729-shape grid against torch.matmul (single GPU) ------------------------------------
     grid = None
     if rank == 0 and world == 1 and not args.no_grid:
-        grid = grid_sweep(ctx, torch, hgemm, inputs, stream)
+        grid = grid_sweep(ctx, torch, hgemm, inputs, stream, args.grid_csv)
+        check_status("the grid sweep")
 
     skinny = None
     if rank == 0 and world == 1 and not args.no_grid:
         skinny = skinny_report(ctx, torch, hgemm, inputs, stream)
+        check_status("the projection shapes")
 
     # ---- the CPU oracle on the machine's cores, on a bounded sample -------------------------------------
     cpu = None
@@ -352,15 +379,20 @@ def run_ours(args) -> None:
                "sample": f"first {rows} rows of C for 8192^3 ({rows * 8192 * 8192 / 1e9:.1f} GMAC, {dt:.2f} s wall)"}
 
     if rank == 0:
+        # long arrays first, scalars last: a reader that keeps only the end of the line keeps the figures
+        grid_detail = grid.pop("detail") if grid else None
+        skinny_shapes = skinny.pop("shapes") if skinny else None
         line = {
+            "skinny_shapes": skinny_shapes, "grid_detail": grid_detail, "per_shape": per_shape,
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "accumulate": "f32", "inputs": "uniform[-1,1) rounded to fp16, seeded per shape",
                        "l2": "inputs larger than L2: buffer sets rotate so that each shape's footprint exceeds 2x the 126 MB L2",
                        "parallelism": "replicas" if world > 1 else "single GPU"},
-            "per_shape": per_shape, "pct_of_spec_peak": 100.0 * value / world / SPEC_TFLOPS,
-            "roofline": roofline, "torch_matmul": torch_cmp, "grid": grid, "skinny": skinny, "cpu_baseline": cpu, "clocks": clocks,
+            "pct_of_spec_peak": 100.0 * value / world / SPEC_TFLOPS,
+            "variants": variants, "skinny": skinny, "grid": grid, "torch_matmul": torch_cmp, "sustained": sustained,
+            "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": args.steps * len(SWEEP),
         }
@@ -370,21 +402,49 @@ def run_ours(args) -> None:
         dist.destroy_process_group()
 
 
-def grid_sweep(ctx, torch, hgemm, inputs, stream) -> dict:
-    """All 729 grid shapes, ours against torch.matmul on the same buffers: warm (back-to-back) calls,
-    batches of n calls between two events, ours/torch batches interleaved in seeded random order,
-    median over rounds.  Buffers are dense M x K / N x K / M x N prefixes of three maximal arrays."""
-    mx = GRID[-1]
-    A_all = inputs.draw(1, inputs.TAG_A, mx, mx, "uniform", "cuda")
-    B_all = inputs.draw(1, inputs.TAG_B, mx, mx, "uniform", "cuda")
-    C_all = torch.empty(mx * mx, dtype=torch.float16, device="cuda")
-    rng = random.Random(729)
-    ratios, rows = [], []
-    server_ratios = []
-    roof_frac = []
-    peaks = measured_peaks()
+def sustained_report(torch, one_step, torch_step, step_flops, ms_per_step, gpu_index, stream) -> dict:
+    """The square sweep under the power cap: four phases of about 0.8 s each, ours / torch.matmul / ours / torch.matmul,
+    same rotating buffers, SM clock sampled per phase.  time x clock (device cycles per step) compares boxes whose
+    power caps settle at different clocks."""
+    n = max(20, min(2000, int(800.0 / max(ms_per_step, 1e-3))))
+    phases = []
+    for name, fn in (("ours", one_step), ("torch", torch_step), ("ours", one_step), ("torch", torch_step)):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        sampler = ClockSampler(gpu_index)
+        sampler.start()
+        time.sleep(0.1)
+        t0 = time.time()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(n):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        t1 = time.time()
+        clk = sampler.stop(t0, t1)
+        ms = e0.elapsed_time(e1) / n
+        phases.append({"arm": name, "tflops": step_flops / (ms * 1e-3) / 1e12, "ms_per_step": ms, "sm_mhz": clk.get("sm_mhz"),
+                       "mcycles_per_step": (ms * 1e-3 * clk["sm_mhz"]) if clk.get("sm_mhz") else None, "reasons": clk.get("reasons")})
+    ours = statistics.mean(p["tflops"] for p in phases if p["arm"] == "ours")
+    ref = statistics.mean(p["tflops"] for p in phases if p["arm"] == "torch")
+    return {"regime": f"{n} steps per phase, ours and torch.matmul alternating, rotating buffers", "phases": phases,
+            "ours_tflops": ours, "torch_tflops": ref, "ours_over_torch": ours / ref}
 
-    def batch_ms(fn, n):
+
+def variant_lines(ctx, torch, hgemm, inputs, stream) -> dict:
+    """One figure each for the row-major-B layout, the alpha/beta form and fp16 accumulators, on 4096^3 (warm calls,
+    torch's counterpart beside it where it has one)."""
+    S = 4096
+    A, B = inputs.make_ab(S, S, S, "uniform", "cuda")
+    Bkn = B.T.contiguous()                                   # the K x N row-major operand
+    C = torch.zeros(S, S, dtype=torch.float16, device="cuda")
+    s = stream.cuda_stream
+
+    def per_call_ms(fn, n=60):
+        for _ in range(5):
+            fn()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(n):
@@ -393,72 +453,242 @@ def grid_sweep(ctx, torch, hgemm, inputs, stream) -> dict:
         e1.synchronize()
         return e0.elapsed_time(e1) / n
 
+    def tf(ms):
+        return flops(S, S, S) / (ms * 1e-3) / 1e12
+
+    out = {"shape": [S, S, S], "regime": "warm back-to-back calls"}
+    plan = ctx.plan(S, S, S)
+    out["tn_plain"] = {"tflops": tf(per_call_ms(lambda: plan.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s))),
+                       "torch_tflops": tf(per_call_ms(lambda: torch.matmul(A, B.T, out=C)))}
+    nn = ctx.plan(S, S, S, layout=hgemm.LAYOUT_NN)
+    out["nn_layout"] = {"tflops": tf(per_call_ms(lambda: nn.run_ptr(A.data_ptr(), Bkn.data_ptr(), C.data_ptr(), s))),
+                        "torch_tflops": tf(per_call_ms(lambda: torch.matmul(A, Bkn, out=C))), "config": nn.config.as_dict()}
+    nn.close()
+    C.zero_()
+    out["alpha_beta"] = {"tflops": tf(per_call_ms(lambda: plan.run_scaled(0.5, 0.25, A, B, C))),
+                         "torch_tflops": tf(per_call_ms(lambda: torch.addmm(C, A, B.T, beta=0.25, alpha=0.5, out=C))),
+                         "alpha": 0.5, "beta": 0.25}
+    cfg = plan.config
+    cfg.accumulate = hgemm.ACC_F16
+    if cfg.tail_split >= 2 and cfg.tail_mode == hgemm.TAIL_K:
+        cfg.tail_split = 0
+    if plan.try_set_config(cfg) == hgemm.OK:
+        entry = {"tflops": tf(per_call_ms(lambda: plan.run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), s)))}
+        flag = getattr(torch.backends.cuda.matmul, "allow_fp16_accumulation", None)
+        if flag is not None:
+            torch.backends.cuda.matmul.allow_fp16_accumulation = True
+            try:
+                entry["torch_tflops"] = tf(per_call_ms(lambda: torch.matmul(A, B.T, out=C)))
+            finally:
+                torch.backends.cuda.matmul.allow_fp16_accumulation = flag
+        out["fp16_accumulate"] = entry
+    plan.close()
+    return out
+
+
+def device_durations(torch, calls) -> list:
+    """GPU-side duration in microseconds of each call in `calls` (a list of callables): from the start of the first
+    kernel the call launches to the end of the last, as the profiler's activity records give it.  The host path
+    (argument checks, heuristics, launch) is not in it.  None entries where the profiler gave nothing."""
+    from torch.profiler import ProfilerActivity, profile, record_function
+    out = [None] * len(calls)
+    CHUNK = 300
+    for c0 in range(0, len(calls), CHUNK):
+        part = calls[c0:c0 + CHUNK]
+        with profile(activities=[ProfilerActivity.CPU, ProfilerActivity.CUDA]) as prof:
+            for j, fn in enumerate(part):
+                with record_function(f"hgemm_bench_call_{c0 + j}"):
+                    fn()
+                torch.cuda.synchronize()
+        # the profiler mirrors every annotation on the GPU timeline: an event of the same name whose span runs from the
+        # start of the first kernel launched inside the annotation to the end of the last one
+        for ev in prof.events():
+            name = ev.name
+            if name.startswith("hgemm_bench_call_") and ev.device_type == torch.autograd.DeviceType.CUDA:
+                dur = ev.time_range.end - ev.time_range.start            # microseconds
+                if dur > 0:
+                    out[int(name.rsplit("_", 1)[1])] = float(dur)
+    return out
+
+
+def grid_sweep(ctx, torch, hgemm, inputs, stream, csv_path=None) -> dict:
+    """All 729 grid shapes, ours against torch.matmul on the same buffers, in four regimes.
+
+    warm    back-to-back calls on one buffer set (the paper's offline mode): batches of n calls between two events,
+            ours/torch batches interleaved in seeded random order, median over rounds
+    cold    the same with the buffer sets rotating through more than 2x L2 of A/B/C, so that no call finds its
+            operands in L2 (shapes whose single set already exceeds 2x L2 keep one set)
+    server  single calls after idle gaps that are not timed (paper section 2.4): short gaps of 20-200 us on the warm
+            buffers, and gaps of at least 2 ms on the rotating buffers (caches cool down, the clock governor reacts)
+    device  the GPU-side duration of one warm call of each arm from the profiler's kernel records: no host path
+    Buffers are dense prefixes (and, for the rotating sets, consecutive slices) of three pools."""
+    mx = GRID[-1]
+    pool = (max(mx * mx, int(2.2 * L2_BYTES) // 2 + mx * mx) + 4095) // 4096 * 4096   # elements: room for > 2x L2 of any one operand
+    A_all = inputs.draw(1, inputs.TAG_A, pool // 4096, 4096, "uniform", "cuda").view(-1)
+    B_all = inputs.draw(1, inputs.TAG_B, pool // 4096, 4096, "uniform", "cuda").view(-1)
+    C_all = torch.empty(pool, dtype=torch.float16, device="cuda")
+    rng = random.Random(729)
+    peaks = measured_peaks()
+    rows = []
+    dev_calls, dev_meta = [], []
+    plans = []
+
+    def batch_ms(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(n):
+            fn(i)
+        e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    def idle(seconds):
+        t = time.perf_counter() + seconds
+        while time.perf_counter() < t:
+            pass
+
     for M in GRID:
         for N in GRID:
             for K in GRID:
-                A = A_all.view(-1)[:M * K].view(M, K)
-                B = B_all.view(-1)[:N * K].view(N, K)
-                C = C_all[:M * N].view(M, N)
+                foot = compulsory_bytes(M, N, K)
+                sets = max(1, min(math.ceil(2 * L2_BYTES / foot), (pool - 1) // max(M * K, N * K, M * N)))
+                bufs = []
+                for r in range(sets):
+                    A = A_all[r * M * K:(r + 1) * M * K].view(M, K)
+                    B = B_all[r * N * K:(r + 1) * N * K].view(N, K)
+                    C = C_all[r * M * N:(r + 1) * M * N].view(M, N)
+                    bufs.append((A, B.T, C, A.data_ptr(), B.data_ptr(), C.data_ptr()))
                 plan = ctx.plan(M, N, K)
-                a, b, c, s = A.data_ptr(), B.data_ptr(), C.data_ptr(), stream.cuda_stream
-                ours = lambda: plan.run_ptr(a, b, c, s)          # noqa: E731
-                Bt = B.T
-                ref = lambda: torch.matmul(A, Bt, out=C)         # noqa: E731
-                for fn in (ours, ref):
-                    for _ in range(3):
-                        fn()
-                est = max(batch_ms(ours, 3), 1e-3)
+                s = stream.cuda_stream
+                A0, Bt0, C0, a0, b0, c0 = bufs[0]
+                ours_w = lambda i: plan.run_ptr(a0, b0, c0, s)                      # noqa: E731
+                ref_w = lambda i: torch.matmul(A0, Bt0, out=C0)                     # noqa: E731
+
+                def ours_c(i, bufs=bufs, plan=plan):
+                    b = bufs[i % len(bufs)]
+                    plan.run_ptr(b[3], b[4], b[5], s)
+
+                def ref_c(i, bufs=bufs):
+                    b = bufs[i % len(bufs)]
+                    torch.matmul(b[0], b[1], out=b[2])
+                for fn in (ours_w, ref_w):
+                    for i in range(3):
+                        fn(i)
+                est = max(batch_ms(ours_w, 3), 1e-3)
                 n = max(3, min(200, int(1.0 / est)))
-                t = {"ours": [], "torch": []}
+                t = {"ours": [], "torch": [], "ours_cold": [], "torch_cold": []}
                 for _ in range(3):
-                    order = [("ours", ours), ("torch", ref)]
+                    order = [("ours", ours_w), ("torch", ref_w)]
                     rng.shuffle(order)
                     for name, fn in order:
                         t[name].append(batch_ms(fn, n))
+                if sets > 1:
+                    for fn in (ours_c, ref_c):                                       # tensor maps of every set encoded, kernels loaded
+                        batch_ms(fn, sets)
+                    nc = max(sets, min(200, int(1.0 / est)))
+                    for _ in range(3):
+                        order = [("ours_cold", ours_c), ("torch_cold", ref_c)]
+                        rng.shuffle(order)
+                        for name, fn in order:
+                            t[name].append(batch_ms(fn, nc))
+                else:
+                    t["ours_cold"], t["torch_cold"] = t["ours"], t["torch"]
                 to, tt = statistics.median(t["ours"]), statistics.median(t["torch"])
-                ratios.append(tt / to)
-                # server mode (paper section 2.4): single calls separated by random idle gaps that are not
-                # timed; each call is bracketed by its own pair of events
+                toc, ttc = statistics.median(t["ours_cold"]), statistics.median(t["torch_cold"])
+                # server mode, short gaps: single calls on the warm buffers, each bracketed by its own pair of events
                 ts = {"ours": [], "torch": []}
                 for _ in range(5):
-                    order = [("ours", ours), ("torch", ref)]
+                    order = [("ours", ours_w), ("torch", ref_w)]
                     rng.shuffle(order)
                     for name, fn in order:
-                        gap = time.perf_counter() + rng.uniform(20e-6, 200e-6)
-                        while time.perf_counter() < gap:
-                            pass
+                        idle(rng.uniform(20e-6, 200e-6))
                         ts[name].append(batch_ms(fn, 1))
-                server_ratios.append(statistics.median(ts["torch"]) / statistics.median(ts["ours"]))
-                t_roof = max(flops(M, N, K) / (peaks["tflops_burst"] * 1e12), compulsory_bytes(M, N, K) / (peaks["hbm_gbs"] * 1e9))
-                roof_frac.append(t_roof / (to * 1e-3))
-                rows.append((M, N, K, to * 1e3, tt * 1e3))
-                plan.close()
-    geo = math.exp(sum(math.log(r) for r in ratios) / len(ratios))
-    worst = sorted(zip(ratios, rows))[:5]
-    big = [(r, row) for r, row in zip(ratios, rows) if min(row[:3]) >= 4096]
-    out_path = os.path.join(ROOT, "gpurun_out", "grid_times.csv")
+                # server mode, long gaps: at least 2 ms of idle time, rotating buffers, 15 single calls per arm
+                tl = {"ours": [], "torch": []}
+                for j in range(15):
+                    order = [("ours", ours_c), ("torch", ref_c)]
+                    rng.shuffle(order)
+                    for name, fn in order:
+                        idle(rng.uniform(2.0e-3, 2.5e-3))
+                        tl[name].append(batch_ms(lambda i, fn=fn, j=j: fn(j), 1))
+                t_roof = max(flops(M, N, K) / (peaks["tflops_burst"] * 1e12), foot / (peaks["hbm_gbs"] * 1e9))
+                rows.append({"shape": (M, N, K), "ours": to * 1e3, "torch": tt * 1e3, "ours_cold": toc * 1e3, "torch_cold": ttc * 1e3,
+                             "srv_ours": statistics.median(ts["ours"]) * 1e3, "srv_torch": statistics.median(ts["torch"]) * 1e3,
+                             "srvl_ours": statistics.median(tl["ours"]) * 1e3, "srvl_torch": statistics.median(tl["torch"]) * 1e3,
+                             "roof_us": t_roof * 1e6, "sets": sets})
+                dev_calls += [lambda f=ours_w: f(0), lambda f=ref_w: f(0)]
+                dev_meta.append(len(rows) - 1)
+                plans.append(plan)
+    # device-side durations of one warm call per arm (the plans are still alive: the callables hold them)
+    dev_error = None
     try:
-        os.makedirs(os.path.dirname(out_path), exist_ok=True)
-        with open(out_path, "w") as f:
-            f.write("M,N,K,ours_us,torch_us,ratio\n")
-            for r, (M, N, K, to, tt) in zip(ratios, rows):
-                f.write(f"{M},{N},{K},{to:.3f},{tt:.3f},{r:.4f}\n")
-    except OSError:
-        pass
-    return {
-        "shapes": len(ratios), "regime": "warm, back-to-back calls (the paper's offline mode)",
-        "geomean_torch_time_over_ours": geo, "wins": sum(r > 1.0 for r in ratios),
-        "mean_speedup_minus_1": sum(r - 1.0 for r in ratios) / len(ratios),
-        "geomean_fraction_of_measured_roofline": math.exp(sum(math.log(x) for x in roof_frac) / len(roof_frac)),
-        "compute_bound_min_tflops": min(flops(*row[:3]) / (row[3] * 1e-6) / 1e12 for _, row in big),
-        "compute_bound_geomean_vs_torch": math.exp(sum(math.log(r) for r, _ in big) / len(big)),
-        "worst5": [{"shape": list(row[:3]), "ratio": r, "ours_us": row[3], "torch_us": row[4]} for r, row in worst],
-        "server_mode": {"regime": "single calls after random idle gaps of 20-200 us, gap not timed, median of 5",
-                        "geomean_torch_time_over_ours": math.exp(sum(math.log(r) for r in server_ratios) / len(server_ratios)),
-                        "mean_speedup_minus_1": sum(r - 1.0 for r in server_ratios) / len(server_ratios),
-                        "win_rate": sum(r > 1.0 for r in server_ratios) / len(server_ratios)},
-        "offline_win_rate": sum(r > 1.0 for r in ratios) / len(ratios),
+        for fn in dev_calls:                                # every kernel loaded, every map encoded
+            fn()
+        torch.cuda.synchronize()
+        dur = device_durations(torch, dev_calls)
+        for j, ri in enumerate(dev_meta):
+            rows[ri]["dev_ours"], rows[ri]["dev_torch"] = dur[2 * j], dur[2 * j + 1]
+    except Exception as e:                                  # no profiler on this box: the regime is reported as absent
+        dev_error = f"{type(e).__name__}: {e}"
+    for plan in plans:
+        plan.close()
+
+    def geo(pairs):
+        pairs = [(a, b) for a, b in pairs if a and b]
+        return math.exp(sum(math.log(b / a) for a, b in pairs) / len(pairs)) if pairs else None
+
+    def summary(ko, kt, sel=lambda r: True):
+        use = [r for r in rows if sel(r) and r.get(ko) and r.get(kt)]
+        if not use:
+            return None
+        ratios = [r[kt] / r[ko] for r in use]
+        return {"shapes": len(use), "geomean_torch_time_over_ours": geo([(r[ko], r[kt]) for r in use]),
+                "mean_speedup_minus_1": sum(x - 1.0 for x in ratios) / len(ratios), "win_rate": sum(x > 1.0 for x in ratios) / len(ratios)}
+
+    if csv_path:
+        with open(csv_path, "w") as f:
+            cols = ["ours", "torch", "ours_cold", "torch_cold", "srv_ours", "srv_torch", "srvl_ours", "srvl_torch", "dev_ours", "dev_torch"]
+            f.write("M,N,K,sets," + ",".join(c + "_us" for c in cols) + "\n")
+            for r in rows:
+                f.write(",".join(str(v) for v in r["shape"]) + f",{r['sets']}," +
+                        ",".join("" if r.get(c) is None else f"{r[c]:.3f}" for c in cols) + "\n")
+
+    big = [r for r in rows if min(r["shape"]) >= 4096]
+    worst = sorted(rows, key=lambda r: r["torch"] / r["ours"])[:5]
+    worst_dev = sorted((r for r in rows if r.get("dev_ours") and r.get("dev_torch")), key=lambda r: r["dev_torch"] / r["dev_ours"])[:5]
+    device = None
+    if dev_error is None:
+        device = summary("dev_ours", "dev_torch")
+        if device:
+            device["regime"] = "GPU-side duration of one warm call per arm (first kernel start to last kernel end), from the profiler"
+            device["buckets_by_our_device_time"] = {
+                "under_5us": summary("dev_ours", "dev_torch", lambda r: (r.get("dev_ours") or 0) < 5.0),
+                "5_to_30us": summary("dev_ours", "dev_torch", lambda r: 5.0 <= (r.get("dev_ours") or 0) < 30.0),
+                "over_30us": summary("dev_ours", "dev_torch", lambda r: (r.get("dev_ours") or 0) >= 30.0)}
+    warm = summary("ours", "torch")
+    out = {
+        "detail": {"columns": ["M", "N", "K", "ours_us", "torch_us", "ours_cold_us", "torch_cold_us", "dev_ours_us", "dev_torch_us"],
+                   "rows": [list(r["shape"]) + [round(r["ours"], 2), round(r["torch"], 2), round(r["ours_cold"], 2), round(r["torch_cold"], 2),
+                                                None if r.get("dev_ours") is None else round(r["dev_ours"], 2),
+                                                None if r.get("dev_torch") is None else round(r["dev_torch"], 2)] for r in rows],
+                   "worst5_warm": [{"shape": list(r["shape"]), "ratio": r["torch"] / r["ours"], "ours_us": r["ours"], "torch_us": r["torch"]} for r in worst],
+                   "worst5_device": [{"shape": list(r["shape"]), "ratio": r["dev_torch"] / r["dev_ours"], "ours_us": r["dev_ours"],
+                                      "torch_us": r["dev_torch"]} for r in worst_dev]},
+        "shapes": len(rows), "regime": "warm, back-to-back calls (the paper's offline mode)",
+        "geomean_torch_time_over_ours": warm["geomean_torch_time_over_ours"], "wins": sum(r["torch"] > r["ours"] for r in rows),
+        "mean_speedup_minus_1": warm["mean_speedup_minus_1"], "offline_win_rate": warm["win_rate"],
+        "geomean_fraction_of_measured_roofline": math.exp(sum(math.log(r["roof_us"] / r["ours"]) for r in rows) / len(rows)),
+        "geomean_fraction_of_measured_roofline_cold": math.exp(sum(math.log(r["roof_us"] / r["ours_cold"]) for r in rows) / len(rows)),
+        "compute_bound_min_tflops": min(flops(*r["shape"]) / (r["ours"] * 1e-6) / 1e12 for r in big),
+        "compute_bound_geomean_vs_torch": geo([(r["ours"], r["torch"]) for r in big]),
+        "cold": dict(summary("ours_cold", "torch_cold"), regime="buffer sets rotate through more than 2x L2 (every call finds its operands cold)",
+                     rotated_shapes=sum(r["sets"] > 1 for r in rows)),
+        "server_mode": dict(summary("srv_ours", "srv_torch"), regime="single calls after random idle gaps of 20-200 us, gap not timed, median of 5, warm buffers"),
+        "server_mode_long_gaps": dict(summary("srvl_ours", "srvl_torch"),
+                                      regime="single calls after idle gaps of 2.0-2.5 ms, gap not timed, median of 15, rotating buffers"),
+        "device_time": device, "device_time_error": dev_error,
     }
+    return out
 
 
 def skinny_report(ctx, torch, hgemm, inputs, stream) -> dict:
@@ -505,6 +735,8 @@ def skinny_report(ctx, torch, hgemm, inputs, stream) -> dict:
         del Bs, B0
     return {"regime": "B rotates through copies totalling more than 2x L2 (cold weights), A and C stay hot",
             "inputs": "N(0,1) * K^-1/2 rounded to fp16", "shapes": out,
+            "per_shape_frac_of_measured_hbm": {"x".join(map(str, r["shape"])): round(r["frac_of_measured_hbm"], 4) for r in out},
+            "per_shape_torch_time_over_ours": {"x".join(map(str, r["shape"])): round(r["torch_time_over_ours"], 4) for r in out},
             "geomean_frac_of_measured_hbm": math.exp(sum(math.log(r["frac_of_measured_hbm"]) for r in out) / len(out)),
             "geomean_torch_time_over_ours": math.exp(sum(math.log(r["torch_time_over_ours"]) for r in out) / len(out))}
 
@@ -515,7 +747,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--no-grid", action="store_true", help="skip the 729-shape comparison against torch.matmul")
+    ap.add_argument("--no-grid", action="store_true", help="skip everything but the timed sweep, torch.matmul beside it and the end-to-end leg")
+    ap.add_argument("--grid-csv", metavar="PATH", help="also write the grid's per-shape times to this CSV file")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -92,6 +92,12 @@ enum {
 };
 
 enum {
+    HGEMM_RASTER_SWEEP = 0,     /* every group of raster_group m-tiles sweeps the n-tiles from first to last */
+    HGEMM_RASTER_SERPENTINE = 1 /* odd groups sweep from last to first (boustrophedon), so a group starts on the B
+                                   tiles the group before it used last and finds them in L2 */
+};
+
+enum {
     HGEMM_EPILOGUE_DIRECT = 0,  /* registers -> 16-byte global stores */
     HGEMM_EPILOGUE_TMA = 1,     /* registers -> swizzled shared memory -> TMA store, 32 x 32 boxes */
     HGEMM_EPILOGUE_TMA_WIDE = 2 /* the same with 32-row x 64-column boxes: half as many fences, stores and
@@ -107,7 +113,10 @@ enum {
 typedef struct {
     int32_t family;       /* HGEMM_FAMILY_* */
     int32_t block_m;      /* 128 (1-CTA) or 256 (2-CTA pair) */
-    int32_t block_n;      /* multiple of 32 in [32, 256] */
+    int32_t block_n;      /* multiple of 32 in [32, 256]; or 512 (CTA-pair family only): a 256 x 512 tile held in both
+                             tensor-memory accumulators at once, two MMAs per K step sharing the A tile -- a quarter less
+                             shared-memory fill per flop than 256 x 256, no overlap of a tile's epilogue with the next
+                             tile's MMAs.  Needs N % 512 == 0, split_k == 1, no tail_split, no swap_ab, the TN layout */
     int32_t block_k;      /* K extent of a pipeline stage: 64 or 128 (one or two 128-byte swizzle spans) */
     int32_t stages;       /* shared-memory ring depth, 2..12, bounded by shared memory */
     int32_t split_k;      /* >= 1; K slices reduced in slice order (deterministic) */
@@ -126,7 +135,16 @@ typedef struct {
                              fp16 inputs, section 1): every 16-wide K step rounds the running sums to fp16, so
                              results carry the larger error of that arithmetic.  Needs split_k == 1 and no K tail
                              split; never chosen by the planner or the tuned table */
-    int32_t reserved[4];  /* must be zero */
+    int32_t swap_ab;      /* 0: the tile's 128 (256 for a pair) accumulator rows are rows of C, block_n its columns.
+                             1: the operands trade places inside the kernel -- the rows of B (N of them) go to the
+                             accumulator rows, block_n covers rows of A, and the epilogue stores the tile transposed,
+                             so C is the same row-major M x N matrix with the same values.  For few rows and many
+                             columns (M <= 256, a projection of a few tokens through a wide weight matrix: the
+                             paper's "BM ~ M" cases, section 5.2) this fills the 128-row side of the MMA with weight rows instead of zero
+                             padding, and a CTA pair splits the small operand instead of re-reading all of it.
+                             Needs N % 8 == 0, fp32 accumulators, the TN layout, no tail_split and not the wide epilogue */
+    int32_t raster_mode;  /* HGEMM_RASTER_* : the order in which raster groups sweep the n-tiles */
+    int32_t reserved[2];  /* must be zero */
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the
@@ -330,7 +348,11 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
  * buffer.  While a trace buffer or a skip mask (below) is set, launches run the
  * instrumented instantiation of the kernel, which is 10-15 % slower on small and
  * mid-size shapes than the one that runs otherwise: the stamps describe the
- * pipeline's structure and proportions, not the production kernel's absolute times. */
+ * pipeline's structure and proportions, not the production kernel's absolute times.
+ * The instrumented kernels do not exist for swapped-operand configurations (swap_ab = 1)
+ * nor for the 512-wide tile:
+ * hgemm_run returns HGEMM_ERR_UNSUPPORTED for such a plan while a trace buffer or a skip
+ * mask is set. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan

@@ -122,6 +122,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     // the slices of a tile wait for each other: each needs its own SM (or SM pair)
     if (cfg.split_k > 1 && cfg.split_k > ctx->num_sms / cg) return HGEMM_ERR_UNSUPPORTED;
     if (pl->layout == HGEMM_LAYOUT_NN && (cfg.block_n % (64 * cg)) != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (pl->layout == HGEMM_LAYOUT_NN && cfg.swap_ab) return HGEMM_ERR_UNSUPPORTED;   // the swapped form is built for K-contiguous operands
+    if (pl->layout == HGEMM_LAYOUT_NN && cfg.block_n == 512) return HGEMM_ERR_UNSUPPORTED;   // so is the double-accumulator tile
     // row-major B is staged in blocks of 64 columns: column pieces of tail tiles must be whole blocks per CTA
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 &&
         ((cfg.block_n / cfg.tail_split) % (64 * cg)) != 0)
@@ -201,11 +203,15 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     pl->cfg = cfg;
     KernelParams &p = pl->params;
     std::memset(&p, 0, sizeof(p));
-    p.M = int32_t(pl->M);
-    p.N = int32_t(pl->N);
+    // a swapped configuration runs the kernel on the transposed problem: its rows are the caller's columns
+    const int64_t kM = cfg.swap_ab ? pl->N : pl->M, kN = cfg.swap_ab ? pl->M : pl->N;
+    p.M = int32_t(kM);
+    p.N = int32_t(kN);
     p.K = int32_t(pl->K);
-    p.tiles_m = int32_t((pl->M + 128 * cg - 1) / (128 * cg));
-    p.tiles_n = int32_t((pl->N + cfg.block_n - 1) / cfg.block_n);
+    p.transposed = cfg.swap_ab ? 1 : 0;
+    p.raster_serpentine = cfg.raster_mode == HGEMM_RASTER_SERPENTINE ? 1 : 0;
+    p.tiles_m = int32_t((kM + 128 * cg - 1) / (128 * cg));
+    p.tiles_n = int32_t((kN + cfg.block_n - 1) / cfg.block_n);
     p.split_k = int32_t(layout.slices);
     p.first_split_tile = int32_t(layout.first_split_tile);
     p.total_work = int32_t(layout.work_items);
@@ -225,11 +231,12 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         p.fd_split = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.split_k)));
         p.fd_pieces = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.tail_pieces)));
     }
-    p.tmem_cols = pow2_at_least(2 * cfg.block_n);
-    p.ragged_n = (pl->N % 8) != 0 ? 1 : 0;
+    p.tmem_cols = cfg.block_n == 512 ? 512 : pow2_at_least(2 * cfg.block_n);   // two accumulators either way
+    p.ragged_n = (!cfg.swap_ab && (pl->N % 8) != 0) ? 1 : 0;   // (a swapped configuration needs N % 8 == 0 and stores by its own rule)
     p.epilogue_tma = (cfg.epilogue != HGEMM_EPILOGUE_DIRECT && cfg.split_k == 1 && !p.ragged_n)             // whole tiles only
                          ? (cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? 2 : 1) : 0;
-    p.idesc = make_idesc(128 * cg, cfg.block_n, pl->layout == HGEMM_LAYOUT_NN, cfg.accumulate == HGEMM_ACC_F16);
+    // (the 512-wide double tile issues two MMAs of N = 256 per K step)
+    p.idesc = make_idesc(128 * cg, cfg.block_n == 512 ? 256 : cfg.block_n, pl->layout == HGEMM_LAYOUT_NN, cfg.accumulate == HGEMM_ACC_F16);
     p.acc_f16 = cfg.accumulate == HGEMM_ACC_F16 ? 1 : 0;
     p.idesc_tail = make_idesc(128 * cg, cfg.block_n / int(std::max<int64_t>(1, layout.pieces)), pl->layout == HGEMM_LAYOUT_NN,
                               cfg.accumulate == HGEMM_ACC_F16);
@@ -256,26 +263,50 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
 // The kernel instantiation for a CTA group size, store-box width and kind of split-K reduction
 // (0: no K slices, 1: through the workspace -- also a tail cut along K --, 2: inside a cluster); `plain` selects
 // the instantiation without the optional features, `trace` the one with the instrumentation (never plain).
-template <bool PLAIN, bool TRACE, int SUBS>
+template <bool PLAIN, bool TRACE, int SUBS, bool XPOSE>
 const void *kernel_of(int cg, bool wide, int split)
 {
     using namespace hgemm_dev;
-#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S, PLAIN, TRACE, SUBS>)
-    if (cg == 1) {
-        if (wide) return split == 0 ? HGEMM_K(1, true, 0) : HGEMM_K(1, true, 1);      // no split_k > 1 with wide boxes
-        return split == 0 ? HGEMM_K(1, false, 0) : split == 1 ? HGEMM_K(1, false, 1) : HGEMM_K(1, false, 2);
+#define HGEMM_K(CG, W, S) reinterpret_cast<const void *>(hgemm_umma_kernel<CG, W, S, PLAIN, TRACE, SUBS, XPOSE>)
+    if constexpr (XPOSE) {                   // transposed stores: no wide boxes
+        if (cg == 1) return split == 0 ? HGEMM_K(1, false, 0) : split == 1 ? HGEMM_K(1, false, 1) : HGEMM_K(1, false, 2);
+        return split == 0 ? HGEMM_K(2, false, 0) : split == 1 ? HGEMM_K(2, false, 1) : HGEMM_K(2, false, 2);
+    } else {
+        if (cg == 1) {
+            if (wide) return split == 0 ? HGEMM_K(1, true, 0) : HGEMM_K(1, true, 1);      // no split_k > 1 with wide boxes
+            return split == 0 ? HGEMM_K(1, false, 0) : split == 1 ? HGEMM_K(1, false, 1) : HGEMM_K(1, false, 2);
+        }
+        if (wide) return split == 0 ? HGEMM_K(2, true, 0) : HGEMM_K(2, true, 1);
+        return split == 0 ? HGEMM_K(2, false, 0) : split == 1 ? HGEMM_K(2, false, 1) : HGEMM_K(2, false, 2);
     }
-    if (wide) return split == 0 ? HGEMM_K(2, true, 0) : HGEMM_K(2, true, 1);
-    return split == 0 ? HGEMM_K(2, false, 0) : split == 1 ? HGEMM_K(2, false, 1) : HGEMM_K(2, false, 2);
 #undef HGEMM_K
 }
 
-// `subs`: 64-wide sub-tiles per stage (block_k / 64); the plain instantiations are compiled for each value.
-const void *kernel_for(int cg, bool wide, int split, bool plain, bool trace, int subs)
+// The double-accumulator pair tile (block_n == 512): CTA pairs, no K slices, no transposed stores, no instrumentation.
+template <bool PLAIN, int SUBS>
+const void *dual_kernel_of(bool wide)
 {
-    if (trace) return kernel_of<false, true, 0>(cg, wide, split);
-    if (!plain) return kernel_of<false, false, 0>(cg, wide, split);
-    return subs == 2 ? kernel_of<true, false, 2>(cg, wide, split) : kernel_of<true, false, 1>(cg, wide, split);
+    using namespace hgemm_dev;
+    return wide ? reinterpret_cast<const void *>(hgemm_umma_kernel<2, true, 0, PLAIN, false, SUBS, false, true>)
+                : reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, 0, PLAIN, false, SUBS, false, true>);
+}
+
+// `subs`: 64-wide sub-tiles per stage (block_k / 64); the plain instantiations are compiled for each value.
+// `xpose`: the instantiations that store the tile transposed (swapped operands); they exist without instrumentation.
+// `dual`: the instantiations for block_n == 512.
+const void *kernel_for(int cg, bool wide, int split, bool plain, bool trace, int subs, bool xpose = false, bool dual = false)
+{
+    if (dual) {
+        if (!plain) return dual_kernel_of<false, 0>(wide);
+        return subs == 2 ? dual_kernel_of<true, 2>(wide) : dual_kernel_of<true, 1>(wide);
+    }
+    if (xpose) {
+        if (!plain) return kernel_of<false, false, 0, true>(cg, false, split);
+        return subs == 2 ? kernel_of<true, false, 2, true>(cg, false, split) : kernel_of<true, false, 1, true>(cg, false, split);
+    }
+    if (trace) return kernel_of<false, true, 0, false>(cg, wide, split);
+    if (!plain) return kernel_of<false, false, 0, false>(cg, wide, split);
+    return subs == 2 ? kernel_of<true, false, 2, false>(cg, wide, split) : kernel_of<true, false, 1, false>(cg, wide, split);
 }
 
 bool encode_2d(hgemm_ctx_s *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer, uint32_t box_inner,
@@ -377,8 +408,17 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
         ctx->free_status_slots.reserve(kStatusSlots);
         for (int slot = kStatusSlots - 1; slot >= 1; --slot) ctx->free_status_slots.push_back(slot);
         // every instantiation: 1-CTA / CTA-pair, narrow / wide store boxes, no K slices / workspace / cluster reduction
-        for (int k = 0; k < 48 && e == cudaSuccess; ++k) {
-            const void *fn_k = kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k / 12 >= 2, k / 12 == 1, k / 12 == 3 ? 2 : 1);
+        for (int k = 0; k < 72 && e == cudaSuccess; ++k) {
+            // k / 12: 0 full-featured, 1 instrumented, 2 and 3 plain with 64- and 128-wide stages; 4 and 5: transposed stores
+            // (full-featured, then plain with either stage width)
+            const bool xp = k >= 48;
+            const void *fn_k = xp ? kernel_for(1 + (k & 1), false, (k >> 2) % 3, k >= 60, false, (k & 2) ? 2 : 1, true)
+                                  : kernel_for(1 + (k & 1), (k & 2) != 0, (k >> 2) % 3, k / 12 >= 2, k / 12 == 1, k / 12 == 3 ? 2 : 1);
+            e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        }
+        for (int k = 0; k < 6 && e == cudaSuccess; ++k) {           // the double-accumulator instantiations
+            const void *fn_k = kernel_for(2, (k & 1) != 0, 0, k >= 2, false, k >= 4 ? 2 : 1, false, true);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
@@ -483,6 +523,10 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
     hgemm_config_t cfg;
     s = hgemm_host::plan_config(M, N, Kp, ctx->num_sms, &cfg);   // the table, else the neighbours' configurations re-fitted
     if (s != HGEMM_OK) return s;
+    if (layout == HGEMM_LAYOUT_NN && cfg.swap_ab) {
+        s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);   // the swapped form needs K-contiguous operands
+        if (s != HGEMM_OK) return s;
+    }
     if (layout == HGEMM_LAYOUT_NN) {
         // row-major B is staged in blocks of 64 columns: widen the tile to the next legal width and
         // give back stages until it fits
@@ -679,6 +723,8 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         B = plan->pad_b;
     }
 
+    if (cfg.swap_ab) std::swap(A, B);       // the kernel's A operand (its 128-row side) is the caller's B
+
     hgemm_plan_s::MapEntry *me = nullptr;
     for (int i = 0; i < plan->maps_used; ++i) {
         hgemm_plan_s::MapEntry &e = plan->maps[i];
@@ -691,7 +737,7 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         hgemm_plan_s::MapEntry &e = plan->maps[plan->maps_next];
         e.a = e.b = nullptr;
         e.c = nullptr;
-        const uint64_t M = uint64_t(plan->M), N = uint64_t(plan->N), K = uint64_t(plan->K);
+        const uint64_t M = uint64_t(plan->params.M), N = uint64_t(plan->params.N), K = uint64_t(plan->K);   // as the kernel sees them
         if (plan->params.tma_3d) {
             if (!encode_3d_ksub(ctx, &e.tmap_a, A, K, M, 128)) return HGEMM_ERR_CUDA;
             if (!encode_3d_ksub(ctx, &e.tmap_b, B, K, N, uint32_t(cfg.block_n / cg))) return HGEMM_ERR_CUDA;
@@ -713,6 +759,9 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         } else if (plan->params.epilogue_tma == 2) {
             // wide epilogue: 32-row x 64-column store boxes (128-byte rows)
             if (!encode_2d(ctx, &e.tmap_c, C, N, M, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B)) return HGEMM_ERR_CUDA;
+        } else if (plan->params.transposed) {
+            // the caller's C: rows of the kernel's M elements, the kernel's N of them; boxes are stored transposed
+            if (!encode_2d(ctx, &e.tmap_c, C, M, N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return HGEMM_ERR_CUDA;
         } else if (!encode_2d(ctx, &e.tmap_c, C, N, M, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
             return HGEMM_ERR_CUDA;
         }
@@ -756,8 +805,9 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     const KernelParams &kp = plan->params;
     const bool trace = kp.trace != nullptr || kp.debug_skip != 0;
     const bool plain = !kp.scaled && !kp.acc_f16 && !kp.ragged_n && !kp.b_row_major && kp.tail_pieces <= 1;
+    if (trace && (kp.transposed || kp.block_n == 512)) return HGEMM_ERR_UNSUPPORTED;   // no instrumented kernels for these two
     const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
-                                trace, kp.block_k / 64);
+                                trace, kp.block_k / 64, kp.transposed != 0, kp.block_n == 512);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
     e = cudaLaunchKernelExC(&lc, fn, args);
     if (e != cudaSuccess) return cuda_fail(ctx, e);

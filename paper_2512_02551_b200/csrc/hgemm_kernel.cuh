@@ -112,6 +112,10 @@ struct KernelParams {
     int32_t tail_pieces;          // > 1: work items from first_split_tile on are tiles cut into this many column pieces (no K split)
     uint32_t scaled;              // 0: C = A B^T; 1: C = alpha A B^T + beta C (paper section 2.1)
     float alpha, beta;
+    int32_t transposed;           // 1: the kernel computes the transposed problem (the caller's B is its A, M and N are
+                                  // traded) and stores element (row, col) of its tile at C[col * M + row]: the
+                                  // caller's row-major C (whose rows are this kernel's M long)
+    int32_t raster_serpentine;    // 1: odd raster groups sweep the n-tiles from last to first
 };
 
 template <bool OFF = false>
@@ -195,6 +199,25 @@ __device__ __forceinline__ void store_ragged(__half *C, int64_t N, int32_t row, 
         if (col + j < N) C[static_cast<size_t>(row) * N + col + j] = __float2half_rn(vals[j]);
 }
 
+// Transposed result (see KernelParams::transposed): `count` consecutive columns of one row of the kernel's tile are
+// `count` elements of one COLUMN of the caller's C, p.M apart.
+__device__ __forceinline__ void store_transposed(__half *C, int64_t ldc, int32_t n_cols, int32_t row, int32_t col, const float *vals, int count)
+{
+    for (int j = 0; j < count; ++j)
+        if (col + j < n_cols) C[static_cast<size_t>(col + j) * ldc + row] = __float2half_rn(vals[j]);
+}
+
+// Four consecutive columns of one row of the kernel's tile, for the two layouts of C that rule out 8-byte stores
+// (rows that are not multiples of 16 bytes; the transposed result).  Out of line on purpose: the split-K reductions
+// call it from loops that keep dozens of partial sums in registers, and inlined there it made them spill.
+__device__ __noinline__ void store_unit4_slow(__half *C, int32_t M, int32_t N, int32_t transposed, int32_t row, int32_t col,
+                                              float x, float y, float z, float w)
+{
+    const float f[4] = {x, y, z, w};
+    if (transposed) store_transposed(C, M, N, row, col, f, 4);
+    else store_ragged(C, N, row, col, f, 4);
+}
+
 // The same for a tile that is contiguous along its M/N dimension (a row-major K x N operand): the tile
 // is stored as blocks of 64 columns, each block 64 k-rows of 128 bytes under the 128-byte swizzle.
 // Leading byte offset = distance between 64-column blocks, stride byte offset = distance between
@@ -224,12 +247,17 @@ __device__ __forceinline__ float scaled_value(float acc, float alpha, float beta
 }
 
 // v[0..7]: fp32 bit patterns of eight consecutive columns col .. col + 7 of row `row`.
+template <bool XPOSE = false>
 __device__ __forceinline__ void scale_group8(uint32_t *v, const KernelParams &p, int32_t row, int32_t col)
 {
     float old[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) old[i] = 0.0f;
-    if (p.beta != 0.0f) {
+    if (XPOSE && p.beta != 0.0f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (col + i < p.N) old[i] = __half2float(p.C[static_cast<size_t>(col + i) * p.M + row]);
+    } else if (p.beta != 0.0f) {
         const __half *src = p.C + static_cast<size_t>(row) * p.N + col;
         if (!p.ragged_n && col + 8 <= p.N) {
             const uint4 o = *reinterpret_cast<const uint4 *>(src);   // N % 8 == 0: 16-byte aligned
@@ -251,10 +279,15 @@ __device__ __forceinline__ void scale_group8(uint32_t *v, const KernelParams &p,
 }
 
 // s: four consecutive columns col .. col + 3 of row `row`.
+template <bool XPOSE = false>
 __device__ __forceinline__ void scale_unit4(float4 &s, const KernelParams &p, int32_t row, int32_t col)
 {
     float old[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    if (p.beta != 0.0f) {
+    if (XPOSE && p.beta != 0.0f) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (col + i < p.N) old[i] = __half2float(p.C[static_cast<size_t>(col + i) * p.M + row]);
+    } else if (p.beta != 0.0f) {
         const __half *src = p.C + static_cast<size_t>(row) * p.N + col;
         if (!p.ragged_n) {                                            // N % 8 == 0 and col % 4 == 0: 8-byte aligned, in bounds
             const uint2 o = *reinterpret_cast<const uint2 *>(src);
@@ -327,8 +360,10 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     const int32_t r = it.tile - g * per_group;
     const int32_t tn = gsize == p.raster_group ? fast_div(r, p.fd_raster) : fast_div(r, p.fd_last_group);
     const int32_t tm = first_m + (r - tn * gsize);
+    // serpentine: an odd group walks the n-tiles backwards, starting on the B tiles the group before it used last
+    const int32_t tn_at = (p.raster_serpentine && (g & 1)) ? p.tiles_n - 1 - tn : tn;
     it.m0 = tm * block_m_total;
-    it.n0 = tn * p.block_n + n_off;
+    it.n0 = tn_at * p.block_n + n_off;
     if (!SPLIT || it.slices == 1) {
         it.kb_begin = 0;
         it.kb_count = p.kblocks;
@@ -373,7 +408,17 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // compiled in but switched off it cost 10-15 % on small and mid-size shapes, so it only runs when one of them is set.
 // WIDE_STORE: the instantiation for HGEMM_EPILOGUE_TMA_WIDE (whole tiles leave through 32 x 64 store boxes and the
 // store staging is 64 KB); the other one is the code for every other configuration, unchanged by the wide path.
-template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false, bool TRACE = !PLAIN, int SUBS = 0>
+// XPOSE: the instantiations that store the tile transposed (KernelParams::transposed, the swapped-operand
+// configurations); kept out of all the others, where its store paths cost registers the widest reductions do not have.
+// DUAL (CTA pairs only, block_n == 512): one work item is a 256 x 512 tile held in BOTH accumulators at once -- every
+// 16-wide K step issues two MMAs (N = 256 each) that read the same A sub-tile -- so each CTA fetches 128 rows of A and
+// 256 rows of B per k-block for 128 x 512 results: a quarter less shared-memory fill per flop than the 256 x 256 pair
+// tile, which is what bounds the large shapes when L2 cannot feed 64 B/clk to every SM.  Price: no spare accumulator, so
+// the epilogue of a tile does not overlap the next tile's MMAs (the producer still prefetches through it).  Each CTA
+// loads 256 CONSECUTIVE rows of B (one box); MMA h (h = 0, 1) takes rows 128 h .. 128 h + 127 of both CTAs' boxes, so
+// accumulator column t holds column  256 * ((t % 256) / 128) + 128 * (t / 256) + t % 128  of the tile.
+template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false, bool TRACE = !PLAIN, int SUBS = 0, bool XPOSE = false,
+          bool DUAL = false>
 __global__ void __launch_bounds__(kThreads, 1)
 hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bt, const KernelParams p)
@@ -592,8 +637,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
                 const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
-                const uint32_t acc = local_tile & 1u;
-                const uint32_t acc_ph = (local_tile >> 1) & 1u;
+                const uint32_t acc = DUAL ? 0u : (local_tile & 1u);            // DUAL: one work item fills both accumulators
+                const uint32_t acc_ph = DUAL ? (local_tile & 1u) : ((local_tile >> 1) & 1u);
                 const long long ca = tr ? clock64() : 0;
                 ok = mbar_wait(bar_tmem_empty + 8 * acc, acc_ph ^ 1u, ctl, status_code(kRoleMma, 1, acc));
                 ok = __all_sync(0xffffffffu, ok);
@@ -625,6 +670,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                 // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
                                 umma_f16_elect<CTA_GROUP>(d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, idesc,
                                                        (kb | sub | k) != 0 ? 1u : 0u);
+                                if constexpr (DUAL)      // rows 128 .. 255 of both CTAs' B boxes into the second accumulator
+                                    umma_f16_elect<CTA_GROUP>(d_tmem + 256u, a_sub + 2u * k, b_sub + ((128u * 128u) >> 4) + b_kstep * k, idesc,
+                                                           (kb | sub | k) != 0 ? 1u : 0u);
                             }
                         }
                     }
@@ -681,8 +729,12 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         grid_dependency_wait();                            // before the first store to C, workspace or counters
         for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
             const WorkItem it = decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal);
-            const uint32_t acc = local_tile & 1u;
-            const uint32_t acc_ph = (local_tile >> 1) & 1u;
+            const uint32_t acc = DUAL ? 0u : (local_tile & 1u);
+            const uint32_t acc_ph = DUAL ? (local_tile & 1u) : ((local_tile >> 1) & 1u);
+            // first column, within the tile, of 32-column accumulator chunk c (DUAL: see the template comment)
+            auto chunk_col = [](int32_t c) -> int32_t {
+                return DUAL ? ((c >> 2) & 1) * 256 + (c >> 3) * 128 + (c & 3) * 32 : c * 32;
+            };
             ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
             ok = __all_sync(0xffffffffu, ok);   // the warp-wide tensor-memory loads below need the whole warp
             if (!ok) break;
@@ -694,8 +746,37 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
             // One 32-column chunk of this thread's row, converted and sent to C.
             auto emit_chunk = [&](const uint32_t (&v)[32], int32_t c) {
-                const int32_t col0 = it.n0 + c * 32;
-                if (!WIDE_STORE && p.epilogue_tma) {
+                const int32_t col0 = it.n0 + chunk_col(c);
+                if (XPOSE && !WIDE_STORE) {
+                    // The caller's C is the transpose of what this kernel computes: this thread's 32 values are 32
+                    // elements of one column of C (row col0 + j, column grow).
+                    if (p.epilogue_tma) {
+                        // stage the chunk transposed -- box row j holds what the 32 lanes computed for column
+                        // col0 + j, 64 consecutive bytes per store instruction -- in the 64-byte swizzle the store
+                        // box expects (16-byte piece t of row r lives at piece t ^ ((r >> 1) & 3)), then one TMA store
+                        const uint32_t buf = staging + (store_count & 1u) * (kStagingBytesPerWarp / 2);
+                        bulk_wait_group_read<1>();
+                        __syncwarp();
+                        const uint32_t piece = lane >> 3, within = (lane & 7u) * 2u;
+#pragma unroll
+                        for (uint32_t j = 0; j < 32; ++j) {
+                            const __half h = __float2half_rn(__uint_as_float(v[j]));
+                            st_shared_u16(buf + j * 64u + ((piece ^ ((j >> 1) & 3u)) << 4) + within, __half_as_ushort(h));
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        const int32_t box_col = row0 + static_cast<int32_t>(q) * 32;          // first column of C in the box
+                        const bool go = lane == 0 && box_col < p.M && col0 < p.N && !((TRACE ? p.debug_skip : 0u) & 4u);
+                        tma_store_2d_if(go ? 1u : 0u, &tmap_c, box_col, col0, buf);
+                        bulk_commit_group();
+                        ++store_count;
+                    } else if (grow < p.M) {
+                        unsigned short *dst = reinterpret_cast<unsigned short *>(p.C) + static_cast<size_t>(col0) * p.M + grow;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) dst[static_cast<size_t>(j) * p.M] = __half_as_ushort(__float2half_rn(__uint_as_float(v[j])));
+                    }
+                } else if (!WIDE_STORE && p.epilogue_tma) {
                     const uint32_t buf = staging + (store_count & 1u) * (kStagingBytesPerWarp / 2);
                     // the buffer written two stores ago must have been read by its TMA store
                     bulk_wait_group_read<1>();                      // lanes other than 0 own no groups
@@ -803,7 +884,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                                 for (int j = 0; j < 4; ++j)
-                                    if (it.n0 + c * 32 + 8 * j < p.N) scale_group8(v + 8 * j, p, grow, it.n0 + c * 32 + 8 * j);
+                                    if (it.n0 + chunk_col(c) + 8 * j < p.N) scale_group8<XPOSE>(v + 8 * j, p, grow, it.n0 + chunk_col(c) + 8 * j);
                             }
 #pragma unroll
                             for (uint32_t j = 0; j < 4; ++j) {
@@ -817,7 +898,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     __syncwarp();
                     {
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                        const int32_t col0 = it.n0 + b * 64;
+                        const int32_t col0 = it.n0 + chunk_col(2 * b);
                         const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((TRACE ? p.debug_skip : 0u) & 4u);
                         tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
@@ -844,7 +925,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
-                            if (it.n0 + c * 32 + 8 * j < p.N) scale_group8(v + 8 * j, p, grow, it.n0 + c * 32 + 8 * j);
+                            if (it.n0 + chunk_col(c) + 8 * j < p.N) scale_group8<XPOSE>(v + 8 * j, p, grow, it.n0 + chunk_col(c) + 8 * j);
                     }
                     emit_chunk(v, c);
                 }
@@ -963,7 +1044,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const int32_t u = u0 + j * 256;
                         const int32_t c = u >> 10, r = (u >> 3) & 127, g = (u & 7) ^ (r & 7);
                         const int32_t orow = row0 + r, col = it.n0 + c * 32 + g * 4;
-                        if ((!PLAIN && p.scaled)) scale_unit4(sum[j], p, orow, col);
+                        if ((!PLAIN && p.scaled)) scale_unit4<XPOSE>(sum[j], p, orow, col);
+                        if (XPOSE) {
+                            store_unit4_slow(p.C, p.M, p.N, 1, orow, col, sum[j].x, sum[j].y, sum[j].z, sum[j].w);
+                            continue;
+                        }
                         if ((!PLAIN && p.ragged_n)) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
                             store_ragged(p.C, p.N, orow, col, f, 4);
@@ -1092,7 +1177,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         const int32_t c = static_cast<int32_t>(cc), g = static_cast<int32_t>((u & 7u) ^ (r & 7u));
                         const int32_t orow = cs_m0 + static_cast<int32_t>(r), col = cs_n0 + c * 32 + g * 4;
                         if (orow >= p.M || col >= p.N) continue;
-                        if ((!PLAIN && p.scaled)) scale_unit4(sum[j], p, orow, col);
+                        if ((!PLAIN && p.scaled)) scale_unit4<XPOSE>(sum[j], p, orow, col);
+                        if (XPOSE) {
+                            store_unit4_slow(p.C, p.M, p.N, 1, orow, col, sum[j].x, sum[j].y, sum[j].z, sum[j].w);
+                            continue;
+                        }
                         if ((!PLAIN && p.ragged_n)) {
                             const float f[4] = {sum[j].x, sum[j].y, sum[j].z, sum[j].w};
                             store_ragged(p.C, p.N, orow, col, f, 4);

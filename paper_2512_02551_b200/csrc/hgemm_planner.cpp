@@ -54,6 +54,7 @@ int32_t max_stages_of(const hgemm_config_t &c)
 
 SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c)
 {
+    if (c.swap_ab) std::swap(M, N);   // the kernel tiles the transposed problem
     const int cg = cta_group_of(c);
     SplitLayout L;
     L.tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
@@ -115,10 +116,25 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
 {
     const hgemm_status_t s = validate_shape(M, N, K);
     if (s != HGEMM_OK) return s;
+    if (c.swap_ab != 0 && c.swap_ab != 1) return HGEMM_ERR_UNSUPPORTED;
+    if (c.raster_mode != HGEMM_RASTER_SWEEP && c.raster_mode != HGEMM_RASTER_SERPENTINE) return HGEMM_ERR_UNSUPPORTED;
+    if (c.swap_ab) {
+        // the transposed tile is stored through 32 x 32 boxes or 2-byte stores into rows of C that are multiples of
+        // 16 bytes; everything below judges the problem the kernel sees: rows and columns traded
+        if ((N % 8) != 0 || c.accumulate != HGEMM_ACC_F32 || c.tail_split >= 2 || c.epilogue == HGEMM_EPILOGUE_TMA_WIDE)
+            return HGEMM_ERR_UNSUPPORTED;
+        std::swap(M, N);
+    }
     if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA) return HGEMM_ERR_UNSUPPORTED;
     const int cg = cta_group_of(c);
     if (c.block_m != 128 * cg || (c.block_k != 64 && c.block_k != 128)) return HGEMM_ERR_UNSUPPORTED;
-    if (c.block_n < 32 || c.block_n > 256 || (c.block_n % 32) != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (c.block_n == 512) {
+        // the double-accumulator pair tile (256 x 512): whole tiles only, nothing that needs a spare accumulator or
+        // another column order
+        if (cg != 2 || c.split_k != 1 || c.tail_split >= 2 || c.swap_ab || (N % 512) != 0) return HGEMM_ERR_UNSUPPORTED;
+    } else if (c.block_n < 32 || c.block_n > 256 || (c.block_n % 32) != 0) {
+        return HGEMM_ERR_UNSUPPORTED;
+    }
     if (c.stages < 1 || c.stages > 12) return HGEMM_ERR_UNSUPPORTED;
     if (smem_bytes(c) > kSmemOptInBytes) return HGEMM_ERR_UNSUPPORTED;
     if (c.split_k < 1 || c.split_k > ceil_div(K, c.block_k)) return HGEMM_ERR_UNSUPPORTED;
@@ -132,7 +148,7 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
         if (c.split_k != 1 || (c.block_n % 64) != 0) return HGEMM_ERR_UNSUPPORTED;
         if (c.tail_split >= 2 && c.tail_mode == HGEMM_TAIL_N && (c.block_n % (64 * c.tail_split)) != 0) return HGEMM_ERR_UNSUPPORTED;
     }
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 2; ++i)
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
     if (c.accumulate != HGEMM_ACC_F32 && c.accumulate != HGEMM_ACC_F16) return HGEMM_ERR_UNSUPPORTED;
     // fp16 accumulators: no fp16 partial sums are exchanged, so no split along K
@@ -154,7 +170,9 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     }
     const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, c.block_n);
     if (tiles * c.split_k >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
-    if (workspace_bytes(M, N, K, c) > kMaxWorkspaceBytes) return HGEMM_ERR_UNSUPPORTED;
+    if (c.split_k > 1 && c.split_mode == HGEMM_SPLIT_WORKSPACE &&
+        tiles * c.split_k * cg * 128 * int64_t(c.block_n) * 4 > kMaxWorkspaceBytes)
+        return HGEMM_ERR_UNSUPPORTED;
     return HGEMM_OK;
 }
 
@@ -181,7 +199,8 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
 
     const int cg = cta_group_of(c);
     const int64_t units = std::max(1, num_sms / cg);
-    const SplitLayout L = split_layout(M, N, K, num_sms, c);
+    const SplitLayout L = split_layout(M, N, K, num_sms, c);   // (trades M and N itself for a swapped configuration)
+    if (c.swap_ab) std::swap(M, N);                            // from here on: the problem as the kernel tiles it
     const int64_t work = L.work_items;
     // a cut tail wave costs 1 / slices of a wave (plus the reduction, added below), or a little more than
     // 1 / pieces (narrower tiles run below the wide ones' rate)
@@ -293,14 +312,20 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
     auto add = [&](const hgemm_config_t &c) {
         if (validate(M, N, K, c) == HGEMM_OK) all.emplace_back(estimate_cycles(M, N, K, num_sms, c), c);
     };
+    // swap == 1: the operands trade places (few rows, many columns: the rows of B fill the MMA's 128-row side)
+    for (int swap = 0; swap < 2; ++swap) {
+    if (swap == 1 && !(M <= 256 && N >= 512 && (N % 8) == 0)) continue;
+    const int64_t Mk = swap ? N : M, Nk = swap ? M : N;              // the problem as the kernel tiles it
     for (int family = 0; family < 2; ++family) {
         const int cg = family == HGEMM_FAMILY_UMMA_2CTA ? 2 : 1;
         const int64_t units = std::max(1, num_sms / cg);
-        for (int32_t bn = 32; bn <= 256; bn += 32) {
-            if (bn > 32 && bn - 32 >= N) break;                       // a wider tile would only add padding
-            const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, bn);
+        for (int32_t bn = 32; bn <= 512; bn += (bn == 256 ? 256 : 32)) {      // 32 .. 256, then the 512-wide double tile
+            if (bn > 32 && bn - 32 >= Nk) break;                       // a wider tile would only add padding
+            if (bn == 512 && (cg != 2 || swap || (Nk % 512) != 0)) continue;
+            const int64_t tiles = ceil_div(Mk, 128 * cg) * ceil_div(Nk, bn);
             const int64_t tail = tiles % units;
             for (int32_t bk = 64; bk <= 128; bk += 64) {
+                if (bn == 512 && bk == 128) continue;                 // two stages only: not worth a candidate
                 if (bk == 128 && K < 128) continue;
                 const int64_t kb = ceil_div(K, bk);
                 for (int32_t split : kSplits) {
@@ -310,7 +335,7 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                         if (mode == 1 && (split == 1 || split * cg > 16)) continue;
                         for (int epi = 0; epi < 3; ++epi) {
                             if (split > 1 && epi != HGEMM_EPILOGUE_DIRECT) continue;
-                            if (epi == HGEMM_EPILOGUE_TMA_WIDE && (bn % 64) != 0) continue;
+                            if (epi == HGEMM_EPILOGUE_TMA_WIDE && ((bn % 64) != 0 || swap)) continue;
                             hgemm_config_t c;
                             std::memset(&c, 0, sizeof(c));
                             c.family = family;
@@ -320,11 +345,12 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                             c.split_k = split;
                             c.split_mode = mode;
                             c.epilogue = epi;
+                            c.swap_ab = swap;
                             c.stages = std::min<int32_t>(max_stages_of(c), 8);
                             if (c.stages < 1) continue;
-                            c.raster_group = raster_group_for(M, num_sms, c);
+                            c.raster_group = raster_group_for(Mk, num_sms, c);
                             add(c);
-                            if (split == 1 && tiles > units && tail > 0 && tail <= units / 2) {
+                            if (split == 1 && !swap && tiles > units && tail > 0 && tail <= units / 2) {
                                 const int32_t ts = int32_t(std::min<int64_t>(std::min<int64_t>(units / tail, 8), kb));
                                 if (ts >= 2) {
                                     hgemm_config_t t = c;
@@ -345,6 +371,7 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                 }
             }
         }
+    }
     }
     std::stable_sort(all.begin(), all.end(), [](const auto &a, const auto &b) { return a.first < b.first; });
     const int32_t n = int32_t(std::min<size_t>(all.size(), size_t(max)));
@@ -393,7 +420,7 @@ hgemm_status_t plan_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hge
     for (int i = 0; i < count; ++i) {
         const double scale = calib[i] > 0.0 ? calib[i] : calib_mean;
         hgemm_config_t c = nb[i].cfg;
-        c.raster_group = raster_group_for(M, num_sms, c);
+        c.raster_group = raster_group_for(c.swap_ab ? N : M, num_sms, c);
         c.tail_split = 0;
         c.tail_mode = HGEMM_TAIL_K;
         c.stages = std::min(c.stages, max_stages_of(c));
@@ -414,7 +441,7 @@ hgemm_status_t plan_config(int64_t M, int64_t N, int64_t K, int32_t num_sms, hge
                 d.epilogue = nb[i].cfg.split_k > 1 ? HGEMM_EPILOGUE_TMA : d.epilogue;
             }
             consider(d, scale);
-            if (d.split_k == 1) {
+            if (d.split_k == 1 && !d.swap_ab) {
                 // the last wave's tiles as column pieces, where the wave is at most half full
                 const int64_t units = std::max(1, num_sms / cg);
                 const int64_t tiles = ceil_div(M, 128 * cg) * ceil_div(N, d.block_n);

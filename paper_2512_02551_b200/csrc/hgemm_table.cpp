@@ -13,10 +13,11 @@ struct Entry {
     int32_t family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue;
     int32_t tail_mode;   // after the original columns, so that rows written before it existed still read as 0
     float us;            // time the tuner measured (0 in rows written before the column existed)
+    int32_t swap_ab, raster_mode;   // later columns again: absent from older rows, which then read 0
 };
 const Entry kTable[] = {
 #include "hgemm_table.inc"
-    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0.0f}   // sentinel
+    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0.0f, 0, 0}   // sentinel
 };
 } // namespace
 
@@ -36,6 +37,8 @@ hgemm_config_t config_of(const Entry &e)
     c.tail_mode = e.tail_mode;
     c.raster_group = e.raster_group;
     c.epilogue = e.epilogue;
+    c.swap_ab = e.swap_ab;
+    c.raster_mode = e.raster_mode;
     return c;
 }
 

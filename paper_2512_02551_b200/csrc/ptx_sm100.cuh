@@ -463,6 +463,11 @@ __device__ __forceinline__ uint32_t pack_half2_rn(uint32_t a_f32_bits, uint32_t 
     return *reinterpret_cast<uint32_t *>(&h);
 }
 
+__device__ __forceinline__ void st_shared_u16(uint32_t addr, unsigned short v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");

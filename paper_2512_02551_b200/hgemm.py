@@ -20,6 +20,7 @@ SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
 TAIL_K, TAIL_N = 0, 1
 ACC_F32, ACC_F16 = 0, 1
 LAYOUT_TN, LAYOUT_NN = 0, 1
+RASTER_SWEEP, RASTER_SERPENTINE = 0, 1
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
@@ -42,14 +43,16 @@ class Config(ctypes.Structure):
     _fields_ = [("family", ctypes.c_int32), ("block_m", ctypes.c_int32), ("block_n", ctypes.c_int32),
                 ("block_k", ctypes.c_int32), ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32),
                 ("raster_group", ctypes.c_int32), ("epilogue", ctypes.c_int32), ("split_mode", ctypes.c_int32),
-                ("tail_split", ctypes.c_int32), ("tail_mode", ctypes.c_int32), ("accumulate", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4)]
+                ("tail_split", ctypes.c_int32), ("tail_mode", ctypes.c_int32), ("accumulate", ctypes.c_int32),
+                ("swap_ab", ctypes.c_int32), ("raster_mode", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
 
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
 
     @classmethod
     def make(cls, family=FAMILY_UMMA_1CTA, block_n=128, stages=4, split_k=1, raster_group=8,
-             epilogue=EPILOGUE_DIRECT, block_k=64, split_mode=0, tail_split=0, tail_mode=0, accumulate=0) -> "Config":
+             epilogue=EPILOGUE_DIRECT, block_k=64, split_mode=0, tail_split=0, tail_mode=0, accumulate=0, swap_ab=0,
+             raster_mode=0) -> "Config":
         c = cls()
         c.family = family
         c.block_m = 256 if family == FAMILY_UMMA_2CTA else 128
@@ -63,6 +66,8 @@ class Config(ctypes.Structure):
         c.tail_split = tail_split
         c.tail_mode = tail_mode
         c.accumulate = accumulate
+        c.swap_ab = swap_ab
+        c.raster_mode = raster_mode
         return c
 
 

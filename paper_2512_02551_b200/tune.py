@@ -1,8 +1,10 @@
 """Per-shape tuner: times candidate configurations on the GPU and writes the planner's table.
 
-    python -m paper_2512_02551_b200.tune [--out DIR] [--shapes MxNxK ...] [--top 20] [--resume]
+    python -m paper_2512_02551_b200.tune [--out DIR] [--shapes MxNxK ...] [--grid10] [--top 20] [--resume]
+                                         [--time-limit SECONDS] [--merge-into csrc/hgemm_table.inc]
 
-For every shape of the 9 x 9 x 9 grid (or the shapes given) it ranks the legal configurations with
+For every shape of the 9 x 9 x 9 grid (with --grid10: the 271 shapes that the paper's tenth grid value,
+16384, adds; or the shapes given) it ranks the legal configurations with
 the planner's cost model, times the best `--top` of them plus the heuristic's own choice, checks
 the winner against torch.matmul, and writes
   DIR/tune.jsonl        one line per shape (resumable with --resume)
@@ -40,15 +42,27 @@ def max_stages(family: int, bn: int, bk: int, epilogue: int = hgemm.EPILOGUE_TMA
 
 def candidates(M: int, N: int, K: int):
     out = []
+    for swap in (0, 1):
+        if swap and not (M <= 256 and N >= 512 and N % 8 == 0):
+            continue
+        out += _candidates(M, N, K, swap)
+    return out
+
+
+def _candidates(M: int, N: int, K: int, swap: int):
+    """The configurations of one orientation; with swap = 1 the kernel tiles the transposed problem."""
+    out = []
+    Mk, Nk = (N, M) if swap else (M, N)
     for family in (0, 1):
         cg = family + 1
         units = NUM_SMS // cg
-        for bn in range(32, 257, 32):
-            if bn > 32 and bn - 32 >= N:
+        widths = list(range(32, 257, 32)) + ([512] if family == 1 and not swap and Nk % 512 == 0 else [])   # 512: the double tile
+        for bn in widths:
+            if bn > 32 and bn - 32 >= Nk:
                 break
-            tiles = -(-M // (128 * cg)) * -(-N // bn)
+            tiles = -(-Mk // (128 * cg)) * -(-Nk // bn)
             for bk in (64, 128):
-                if bk == 128 and K < 128:
+                if bk == 128 and (K < 128 or bn == 512):
                     continue
                 st = min(max_stages(family, bn, bk), 8)
                 if st < 1:
@@ -58,20 +72,22 @@ def candidates(M: int, N: int, K: int):
                         break
                     if split > 1 and tiles * split > 2 * units:
                         continue
-                    rg = max(1, min(-(-M // (128 * cg)), round((units * bn / (128.0 * cg)) ** 0.5)))
+                    rg = max(1, min(-(-Mk // (128 * cg)), round((units * bn / (128.0 * cg)) ** 0.5)))
                     modes = (0,) if split == 1 else ((0, 1) if split * cg <= 16 else (0,))
                     for mode in modes:
                         epis = (hgemm.EPILOGUE_DIRECT,)
                         if split == 1:
-                            epis = (hgemm.EPILOGUE_TMA, hgemm.EPILOGUE_DIRECT) + ((hgemm.EPILOGUE_TMA_WIDE,) if bn % 64 == 0 else ())
+                            epis = (hgemm.EPILOGUE_TMA, hgemm.EPILOGUE_DIRECT) + ((hgemm.EPILOGUE_TMA_WIDE,) if bn % 64 == 0 and not swap else ())
                         for epi in epis:
                             st = min(max_stages(family, bn, bk, epi), 8)      # the wide epilogue's staging leaves fewer stages
                             if st < 1:
                                 continue
                             c = hgemm.Config.make(family=family, block_n=bn, stages=st, split_k=split, raster_group=rg,
-                                                  epilogue=epi, block_k=bk, split_mode=mode)
+                                                  epilogue=epi, block_k=bk, split_mode=mode, swap_ab=swap)
                             if hgemm.validate_config(M, N, K, c) == hgemm.OK:
                                 out.append(c)
+                            if swap:
+                                continue                      # no tail cuts in the swapped orientation
                             tail = tiles % units
                             if split == 1 and tiles > units and 0 < tail <= units // 2:
                                 ts = min(units // tail, 8, -(-K // bk))
@@ -102,9 +118,15 @@ def batch_ms(fn, n: int, stream) -> float:
     return e0.elapsed_time(e1) / n
 
 
+def ctypes_copy(dst: hgemm.Config, src: hgemm.Config) -> None:
+    import ctypes
+    ctypes.memmove(ctypes.byref(dst), ctypes.byref(src), ctypes.sizeof(hgemm.Config))
+
+
 def key(c: hgemm.Config):
     d = c.as_dict()
-    return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "tail_mode", "raster_group", "epilogue"))
+    return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "tail_mode", "raster_group", "epilogue",
+                                "swap_ab", "raster_mode"))
 
 
 def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, stream, explore: int = 0) -> dict:
@@ -167,6 +189,35 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
             sustained[key(c)] = batch_ms(run, n, stream)
         final = sorted(((sustained[key(c)], e, c) for _, e, c in final), key=lambda r: r[0])
     best_t, _, best = final[0]
+    # The tile order of the winner: the candidates above all carry the raster group of a square-ish wave; with more
+    # tiles than SMs other groups, and the serpentine sweep, change what stays in L2 between waves.  Timed the same
+    # way as the finalists (sustained for long kernels), the winner's own order included again.
+    cg = best.family + 1
+    tiles_m = -(-(N if best.swap_ab else M) // (128 * cg))
+    tiles_n = -(-(M if best.swap_ab else N) // best.block_n)
+    if tiles_m > 1 and tiles_n > 1 and tiles_m * tiles_n > NUM_SMS // cg and best.split_k == 1:
+        sustained = best_t > 0.08
+        orders = {(best.raster_group, best.raster_mode)}
+        for rg in (1, 2, 4, 8, 16, tiles_m):
+            for rm in (hgemm.RASTER_SWEEP, hgemm.RASTER_SERPENTINE):
+                orders.add((min(rg, tiles_m), rm))
+        timed = []
+        order_list = sorted(orders)
+        rng.shuffle(order_list)
+        for rg, rm in order_list:
+            c = hgemm.Config()
+            ctypes_copy(c, best)
+            c.raster_group, c.raster_mode = rg, rm
+            if plan.try_set_config(c) != hgemm.OK:
+                continue
+            for _ in range(3):
+                run()
+            n = max(5, min(2000, int(0.25 / (best_t * 1e-3)))) if sustained else max(3, min(100, int(0.6 / max(best_t, 1e-3))))
+            t = batch_ms(run, n, stream) if sustained else statistics.median(batch_ms(run, n, stream) for _ in range(3))
+            timed.append((t, c))
+        timed.sort(key=lambda r: r[0])
+        if timed and timed[0][0] < 0.995 * min(t for t, c in timed if (c.raster_group, c.raster_mode) == (best.raster_group, best.raster_mode)):
+            best_t, best = timed[0]
     plan.set_config(best)
     C.zero_()
     run()
@@ -195,13 +246,41 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
 def write_table(rows, path):
     with open(path, "w") as f:
         f.write("// Tuned per-shape configurations for B200, written by tune.py on the GPU box.\n")
-        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode, measured us}\n")
+        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode, measured us, swap_ab, raster_mode}\n")
         for r in rows:
             if not r["ok"]:
                 continue
             b = r["best"]
             f.write(f"{{{r['M']}, {r['N']}, {r['K']}, {b['family']}, {b['block_n']}, {b['block_k']}, {b['stages']}, "
-                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}, {b.get('tail_mode', 0)}, {r['us']:.2f}f}},\n")
+                    f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}, {b.get('tail_mode', 0)}, {r['us']:.2f}f, "
+                    f"{b.get('swap_ab', 0)}, {b.get('raster_mode', 0)}}},\n")
+
+
+def merge_table(new_rows, path):
+    """Rewrites the table at `path`: rows of shapes in `new_rows` are replaced, every other row is kept."""
+    import re
+    fresh = {(r["M"], r["N"], r["K"]): r for r in new_rows if r["ok"]}
+    kept, header = [], []
+    if os.path.exists(path):
+        for line in open(path):
+            m = re.match(r"\{(\d+), (\d+), (\d+),", line)
+            if m is None:
+                if line.startswith("//"):
+                    header.append(line)
+                continue
+            if tuple(int(v) for v in m.groups()) not in fresh:
+                kept.append(line)
+    tmp = path + ".new"
+    write_table(list(fresh.values()), tmp)
+    body = [line for line in open(tmp) if not line.startswith("//")]
+    head = [line for line in open(tmp) if line.startswith("//")]
+    os.remove(tmp)
+
+    def shape_key(line):
+        return tuple(int(v) for v in re.match(r"\{(\d+), (\d+), (\d+),", line).groups())
+    with open(path, "w") as f:
+        f.writelines(head)
+        f.writelines(sorted(kept + body, key=shape_key))
 
 
 def main():
@@ -211,10 +290,18 @@ def main():
     ap.add_argument("--top", type=int, default=20)
     ap.add_argument("--resume", action="store_true")
     ap.add_argument("--explore", type=int, default=0, help="also time this many randomly drawn candidates per shape")
+    ap.add_argument("--grid10", action="store_true", help="the 271 shapes of the ten-value grid that contain 16384")
+    ap.add_argument("--time-limit", type=float, default=0.0, help="stop starting new shapes after this many seconds (resume later)")
+    ap.add_argument("--merge-into", metavar="TABLE", help="replace these shapes' rows in an existing table file, keep its other rows")
     args = ap.parse_args()
     os.makedirs(args.out, exist_ok=True)
-    shapes = ([tuple(int(v) for v in s.lower().split("x")) for s in args.shapes] if args.shapes
-              else [(M, N, K) for M in GRID for N in GRID for K in GRID])
+    if args.shapes:
+        shapes = [tuple(int(v) for v in s.lower().split("x")) for s in args.shapes]
+    elif args.grid10:
+        g10 = GRID + [16384]
+        shapes = [(M, N, K) for M in g10 for N in g10 for K in g10 if 16384 in (M, N, K)]
+    else:
+        shapes = [(M, N, K) for M in GRID for N in GRID for K in GRID]
     log_path = os.path.join(args.out, "tune.jsonl")
     done = {}
     if args.resume and os.path.exists(log_path):
@@ -229,15 +316,21 @@ def main():
     C_all = torch.empty(mx_mn, dtype=torch.float16, device="cuda")
     rng = random.Random(2512)
     rows = []
+    import time
+    started = time.time()
     with hgemm.Context(0) as ctx, open(log_path, "a" if args.resume else "w") as log:
         for (M, N, K) in shapes:
             r = done.get((M, N, K))
             if r is None:
+                if args.time_limit > 0 and time.time() - started > args.time_limit:
+                    continue                                   # out of time: left for a later --resume run
                 r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream, args.explore)
                 log.write(json.dumps(r) + "\n")
                 log.flush()
             rows.append(r)
     write_table(rows, os.path.join(args.out, "hgemm_table.inc"))
+    if args.merge_into:
+        merge_table(rows, args.merge_into)
     import math
     g = math.exp(sum(math.log(r["torch_us"] / r["us"]) for r in rows) / len(rows))
     bad = [r for r in rows if not r["ok"]]

@@ -198,6 +198,171 @@ def test_unit_shapes_wide_stages_and_cluster_split(ctx, gu, case):
         plan.close()
 
 
+# ---- swapped operands: the rows of B on the MMA's 128-row side, the tile stored transposed ----------------------
+
+SWAP_CASES = [
+    # M, N, K, family, bn (covers rows of A), stages, split, block_k, split mode, epilogue
+    (64, 128, 64, F1, 64, 2, 1, 64, WORKSPACE, TMA),          # one tile
+    (64, 256, 256, F2, 64, 4, 1, 64, WORKSPACE, TMA),         # one pair tile: each CTA stages 32 rows of A
+    (64, 4096, 1024, F2, 64, 4, 1, 128, WORKSPACE, TMA),      # the skinny projection case, 16 pair tiles
+    (128, 2048, 512, F2, 128, 4, 1, 64, WORKSPACE, DIRECT),   # 2-byte transposed stores
+    (256, 1536, 384, F2, 256, 3, 1, 128, WORKSPACE, TMA),
+    (200, 1000, 328, F1, 224, 3, 1, 64, WORKSPACE, TMA),      # ragged M, N (a multiple of 8) and K
+    (37, 520, 200, F2, 64, 4, 1, 64, WORKSPACE, TMA),         # fewer rows than one box; the last pair tile is mostly empty
+    (37, 520, 200, F1, 32, 4, 1, 64, WORKSPACE, DIRECT),      # two column tiles of the kernel's problem
+    (96, 2048, 4096, F1, 96, 4, 4, 64, CLUSTER, DIRECT),      # K slices summed inside a cluster, stored transposed
+    (64, 1024, 8192, F2, 64, 4, 4, 64, CLUSTER, DIRECT),      # clusters of four pairs
+    (128, 512, 2048, F1, 128, 4, 3, 64, WORKSPACE, DIRECT),   # K slices through the workspace
+    (256, 768, 1152, F2, 128, 4, 2, 128, WORKSPACE, DIRECT),  # two column tiles per pair row, uneven slices
+    (1000, 136, 320, F1, 128, 4, 1, 64, WORKSPACE, TMA),      # many rows of A after all: eight column tiles, raster groups
+]
+
+
+@pytest.mark.parametrize("case", SWAP_CASES, ids=lambda c: "x".join(map(str, c[:3])) + f"-f{c[3]}bn{c[4]}k{c[6]}m{c[8]}e{c[9]}")
+def test_swapped_operands(ctx, gu, case):
+    """swap_ab = 1 computes the same C: exact on integer inputs, the contract on random ones, nothing written
+    outside C (guard bands), every element written (sentinel)."""
+    import oracle
+    M, N, K, family, bn, stages, split, bk, mode, epi = case
+    cfg = hgemm.Config.make(family=family, block_n=bn, stages=stages, split_k=split, raster_group=3, epilogue=epi, block_k=bk,
+                            split_mode=mode, swap_ab=1, raster_mode=hgemm.RASTER_SERPENTINE if M > 256 else hgemm.RASTER_SWEEP)
+    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    assert plan.config.swap_ab == 1
+    gu.assert_close_full(C, A, B, f"swapped {case}")
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"swapped {case} integers")
+    # the general form through the same configuration (exact: 0/1 operands, small integers in C)
+    Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
+    C0 = inputs.draw(33, inputs.TAG_A, M, N, "int5", "cuda")
+    buf, Cs = gu.alloc_c_with_guards(M, N)
+    Cs.copy_(C0)
+    plan.run_scaled(2.0, -3.0, Ab, Bb, Cs)
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    assert gu.guards_intact(buf, M, N)
+    gu.assert_exact(Cs, oracle.hgemm_scaled_full(inputs.bits(Ab), inputs.bits(Bb), inputs.bits(C0), 2.0, -3.0), f"swapped {case} scaled")
+    plan.close()
+
+
+def test_swapped_operands_rules(ctx):
+    ok = hgemm.Config.make(family=F2, block_n=64, stages=4, epilogue=TMA, swap_ab=1)
+    assert hgemm.validate_config(64, 4096, 4096, ok) == hgemm.OK
+    assert hgemm.validate_config(64, 4100, 4096, ok) == hgemm.ERR_UNSUPPORTED            # rows of C must be multiples of 16 bytes
+    for kw in (dict(epilogue=WIDE), dict(accumulate=hgemm.ACC_F16), dict(tail_split=2), dict(swap_ab=2)):
+        c = hgemm.Config.make(**{**dict(family=F2, block_n=64, stages=4, epilogue=TMA, swap_ab=1), **kw})
+        assert hgemm.validate_config(64, 4096, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
+    # K that needs padded copies works too: the copies trade places with the operands
+    plan = ctx.plan(48, 264, 100)
+    plan.set_config(hgemm.Config.make(family=F1, block_n=64, stages=3, epilogue=TMA, swap_ab=1))
+    A, B = inputs.make_ab(48, 264, 100, "int5", "cuda")
+    C = torch.zeros(48, 264, dtype=torch.float16, device="cuda")
+    plan.run(A, B, C)
+    torch.cuda.synchronize()
+    assert torch.equal(C.float(), A.float() @ B.float().T)
+    # the NN layout has no swapped form
+    nn = ctx.plan(64, 512, 256, layout=hgemm.LAYOUT_NN)
+    assert nn.try_set_config(hgemm.Config.make(family=F1, block_n=64, stages=3, epilogue=TMA, swap_ab=1)) == hgemm.ERR_UNSUPPORTED
+    nn.close()
+    plan.close()
+
+
+@pytest.mark.parametrize("family", [F1, F2])
+@pytest.mark.parametrize("shape,bn,raster", [((1024, 2048, 128), 32, 3), ((2048, 1536, 256), 128, 4), ((1300, 1000, 192), 96, 2),
+                                              ((4096, 4096, 512), 256, 5)])
+def test_serpentine_raster(ctx, gu, family, shape, bn, raster):
+    """The serpentine tile order visits every tile exactly once: same results as the plain sweep, bit for bit, with
+    full and ragged last raster groups and more tiles than SMs."""
+    import oracle
+    M, N, K = shape
+    A, B = inputs.make_ab(M, N, K, "int5", "cuda")
+    want = oracle.hgemm_full(inputs.bits(A), inputs.bits(B))
+    for epi in (TMA, DIRECT):
+        cfg = hgemm.Config.make(family=family, block_n=bn, stages=3, raster_group=raster, epilogue=epi, raster_mode=hgemm.RASTER_SERPENTINE)
+        C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+        gu.assert_exact(C, want, f"serpentine {shape} family={family} epi={epi}")
+        plan.close()
+    assert hgemm.validate_config(M, N, K, hgemm.Config.make(block_n=bn, stages=3, raster_mode=2)) == hgemm.ERR_UNSUPPORTED
+
+
+# ---- the 256 x 512 pair tile that fills both accumulators ---------------------------------------------------------
+
+DUAL_CASES = [
+    # M, N, K, block_k, stages, epilogue, raster
+    (256, 512, 64, 64, 2, TMA, 1),          # one tile, one k-block
+    (256, 512, 1024, 64, 4, TMA, 1),        # ring wraps
+    (300, 1024, 200, 64, 3, DIRECT, 1),     # ragged M and K: dead rows, zero-filled k tail
+    (512, 1536, 384, 128, 2, TMA, 2),       # 128-wide stages (two of them fill shared memory)
+    (4096, 8192, 128, 64, 4, TMA, 4),       # 256 tiles on 74 pairs: up to four tiles per pair, the accumulators' phase alternates
+    (2048, 4096, 256, 64, 3, WIDE, 3),      # 64-column store boxes
+    (100, 512, 72, 64, 4, TMA, 1),          # fewer rows than one CTA's 128
+]
+
+
+@pytest.mark.parametrize("case", DUAL_CASES, ids=lambda c: "x".join(map(str, c[:3])) + f"-bk{c[3]}s{c[4]}e{c[5]}")
+def test_double_accumulator_tile(ctx, gu, case):
+    """block_n = 512: each accumulator column must land in the column of C that the two-MMA layout assigns it --
+    a wrong permutation fails the integer case on nearly every element."""
+    import oracle
+    M, N, K, bk, stages, epi, raster = case
+    cfg = hgemm.Config.make(family=F2, block_n=512, stages=stages, raster_group=raster, epilogue=epi, block_k=bk,
+                            raster_mode=hgemm.RASTER_SERPENTINE if raster > 1 else hgemm.RASTER_SWEEP)
+    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, plan = gu.run_gemm(ctx, Ai, Bi, cfg)
+    assert plan.config.block_n == 512
+    if M * N * K <= gu.FULL_CHECK_VOLUME // 4:
+        gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"double tile {case} integers")
+        A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+        C, _, _ = gu.run_gemm(ctx, A, B, plan=plan)
+        gu.assert_close_full(C, A, B, f"double tile {case}")
+    else:
+        # sampled: 4096 seeded entries, one full row, one full column -- exact values on integer inputs
+        ii, jj, row, col = inputs.sample_indices(11, M, N, 4096)
+        ii = np.concatenate([ii, np.full(N, row, dtype=np.int64), np.arange(M, dtype=np.int64)])
+        jj = np.concatenate([jj, np.arange(N, dtype=np.int64), np.full(M, col, dtype=np.int64)])
+        ref = oracle.hgemm_sampled(inputs.bits(Ai), inputs.bits(Bi), ii, jj)
+        got = gu.bits_to_f64(inputs.bits(Ci[torch.from_numpy(ii).cuda(), torch.from_numpy(jj).cuda()]))
+        assert np.array_equal(got, ref), f"double tile {case}: sampled integer entries differ"
+        # and every entry against the library's own 256-wide pair tile (bit for bit: the same fp32 sums in the same order)
+        C2, _, _ = gu.run_gemm(ctx, Ai, Bi, hgemm.Config.make(family=F2, block_n=256, stages=3, raster_group=4, epilogue=TMA), plan=plan)
+        assert torch.equal(Ci.view(torch.int16), C2.view(torch.int16))
+    plan.close()
+
+
+def test_double_accumulator_tile_other_forms(ctx, gu):
+    import oracle
+    M, N, K = 384, 1024, 320
+    cfg = hgemm.Config.make(family=F2, block_n=512, stages=4, raster_group=1, epilogue=TMA, block_k=64)
+    plan = ctx.plan(M, N, K)
+    plan.set_config(cfg)
+    # alpha / beta (exact: 0/1 operands, small integers in C)
+    Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
+    C0 = inputs.draw(35, inputs.TAG_A, M, N, "int5", "cuda")
+    buf, Cs = gu.alloc_c_with_guards(M, N)
+    Cs.copy_(C0)
+    plan.run_scaled(-1.0, 2.0, Ab, Bb, Cs)
+    assert ctx.last_device_status() == (hgemm.OK, 0) and gu.guards_intact(buf, M, N)
+    gu.assert_exact(Cs, oracle.hgemm_scaled_full(inputs.bits(Ab), inputs.bits(Bb), inputs.bits(C0), -1.0, 2.0), "double tile scaled")
+    # fp16 accumulators
+    cfg.accumulate = hgemm.ACC_F16
+    plan.set_config(cfg)
+    C, _, _ = gu.run_gemm(ctx, Ab, Bb, plan=plan)
+    gu.assert_exact(C, oracle.hgemm_full(inputs.bits(Ab), inputs.bits(Bb)), "double tile, fp16 accumulators, 0/1 operands")
+    plan.close()
+    # rules
+    ok = hgemm.Config.make(family=F2, block_n=512, stages=4, epilogue=TMA)
+    assert hgemm.validate_config(512, 1024, 512, ok) == hgemm.OK
+    assert hgemm.validate_config(512, 1000, 512, ok) == hgemm.ERR_UNSUPPORTED                       # N must be a multiple of 512
+    for kw in (dict(family=F1), dict(split_k=2), dict(tail_split=2), dict(swap_ab=1), dict(stages=5)):
+        c = hgemm.Config.make(**{**dict(family=F2, block_n=512, stages=4, epilogue=TMA), **kw})
+        assert hgemm.validate_config(512, 1024, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
+    nn = ctx.plan(512, 1024, 512, layout=hgemm.LAYOUT_NN)
+    assert nn.try_set_config(ok) == hgemm.ERR_UNSUPPORTED
+    nn.close()
+
+
 def test_dependent_launch_keeps_stream_order(ctx, gu):
     """Launches may become resident before the kernel ahead of them has finished.  A chain in which each
     GEMM consumes the previous GEMM's output must still see stream order: C1 = A B1^T, C2 = C1 B2^T."""

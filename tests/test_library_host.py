@@ -72,7 +72,7 @@ def test_validate_rejects_illegal_configs(lib):
     c.block_m = 256                           # wrong for the 1-CTA family
     assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
     c = hgemm.Config.make(block_n=128, stages=4)
-    c.reserved[3] = 1
+    c.reserved[1] = 1
     assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
     # cluster split-K: at most 16 CTAs per cluster (16 slices, 8 for CTA pairs), the ring must hold the fp32 partial
     assert hgemm.validate_config(M, N, 4096, hgemm.Config.make(block_n=128, stages=4, split_k=8, split_mode=1)) == hgemm.OK
