@@ -61,7 +61,11 @@ typedef enum {
  * for small and for large shapes; the families here are this library's own). */
 enum {
     HGEMM_FAMILY_UMMA_1CTA = 0, /* persistent, warp-specialised, 128 x block_n tiles, one CTA per tile */
-    HGEMM_FAMILY_UMMA_2CTA = 1  /* the same with CTA pairs: 256 x block_n tiles, B split across the pair */
+    HGEMM_FAMILY_UMMA_2CTA = 1, /* the same with CTA pairs: 256 x block_n tiles, B split across the pair */
+    HGEMM_FAMILY_LIGHT = 2      /* the small-problem kernel: one 128 x block_n tile per CTA, no persistent loop, one
+                                   accumulator, six warps, only the shared memory it uses; its first loads leave before
+                                   the CTA's set-up has finished.  Needs K % 8 == 0 and N % 8 == 0, split_k == 1, no
+                                   tail_split, no swap_ab, fp32 accumulators, the TN layout, HGEMM_EPILOGUE_TMA */
 };
 
 /* Where the fp32 partial sums of a split-K tile meet.  Both sum the slices in slice
@@ -112,7 +116,7 @@ enum {
  * count and block-swizzle stride of sections 5.2 and 6, plus split-K). */
 typedef struct {
     int32_t family;       /* HGEMM_FAMILY_* */
-    int32_t block_m;      /* 128 (1-CTA) or 256 (2-CTA pair) */
+    int32_t block_m;      /* 128 (1-CTA and light families) or 256 (2-CTA pair) */
     int32_t block_n;      /* multiple of 32 in [32, 256]; or 512 (CTA-pair family only): a 256 x 512 tile held in both
                              tensor-memory accumulators at once, two MMAs per K step sharing the A tile -- a quarter less
                              shared-memory fill per flop than 256 x 256, no overlap of a tile's epilogue with the next
@@ -155,7 +159,8 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device);
 /* Free the context, every plan it still owns and their workspaces. */
 hgemm_status_t hgemm_destroy(hgemm_ctx_t *ctx);
 
-/* Plan one (M, N, K): picks a configuration (tuned table, else heuristic) and
+/* Plan one (M, N, K): picks a configuration (tuned table, else heuristic; rows of a table file named
+ * by the environment variable HGEMM_TABLE, in the syntax the tuner writes, override the built-in table) and
  * allocates the split-K workspace if the configuration needs one.  May call
  * cudaMalloc/cudaMemset (synchronising); call it outside timed regions and
  * outside stream capture. */
@@ -349,8 +354,8 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
  * instrumented instantiation of the kernel, which is 10-15 % slower on small and
  * mid-size shapes than the one that runs otherwise: the stamps describe the
  * pipeline's structure and proportions, not the production kernel's absolute times.
- * The instrumented kernels do not exist for swapped-operand configurations (swap_ab = 1)
- * nor for the 512-wide tile:
+ * The instrumented kernels do not exist for swapped-operand configurations (swap_ab = 1),
+ * for the 512-wide tile or for the light family:
  * hgemm_run returns HGEMM_ERR_UNSUPPORTED for such a plan while a trace buffer or a skip
  * mask is set. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);

@@ -10,6 +10,7 @@
 
 #include "../../include/hgemm.h"
 #include "hgemm_kernel.cuh"
+#include "hgemm_light_kernel.cuh"
 #include "hgemm_planner.h"
 
 using hgemm_dev::KernelParams;
@@ -124,6 +125,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     if (pl->layout == HGEMM_LAYOUT_NN && (cfg.block_n % (64 * cg)) != 0) return HGEMM_ERR_UNSUPPORTED;
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.swap_ab) return HGEMM_ERR_UNSUPPORTED;   // the swapped form is built for K-contiguous operands
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.block_n == 512) return HGEMM_ERR_UNSUPPORTED;   // so is the double-accumulator tile
+    if (pl->layout == HGEMM_LAYOUT_NN && cfg.family == HGEMM_FAMILY_LIGHT) return HGEMM_ERR_UNSUPPORTED;   // and the light kernel
     // row-major B is staged in blocks of 64 columns: column pieces of tail tiles must be whole blocks per CTA
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 &&
         ((cfg.block_n / cfg.tail_split) % (64 * cg)) != 0)
@@ -232,6 +234,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         p.fd_pieces = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.tail_pieces)));
     }
     p.tmem_cols = cfg.block_n == 512 ? 512 : pow2_at_least(2 * cfg.block_n);   // two accumulators either way
+    if (cfg.family == HGEMM_FAMILY_LIGHT) p.tmem_cols = pow2_at_least(cfg.block_n);   // ... except in the light kernel: one
     p.ragged_n = (!cfg.swap_ab && (pl->N % 8) != 0) ? 1 : 0;   // (a swapped configuration needs N % 8 == 0 and stores by its own rule)
     p.epilogue_tma = (cfg.epilogue != HGEMM_EPILOGUE_DIRECT && cfg.split_k == 1 && !p.ragged_n)             // whole tiles only
                          ? (cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? 2 : 1) : 0;
@@ -245,7 +248,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.counters = pl->counters;
     p.status = ctx->d_status + pl->status_slot;
     p.cluster_split = cluster_split ? 1 : 0;
-    p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d && pl->layout == HGEMM_LAYOUT_TN) ? 1 : 0;
+    p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d && pl->layout == HGEMM_LAYOUT_TN && cfg.family != HGEMM_FAMILY_LIGHT) ? 1 : 0;
     p.C = nullptr;
     p.wait_budget = ctx->wait_budget;
     const int units = std::max(1, ctx->num_sms / cg);
@@ -256,6 +259,12 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     // CTAs can never wait on each other's tensor-memory allocation.  (Letting small configurations ask for what
     // they use, so that the next call's CTAs become resident beside this call's, made those calls slower.)
     pl->smem = int(hgemm_host::kSmemOptInBytes);
+    if (cfg.family == HGEMM_FAMILY_LIGHT) {
+        // one CTA per tile, and only the shared memory the configuration uses
+        pl->grid = p.tiles_m * p.tiles_n;
+        pl->cluster_dim = 1;
+        pl->smem = int(hgemm_host::smem_bytes(cfg));
+    }
     pl->maps_used = pl->maps_next = 0;   // the B box depends on the configuration
     return HGEMM_OK;
 }
@@ -417,6 +426,8 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
         for (int k = 0; k < 6 && e == cudaSuccess; ++k) {           // the double-accumulator instantiations
             const void *fn_k = kernel_for(2, (k & 1) != 0, 0, k >= 2, false, k >= 4 ? 2 : 1, false, true);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
@@ -805,11 +816,18 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     const KernelParams &kp = plan->params;
     const bool trace = kp.trace != nullptr || kp.debug_skip != 0;
     const bool plain = !kp.scaled && !kp.acc_f16 && !kp.ragged_n && !kp.b_row_major && kp.tail_pieces <= 1;
-    if (trace && (kp.transposed || kp.block_n == 512)) return HGEMM_ERR_UNSUPPORTED;   // no instrumented kernels for these two
+    const bool light = plan->cfg.family == HGEMM_FAMILY_LIGHT;
+    if (trace && (kp.transposed || kp.block_n == 512 || light)) return HGEMM_ERR_UNSUPPORTED;   // no instrumented kernels for these
     const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
                                 trace, kp.block_k / 64, kp.transposed != 0, kp.block_n == 512);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
-    e = cudaLaunchKernelExC(&lc, fn, args);
+    if (light) {
+        void *largs[4] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &plan->params};
+        lc.blockDim = dim3(hgemm_dev::kLightThreads, 1, 1);
+        e = cudaLaunchKernelExC(&lc, reinterpret_cast<const void *>(hgemm_dev::hgemm_light_kernel), largs);
+    } else {
+        e = cudaLaunchKernelExC(&lc, fn, args);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;
 }

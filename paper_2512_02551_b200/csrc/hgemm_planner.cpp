@@ -27,6 +27,7 @@ int64_t stage_bytes(const hgemm_config_t &c)
 // Store staging of the eight epilogue warps: two 2 KB boxes each, or two 4 KB ones for the wide TMA epilogue.
 int64_t staging_bytes(const hgemm_config_t &c)
 {
+    if (c.family == HGEMM_FAMILY_LIGHT) return kStagingBytes / 2;        // four epilogue warps
     return c.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? 2 * kStagingBytes : kStagingBytes;
 }
 
@@ -125,7 +126,13 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
             return HGEMM_ERR_UNSUPPORTED;
         std::swap(M, N);
     }
-    if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA) return HGEMM_ERR_UNSUPPORTED;
+    if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA && c.family != HGEMM_FAMILY_LIGHT) return HGEMM_ERR_UNSUPPORTED;
+    if (c.family == HGEMM_FAMILY_LIGHT) {
+        // one plain tile per CTA: nothing that needs the persistent kernel's extra paths
+        if (c.split_k != 1 || c.tail_split >= 2 || c.swap_ab || c.accumulate != HGEMM_ACC_F32 || c.epilogue != HGEMM_EPILOGUE_TMA ||
+            c.raster_mode != HGEMM_RASTER_SWEEP || c.block_n > 256 || (K % 8) != 0 || (N % 8) != 0)
+            return HGEMM_ERR_UNSUPPORTED;
+    }
     const int cg = cta_group_of(c);
     if (c.block_m != 128 * cg || (c.block_k != 64 && c.block_k != 128)) return HGEMM_ERR_UNSUPPORTED;
     if (c.block_n == 512) {
@@ -239,6 +246,12 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
         }
     }
     t = std::max(t, bytes / kHbmBytesPerClk);
+    if (c.family == HGEMM_FAMILY_LIGHT) {
+        // not persistent: every wave of CTAs pays its own start, and nothing overlaps a tile's epilogue; in exchange
+        // the set-up is shorter (its first loads overlap it).  Not fitted: a ranking hint so that the tuner times it
+        const double waves = double(ceil_div(L.tiles, units));
+        t = t - 600.0 + (waves - 1.0) * (epilogue + 0.5 * kFillLatency);
+    }
     return t + kLaunch;
 }
 
@@ -316,12 +329,14 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
     for (int swap = 0; swap < 2; ++swap) {
     if (swap == 1 && !(M <= 256 && N >= 512 && (N % 8) == 0)) continue;
     const int64_t Mk = swap ? N : M, Nk = swap ? M : N;              // the problem as the kernel tiles it
-    for (int family = 0; family < 2; ++family) {
+    for (int family = 0; family < 3; ++family) {
+        const bool light = family == HGEMM_FAMILY_LIGHT;
+        if (light && (swap || (K % 8) != 0 || (N % 8) != 0)) continue;
         const int cg = family == HGEMM_FAMILY_UMMA_2CTA ? 2 : 1;
         const int64_t units = std::max(1, num_sms / cg);
         for (int32_t bn = 32; bn <= 512; bn += (bn == 256 ? 256 : 32)) {      // 32 .. 256, then the 512-wide double tile
             if (bn > 32 && bn - 32 >= Nk) break;                       // a wider tile would only add padding
-            if (bn == 512 && (cg != 2 || swap || (Nk % 512) != 0)) continue;
+            if (bn == 512 && (family != HGEMM_FAMILY_UMMA_2CTA || swap || (Nk % 512) != 0)) continue;
             const int64_t tiles = ceil_div(Mk, 128 * cg) * ceil_div(Nk, bn);
             const int64_t tail = tiles % units;
             for (int32_t bk = 64; bk <= 128; bk += 64) {
@@ -330,11 +345,12 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                 const int64_t kb = ceil_div(K, bk);
                 for (int32_t split : kSplits) {
                     if (split > kb) break;
-                    if (split > 1 && tiles * split > 2 * units) continue;   // split-K only to fill an under-full machine
+                    if (split > 1 && (light || tiles * split > 2 * units)) continue;   // split-K only to fill an under-full machine
                     for (int mode = 0; mode < 2; ++mode) {
                         if (mode == 1 && (split == 1 || split * cg > 16)) continue;
                         for (int epi = 0; epi < 3; ++epi) {
                             if (split > 1 && epi != HGEMM_EPILOGUE_DIRECT) continue;
+                            if (light && epi != HGEMM_EPILOGUE_TMA) continue;
                             if (epi == HGEMM_EPILOGUE_TMA_WIDE && ((bn % 64) != 0 || swap)) continue;
                             hgemm_config_t c;
                             std::memset(&c, 0, sizeof(c));
@@ -347,10 +363,11 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                             c.epilogue = epi;
                             c.swap_ab = swap;
                             c.stages = std::min<int32_t>(max_stages_of(c), 8);
+                            if (light) c.stages = int32_t(std::min<int64_t>(std::min<int32_t>(max_stages_of(c), 12), kb));   // no more stages than k-blocks
                             if (c.stages < 1) continue;
-                            c.raster_group = raster_group_for(Mk, num_sms, c);
+                            c.raster_group = light ? 1 : raster_group_for(Mk, num_sms, c);
                             add(c);
-                            if (split == 1 && !swap && tiles > units && tail > 0 && tail <= units / 2) {
+                            if (split == 1 && !swap && !light && tiles > units && tail > 0 && tail <= units / 2) {
                                 const int32_t ts = int32_t(std::min<int64_t>(std::min<int64_t>(units / tail, 8), kb));
                                 if (ts >= 2) {
                                     hgemm_config_t t = c;

@@ -1,7 +1,11 @@
 // Tuned-table lookup (see hgemm_planner.h).  The table itself is generated on the GPU machine
 // by the tuner and compiled in; an untabulated shape falls back to the heuristic.
 #include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "hgemm_planner.h"
 
@@ -19,6 +23,38 @@ const Entry kTable[] = {
 #include "hgemm_table.inc"
     {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0.0f, 0, 0}   // sentinel
 };
+// Rows read at run time from the file named by the environment variable HGEMM_TABLE (same row syntax as
+// hgemm_table.inc, as the tuner writes it; lines that do not start with '{' are skipped): they take precedence over
+// the compiled-in rows, so a table re-tuned on another box can be tried without rebuilding the library.
+std::vector<Entry> g_file_rows;
+std::once_flag g_file_once;
+
+void load_file_rows()
+{
+    const char *path = std::getenv("HGEMM_TABLE");
+    if (!path || !*path) return;
+    FILE *f = std::fopen(path, "r");
+    if (!f) return;
+    char line[512];
+    while (std::fgets(line, sizeof(line), f)) {
+        const char *p = line;
+        while (*p == ' ' || *p == '\t') ++p;
+        if (*p != '{') continue;
+        Entry e;
+        std::memset(&e, 0, sizeof(e));
+        const int n = std::sscanf(p, "{%d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %ff, %d, %d", &e.M, &e.N, &e.K, &e.family, &e.block_n,
+                                  &e.block_k, &e.stages, &e.split_k, &e.split_mode, &e.tail_split, &e.raster_group, &e.epilogue, &e.tail_mode,
+                                  &e.us, &e.swap_ab, &e.raster_mode);
+        if (n >= 12 && e.M > 0 && e.N > 0 && e.K > 0) g_file_rows.push_back(e);
+    }
+    std::fclose(f);
+}
+
+const std::vector<Entry> &file_rows()
+{
+    std::call_once(g_file_once, load_file_rows);
+    return g_file_rows;
+}
 } // namespace
 
 namespace {
@@ -47,14 +83,16 @@ hgemm_config_t config_of(const Entry &e)
 int table_neighbours(int64_t M, int64_t N, int64_t K, TableNeighbour *out, int max_out)
 {
     // the max_out tabulated shapes nearest in log space: distance |log M/M'| + |log N/N'| + |log K/K'|
-    const int n = int(sizeof(kTable) / sizeof(kTable[0])) - 1;
+    const std::vector<Entry> &extra = file_rows();
+    const int nt = int(sizeof(kTable) / sizeof(kTable[0])) - 1, n = nt + int(extra.size());
+    auto row = [&](int i) -> const Entry & { return i < nt ? kTable[i] : extra[size_t(i - nt)]; };
     if (n <= 0 || max_out <= 0) return 0;
     if (max_out > 8) max_out = 8;
     double dist[8];
     int idx[8];
     int count = 0;
     for (int i = 0; i < n; ++i) {
-        const Entry &e = kTable[i];
+        const Entry &e = row(i);
         const double d = std::fabs(std::log(double(M) / double(e.M))) + std::fabs(std::log(double(N) / double(e.N))) +
                          std::fabs(std::log(double(K) / double(e.K)));
         int pos = count;
@@ -70,7 +108,7 @@ int table_neighbours(int64_t M, int64_t N, int64_t K, TableNeighbour *out, int m
         if (count < max_out) ++count;
     }
     for (int j = 0; j < count; ++j) {
-        const Entry &e = kTable[idx[j]];
+        const Entry &e = row(idx[j]);
         out[j].M = e.M;
         out[j].N = e.N;
         out[j].K = e.K;
@@ -82,6 +120,14 @@ int table_neighbours(int64_t M, int64_t N, int64_t K, TableNeighbour *out, int m
 
 bool table_lookup(int64_t M, int64_t N, int64_t K, hgemm_config_t *out)
 {
+    for (const Entry &e : file_rows()) {                     // rows from the HGEMM_TABLE file first
+        if (e.M == M && e.N == N && e.K == K) {
+            const hgemm_config_t c = config_of(e);
+            if (validate(M, N, K, c) != HGEMM_OK) break;     // an illegal row is ignored: the compiled-in table answers
+            *out = c;
+            return true;
+        }
+    }
     const int n = int(sizeof(kTable) / sizeof(kTable[0])) - 1;
     for (int i = 0; i < n; ++i) {
         const Entry &e = kTable[i];

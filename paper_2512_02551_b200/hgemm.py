@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhgemm.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_SCRATCH_LIMIT = range(8)
-FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA = 0, 1
+FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA, FAMILY_LIGHT = 0, 1, 2
 EPILOGUE_DIRECT, EPILOGUE_TMA, EPILOGUE_TMA_WIDE = 0, 1, 2
 SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
 TAIL_K, TAIL_N = 0, 1

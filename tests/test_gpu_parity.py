@@ -363,6 +363,85 @@ def test_double_accumulator_tile_other_forms(ctx, gu):
     nn.close()
 
 
+# ---- the light family: one tile per CTA, for the latency-bound shapes ----------------------------------------------
+
+LIGHT = hgemm.FAMILY_LIGHT
+LIGHT_CASES = [
+    # M, N, K, bn, block_k, stages
+    (128, 128, 64, 128, 64, 1),         # one tile, one k-block, one stage
+    (128, 128, 1024, 128, 64, 3),       # the ring wraps five times
+    (64, 64, 64, 32, 64, 1),            # half-empty tile rows, two column tiles
+    (8, 8, 8, 32, 64, 1),               # smallest legal shape: tails in all three dimensions
+    (100, 136, 72, 64, 64, 2),          # ragged M, N and K (multiples of 8)
+    (512, 512, 512, 32, 64, 8),         # every k-block has its own stage: no stage is ever freed
+    (512, 512, 512, 64, 128, 4),        # 128-wide stages
+    (256, 256, 4096, 256, 128, 2),      # widest tile, long K through two stages
+    (1024, 2048, 128, 32, 64, 2),       # 512 CTAs on 148 SMs: several waves
+    (384, 416, 192, 96, 64, 3),         # tile width that is not a power of two
+    (130, 264, 200, 256, 64, 4),        # one row group / a few columns past a tile edge
+]
+
+
+@pytest.mark.parametrize("case", LIGHT_CASES, ids=lambda c: "x".join(map(str, c[:3])) + f"-bn{c[3]}bk{c[4]}s{c[5]}")
+def test_light_family(ctx, gu, case):
+    import oracle
+    M, N, K, bn, bk, stages = case
+    cfg = hgemm.Config.make(family=LIGHT, block_n=bn, stages=stages, raster_group=1, epilogue=TMA, block_k=bk)
+    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    assert plan.config.family == LIGHT
+    gu.assert_close_full(C, A, B, f"light {case}")
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"light {case} integers")
+    # the general form (exact: 0/1 operands, small integers in C)
+    Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
+    C0 = inputs.draw(37, inputs.TAG_A, M, N, "int5", "cuda")
+    buf, Cs = gu.alloc_c_with_guards(M, N)
+    Cs.copy_(C0)
+    plan.run_scaled(2.0, -1.0, Ab, Bb, Cs)
+    assert ctx.last_device_status() == (hgemm.OK, 0) and gu.guards_intact(buf, M, N)
+    gu.assert_exact(Cs, oracle.hgemm_scaled_full(inputs.bits(Ab), inputs.bits(Bb), inputs.bits(C0), 2.0, -1.0), f"light {case} scaled")
+    plan.close()
+
+
+def test_light_family_rules_and_stream_order(ctx, gu):
+    import oracle
+    ok = hgemm.Config.make(family=LIGHT, block_n=64, stages=4, epilogue=TMA)
+    assert hgemm.validate_config(512, 512, 512, ok) == hgemm.OK
+    assert hgemm.validate_config(512, 516, 512, ok) == hgemm.ERR_UNSUPPORTED            # rows of C: multiples of 16 bytes
+    assert hgemm.validate_config(512, 512, 516, ok) == hgemm.ERR_UNSUPPORTED            # rows of A and B too (no padded copies here)
+    for kw in (dict(split_k=2), dict(epilogue=DIRECT), dict(epilogue=WIDE), dict(accumulate=hgemm.ACC_F16), dict(tail_split=2),
+               dict(swap_ab=1), dict(block_n=512), dict(raster_mode=1)):
+        c = hgemm.Config.make(**{**dict(family=LIGHT, block_n=64, stages=4, epilogue=TMA), **kw})
+        assert hgemm.validate_config(512, 512, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
+    nn = ctx.plan(256, 512, 256, layout=hgemm.LAYOUT_NN)
+    assert nn.try_set_config(ok) == hgemm.ERR_UNSUPPORTED
+    nn.close()
+    # a chain of dependent launches through light plans: C1 = A B1^T, C2 = C1 B2^T, stream order kept
+    M, K1, N1, N2 = 512, 64, 64, 384
+    A = inputs.draw(1, inputs.TAG_A, M, K1, "int5", "cuda")
+    B1 = inputs.draw(2, inputs.TAG_B, N1, K1, "int5", "cuda")
+    B2 = inputs.draw(3, inputs.TAG_B, N2, N1, "int5", "cuda")
+    c1_ref = oracle.hgemm_full(inputs.bits(A), inputs.bits(B1))
+    c2_ref = oracle.hgemm_full(oracle.f64_to_f16_bits(c1_ref.ravel()).reshape(M, N1), inputs.bits(B2))
+    p1, p2 = ctx.plan(M, N1, K1), ctx.plan(M, N2, N1)
+    p1.set_config(hgemm.Config.make(family=LIGHT, block_n=64, stages=1, epilogue=TMA))
+    p2.set_config(hgemm.Config.make(family=LIGHT, block_n=96, stages=1, epilogue=TMA))
+    for rep in range(25):
+        C1 = torch.zeros(M, N1, dtype=torch.float16, device="cuda")
+        C2 = torch.zeros(M, N2, dtype=torch.float16, device="cuda")
+        p1.run(A, B1, C1)
+        p2.run(C1, B2, C2)
+        p1.run(A, B1, C1)
+        torch.cuda.synchronize()
+        gu.assert_exact(C2, c2_ref, f"light chain, repetition {rep}")
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    p1.close()
+    p2.close()
+
+
 def test_dependent_launch_keeps_stream_order(ctx, gu):
     """Launches may become resident before the kernel ahead of them has finished.  A chain in which each
     GEMM consumes the previous GEMM's output must still see stream order: C1 = A B1^T, C2 = C1 B2^T."""

@@ -143,7 +143,7 @@ def test_every_grid_shape_plans_to_a_legal_configuration(lib):
                 assert hgemm.validate_config(M, N, K, c) == hgemm.OK, (M, N, K, c.as_dict())
                 assert hgemm.config_smem_bytes(c) <= 232448
                 families.add(c.family)
-    assert families == {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA}
+    assert {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA} <= families <= {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA, hgemm.FAMILY_LIGHT}
 
 
 def test_candidate_configs_are_legal_ranked_and_distinct(lib):
@@ -156,10 +156,34 @@ def test_candidate_configs_are_legal_ranked_and_distinct(lib):
         assert all(hgemm.validate_config(M, N, Kp, c) == hgemm.OK for c in cands)
         keys = {tuple(sorted(c.as_dict().items())) for c in cands}
         assert len(keys) == len(cands)
-    # both families, both stage widths, split-K and the wide epilogue all occur among the candidates of a shape that admits them
+    # all three families, both stage widths, split-K and the wide epilogue all occur among the candidates of a shape that admits them
     pool = hgemm.candidate_configs(512, 512, 4096, max_count=256)
-    assert {c.family for c in pool} == {0, 1} and {c.block_k for c in pool} == {64, 128}
+    assert {c.family for c in pool} == {0, 1, 2} and {c.block_k for c in pool} == {64, 128}
+    assert all(c.split_k == 1 and c.epilogue == hgemm.EPILOGUE_TMA for c in pool if c.family == hgemm.FAMILY_LIGHT)
+    big = hgemm.candidate_configs(8192, 8192, 8192, max_count=256)
+    assert any(c.block_n == 512 and c.family == hgemm.FAMILY_UMMA_2CTA for c in big)          # the double-accumulator tile
+    skinny = hgemm.candidate_configs(64, 12288, 4096, max_count=256)
+    assert any(c.swap_ab == 1 for c in skinny) and not any(c.swap_ab for c in big)            # swapped operands: few rows only
     assert any(c.split_k > 1 and c.split_mode == 1 for c in pool) and any(c.split_k > 1 and c.split_mode == 0 for c in pool)
     assert any(c.epilogue == hgemm.EPILOGUE_TMA_WIDE for c in pool)
     assert hgemm.candidate_configs(0, 64, 64) == [] and hgemm.candidate_configs(64, 64, 1 << 30) == []
 
+
+
+def test_table_file_overrides_the_built_in_table(lib, tmp_path):
+    """HGEMM_TABLE names a file of tuner rows that take precedence over the compiled-in table (read once per process,
+    so the check runs in a child process)."""
+    import subprocess
+    import sys
+    table = tmp_path / "table.inc"
+    table.write_text("// a comment line\n"
+                     "{4096, 4096, 4096, 0, 96, 64, 5, 1, 0, 0, 7, 0, 0, 123.00f, 0, 1},\n"      # a tabulated shape, overridden
+                     "{1000, 2000, 3000, 1, 128, 128, 3, 1, 0, 0, 4, 1, 0, 50.00f},\n"            # an off-grid shape, old row format
+                     "{64, 64, 64, 0, 48, 64, 2, 1, 0, 0, 1, 0, 0, 1.00f, 0, 0},\n")              # an illegal row: ignored
+    code = ("from paper_2512_02551_b200 import hgemm\n"
+            "a = hgemm.planned_config(4096, 4096, 4096); b = hgemm.planned_config(1000, 2000, 3000); c = hgemm.planned_config(64, 64, 64)\n"
+            "print(a.family, a.block_n, a.stages, a.raster_group, a.raster_mode, b.family, b.block_n, b.block_k, c.block_n)")
+    env = dict(os.environ, HGEMM_TABLE=str(table), PYTHONPATH=ROOT)
+    out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, check=True).stdout.split()
+    assert out[:8] == ["0", "96", "5", "7", "1", "1", "128", "128"]
+    assert out[8] != "48"
