@@ -561,8 +561,9 @@ def grid_sweep(ctx, torch, hgemm, inputs, stream, csv_path=None) -> dict:
                 plan = ctx.plan(M, N, K)
                 s = stream.cuda_stream
                 A0, Bt0, C0, a0, b0, c0 = bufs[0]
-                ours_w = lambda i: plan.run_ptr(a0, b0, c0, s)                      # noqa: E731
-                ref_w = lambda i: torch.matmul(A0, Bt0, out=C0)                     # noqa: E731
+                # (defaults bind this iteration's plan and buffers: the callables are used again after the loop)
+                ours_w = lambda i, plan=plan, a0=a0, b0=b0, c0=c0: plan.run_ptr(a0, b0, c0, s)      # noqa: E731
+                ref_w = lambda i, A0=A0, Bt0=Bt0, C0=C0: torch.matmul(A0, Bt0, out=C0)            # noqa: E731
 
                 def ours_c(i, bufs=bufs, plan=plan):
                     b = bufs[i % len(bufs)]

@@ -62,10 +62,15 @@ typedef enum {
 enum {
     HGEMM_FAMILY_UMMA_1CTA = 0, /* persistent, warp-specialised, 128 x block_n tiles, one CTA per tile */
     HGEMM_FAMILY_UMMA_2CTA = 1, /* the same with CTA pairs: 256 x block_n tiles, B split across the pair */
-    HGEMM_FAMILY_LIGHT = 2      /* the small-problem kernel: one 128 x block_n tile per CTA, no persistent loop, one
-                                   accumulator, six warps, only the shared memory it uses; its first loads leave before
-                                   the CTA's set-up has finished.  Needs K % 8 == 0 and N % 8 == 0, split_k == 1, no
-                                   tail_split, no swap_ab, fp32 accumulators, the TN layout, HGEMM_EPILOGUE_TMA */
+    HGEMM_FAMILY_LIGHT = 2,     /* the small-problem kernel: one 128 x block_n tile per CTA, no persistent loop, one
+                                   accumulator, no CTA-wide barrier at the end, only the shared memory it uses; its first
+                                   loads leave before the CTA's set-up has finished.  Needs K % 8 == 0 and N % 8 == 0, split_k == 1, no
+                                   tail_split, no swap_ab, fp32 accumulators, the TN layout, HGEMM_EPILOGUE_DIRECT or HGEMM_EPILOGUE_TMA */
+    HGEMM_FAMILY_SMALL = 3      /* the register-accumulator kernel for the smallest problems: 64 x 64 tiles, cp.async + ldmatrix
+                                   + mma.sync with fp32 accumulators in registers -- no tensor memory to allocate (0.7 us on
+                                   B200), no tensor maps, no mbarriers.  One fixed configuration: block_m = block_n = block_k
+                                   = 64, stages = 3, split_k = 1, HGEMM_EPILOGUE_DIRECT.  Needs K % 8 == 0 and N % 8 == 0, no
+                                   tail_split, no swap_ab, fp32 accumulators, the TN layout */
 };
 
 /* Where the fp32 partial sums of a split-K tile meet.  Both sum the slices in slice
@@ -116,7 +121,7 @@ enum {
  * count and block-swizzle stride of sections 5.2 and 6, plus split-K). */
 typedef struct {
     int32_t family;       /* HGEMM_FAMILY_* */
-    int32_t block_m;      /* 128 (1-CTA and light families) or 256 (2-CTA pair) */
+    int32_t block_m;      /* 128 (1-CTA and light families), 256 (2-CTA pair) or 64 (small family) */
     int32_t block_n;      /* multiple of 32 in [32, 256]; or 512 (CTA-pair family only): a 256 x 512 tile held in both
                              tensor-memory accumulators at once, two MMAs per K step sharing the A tile -- a quarter less
                              shared-memory fill per flop than 256 x 256, no overlap of a tile's epilogue with the next
@@ -355,9 +360,13 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream);
  * mid-size shapes than the one that runs otherwise: the stamps describe the
  * pipeline's structure and proportions, not the production kernel's absolute times.
  * The instrumented kernels do not exist for swapped-operand configurations (swap_ab = 1),
- * for the 512-wide tile or for the light family:
- * hgemm_run returns HGEMM_ERR_UNSUPPORTED for such a plan while a trace buffer or a skip
- * mask is set. */
+ * for the 512-wide tile or for the small family: hgemm_run returns HGEMM_ERR_UNSUPPORTED for such a plan while a
+ * trace buffer or a skip mask is set.  The light family writes its own stamps, SM-clock
+ * values (clock64) of CTA 0 in slots 0..12: 0 entry, 1 first barriers initialised, 2 first
+ * loads issued, 3 tensor memory allocated, 4 set-up barrier passed, 5 first k-block landed,
+ * 6 last MMA issued, 7 accumulator ready, 8 first chunk converted, 9 last store issued,
+ * 10 epilogue warp done, 11 tensor memory read by every epilogue warp, 12 tensor memory
+ * freed; it has no skip mask. */
 hgemm_status_t hgemm_debug_set_trace(hgemm_plan_t *plan, void *device_buf);
 
 /* Instrumentation for bottleneck analysis: bit 0 makes later launches of this plan

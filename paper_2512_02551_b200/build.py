@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhgemm.so")
 SOURCES = ["hgemm_api.cu", "hgemm_static_scratch.cu", "hgemm_planner.cpp", "hgemm_table.cpp"]
-DEPS = SOURCES + ["hgemm_kernel.cuh", "hgemm_light_kernel.cuh", "ptx_sm100.cuh", "hgemm_planner.h", "hgemm_table.inc",
+DEPS = SOURCES + ["hgemm_kernel.cuh", "hgemm_light_kernel.cuh", "hgemm_small_kernel.cuh", "ptx_sm100.cuh", "hgemm_planner.h", "hgemm_table.inc",
                   os.path.join("..", "..", "include", "hgemm.h")]
 
 

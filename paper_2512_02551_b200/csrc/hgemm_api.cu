@@ -11,6 +11,7 @@
 #include "../../include/hgemm.h"
 #include "hgemm_kernel.cuh"
 #include "hgemm_light_kernel.cuh"
+#include "hgemm_small_kernel.cuh"
 #include "hgemm_planner.h"
 
 using hgemm_dev::KernelParams;
@@ -125,7 +126,7 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     if (pl->layout == HGEMM_LAYOUT_NN && (cfg.block_n % (64 * cg)) != 0) return HGEMM_ERR_UNSUPPORTED;
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.swap_ab) return HGEMM_ERR_UNSUPPORTED;   // the swapped form is built for K-contiguous operands
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.block_n == 512) return HGEMM_ERR_UNSUPPORTED;   // so is the double-accumulator tile
-    if (pl->layout == HGEMM_LAYOUT_NN && cfg.family == HGEMM_FAMILY_LIGHT) return HGEMM_ERR_UNSUPPORTED;   // and the light kernel
+    if (pl->layout == HGEMM_LAYOUT_NN && (cfg.family == HGEMM_FAMILY_LIGHT || cfg.family == HGEMM_FAMILY_SMALL)) return HGEMM_ERR_UNSUPPORTED;   // and the two small-problem kernels
     // row-major B is staged in blocks of 64 columns: column pieces of tail tiles must be whole blocks per CTA
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 &&
         ((cfg.block_n / cfg.tail_split) % (64 * cg)) != 0)
@@ -259,6 +260,14 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     // CTAs can never wait on each other's tensor-memory allocation.  (Letting small configurations ask for what
     // they use, so that the next call's CTAs become resident beside this call's, made those calls slower.)
     pl->smem = int(hgemm_host::kSmemOptInBytes);
+    if (cfg.family == HGEMM_FAMILY_SMALL) {
+        // 64 x 64 tiles, one CTA each, static shared memory, no tensor maps
+        p.tiles_m = int32_t((pl->M + 63) / 64);
+        p.tiles_n = int32_t((pl->N + 63) / 64);
+        pl->grid = p.tiles_m * p.tiles_n;
+        pl->cluster_dim = 1;
+        pl->smem = 0;
+    }
     if (cfg.family == HGEMM_FAMILY_LIGHT) {
         // one CTA per tile, and only the shared memory the configuration uses
         pl->grid = p.tiles_m * p.tiles_n;
@@ -427,7 +436,9 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         }
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+            e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
         for (int k = 0; k < 6 && e == cudaSuccess; ++k) {           // the double-accumulator instantiations
             const void *fn_k = kernel_for(2, (k & 1) != 0, 0, k >= 2, false, k >= 4 ? 2 : 1, false, true);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
@@ -734,6 +745,36 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         B = plan->pad_b;
     }
 
+    if (cfg.family == HGEMM_FAMILY_SMALL) {
+        // the register-accumulator kernel: plain pointers, no tensor maps, no cluster
+        if (plan->trace != nullptr || plan->debug_skip != 0) return HGEMM_ERR_UNSUPPORTED;       // it has no instrumentation
+        hgemm_dev::SmallParams sp;
+        sp.A = static_cast<const __half *>(A);
+        sp.B = static_cast<const __half *>(B);
+        sp.C = static_cast<__half *>(C);
+        sp.M = int32_t(plan->M);
+        sp.N = int32_t(plan->N);
+        sp.K = int32_t(plan->K);
+        sp.tiles_m = plan->params.tiles_m;
+        sp.scaled = scaled ? 1u : 0u;
+        sp.alpha = alpha;
+        sp.beta = beta;
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof(lc));
+        lc.gridDim = dim3(unsigned(plan->grid), 1, 1);
+        lc.blockDim = dim3(hgemm_dev::kSmallThreads, 1, 1);
+        lc.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = ctx->dependent_launch ? 1 : 0;
+        void *sargs[1] = {&sp};
+        cudaError_t e = cudaLaunchKernelExC(&lc, reinterpret_cast<const void *>(hgemm_dev::hgemm_small_kernel), sargs);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        return HGEMM_OK;
+    }
+
     if (cfg.swap_ab) std::swap(A, B);       // the kernel's A operand (its 128-row side) is the caller's B
 
     hgemm_plan_s::MapEntry *me = nullptr;
@@ -817,14 +858,18 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     const bool trace = kp.trace != nullptr || kp.debug_skip != 0;
     const bool plain = !kp.scaled && !kp.acc_f16 && !kp.ragged_n && !kp.b_row_major && kp.tail_pieces <= 1;
     const bool light = plan->cfg.family == HGEMM_FAMILY_LIGHT;
-    if (trace && (kp.transposed || kp.block_n == 512 || light)) return HGEMM_ERR_UNSUPPORTED;   // no instrumented kernels for these
+    if (trace && (kp.transposed || kp.block_n == 512)) return HGEMM_ERR_UNSUPPORTED;   // no instrumented kernels for these
+    if (light && kp.debug_skip != 0) return HGEMM_ERR_UNSUPPORTED;                       // the light kernel has stamps, no skip mask
     const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
                                 trace, kp.block_k / 64, kp.transposed != 0, kp.block_n == 512);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
     if (light) {
         void *largs[4] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &plan->params};
         lc.blockDim = dim3(hgemm_dev::kLightThreads, 1, 1);
-        e = cudaLaunchKernelExC(&lc, reinterpret_cast<const void *>(hgemm_dev::hgemm_light_kernel), largs);
+        lc.attrs = attr + 1;                         // no cluster attribute: a plain grid, with or without the dependent-launch one
+        lc.numAttrs = ctx->dependent_launch ? 1 : 0;
+        e = cudaLaunchKernelExC(&lc, kp.trace != nullptr ? reinterpret_cast<const void *>(hgemm_dev::hgemm_light_kernel<true>)
+                                                         : reinterpret_cast<const void *>(hgemm_dev::hgemm_light_kernel<false>), largs);
     } else {
         e = cudaLaunchKernelExC(&lc, fn, args);
     }

@@ -27,12 +27,13 @@ int64_t stage_bytes(const hgemm_config_t &c)
 // Store staging of the eight epilogue warps: two 2 KB boxes each, or two 4 KB ones for the wide TMA epilogue.
 int64_t staging_bytes(const hgemm_config_t &c)
 {
-    if (c.family == HGEMM_FAMILY_LIGHT) return kStagingBytes / 2;        // four epilogue warps
+    if (c.family == HGEMM_FAMILY_LIGHT) return c.epilogue == HGEMM_EPILOGUE_DIRECT ? 0 : kStagingBytes;   // direct stores stage nothing
     return c.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? 2 * kStagingBytes : kStagingBytes;
 }
 
 int64_t smem_bytes(const hgemm_config_t &c)
 {
+    if (c.family == HGEMM_FAMILY_SMALL) return 3 * 2 * 64 * 64 * 2;      // its static ring: three stages of A and B tiles
     return kAlignSlack + int64_t(c.stages) * stage_bytes(c) + staging_bytes(c) + kCtrlBytes;
 }
 
@@ -55,6 +56,15 @@ int32_t max_stages_of(const hgemm_config_t &c)
 
 SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c)
 {
+    if (c.family == HGEMM_FAMILY_SMALL) {
+        SplitLayout S;
+        S.tiles = ceil_div(M, 64) * ceil_div(N, 64);
+        S.first_split_tile = S.tiles;
+        S.slices = 1;
+        S.pieces = 1;
+        S.work_items = S.tiles;
+        return S;
+    }
     if (c.swap_ab) std::swap(M, N);   // the kernel tiles the transposed problem
     const int cg = cta_group_of(c);
     SplitLayout L;
@@ -126,10 +136,22 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
             return HGEMM_ERR_UNSUPPORTED;
         std::swap(M, N);
     }
+    if (c.family == HGEMM_FAMILY_SMALL) {
+        // one fixed configuration
+        for (int i = 0; i < 2; ++i)
+            if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+        if (c.block_m != 64 || c.block_n != 64 || c.block_k != 64 || c.stages != 3 || c.split_k != 1 || c.tail_split >= 2 || c.swap_ab ||
+            c.accumulate != HGEMM_ACC_F32 || c.epilogue != HGEMM_EPILOGUE_DIRECT || c.raster_mode != HGEMM_RASTER_SWEEP || c.raster_group < 1 ||
+            (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) || (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N) ||
+            (K % 8) != 0 || (N % 8) != 0)
+            return HGEMM_ERR_UNSUPPORTED;
+        if (ceil_div(M, 64) * ceil_div(N, 64) >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
+        return HGEMM_OK;
+    }
     if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA && c.family != HGEMM_FAMILY_LIGHT) return HGEMM_ERR_UNSUPPORTED;
     if (c.family == HGEMM_FAMILY_LIGHT) {
         // one plain tile per CTA: nothing that needs the persistent kernel's extra paths
-        if (c.split_k != 1 || c.tail_split >= 2 || c.swap_ab || c.accumulate != HGEMM_ACC_F32 || c.epilogue != HGEMM_EPILOGUE_TMA ||
+        if (c.split_k != 1 || c.tail_split >= 2 || c.swap_ab || c.accumulate != HGEMM_ACC_F32 || c.epilogue == HGEMM_EPILOGUE_TMA_WIDE ||
             c.raster_mode != HGEMM_RASTER_SWEEP || c.block_n > 256 || (K % 8) != 0 || (N % 8) != 0)
             return HGEMM_ERR_UNSUPPORTED;
     }
@@ -185,6 +207,12 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
 
 double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c)
 {
+    if (c.family == HGEMM_FAMILY_SMALL) {
+        // Not fitted: a ranking hint.  Per 64-wide k-block a CTA moves 16 KB into shared memory and issues 128 MMAs of
+        // 16 x 8 x 16 (about 1024 MACs per clock and SM on the register path); four CTAs share an SM; a short fixed part.
+        const double waves = std::ceil(double(ceil_div(M, 64) * ceil_div(N, 64)) / (4.0 * std::max(1, num_sms)));
+        return 1400.0 + waves * (double(ceil_div(K, 64)) * 300.0 * 4.0 / 4.0 + 600.0);
+    }
     // Rough machine model, in SM clock cycles: a ranking aid, not a prediction.  Its form follows the kernel
     // (waves of tiles, k-blocks bounded by the tensor pipe, the stage hand-off, the fill rate of one SM, the
     // aggregate L2 rate or the latency the stage ring can hide; a drain, a reduction for split-K); its constants
@@ -325,6 +353,16 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
     auto add = [&](const hgemm_config_t &c) {
         if (validate(M, N, K, c) == HGEMM_OK) all.emplace_back(estimate_cycles(M, N, K, num_sms, c), c);
     };
+    {
+        hgemm_config_t c;
+        std::memset(&c, 0, sizeof(c));
+        c.family = HGEMM_FAMILY_SMALL;
+        c.block_m = c.block_n = c.block_k = 64;
+        c.stages = 3;
+        c.split_k = 1;
+        c.raster_group = 1;
+        add(c);                                                     // (validate() keeps it to K % 8 == 0 and N % 8 == 0)
+    }
     // swap == 1: the operands trade places (few rows, many columns: the rows of B fill the MMA's 128-row side)
     for (int swap = 0; swap < 2; ++swap) {
     if (swap == 1 && !(M <= 256 && N >= 512 && (N % 8) == 0)) continue;
@@ -350,7 +388,7 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                         if (mode == 1 && (split == 1 || split * cg > 16)) continue;
                         for (int epi = 0; epi < 3; ++epi) {
                             if (split > 1 && epi != HGEMM_EPILOGUE_DIRECT) continue;
-                            if (light && epi != HGEMM_EPILOGUE_TMA) continue;
+                            if (light && epi == HGEMM_EPILOGUE_TMA_WIDE) continue;
                             if (epi == HGEMM_EPILOGUE_TMA_WIDE && ((bn % 64) != 0 || swap)) continue;
                             hgemm_config_t c;
                             std::memset(&c, 0, sizeof(c));

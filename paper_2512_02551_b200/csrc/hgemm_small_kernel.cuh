@@ -1,0 +1,175 @@
+// The register-accumulator kernel for the smallest problems.
+//
+// A tcgen05 kernel pays fixed costs before and after its MMAs that do not shrink with the problem: allocating
+// and freeing tensor memory alone measures about 0.7 us on B200 (an empty kernel: 0.9 us), tensor-map fetches
+// and mbarrier round trips add more.  For problems that are a handful of 64 x 64 tiles with a short K loop -- the
+// corner of the shape grid where the paper found its largest gains, and where it picks a lighter kernel structure
+// (section 5.1) -- those costs are most of the call.  This kernel has none of them: cp.async into swizzled shared
+// memory, ldmatrix, mma.sync.m16n8k16 (fp16 x fp16 -> fp32) with the accumulators in registers, 4-byte stores.
+// The tensor cores still do the contraction; what is dropped is everything around them.
+//
+//   CTA: 128 threads = 2 x 2 warps, one 64 x 64 tile of C; each warp a 32 x 32 quarter (2 x 4 MMA tiles)
+//   K loop: 64-wide k-blocks through a 3-stage cp.async ring (8 KB of A + 8 KB of B per stage)
+//   shared memory: rows of 128 bytes; 16-byte piece c of row r lives at piece c ^ (r & 7), so that the eight
+//   row addresses of an ldmatrix fall on different banks
+//
+// Same arithmetic as the tcgen05 kernels: exact fp16 products, fp32 accumulation, one rounding to fp16 (or the
+// alpha / beta form before it).  Needs K % 8 == 0 and N % 8 == 0; rows and columns beyond M, N and K are
+// zero-filled on the way in and never stored.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+#include "ptx_sm100.cuh"
+
+namespace hgemm_dev {
+
+constexpr int kSmallTile = 64;        // rows and columns of C per CTA
+constexpr int kSmallBk = 64;          // K extent of a stage
+constexpr int kSmallStages = 3;
+constexpr int kSmallThreads = 128;
+
+struct SmallParams {
+    const __half *A;                  // M x K, K-contiguous
+    const __half *B;                  // N x K, K-contiguous
+    __half *C;                        // M x N row-major
+    int32_t M, N, K;
+    int32_t tiles_m;                  // ceil(M / 64): CTA b computes tile (b % tiles_m, b / tiles_m)
+    uint32_t scaled;                  // 1: C = alpha A B^T + beta C
+    float alpha, beta;
+};
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
+{
+    // src_bytes == 0 writes sixteen zero bytes and reads nothing
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+
+__device__ __forceinline__ void mma_m16n8k16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(kSmallThreads)
+hgemm_small_kernel(const SmallParams p)
+{
+    __shared__ __align__(128) uint8_t smem[kSmallStages * 2 * kSmallTile * kSmallBk * 2];     // 48 KB: [stage][A | B][64 rows][128 bytes]
+    const uint32_t smem_base = smem_addr(smem);
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t wm = warp & 1u, wn = warp >> 1;                      // this warp's 32 x 32 quarter of the tile
+    const int32_t tile = static_cast<int32_t>(blockIdx.x);
+    const int32_t tn = tile / p.tiles_m, tm = tile - tn * p.tiles_m;
+    const int32_t m0 = tm * kSmallTile, n0 = tn * kSmallTile;
+    const int32_t kblocks = (p.K + kSmallBk - 1) / kSmallBk;
+    constexpr uint32_t kTileBytes = kSmallTile * kSmallBk * 2;          // 8 KB
+
+    grid_launch_dependents();          // the next kernel in the stream may start its own set-up
+    grid_dependency_wait();            // ... and this one reads nothing before the kernels ahead of it are complete
+
+    // One stage: 64 rows x eight 16-byte pieces of A and of B, four pieces of each per thread.
+    auto load_stage = [&](int32_t kb, int32_t s) {
+        const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * 2u * kTileBytes;
+        const uint32_t b_dst = a_dst + kTileBytes;
+        const int32_t k0 = kb * kSmallBk;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t piece = tid + static_cast<uint32_t>(i) * kSmallThreads;       // 0 .. 511
+            const uint32_t r = piece >> 3, c = piece & 7u;
+            const int32_t k = k0 + static_cast<int32_t>(c) * 8;
+            const uint32_t off = r * 128u + ((c ^ (r & 7u)) << 4);
+            const bool k_in = k < p.K;                                                     // K % 8 == 0: a piece is inside or outside
+            const int32_t ar = m0 + static_cast<int32_t>(r), br = n0 + static_cast<int32_t>(r);
+            const bool a_in = k_in && ar < p.M, b_in = k_in && br < p.N;
+            // (an address inside the matrix even when nothing is read from it)
+            cp_async_16(a_dst + off, p.A + (a_in ? static_cast<size_t>(ar) * p.K + k : 0), a_in ? 16u : 0u);
+            cp_async_16(b_dst + off, p.B + (b_in ? static_cast<size_t>(br) * p.K + k : 0), b_in ? 16u : 0u);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    float acc[2][4][4];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.0f;
+
+    // prologue: two stages in flight (an empty group where K is shorter, so that the group count stays uniform)
+    for (int32_t s = 0; s < kSmallStages - 1; ++s) {
+        if (s < kblocks) load_stage(s, s);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+
+    for (int32_t kb = 0; kb < kblocks; ++kb) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(kSmallStages - 2) : "memory");      // k-block kb has landed (this thread's part)
+        __syncthreads();                                                                  // ... everyone's; and stage (kb - 1) % 3 is free
+        if (kb + kSmallStages - 1 < kblocks) load_stage(kb + kSmallStages - 1, (kb + kSmallStages - 1) % kSmallStages);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        const uint32_t a_tile = smem_base + static_cast<uint32_t>(kb % kSmallStages) * 2u * kTileBytes;
+        const uint32_t b_tile = a_tile + kTileBytes;
+#pragma unroll
+        for (uint32_t kk = 0; kk < kSmallBk / 16; ++kk) {
+            // A fragments: rows 16 i .. 16 i + 15 of this warp's 32; matrices in the order (rows 0-7, k 0-7),
+            // (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15) = registers a0..a3 of the MMA
+            uint32_t a[2][4];
+#pragma unroll
+            for (uint32_t i = 0; i < 2; ++i) {
+                const uint32_t row = wm * 32u + i * 16u + (lane & 7u) + ((lane >> 3) & 1u) * 8u;
+                const uint32_t piece = kk * 2u + (lane >> 4);
+                ldmatrix_x4(a_tile + row * 128u + ((piece ^ (row & 7u)) << 4), a[i][0], a[i][1], a[i][2], a[i][3]);
+            }
+            // B fragments: two 8-column tiles per ldmatrix; matrices (n 0-7, k 0-7), (n 0-7, k 8-15), (n 8-15, k 0-7),
+            // (n 8-15, k 8-15) = b0, b1 of the first tile, b0, b1 of the second
+            uint32_t b[4][2];
+#pragma unroll
+            for (uint32_t j = 0; j < 2; ++j) {
+                const uint32_t row = wn * 32u + j * 16u + (lane & 7u) + (lane >> 4) * 8u;
+                const uint32_t piece = kk * 2u + ((lane >> 3) & 1u);
+                ldmatrix_x4(b_tile + row * 128u + ((piece ^ (row & 7u)) << 4), b[2 * j][0], b[2 * j][1], b[2 * j + 1][0], b[2 * j + 1][1]);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) mma_m16n8k16(acc[i][j], a[i], b[j][0], b[j][1]);
+        }
+    }
+
+    // epilogue: accumulator element pairs (row l / 4 [+ 8], columns 2 (l % 4), + 1) -> half2 -> 4-byte stores
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int32_t row = m0 + static_cast<int32_t>(wm * 32u + i * 16u + h * 8u + (lane >> 2));
+            if (row >= p.M) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int32_t col = n0 + static_cast<int32_t>(wn * 32u + j * 8u + (lane & 3u) * 2u);
+                if (col >= p.N) continue;                                 // N is even: the pair is inside or outside
+                float x = acc[i][j][2 * h], y = acc[i][j][2 * h + 1];
+                __half2 *dst = reinterpret_cast<__half2 *>(p.C + static_cast<size_t>(row) * p.N + col);
+                if (p.scaled) {
+                    float ox = 0.0f, oy = 0.0f;
+                    if (p.beta != 0.0f) {
+                        const float2 o = __half22float2(*dst);
+                        ox = o.x;
+                        oy = o.y;
+                    }
+                    x = fmaf(p.beta, ox, p.alpha * x);
+                    y = fmaf(p.beta, oy, p.alpha * y);
+                }
+                *dst = __floats2half2_rn(x, y);
+            }
+        }
+    }
+}
+
+} // namespace hgemm_dev

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libhgemm.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_SCRATCH_LIMIT = range(8)
-FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA, FAMILY_LIGHT = 0, 1, 2
+FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA, FAMILY_LIGHT, FAMILY_SMALL = 0, 1, 2, 3
 EPILOGUE_DIRECT, EPILOGUE_TMA, EPILOGUE_TMA_WIDE = 0, 1, 2
 SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
 TAIL_K, TAIL_N = 0, 1
@@ -46,6 +46,11 @@ class Config(ctypes.Structure):
                 ("tail_split", ctypes.c_int32), ("tail_mode", ctypes.c_int32), ("accumulate", ctypes.c_int32),
                 ("swap_ab", ctypes.c_int32), ("raster_mode", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
 
+    @classmethod
+    def small(cls) -> "Config":
+        """The one configuration of the register-accumulator kernel for the smallest problems."""
+        return cls.make(family=FAMILY_SMALL, block_n=64, stages=3, split_k=1, raster_group=1, epilogue=EPILOGUE_DIRECT, block_k=64)
+
     def as_dict(self) -> dict:
         return {k: int(getattr(self, k)) for k, _ in self._fields_ if k != "reserved"}
 
@@ -55,7 +60,7 @@ class Config(ctypes.Structure):
              raster_mode=0) -> "Config":
         c = cls()
         c.family = family
-        c.block_m = 256 if family == FAMILY_UMMA_2CTA else 128
+        c.block_m = 256 if family == FAMILY_UMMA_2CTA else 64 if family == FAMILY_SMALL else 128
         c.block_n = block_n
         c.block_k = block_k
         c.stages = stages

@@ -42,6 +42,9 @@ def max_stages(family: int, bn: int, bk: int, epilogue: int = hgemm.EPILOGUE_TMA
 
 def candidates(M: int, N: int, K: int):
     out = []
+    small = hgemm.Config.small()                                  # the register-accumulator kernel's one configuration
+    if hgemm.validate_config(M, N, K, small) == hgemm.OK and M * N * K <= (1 << 31):
+        out.append(small)
     for swap in (0, 1):
         if swap and not (M <= 256 and N >= 512 and N % 8 == 0):
             continue
@@ -82,7 +85,7 @@ def _candidates(M: int, N: int, K: int, swap: int):
                         if split == 1:
                             epis = (hgemm.EPILOGUE_TMA, hgemm.EPILOGUE_DIRECT) + ((hgemm.EPILOGUE_TMA_WIDE,) if bn % 64 == 0 and not swap else ())
                         if light:
-                            epis = (hgemm.EPILOGUE_TMA,)
+                            epis = (hgemm.EPILOGUE_DIRECT, hgemm.EPILOGUE_TMA)
                         for epi in epis:
                             st = min(max_stages(family, bn, bk, epi), 8)      # the wide epilogue's staging leaves fewer stages
                             if light:
@@ -174,7 +177,11 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     cands.sort(key=lambda c: hgemm.estimate_config(M, N, K, c))
     # the wide-store candidates are ranked on their own (8 of them), so that they take no place among the `top`
     wide = [c for c in cands if c.epilogue == hgemm.EPILOGUE_TMA_WIDE][:8]
-    cands = [c for c in cands if c.epilogue != hgemm.EPILOGUE_TMA_WIDE]
+    # so are the double-accumulator tiles and the light kernel's configurations, which the cost model was not fitted on
+    wide += [c for c in cands if c.block_n == 512 and c.epilogue != hgemm.EPILOGUE_TMA_WIDE][:4]
+    wide += [c for c in cands if c.family == hgemm.FAMILY_LIGHT][:8]
+    wide += [c for c in cands if c.family == hgemm.FAMILY_SMALL]
+    cands = [c for c in cands if c.epilogue != hgemm.EPILOGUE_TMA_WIDE and c.block_n != 512 and c.family not in (hgemm.FAMILY_LIGHT, hgemm.FAMILY_SMALL)]
     chosen, seen = [], set()
     extra = rng.sample(cands[top:], min(explore, max(0, len(cands) - top))) if explore > 0 else []   # for refitting the cost model
     for c in [default] + cands[:top] + wide + extra:
@@ -235,7 +242,7 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
             b2b[key(c)] = min(b2b.get(key(c), t), t)
         ranked = sorted(results, key=lambda r: r[0])
         pool, seen_k = [], set()
-        for t, _, c in ranked[:10] + [r for r in ranked if r[2].family == hgemm.FAMILY_LIGHT][:8]:
+        for t, _, c in ranked[:10] + [r for r in ranked if r[2].family in (hgemm.FAMILY_LIGHT, hgemm.FAMILY_SMALL)][:9]:
             if key(c) not in seen_k:
                 seen_k.add(key(c))
                 pool.append(c)

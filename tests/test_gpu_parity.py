@@ -386,15 +386,19 @@ LIGHT_CASES = [
 def test_light_family(ctx, gu, case):
     import oracle
     M, N, K, bn, bk, stages = case
-    cfg = hgemm.Config.make(family=LIGHT, block_n=bn, stages=stages, raster_group=1, epilogue=TMA, block_k=bk)
-    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
-    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
-    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
-    assert plan.config.family == LIGHT
-    gu.assert_close_full(C, A, B, f"light {case}")
-    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
-    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
-    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"light {case} integers")
+    plan = None
+    for epi in (DIRECT, TMA):
+        cfg = hgemm.Config.make(family=LIGHT, block_n=bn, stages=stages, raster_group=1, epilogue=epi, block_k=bk)
+        if epi == TMA and hgemm.validate_config(M, N, K, cfg) != hgemm.OK:
+            cfg.stages = stages - 1                      # the store staging takes the room of a stage
+        assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+        A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+        C, _, plan = gu.run_gemm(ctx, A, B, cfg, plan=plan)
+        assert plan.config.family == LIGHT
+        gu.assert_close_full(C, A, B, f"light {case} epilogue {epi}")
+        Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+        Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+        gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"light {case} epilogue {epi} integers")
     # the general form (exact: 0/1 operands, small integers in C)
     Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
     C0 = inputs.draw(37, inputs.TAG_A, M, N, "int5", "cuda")
@@ -412,7 +416,7 @@ def test_light_family_rules_and_stream_order(ctx, gu):
     assert hgemm.validate_config(512, 512, 512, ok) == hgemm.OK
     assert hgemm.validate_config(512, 516, 512, ok) == hgemm.ERR_UNSUPPORTED            # rows of C: multiples of 16 bytes
     assert hgemm.validate_config(512, 512, 516, ok) == hgemm.ERR_UNSUPPORTED            # rows of A and B too (no padded copies here)
-    for kw in (dict(split_k=2), dict(epilogue=DIRECT), dict(epilogue=WIDE), dict(accumulate=hgemm.ACC_F16), dict(tail_split=2),
+    for kw in (dict(split_k=2), dict(epilogue=WIDE), dict(accumulate=hgemm.ACC_F16), dict(tail_split=2),
                dict(swap_ab=1), dict(block_n=512), dict(raster_mode=1)):
         c = hgemm.Config.make(**{**dict(family=LIGHT, block_n=64, stages=4, epilogue=TMA), **kw})
         assert hgemm.validate_config(512, 512, 4096, c) == hgemm.ERR_UNSUPPORTED, kw
@@ -440,6 +444,63 @@ def test_light_family_rules_and_stream_order(ctx, gu):
     assert ctx.last_device_status() == (hgemm.OK, 0)
     p1.close()
     p2.close()
+
+
+# ---- the small family: register accumulators, for the smallest problems -------------------------------------------
+
+SMALL_CASES = [
+    (64, 64, 64), (8, 8, 8), (64, 64, 8), (128, 128, 128), (100, 136, 72), (64, 64, 4096), (256, 256, 256), (200, 328, 200),
+    (512, 512, 512), (1000, 64, 136), (64, 2048, 64), (320, 192, 1000),
+]
+
+
+@pytest.mark.parametrize("shape", SMALL_CASES, ids=lambda c: "x".join(map(str, c)))
+def test_small_family(ctx, gu, shape):
+    """mma.sync with register accumulators: the same arithmetic as the tcgen05 kernels (exact on integers, the contract
+    on random inputs), tails in every dimension, K shorter and much longer than the cp.async ring."""
+    import oracle
+    M, N, K = shape
+    cfg = hgemm.Config.small()
+    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    assert plan.config.family == hgemm.FAMILY_SMALL
+    gu.assert_close_full(C, A, B, f"small {shape}")
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"small {shape} integers")
+    Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
+    C0 = inputs.draw(39, inputs.TAG_A, M, N, "int5", "cuda")
+    for alpha, beta in ((2.0, -1.0), (0.5, 0.0)):
+        buf, Cs = gu.alloc_c_with_guards(M, N)                 # pre-filled with a NaN pattern
+        if beta != 0.0:
+            Cs.copy_(C0)
+        plan.run_scaled(alpha, beta, Ab, Bb, Cs)
+        assert ctx.last_device_status() == (hgemm.OK, 0) and gu.guards_intact(buf, M, N)
+        gu.assert_exact(Cs, oracle.hgemm_scaled_full(inputs.bits(Ab), inputs.bits(Bb), inputs.bits(C0), alpha, beta), f"small {shape} scaled")
+    plan.close()
+
+
+def test_small_family_rules(ctx, gu):
+    ok = hgemm.Config.small()
+    assert hgemm.validate_config(256, 256, 256, ok) == hgemm.OK
+    assert hgemm.validate_config(256, 260, 256, ok) == hgemm.ERR_UNSUPPORTED and hgemm.validate_config(256, 256, 260, ok) == hgemm.ERR_UNSUPPORTED
+    for field, value in (("block_n", 128), ("stages", 4), ("split_k", 2), ("epilogue", TMA), ("swap_ab", 1), ("block_m", 128), ("accumulate", 1)):
+        c = hgemm.Config.small()
+        setattr(c, field, value)
+        assert hgemm.validate_config(256, 256, 256, c) == hgemm.ERR_UNSUPPORTED, field
+    # K that needs padded copies: the plan pads, the kernel sees a multiple of 8
+    plan = ctx.plan(48, 64, 100)
+    plan.set_config(hgemm.Config.small())
+    A, B = inputs.make_ab(48, 64, 100, "int5", "cuda")
+    C = torch.zeros(48, 64, dtype=torch.float16, device="cuda")
+    plan.run(A, B, C)
+    torch.cuda.synchronize()
+    assert torch.equal(C.float(), A.float() @ B.float().T)
+    plan.close()
+    nn = ctx.plan(64, 512, 256, layout=hgemm.LAYOUT_NN)
+    assert nn.try_set_config(hgemm.Config.small()) == hgemm.ERR_UNSUPPORTED
+    nn.close()
 
 
 def test_dependent_launch_keeps_stream_order(ctx, gu):

@@ -65,7 +65,7 @@ def test_validate_rejects_illegal_configs(lib):
     assert hgemm.validate_config(M, N, K, ok) == hgemm.OK
     for kw in [dict(block_n=48), dict(block_n=288), dict(block_n=0), dict(stages=0), dict(stages=13),
                dict(block_n=256, stages=5), dict(split_k=0), dict(split_k=17), dict(block_k=32), dict(block_k=256), dict(raster_group=0),
-               dict(epilogue=3), dict(family=2)]:
+               dict(epilogue=3), dict(family=4)]:
         c = hgemm.Config.make(**{**dict(block_n=128, stages=4), **kw})
         assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED, kw
     c = hgemm.Config.make(block_n=128, stages=4)
@@ -143,7 +143,7 @@ def test_every_grid_shape_plans_to_a_legal_configuration(lib):
                 assert hgemm.validate_config(M, N, K, c) == hgemm.OK, (M, N, K, c.as_dict())
                 assert hgemm.config_smem_bytes(c) <= 232448
                 families.add(c.family)
-    assert {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA} <= families <= {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA, hgemm.FAMILY_LIGHT}
+    assert {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA} <= families <= {hgemm.FAMILY_UMMA_1CTA, hgemm.FAMILY_UMMA_2CTA, hgemm.FAMILY_LIGHT, hgemm.FAMILY_SMALL}
 
 
 def test_candidate_configs_are_legal_ranked_and_distinct(lib):
@@ -158,8 +158,9 @@ def test_candidate_configs_are_legal_ranked_and_distinct(lib):
         assert len(keys) == len(cands)
     # all three families, both stage widths, split-K and the wide epilogue all occur among the candidates of a shape that admits them
     pool = hgemm.candidate_configs(512, 512, 4096, max_count=256)
-    assert {c.family for c in pool} == {0, 1, 2} and {c.block_k for c in pool} == {64, 128}
-    assert all(c.split_k == 1 and c.epilogue == hgemm.EPILOGUE_TMA for c in pool if c.family == hgemm.FAMILY_LIGHT)
+    assert {c.family for c in pool} == {0, 1, 2, 3} and {c.block_k for c in pool} == {64, 128}
+    assert sum(c.family == hgemm.FAMILY_SMALL for c in pool) == 1                             # one fixed configuration
+    assert all(c.split_k == 1 and c.epilogue != hgemm.EPILOGUE_TMA_WIDE for c in pool if c.family == hgemm.FAMILY_LIGHT)
     big = hgemm.candidate_configs(8192, 8192, 8192, max_count=256)
     assert any(c.block_n == 512 and c.family == hgemm.FAMILY_UMMA_2CTA for c in big)          # the double-accumulator tile
     skinny = hgemm.candidate_configs(64, 12288, 4096, max_count=256)
