@@ -250,6 +250,19 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
 hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t K, int32_t block_n, int32_t split_k,
                                        const void *A, const void *B, void *C, void *stream);
 
+/* Operands that no kernel ahead of the call in its stream writes.  hgemm_run launches with
+ * programmatic stream serialisation (see hgemm_set_dependent_launch): the kernel may become
+ * resident while the kernel ahead of it is still running, but it must not read A or B before that
+ * kernel has completed, because it may be the one that produces them.  A caller who knows better
+ * -- a projection whose weight matrix was written long ago -- can say so: with HGEMM_STATIC_B
+ * (HGEMM_STATIC_A) the first pipeline stages' loads of B (A) are issued before the stream
+ * dependency is resolved, so they are in flight while the previous kernel drains; the other
+ * operand's loads and every store still wait.  `which` is a bit mask; 0 (the default) withdraws
+ * the promise.  A wrong promise is a data race on that operand.  Applies to the two persistent
+ * families with K-contiguous operands and K % 8 == 0; ignored elsewhere. */
+enum { HGEMM_STATIC_A = 1, HGEMM_STATIC_B = 2 };
+hgemm_status_t hgemm_plan_set_static_operands(hgemm_plan_t *plan, uint32_t which);
+
 /* Free one plan early (hgemm_destroy frees the rest). */
 hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan);
 

@@ -51,6 +51,7 @@ struct hgemm_plan_s {
     int smem = 0;
     unsigned long long *trace = nullptr;
     uint32_t debug_skip = 0;
+    uint32_t static_operands = 0;  // HGEMM_STATIC_A | HGEMM_STATIC_B as the caller declared them
     void *workspace = nullptr;
     int64_t workspace_bytes = 0;
     uint32_t *counters = nullptr;
@@ -545,8 +546,10 @@ hgemm_status_t hgemm_plan_layout(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t
     hgemm_config_t cfg;
     s = hgemm_host::plan_config(M, N, Kp, ctx->num_sms, &cfg);   // the table, else the neighbours' configurations re-fitted
     if (s != HGEMM_OK) return s;
-    if (layout == HGEMM_LAYOUT_NN && cfg.swap_ab) {
-        s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);   // the swapped form needs K-contiguous operands
+    if (layout == HGEMM_LAYOUT_NN &&
+        (cfg.swap_ab || cfg.block_n == 512 || cfg.family == HGEMM_FAMILY_LIGHT || cfg.family == HGEMM_FAMILY_SMALL)) {
+        // forms that exist only for K-contiguous operands: plan a row-major B from the cost model's own choice instead
+        s = hgemm_host::heuristic(M, N, Kp, ctx->num_sms, &cfg);
         if (s != HGEMM_OK) return s;
     }
     if (layout == HGEMM_LAYOUT_NN) {
@@ -828,6 +831,9 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     plan->params.wait_budget = ctx->wait_budget;
     plan->params.trace = plan->trace;
     plan->params.debug_skip = plan->debug_skip;
+    // a static operand in the caller's terms is the kernel's other operand when the configuration swaps them
+    plan->params.early_ops = cfg.swap_ab ? (((plan->static_operands & 1u) << 1) | ((plan->static_operands >> 1) & 1u)) : plan->static_operands;
+    if (plan->pad_a) plan->params.early_ops = 0u;     // the kernel reads padded copies that this very call has just written
     plan->params.scaled = scaled ? 1u : 0u;
     plan->params.alpha = alpha;
     plan->params.beta = beta;
@@ -904,6 +910,13 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
     if (s != HGEMM_OK) return s;
     e = cudaMemcpyAsync(C_host, plan->stage_c, c_bytes, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_plan_set_static_operands(hgemm_plan_t *plan, uint32_t which)
+{
+    if (!plan || which > 3u) return HGEMM_ERR_INVALID_ARG;
+    plan->static_operands = which;
     return HGEMM_OK;
 }
 

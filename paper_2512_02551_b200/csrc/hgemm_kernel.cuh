@@ -116,6 +116,8 @@ struct KernelParams {
                                   // traded) and stores element (row, col) of its tile at C[col * M + row]: the
                                   // caller's row-major C (whose rows are this kernel's M long)
     int32_t raster_serpentine;    // 1: odd raster groups sweep the n-tiles from last to first
+    uint32_t early_ops;           // bit 0 / bit 1: the kernel's A / B operand is static (no kernel ahead in the stream writes
+                                  // it): its first loads may leave before the stream dependency is resolved
 };
 
 template <bool OFF = false>
@@ -413,8 +415,8 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // DUAL (CTA pairs only, block_n == 512): one work item is a 256 x 512 tile held in BOTH accumulators at once -- every
 // 16-wide K step issues two MMAs (N = 256 each) that read the same A sub-tile -- so each CTA fetches 128 rows of A and
 // 256 rows of B per k-block for 128 x 512 results: a quarter less shared-memory fill per flop than the 256 x 256 pair
-// tile, which is what bounds the large shapes when L2 cannot feed 64 B/clk to every SM.  Price: no spare accumulator, so
-// the epilogue of a tile does not overlap the next tile's MMAs (the producer still prefetches through it).  Each CTA
+// tile, which is what bounds the large shapes when L2 cannot feed 64 B/clk to every SM.  There is no spare accumulator;
+// the epilogue overlaps the MMAs by staggering the two halves instead (see the MMA issuer).  Each CTA
 // loads 256 CONSECUTIVE rows of B (one box); MMA h (h = 0, 1) takes rows 128 h .. 128 h + 127 of both CTAs' boxes, so
 // accumulator column t holds column  256 * ((t % 256) / 128) + 128 * (t / 256) + t % 128  of the tile.
 template <int CTA_GROUP, bool WIDE_STORE = false, int SPLIT = 1, bool PLAIN = false, bool TRACE = !PLAIN, int SUBS = 0, bool XPOSE = false,
@@ -517,6 +519,37 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         long long t_wait = 0, t_work = 0;
         bool ok = true;
         bool dependencies_met = false;
+        // One stage's loads of the plain K-contiguous path, split by operand (for the early loads below): `expect` arms
+        // the stage's barrier with the bytes of BOTH operands, whichever part comes first.
+        auto issue_part = [&](int32_t js, int32_t jk0, int32_t a_row, int32_t b_row, bool expect, bool do_a, bool do_b) {
+            const uint32_t a_dst = smem_base + static_cast<uint32_t>(js) * stage_bytes;
+            const uint32_t b_dst = a_dst + a_stage_bytes;
+            const uint32_t fb = full_leader + 8 * js;
+            if (expect) {
+                if constexpr (CTA_GROUP == 1) mbar_arrive_expect_tx_elect(bar_full + 8 * js, stage_bytes);
+                else if (is_leader) mbar_arrive_expect_tx_elect(bar_full + 8 * js, stage_bytes);
+                else mbar_arrive_expect_tx_cluster_relaxed_elect(fb, stage_bytes);
+            }
+            if (p.tma_3d) {
+                if constexpr (CTA_GROUP == 1) {
+                    if (do_a) tma_load_3d_elect(a_dst, &tmap_a, 0, a_row, jk0 / kSubK, fb);
+                    if (do_b) tma_load_3d_elect(b_dst, &tmap_b, 0, b_row, jk0 / kSubK, fb);
+                } else {
+                    if (do_a) tma_load_3d_pair_elect(a_dst, &tmap_a, 0, a_row, jk0 / kSubK, fb);
+                    if (do_b) tma_load_3d_pair_elect(b_dst, &tmap_b, 0, b_row, jk0 / kSubK, fb);
+                }
+            } else {
+                for (int32_t sub = 0; sub < subs; ++sub) {
+                    if constexpr (CTA_GROUP == 1) {
+                        if (do_a) tma_load_2d_elect(a_dst + sub * kATileBytes, &tmap_a, jk0 + sub * kSubK, a_row, fb);
+                        if (do_b) tma_load_2d_elect(b_dst + sub * b_sub_bytes, &tmap_b, jk0 + sub * kSubK, b_row, fb);
+                    } else {
+                        if (do_a) tma_load_2d_pair_elect(a_dst + sub * kATileBytes, &tmap_a, jk0 + sub * kSubK, a_row, fb);
+                        if (do_b) tma_load_2d_pair_elect(b_dst + sub * b_sub_bytes, &tmap_b, jk0 + sub * kSubK, b_row, fb);
+                    }
+                }
+            }
+        };
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
             const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
@@ -533,11 +566,29 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const int32_t k0 = (it.kb_begin + kb) * p.block_k;
                 const uint32_t fb = full_leader + 8 * s;      // the (leader's) full barrier of this stage
                 if (!dependencies_met) {
+                    // Operands the caller declared static (KernelParams::early_ops: no kernel ahead of this call in the
+                    // stream writes them) may be fetched BEFORE the stream dependency is resolved: the first pass of the
+                    // ring -- every stage is free -- is armed and that operand's loads go out now, the other operand's
+                    // after the wait.  A projection's weights then stream in while the previous kernel drains.
+                    int32_t pre = 0;
+                    if (p.early_ops != 0u && !(TRACE && (p.debug_skip & 1u)) && !(!PLAIN && (p.b_row_major || it.bn != p.block_n))) {
+                        pre = min(it.kb_count, p.stages);
+                        for (int32_t j = 0; j < pre; ++j)
+                            issue_part(j, (it.kb_begin + j) * p.block_k, a_row, b_row, true, (p.early_ops & 1u) != 0u, (p.early_ops & 2u) != 0u);
+                    }
                     grid_dependency_wait();                   // the kernels before this one are complete: global memory may be read
                     dependencies_met = true;
                     if (threadIdx.x == 0) {
                         trace_stamp<!TRACE>(p, 0);
                         trace_stamp<!TRACE>(p, 1);
+                    }
+                    if (pre > 0) {
+                        for (int32_t j = 0; j < pre; ++j)
+                            issue_part(j, (it.kb_begin + j) * p.block_k, a_row, b_row, false, (p.early_ops & 1u) == 0u, (p.early_ops & 2u) == 0u);
+                        if (lane == 0) trace_stamp<!TRACE>(p, 2);
+                        if (pre == p.stages) { s = 0; ph ^= 1u; } else { s = pre; }
+                        kb = pre - 1;                          // the loop's increment moves on to the first k-block not yet issued
+                        continue;
                     }
                 }
                 if ((TRACE ? p.debug_skip : 0u) & 1u) {
@@ -639,6 +690,105 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
                 const uint32_t acc = DUAL ? 0u : (local_tile & 1u);            // DUAL: one work item fills both accumulators
                 const uint32_t acc_ph = DUAL ? (local_tile & 1u) : ((local_tile >> 1) & 1u);
+                if constexpr (DUAL) {
+                    // ---- the 256 x 512 tile: accumulator h (columns 256 h ..) takes rows 128 h .. of both CTAs' B boxes ----
+                    // There is no spare accumulator, so the hand-off to the epilogue is staggered between the halves
+                    // instead: at the head of a tile the first `stages` k-blocks go into accumulator 0 as soon as the
+                    // epilogue has drained it -- while it still drains accumulator 1 -- and only then into accumulator 1;
+                    // at the tail the last `stages` k-blocks finish accumulator 0 first, so that its epilogue runs under
+                    // accumulator 1's last MMAs.  A stage is freed by the MMAs of its second half.  In between both
+                    // halves take each k-block in turn.  (Tiles with fewer than 2 * stages k-blocks are not staggered.)
+                    const int32_t S = p.stages, kbc = it.kb_count;
+                    auto acc_free = [&](uint32_t h) {
+                        ok = mbar_wait(bar_tmem_empty + 8 * h, acc_ph ^ 1u, ctl, status_code(kRoleMma, 1, h));
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (ok) tc_fence_after_sync();
+                    };
+                    auto stage_full = [&](int32_t st, uint32_t par) {
+                        ok = mbar_wait(bar_full + 8 * st, par, ctl, status_code(kRoleMma, 0, st));
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (ok) tc_fence_after_sync();
+                    };
+                    auto issue_half = [&](int32_t st, uint32_t h, bool overwrite) {
+                        const uint64_t a_desc = desc_a0 + static_cast<uint64_t>(static_cast<uint32_t>(st) * desc_stage_step);
+                        const uint64_t b_desc = desc_b0 + static_cast<uint64_t>(static_cast<uint32_t>(st) * desc_stage_step) +
+                                                static_cast<uint64_t>(h * ((128u * 128u) >> 4));
+                        for (int32_t sub = 0; sub < subs; ++sub) {
+                            const uint64_t a_sub = a_desc + static_cast<uint64_t>(static_cast<uint32_t>(sub) * (kATileBytes >> 4));
+                            const uint64_t b_sub = b_desc + static_cast<uint64_t>(static_cast<uint32_t>(sub) * (b_sub_bytes >> 4));
+#pragma unroll
+                            for (int k = 0; k < kSubK / kUmmaK; ++k)
+                                umma_f16_elect<CTA_GROUP>(tmem_base + h * 256u, a_sub + 2u * k, b_sub + 2u * k, p.idesc,
+                                                       (overwrite && (sub | k) == 0) ? 0u : 1u);
+                        }
+                    };
+                    auto advance = [&]() { if (++s == S) { s = 0; ph ^= 1u; } };
+                    if (kbc < 2 * S) {
+                        acc_free(0);
+                        if (ok) acc_free(1);
+                        for (int32_t kb = 0; ok && kb < kbc; ++kb) {
+                            stage_full(s, ph);
+                            if (!ok) break;
+                            issue_half(s, 0, kb == 0);
+                            issue_half(s, 1, kb == 0);
+                            umma_commit_elect<CTA_GROUP>(bar_empty + 8 * s, leader_rank);
+                            advance();
+                        }
+                        if (!ok) break;
+                        umma_commit_elect<CTA_GROUP>(bar_tmem_full, leader_rank);
+                        umma_commit_elect<CTA_GROUP>(bar_tmem_full + 8, leader_rank);
+                    } else {
+                        // head
+                        acc_free(0);
+                        const int s_head = s;
+                        const uint32_t ph_head = ph;
+                        for (int32_t j = 0; ok && j < S; ++j) {
+                            stage_full(s, ph);
+                            if (!ok) break;
+                            issue_half(s, 0, j == 0);
+                            advance();
+                        }
+                        if (ok) acc_free(1);
+                        if (!ok) break;
+                        s = s_head;
+                        ph = ph_head;
+                        for (int32_t j = 0; j < S; ++j) {
+                            issue_half(s, 1, j == 0);
+                            umma_commit_elect<CTA_GROUP>(bar_empty + 8 * s, leader_rank);
+                            advance();
+                        }
+                        // middle
+                        for (int32_t kb = S; ok && kb < kbc - S; ++kb) {
+                            stage_full(s, ph);
+                            if (!ok) break;
+                            issue_half(s, 0, false);
+                            issue_half(s, 1, false);
+                            umma_commit_elect<CTA_GROUP>(bar_empty + 8 * s, leader_rank);
+                            advance();
+                        }
+                        if (!ok) break;
+                        // tail
+                        const int s_tail = s;
+                        const uint32_t ph_tail = ph;
+                        for (int32_t j = 0; ok && j < S; ++j) {
+                            stage_full(s, ph);
+                            if (!ok) break;
+                            issue_half(s, 0, false);
+                            advance();
+                        }
+                        if (!ok) break;
+                        umma_commit_elect<CTA_GROUP>(bar_tmem_full, leader_rank);
+                        s = s_tail;
+                        ph = ph_tail;
+                        for (int32_t j = 0; j < S; ++j) {
+                            issue_half(s, 1, false);
+                            umma_commit_elect<CTA_GROUP>(bar_empty + 8 * s, leader_rank);
+                            advance();
+                        }
+                        umma_commit_elect<CTA_GROUP>(bar_tmem_full + 8, leader_rank);
+                    }
+                    continue;
+                }
                 const long long ca = tr ? clock64() : 0;
                 ok = mbar_wait(bar_tmem_empty + 8 * acc, acc_ph ^ 1u, ctl, status_code(kRoleMma, 1, acc));
                 ok = __all_sync(0xffffffffu, ok);
@@ -670,9 +820,6 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                 // advancing K by 16 fp16 inside the swizzle span = +32 bytes = +2 in the address field
                                 umma_f16_elect<CTA_GROUP>(d_tmem, a_sub + 2u * k, b_sub + b_kstep * k, idesc,
                                                        (kb | sub | k) != 0 ? 1u : 0u);
-                                if constexpr (DUAL)      // rows 128 .. 255 of both CTAs' B boxes into the second accumulator
-                                    umma_f16_elect<CTA_GROUP>(d_tmem + 256u, a_sub + 2u * k, b_sub + ((128u * 128u) >> 4) + b_kstep * k, idesc,
-                                                           (kb | sub | k) != 0 ? 1u : 0u);
                             }
                         }
                     }
@@ -735,11 +882,18 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             auto chunk_col = [](int32_t c) -> int32_t {
                 return DUAL ? ((c >> 2) & 1) * 256 + (c >> 3) * 128 + (c & 3) * 32 : c * 32;
             };
-            ok = mbar_wait(bar_tmem_full + 8 * acc, acc_ph, ctl, status_code(kRoleEpilogue, 2, acc));
-            ok = __all_sync(0xffffffffu, ok);   // the warp-wide tensor-memory loads below need the whole warp
-            if (!ok) break;
+            // DUAL: the two halves of the tile become ready one after the other (see the MMA issuer): each is waited
+            // for, read and released on its own below
+            auto wait_accumulator = [&](uint32_t idx) {
+                ok = mbar_wait(bar_tmem_full + 8 * idx, acc_ph, ctl, status_code(kRoleEpilogue, 2, idx));
+                ok = __all_sync(0xffffffffu, ok);   // the warp-wide tensor-memory loads below need the whole warp
+                if (ok) tc_fence_after_sync();
+            };
+            if constexpr (!DUAL) {
+                wait_accumulator(acc);
+                if (!ok) break;
+            }
             if (w == unit && threadIdx.x == 64) trace_stamp<!TRACE>(p, 5);
-            tc_fence_after_sync();
             const int32_t row0 = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;  // first row of this CTA's 128
             const int32_t grow = row0 + static_cast<int32_t>(row_in_tile);          // this thread's global row
             const uint32_t t_addr = tmem_base + ((q * 32u) << 16) + acc * static_cast<uint32_t>(p.block_n);
@@ -842,14 +996,15 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
             };
-            auto release_accumulator = [&]() {
+            auto release_accumulator = [&](uint32_t idx) {
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) {
-                    if constexpr (CTA_GROUP == 1) mbar_arrive(bar_tmem_empty + 8 * acc);
-                    else mbar_arrive_cluster(tmem_empty_leader + 8 * acc);
+                    if constexpr (CTA_GROUP == 1) mbar_arrive(bar_tmem_empty + 8 * idx);
+                    else mbar_arrive_cluster(tmem_empty_leader + 8 * idx);
                 }
             };
+            constexpr uint32_t kHalves = DUAL ? 2u : 1u;        // DUAL: accumulator h = chunks 8 h .. 8 h + 7 = barrier pair h
 
             // chunks of this tile that hold columns of C, and whether this warp's 32 rows hold rows of C:
             // tiles on the ragged edge (and every tile of a problem with M < 128) skip the dead part
@@ -862,8 +1017,16 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // A box whose second half lies beyond N is staged half empty: the store is clipped there.
                 uint32_t v[32];
                 const int32_t chunks = live_rows ? live_chunks : 0;     // shadows the tile's chunk count
-                const int32_t boxes = (chunks + 1) >> 1;
-                for (int32_t b = static_cast<int32_t>(first_chunk); b < boxes; b += 2) {
+                const int32_t all_boxes = (chunks + 1) >> 1;
+                for (uint32_t hf = 0; ok && hf < kHalves; ++hf) {
+                const uint32_t rel = DUAL ? hf : acc;
+                if constexpr (DUAL) {
+                    wait_accumulator(hf);
+                    if (!ok) break;
+                }
+                const int32_t box_lo = DUAL ? 4 * static_cast<int32_t>(hf) : 0;
+                const int32_t boxes = DUAL ? min(all_boxes, box_lo + 4) : all_boxes;
+                for (int32_t b = box_lo + static_cast<int32_t>(first_chunk); b < boxes; b += 2) {
                     const uint32_t buf = staging + (store_count & 1u) * kWideBoxBytes;
                     bulk_wait_group_read<1>();                      // the box written two stores ago has been read
                     __syncwarp();
@@ -880,7 +1043,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                 for (int j = 0; j < 32; ++j)
                                     v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
                             }
-                            if (b + 2 >= boxes && c + 1 >= min(chunks, 2 * b + 2)) release_accumulator();   // this warp's last load
+                            if (b + 2 >= boxes && c + 1 >= min(chunks, 2 * b + 2)) release_accumulator(rel);   // this warp's last load
                             if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                                 for (int j = 0; j < 4; ++j)
@@ -905,13 +1068,23 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     ++store_count;
                 }
-                if (static_cast<int32_t>(first_chunk) >= boxes) release_accumulator();    // nothing to load
+                if (box_lo + static_cast<int32_t>(first_chunk) >= boxes) release_accumulator(rel);    // nothing to load
+                }
+                if (!ok) break;
             } else if (SPLIT == 0 || it.slices == 1) {
                 // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second
                 // chunk in flight costs more in registers than it hides
                 uint32_t v[32];
-                const int32_t chunks = live_rows ? live_chunks : 0;     // shadows the tile's chunk count
-                for (int32_t c = static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
+                const int32_t all_chunks = live_rows ? live_chunks : 0;
+                for (uint32_t hf = 0; ok && hf < kHalves; ++hf) {
+                const uint32_t rel = DUAL ? hf : acc;
+                if constexpr (DUAL) {
+                    wait_accumulator(hf);
+                    if (!ok) break;
+                }
+                const int32_t chunk_lo = DUAL ? 8 * static_cast<int32_t>(hf) : 0;
+                const int32_t chunks = DUAL ? min(all_chunks, chunk_lo + 8) : all_chunks;     // shadows the tile's chunk count
+                for (int32_t c = chunk_lo + static_cast<int32_t>(first_chunk); c < chunks; c += 2) {
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
                     tmem_ld_wait();
                     if ((!PLAIN && p.acc_f16)) {
@@ -921,7 +1094,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         for (int j = 0; j < 32; ++j)
                             v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
                     }
-                    if (c + 2 >= chunks) release_accumulator();       // every load of this warp has completed
+                    if (c + 2 >= chunks) release_accumulator(rel);    // every load of this warp (from this accumulator) has completed
                     if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
@@ -929,7 +1102,9 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     emit_chunk(v, c);
                 }
-                if (static_cast<int32_t>(first_chunk) >= chunks) release_accumulator();   // nothing to load
+                if (chunk_lo + static_cast<int32_t>(first_chunk) >= chunks) release_accumulator(rel);   // nothing to load
+                }
+                if (!ok) break;
             } else if (SPLIT == 2) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches
@@ -964,7 +1139,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         bulk_commit_group();
                     }
                 }
-                release_accumulator();
+                release_accumulator(acc);
                 if (lane == 0) {
                     bulk_wait_group<0>();                            // this warp's part of the slot is written
                     fence_proxy_async_all();                         // order those writes before the signal below

@@ -21,11 +21,12 @@ TAIL_K, TAIL_N = 0, 1
 ACC_F32, ACC_F16 = 0, 1
 LAYOUT_TN, LAYOUT_NN = 0, 1
 RASTER_SWEEP, RASTER_SERPENTINE = 0, 1
+STATIC_A, STATIC_B = 1, 2
 
 # every symbol include/hgemm.h declares
 EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
-    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_plan_autotune", "hgemm_candidate_configs", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
+    "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_plan_set_static_operands", "hgemm_plan_autotune", "hgemm_candidate_configs", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
     "hgemm_last_device_status", "hgemm_ctx_last_device_status", "hgemm_debug_fail_allocs", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
@@ -101,6 +102,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_plan_destroy": (i32, [p]),
             "hgemm_plan_get_config": (i32, [p, cfgp]),
             "hgemm_plan_set_config": (i32, [p, cfgp]),
+            "hgemm_plan_set_static_operands": (i32, [p, ctypes.c_uint32]),
             "hgemm_plan_autotune": (i32, [p, p, p, p, p, i32, ctypes.POINTER(ctypes.c_float)]),
             "hgemm_heuristic_config": (i32, [i64, i64, i64, i32, cfgp]),
             "hgemm_candidate_configs": (i32, [i64, i64, i64, i32, cfgp, i32]),
@@ -250,6 +252,10 @@ class Plan:
 
     def set_config(self, cfg: Config) -> None:
         _check(lib().hgemm_plan_set_config(self._h, ctypes.byref(cfg)), f"hgemm_plan_set_config({cfg.as_dict()})")
+
+    def set_static_operands(self, a: bool = False, b: bool = False) -> None:
+        """``hgemm_plan_set_static_operands``: promise that no kernel ahead of a call in its stream writes A and/or B."""
+        _check(lib().hgemm_plan_set_static_operands(self._h, (1 if a else 0) | (2 if b else 0)), "hgemm_plan_set_static_operands")
 
     def try_set_config(self, cfg: Config) -> int:
         return int(lib().hgemm_plan_set_config(self._h, ctypes.byref(cfg)))

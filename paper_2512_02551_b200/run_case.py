@@ -1,10 +1,12 @@
 """Run one HGEMM shape a few times through the C ABI and print its device time.
 
     python -m paper_2512_02551_b200.run_case 8192x8192x8192 [--iters 3] [--warmup 2]
-        [--family 0|1 --block-n 256 --stages 4 --split-k 1 --raster 8 --epilogue 0|1]
+        [--family 0|1|2|3 --block-n 256 --block-k 64|128 --stages 4 --split-k 1 --split-mode 0|1 --raster 8
+         --raster-mode 0|1 --epilogue 0|1|2 --swap-ab 0|1]
 
 Small enough to sit under a profiler: it draws the inputs, plans, warms up and launches
-`iters` times.  Without the configuration flags the library's own plan is used.
+`iters` times.  Without the configuration flags the library's own plan is used; with --family the
+configuration starts from a plain one of that family and the other flags refine it.
 """
 from __future__ import annotations
 
@@ -26,6 +28,10 @@ def main() -> None:
     ap.add_argument("--split-k", type=int)
     ap.add_argument("--raster", type=int)
     ap.add_argument("--epilogue", type=int)
+    ap.add_argument("--block-k", type=int)
+    ap.add_argument("--split-mode", type=int)
+    ap.add_argument("--raster-mode", type=int)
+    ap.add_argument("--swap-ab", type=int)
     args = ap.parse_args()
     M, N, K = (int(v) for v in args.shape.lower().split("x"))
     with hgemm.Context(0) as ctx:
@@ -33,12 +39,17 @@ def main() -> None:
         C = torch.empty(M, N, dtype=torch.float16, device="cuda")
         plan = ctx.plan(M, N, K)
         cfg = plan.config
+        if args.family is not None:
+            # an explicit family starts from a clean configuration instead of the plan's own (whose other fields may not apply)
+            cfg = hgemm.Config.small() if args.family == hgemm.FAMILY_SMALL else hgemm.Config.make(
+                family=args.family, block_n=128, stages=4, raster_group=1, epilogue=hgemm.EPILOGUE_TMA)
         for name, attr in (("family", "family"), ("block_n", "block_n"), ("stages", "stages"), ("split_k", "split_k"),
-                           ("raster", "raster_group"), ("epilogue", "epilogue")):
+                           ("raster", "raster_group"), ("epilogue", "epilogue"), ("block_k", "block_k"), ("split_mode", "split_mode"),
+                           ("raster_mode", "raster_mode"), ("swap_ab", "swap_ab")):
             v = getattr(args, name)
             if v is not None:
                 setattr(cfg, attr, v)
-        cfg.block_m = 256 if cfg.family == hgemm.FAMILY_UMMA_2CTA else 128
+        cfg.block_m = 256 if cfg.family == hgemm.FAMILY_UMMA_2CTA else 64 if cfg.family == hgemm.FAMILY_SMALL else 128
         plan.set_config(cfg)
         for _ in range(args.warmup):
             plan.run(A, B, C)

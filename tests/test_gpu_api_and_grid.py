@@ -190,3 +190,20 @@ def test_full_grid_default_plans(ctx, gu):
                 rep = gu.check_shape(ctx, M, N, K, "uniform")
                 worst = max(worst, rep["max_err_over_bound"])
     assert worst < 1.0
+
+
+def test_paper_grid_with_16384_default_plans(ctx, gu):
+    """The 271 shapes that the paper's tenth grid value adds (every (M, N, K) over {64 .. 12288, 16384} with at least one
+    16384), each with the plan the library picks: full-output oracle check up to 2048^3 by volume, 4096 samples + one row
+    + one column above."""
+    g10 = GRID + [16384]
+    worst, count = 0.0, 0
+    for M in g10:
+        for N in g10:
+            for K in g10:
+                if 16384 not in (M, N, K):
+                    continue
+                rep = gu.check_shape(ctx, M, N, K, "uniform")
+                worst = max(worst, rep["max_err_over_bound"])
+                count += 1
+    assert count == 271 and worst < 1.0

@@ -531,6 +531,44 @@ def test_dependent_launch_keeps_stream_order(ctx, gu):
     p2.close()
 
 
+def test_static_operand_promise_keeps_the_other_operand_ordered(ctx, gu):
+    """With HGEMM_STATIC_B the weights' first loads leave before the stream dependency is resolved; the activations,
+    which the kernel ahead produces, must still be read after it: C1 = A B1^T, C2 = C1 B2^T through every persistent
+    path that takes early loads (both families, 64- and 128-wide stages, split-K in a cluster, swapped operands)."""
+    import oracle
+    M, K1, N1, N2 = 256, 512, 1024, 2048
+    A = inputs.draw(1, inputs.TAG_A, M, K1, "binary", "cuda")
+    B1 = inputs.draw(2, inputs.TAG_B, N1, K1, "binary", "cuda")
+    B2 = inputs.draw(3, inputs.TAG_B, N2, N1, "binary", "cuda")
+    c1_ref = oracle.hgemm_full(inputs.bits(A), inputs.bits(B1))                 # <= 512: exact in fp16
+    c2_ref = oracle.hgemm_full(oracle.f64_to_f16_bits(c1_ref.ravel()).reshape(M, N1), inputs.bits(B2))   # < 2^24: exact in fp32
+    p1, p2 = ctx.plan(M, N1, K1), ctx.plan(M, N2, N1)
+    configs = [
+        hgemm.Config.make(family=F1, block_n=128, stages=4, raster_group=1, epilogue=TMA, block_k=64),
+        hgemm.Config.make(family=F2, block_n=256, stages=3, raster_group=1, epilogue=TMA, block_k=128),
+        hgemm.Config.make(family=F1, block_n=128, stages=6, split_k=4, raster_group=1, epilogue=DIRECT, block_k=64, split_mode=CLUSTER),
+        hgemm.Config.make(family=F2, block_n=256, stages=4, raster_group=1, epilogue=TMA, block_k=64, swap_ab=1),
+    ]
+    for cfg in configs:
+        for plan in (p1, p2):
+            plan.set_config(cfg)
+            plan.set_static_operands(b=True)
+        for rep in range(15):
+            C1 = torch.zeros(M, N1, dtype=torch.float16, device="cuda")
+            C2 = torch.zeros(M, N2, dtype=torch.float16, device="cuda")
+            p1.run(A, B1, C1)
+            p2.run(C1, B2, C2)                                                  # reads C1 as its A: not static
+            p1.run(A, B1, C1)
+            torch.cuda.synchronize()
+            gu.assert_exact(C2, c2_ref, f"static B, {cfg.as_dict()}, repetition {rep}")
+            gu.assert_exact(C1, c1_ref, f"static B, first product, repetition {rep}")
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    assert hgemm.lib().hgemm_plan_set_static_operands(p1._h, 4) == hgemm.ERR_INVALID_ARG
+    p1.set_static_operands()
+    p1.close()
+    p2.close()
+
+
 # ---- tail split: only the tiles of the last, partly filled wave are cut along K ------------------------------
 
 @pytest.mark.parametrize("family,bn,bk,stages,tail", [(F2, 256, 64, 6, 2), (F1, 256, 64, 4, 2), (F1, 128, 128, 3, 2), (F2, 128, 128, 4, 3)])
