@@ -66,11 +66,11 @@ enum {
                                    accumulator, no CTA-wide barrier at the end, only the shared memory it uses; its first
                                    loads leave before the CTA's set-up has finished.  Needs K % 8 == 0 and N % 8 == 0, split_k == 1, no
                                    tail_split, no swap_ab, fp32 accumulators, the TN layout, HGEMM_EPILOGUE_DIRECT or HGEMM_EPILOGUE_TMA */
-    HGEMM_FAMILY_SMALL = 3      /* the register-accumulator kernel for the smallest problems: 64 x 64 tiles, cp.async + ldmatrix
-                                   + mma.sync with fp32 accumulators in registers -- no tensor memory to allocate (0.7 us on
-                                   B200), no tensor maps, no mbarriers.  One fixed configuration: block_m = block_n = block_k
-                                   = 64, stages = 3, split_k = 1, HGEMM_EPILOGUE_DIRECT.  Needs K % 8 == 0 and N % 8 == 0, no
-                                   tail_split, no swap_ab, fp32 accumulators, the TN layout */
+    HGEMM_FAMILY_SMALL = 3      /* the register-accumulator kernel for the smallest problems: 64 x 64 or 32 x 32 tiles, cp.async +
+                                   ldmatrix + mma.sync with fp32 accumulators in registers -- no tensor memory to allocate
+                                   (0.7 us on B200), no tensor maps, no mbarriers.  Two fixed configurations: block_m = block_n
+                                   = 64 or 32, block_k = 64, stages = 3, split_k = 1, HGEMM_EPILOGUE_DIRECT.  Needs K % 8 == 0
+                                   and N % 8 == 0, no tail_split, no swap_ab, fp32 accumulators, the TN layout */
 };
 
 /* Where the fp32 partial sums of a split-K tile meet.  Both sum the slices in slice
@@ -121,7 +121,7 @@ enum {
  * count and block-swizzle stride of sections 5.2 and 6, plus split-K). */
 typedef struct {
     int32_t family;       /* HGEMM_FAMILY_* */
-    int32_t block_m;      /* 128 (1-CTA and light families), 256 (2-CTA pair) or 64 (small family) */
+    int32_t block_m;      /* 128 (1-CTA and light families), 256 (2-CTA pair), or block_n (small family) */
     int32_t block_n;      /* multiple of 32 in [32, 256]; or 512 (CTA-pair family only): a 256 x 512 tile held in both
                              tensor-memory accumulators at once, two MMAs per K step sharing the A tile -- a quarter less
                              shared-memory fill per flop than 256 x 256, no overlap of a tile's epilogue with the next

@@ -262,9 +262,9 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     // they use, so that the next call's CTAs become resident beside this call's, made those calls slower.)
     pl->smem = int(hgemm_host::kSmemOptInBytes);
     if (cfg.family == HGEMM_FAMILY_SMALL) {
-        // 64 x 64 tiles, one CTA each, static shared memory, no tensor maps
-        p.tiles_m = int32_t((pl->M + 63) / 64);
-        p.tiles_n = int32_t((pl->N + 63) / 64);
+        // 64 x 64 or 32 x 32 tiles, one CTA each, static shared memory, no tensor maps
+        p.tiles_m = int32_t((pl->M + cfg.block_n - 1) / cfg.block_n);
+        p.tiles_n = int32_t((pl->N + cfg.block_n - 1) / cfg.block_n);
         pl->grid = p.tiles_m * p.tiles_n;
         pl->cluster_dim = 1;
         pl->smem = 0;
@@ -773,7 +773,8 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         lc.attrs = attr;
         lc.numAttrs = ctx->dependent_launch ? 1 : 0;
         void *sargs[1] = {&sp};
-        cudaError_t e = cudaLaunchKernelExC(&lc, reinterpret_cast<const void *>(hgemm_dev::hgemm_small_kernel), sargs);
+        cudaError_t e = cudaLaunchKernelExC(&lc, cfg.block_n == 32 ? reinterpret_cast<const void *>(hgemm_dev::hgemm_small_kernel<32>)
+                                                                   : reinterpret_cast<const void *>(hgemm_dev::hgemm_small_kernel<64>), sargs);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         return HGEMM_OK;
     }

@@ -33,7 +33,7 @@ int64_t staging_bytes(const hgemm_config_t &c)
 
 int64_t smem_bytes(const hgemm_config_t &c)
 {
-    if (c.family == HGEMM_FAMILY_SMALL) return 3 * 2 * 64 * 64 * 2;      // its static ring: three stages of A and B tiles
+    if (c.family == HGEMM_FAMILY_SMALL) return 3 * 2 * int64_t(c.block_n) * 64 * 2;      // its static ring: three stages of A and B tiles
     return kAlignSlack + int64_t(c.stages) * stage_bytes(c) + staging_bytes(c) + kCtrlBytes;
 }
 
@@ -58,7 +58,7 @@ SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const
 {
     if (c.family == HGEMM_FAMILY_SMALL) {
         SplitLayout S;
-        S.tiles = ceil_div(M, 64) * ceil_div(N, 64);
+        S.tiles = ceil_div(M, c.block_n) * ceil_div(N, c.block_n);
         S.first_split_tile = S.tiles;
         S.slices = 1;
         S.pieces = 1;
@@ -137,15 +137,15 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
         std::swap(M, N);
     }
     if (c.family == HGEMM_FAMILY_SMALL) {
-        // one fixed configuration
+        // two fixed configurations: 64 x 64 or 32 x 32 tiles
         for (int i = 0; i < 2; ++i)
             if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
-        if (c.block_m != 64 || c.block_n != 64 || c.block_k != 64 || c.stages != 3 || c.split_k != 1 || c.tail_split >= 2 || c.swap_ab ||
+        if ((c.block_n != 64 && c.block_n != 32) || c.block_m != c.block_n || c.block_k != 64 || c.stages != 3 || c.split_k != 1 || c.tail_split >= 2 || c.swap_ab ||
             c.accumulate != HGEMM_ACC_F32 || c.epilogue != HGEMM_EPILOGUE_DIRECT || c.raster_mode != HGEMM_RASTER_SWEEP || c.raster_group < 1 ||
             (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) || (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N) ||
             (K % 8) != 0 || (N % 8) != 0)
             return HGEMM_ERR_UNSUPPORTED;
-        if (ceil_div(M, 64) * ceil_div(N, 64) >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
+        if (ceil_div(M, c.block_n) * ceil_div(N, c.block_n) >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
         return HGEMM_OK;
     }
     if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA && c.family != HGEMM_FAMILY_LIGHT) return HGEMM_ERR_UNSUPPORTED;
@@ -208,10 +208,11 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
 double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c)
 {
     if (c.family == HGEMM_FAMILY_SMALL) {
-        // Not fitted: a ranking hint.  Per 64-wide k-block a CTA moves 16 KB into shared memory and issues 128 MMAs of
-        // 16 x 8 x 16 (about 1024 MACs per clock and SM on the register path); four CTAs share an SM; a short fixed part.
-        const double waves = std::ceil(double(ceil_div(M, 64) * ceil_div(N, 64)) / (4.0 * std::max(1, num_sms)));
-        return 1400.0 + waves * (double(ceil_div(K, 64)) * 300.0 * 4.0 / 4.0 + 600.0);
+        // Not fitted: a ranking hint.  Per 64-wide k-block a CTA with 64 x 64 tiles moves 16 KB into shared memory and
+        // issues 128 MMAs of 16 x 8 x 16 (a quarter of both with 32 x 32 tiles); a few CTAs share an SM; a short fixed part.
+        const double t = c.block_n == 32 ? 0.3 : 1.0;
+        const double waves = std::ceil(double(ceil_div(M, c.block_n) * ceil_div(N, c.block_n)) / ((c.block_n == 32 ? 8.0 : 4.0) * std::max(1, num_sms)));
+        return 1400.0 + waves * (double(ceil_div(K, 64)) * 600.0 * t + 600.0);
     }
     // Rough machine model, in SM clock cycles: a ranking aid, not a prediction.  Its form follows the kernel
     // (waves of tiles, k-blocks bounded by the tensor pipe, the stage hand-off, the fill rate of one SM, the
@@ -362,6 +363,8 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
         c.split_k = 1;
         c.raster_group = 1;
         add(c);                                                     // (validate() keeps it to K % 8 == 0 and N % 8 == 0)
+        c.block_m = c.block_n = 32;
+        add(c);
     }
     // swap == 1: the operands trade places (few rows, many columns: the rows of B fill the MMA's 128-row side)
     for (int swap = 0; swap < 2; ++swap) {

@@ -8,8 +8,11 @@
 // memory, ldmatrix, mma.sync.m16n8k16 (fp16 x fp16 -> fp32) with the accumulators in registers, 4-byte stores.
 // The tensor cores still do the contraction; what is dropped is everything around them.
 //
-//   CTA: 128 threads = 2 x 2 warps, one 64 x 64 tile of C; each warp a 32 x 32 quarter (2 x 4 MMA tiles)
-//   K loop: 64-wide k-blocks through a 3-stage cp.async ring (8 KB of A + 8 KB of B per stage)
+//   CTA: 128 threads = 2 x 2 warps, one T x T tile of C (T = 64 or 32); each warp a quarter of it (T = 64: 2 x 4 MMA tiles
+//   of 16 x 8; T = 32: 1 x 2).  The register path issues an MMA every few cycles per SM sub-partition, so a CTA's k-block costs
+//   time in proportion to its tile: the 32 x 32 tile spreads a small problem over four times as many SMs and is what the
+//   shortest K loops want, the 64 x 64 tile moves half as many bytes per flop.
+//   K loop: 64-wide k-blocks through a 3-stage cp.async ring (T x 128 bytes of A and of B per stage)
 //   shared memory: rows of 128 bytes; 16-byte piece c of row r lives at piece c ^ (r & 7), so that the eight
 //   row addresses of an ldmatrix fall on different banks
 //
@@ -25,7 +28,6 @@
 
 namespace hgemm_dev {
 
-constexpr int kSmallTile = 64;        // rows and columns of C per CTA
 constexpr int kSmallBk = 64;          // K extent of a stage
 constexpr int kSmallStages = 3;
 constexpr int kSmallThreads = 128;
@@ -35,7 +37,7 @@ struct SmallParams {
     const __half *B;                  // N x K, K-contiguous
     __half *C;                        // M x N row-major
     int32_t M, N, K;
-    int32_t tiles_m;                  // ceil(M / 64): CTA b computes tile (b % tiles_m, b / tiles_m)
+    int32_t tiles_m;                  // ceil(M / T): CTA b computes tile (b % tiles_m, b / tiles_m)
     uint32_t scaled;                  // 1: C = alpha A B^T + beta C
     float alpha, beta;
 };
@@ -58,13 +60,18 @@ __device__ __forceinline__ void mma_m16n8k16(float (&d)[4], const uint32_t (&a)[
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+template <int T>                      // rows and columns of C per CTA: 64 or 32
 __global__ void __launch_bounds__(kSmallThreads)
 hgemm_small_kernel(const SmallParams p)
 {
-    __shared__ __align__(128) uint8_t smem[kSmallStages * 2 * kSmallTile * kSmallBk * 2];     // 48 KB: [stage][A | B][64 rows][128 bytes]
+    static_assert(T == 64 || T == 32, "tile size");
+    constexpr int kSmallTile = T;
+    constexpr int MI = T / 32;        // 16-row MMA tiles per warp
+    constexpr int NI = T / 16;        // 8-column MMA tiles per warp (two per ldmatrix)
+    __shared__ __align__(128) uint8_t smem[kSmallStages * 2 * kSmallTile * kSmallBk * 2];     // 48 or 24 KB: [stage][A | B][T rows][128 bytes]
     const uint32_t smem_base = smem_addr(smem);
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const uint32_t wm = warp & 1u, wn = warp >> 1;                      // this warp's 32 x 32 quarter of the tile
+    const uint32_t wm = warp & 1u, wn = warp >> 1;                      // this warp's quarter of the tile
     const int32_t tile = static_cast<int32_t>(blockIdx.x);
     const int32_t tn = tile / p.tiles_m, tm = tile - tn * p.tiles_m;
     const int32_t m0 = tm * kSmallTile, n0 = tn * kSmallTile;
@@ -74,14 +81,14 @@ hgemm_small_kernel(const SmallParams p)
     grid_launch_dependents();          // the next kernel in the stream may start its own set-up
     grid_dependency_wait();            // ... and this one reads nothing before the kernels ahead of it are complete
 
-    // One stage: 64 rows x eight 16-byte pieces of A and of B, four pieces of each per thread.
+    // One stage: T rows x eight 16-byte pieces of A and of B, T / 16 pieces of each per thread.
     auto load_stage = [&](int32_t kb, int32_t s) {
         const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * 2u * kTileBytes;
         const uint32_t b_dst = a_dst + kTileBytes;
         const int32_t k0 = kb * kSmallBk;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t piece = tid + static_cast<uint32_t>(i) * kSmallThreads;       // 0 .. 511
+        for (int i = 0; i < T / 16; ++i) {
+            const uint32_t piece = tid + static_cast<uint32_t>(i) * kSmallThreads;       // 0 .. 8 T - 1
             const uint32_t r = piece >> 3, c = piece & 7u;
             const int32_t k = k0 + static_cast<int32_t>(c) * 8;
             const uint32_t off = r * 128u + ((c ^ (r & 7u)) << 4);
@@ -95,11 +102,11 @@ hgemm_small_kernel(const SmallParams p)
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
-    float acc[2][4][4];
+    float acc[MI][NI][4];
 #pragma unroll
-    for (int i = 0; i < 2; ++i)
+    for (int i = 0; i < MI; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < NI; ++j)
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.0f;
 
@@ -118,41 +125,41 @@ hgemm_small_kernel(const SmallParams p)
         const uint32_t b_tile = a_tile + kTileBytes;
 #pragma unroll
         for (uint32_t kk = 0; kk < kSmallBk / 16; ++kk) {
-            // A fragments: rows 16 i .. 16 i + 15 of this warp's 32; matrices in the order (rows 0-7, k 0-7),
+            // A fragments: rows 16 i .. 16 i + 15 of this warp's T / 2; matrices in the order (rows 0-7, k 0-7),
             // (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15) = registers a0..a3 of the MMA
-            uint32_t a[2][4];
+            uint32_t a[MI][4];
 #pragma unroll
-            for (uint32_t i = 0; i < 2; ++i) {
-                const uint32_t row = wm * 32u + i * 16u + (lane & 7u) + ((lane >> 3) & 1u) * 8u;
+            for (uint32_t i = 0; i < MI; ++i) {
+                const uint32_t row = wm * (T / 2) + i * 16u + (lane & 7u) + ((lane >> 3) & 1u) * 8u;
                 const uint32_t piece = kk * 2u + (lane >> 4);
                 ldmatrix_x4(a_tile + row * 128u + ((piece ^ (row & 7u)) << 4), a[i][0], a[i][1], a[i][2], a[i][3]);
             }
             // B fragments: two 8-column tiles per ldmatrix; matrices (n 0-7, k 0-7), (n 0-7, k 8-15), (n 8-15, k 0-7),
             // (n 8-15, k 8-15) = b0, b1 of the first tile, b0, b1 of the second
-            uint32_t b[4][2];
+            uint32_t b[NI][2];
 #pragma unroll
-            for (uint32_t j = 0; j < 2; ++j) {
-                const uint32_t row = wn * 32u + j * 16u + (lane & 7u) + (lane >> 4) * 8u;
+            for (uint32_t j = 0; j < NI / 2; ++j) {
+                const uint32_t row = wn * (T / 2) + j * 16u + (lane & 7u) + (lane >> 4) * 8u;
                 const uint32_t piece = kk * 2u + ((lane >> 3) & 1u);
                 ldmatrix_x4(b_tile + row * 128u + ((piece ^ (row & 7u)) << 4), b[2 * j][0], b[2 * j][1], b[2 * j + 1][0], b[2 * j + 1][1]);
             }
 #pragma unroll
-            for (int i = 0; i < 2; ++i)
+            for (int i = 0; i < MI; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) mma_m16n8k16(acc[i][j], a[i], b[j][0], b[j][1]);
+                for (int j = 0; j < NI; ++j) mma_m16n8k16(acc[i][j], a[i], b[j][0], b[j][1]);
         }
     }
 
     // epilogue: accumulator element pairs (row l / 4 [+ 8], columns 2 (l % 4), + 1) -> half2 -> 4-byte stores
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < MI; ++i) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int32_t row = m0 + static_cast<int32_t>(wm * 32u + i * 16u + h * 8u + (lane >> 2));
+            const int32_t row = m0 + static_cast<int32_t>(wm * (T / 2) + i * 16u + h * 8u + (lane >> 2));
             if (row >= p.M) continue;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int32_t col = n0 + static_cast<int32_t>(wn * 32u + j * 8u + (lane & 3u) * 2u);
+            for (int j = 0; j < NI; ++j) {
+                const int32_t col = n0 + static_cast<int32_t>(wn * (T / 2) + j * 8u + (lane & 3u) * 2u);
                 if (col >= p.N) continue;                                 // N is even: the pair is inside or outside
                 float x = acc[i][j][2 * h], y = acc[i][j][2 * h + 1];
                 __half2 *dst = reinterpret_cast<__half2 *>(p.C + static_cast<size_t>(row) * p.N + col);

@@ -49,7 +49,7 @@ def main() -> None:
             v = getattr(args, name)
             if v is not None:
                 setattr(cfg, attr, v)
-        cfg.block_m = 256 if cfg.family == hgemm.FAMILY_UMMA_2CTA else 64 if cfg.family == hgemm.FAMILY_SMALL else 128
+        cfg.block_m = 256 if cfg.family == hgemm.FAMILY_UMMA_2CTA else cfg.block_n if cfg.family == hgemm.FAMILY_SMALL else 128
         plan.set_config(cfg)
         for _ in range(args.warmup):
             plan.run(A, B, C)

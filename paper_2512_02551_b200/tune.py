@@ -42,9 +42,10 @@ def max_stages(family: int, bn: int, bk: int, epilogue: int = hgemm.EPILOGUE_TMA
 
 def candidates(M: int, N: int, K: int):
     out = []
-    small = hgemm.Config.small()                                  # the register-accumulator kernel's one configuration
-    if hgemm.validate_config(M, N, K, small) == hgemm.OK and M * N * K <= (1 << 31):
-        out.append(small)
+    for tile in (64, 32):                                         # the register-accumulator kernel's two configurations
+        small = hgemm.Config.small(tile)
+        if hgemm.validate_config(M, N, K, small) == hgemm.OK and M * N * K <= (1 << 31):
+            out.append(small)
     for swap in (0, 1):
         if swap and not (M <= 256 and N >= 512 and N % 8 == 0):
             continue

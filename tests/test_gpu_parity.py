@@ -454,17 +454,18 @@ SMALL_CASES = [
 ]
 
 
+@pytest.mark.parametrize("tile", [64, 32])
 @pytest.mark.parametrize("shape", SMALL_CASES, ids=lambda c: "x".join(map(str, c)))
-def test_small_family(ctx, gu, shape):
+def test_small_family(ctx, gu, shape, tile):
     """mma.sync with register accumulators: the same arithmetic as the tcgen05 kernels (exact on integers, the contract
     on random inputs), tails in every dimension, K shorter and much longer than the cp.async ring."""
     import oracle
     M, N, K = shape
-    cfg = hgemm.Config.small()
+    cfg = hgemm.Config.small(tile)
     assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
     A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
     C, _, plan = gu.run_gemm(ctx, A, B, cfg)
-    assert plan.config.family == hgemm.FAMILY_SMALL
+    assert plan.config.family == hgemm.FAMILY_SMALL and plan.config.block_n == tile
     gu.assert_close_full(C, A, B, f"small {shape}")
     Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
     Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)

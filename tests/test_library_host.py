@@ -159,7 +159,9 @@ def test_candidate_configs_are_legal_ranked_and_distinct(lib):
     # all three families, both stage widths, split-K and the wide epilogue all occur among the candidates of a shape that admits them
     pool = hgemm.candidate_configs(512, 512, 4096, max_count=256)
     assert {c.family for c in pool} == {0, 1, 2, 3} and {c.block_k for c in pool} == {64, 128}
-    assert sum(c.family == hgemm.FAMILY_SMALL for c in pool) == 1                             # one fixed configuration
+    assert 1 <= sum(c.family == hgemm.FAMILY_SMALL for c in pool) <= 2                        # its two fixed configurations (64 and 32 tiles)
+    tiny = hgemm.candidate_configs(128, 128, 128, max_count=256)
+    assert {c.block_n for c in tiny if c.family == hgemm.FAMILY_SMALL} == {32, 64}
     assert all(c.split_k == 1 and c.epilogue != hgemm.EPILOGUE_TMA_WIDE for c in pool if c.family == hgemm.FAMILY_LIGHT)
     big = hgemm.candidate_configs(8192, 8192, 8192, max_count=256)
     assert any(c.block_n == 512 and c.family == hgemm.FAMILY_UMMA_2CTA for c in big)          # the double-accumulator tile
