@@ -63,7 +63,7 @@ hgemm_config_t config_of(const Entry &e)
     hgemm_config_t c;
     std::memset(&c, 0, sizeof(c));
     c.family = e.family;
-    c.block_m = e.family == HGEMM_FAMILY_UMMA_2CTA ? 256 : 128;
+    c.block_m = e.family == HGEMM_FAMILY_UMMA_2CTA ? 256 : e.family == HGEMM_FAMILY_SMALL ? e.block_n : 128;
     c.block_n = e.block_n;
     c.block_k = e.block_k;
     c.stages = e.stages;

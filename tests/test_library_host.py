@@ -190,3 +190,24 @@ def test_table_file_overrides_the_built_in_table(lib, tmp_path):
     out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, check=True).stdout.split()
     assert out[:8] == ["0", "96", "5", "7", "1", "1", "128", "128"]
     assert out[8] != "48"
+
+
+def test_every_table_row_is_what_the_planner_returns(lib):
+    """A row of the tuned table that failed validation would silently be replaced by its neighbours' configurations:
+    every row of the compiled-in table must come back from the planner field by field."""
+    path = os.path.join(ROOT, "paper_2512_02551_b200", "csrc", "hgemm_table.inc")
+    rows = 0
+    families = set()
+    for line in open(path):
+        if not line.startswith("{"):
+            continue
+        v = [x.strip().rstrip("f") for x in line.strip().rstrip(",").strip("{}").split(",")]
+        M, N, K, family, bn, bk, stages, split, mode, tail, rg, epi, tail_mode = (int(x) for x in v[:13])
+        swap, raster_mode = (int(v[14]), int(v[15])) if len(v) >= 16 else (0, 0)
+        c = hgemm.planned_config(M, N, K)
+        got = (c.family, c.block_n, c.block_k, c.stages, c.split_k, c.split_mode, c.tail_split, c.raster_group, c.epilogue, c.tail_mode,
+               c.swap_ab, c.raster_mode)
+        assert got == (family, bn, bk, stages, split, mode, tail, rg, epi, tail_mode, swap, raster_mode), (M, N, K, got, line)
+        rows += 1
+        families.add(family)
+    assert rows >= 1000 and families == {0, 1, 2, 3}
