@@ -1,5 +1,5 @@
-// The persistent, warp-specialised tcgen05 HGEMM kernel (all kernel families are
-// instances of this one template).
+// The persistent, warp-specialised tcgen05 HGEMM kernel (the 1-CTA and CTA-pair families are
+// instances of this one template; the light and the small family have files of their own).
 //
 // Structure per CTA (320 threads):
 //   warp 0      TMA producer: fills a ring of shared-memory stages with 64-wide
