@@ -232,8 +232,41 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
             sustained[key(c)] = batch_ms(run, n, stream)
         final = sorted(((sustained[key(c)], e, c) for _, e, c in final), key=lambda r: r[0])
     best_t, _, best = final[0]
+    cold_us = None
+    L2 = 126 << 20
+    foot = 2 * (M * K + N * K + M * N)
+    sets = min(-(-2 * L2 // foot), A_all.numel() // max(M * K, 1), B_all.numel() // max(N * K, 1), C_all.numel() // max(M * N, 1))
+    if 0.008 <= best_t <= 0.08 and sets >= 2 and sets * foot >= 2 * L2:
+        # Mid-size kernels whose operands fit in L2 run in two regimes: back to back on the same buffers (everything
+        # above was timed like that), or with operands that come from HBM -- a call between other work.  Among the
+        # finalists within 3 % of the best warm time, take the one with the best geometric mean of the warm time and the
+        # cold time (buffer sets rotating through more than twice the L2): deeper rings win there at no warm cost.
+        ptrs = [(A_all[r * M * K:].data_ptr(), B_all[r * N * K:].data_ptr(), C_all[r * M * N:].data_ptr()) for r in range(sets)]
+
+        def cold_ms(n):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(n):
+                pa, pb, pc = ptrs[i % sets]
+                plan.run_ptr(pa, pb, pc, s)
+            e1.record(stream)
+            e1.synchronize()
+            return e0.elapsed_time(e1) / n
+        scored = []
+        for t, e, c in final:
+            if t > 1.03 * best_t:
+                continue
+            plan.set_config(c)
+            cold_ms(sets)                                           # tensor maps of every set encoded
+            n = max(sets, min(200, int(0.6 / max(t, 1e-3))))
+            tc = statistics.median(cold_ms(n) for _ in range(3))
+            scored.append(((t * tc) ** 0.5, t, tc, e, c))
+        if scored:
+            scored.sort(key=lambda r: r[0])
+            _, best_t, tc, _, best = scored[0]
+            cold_us = tc * 1e3
     dev_us = None
-    if device_metric and best_t < 0.03:
+    if device_metric and best_t < 0.008:
         # Short kernels: back-to-back calls overlap one call's start with the previous call's end and are bounded by
         # the host's launch rate, so many configurations tie.  Among those that tie (within 3 % + 0.1 us of the best),
         # take the one whose kernel is shortest on the device when it runs alone -- what a single call after an idle
@@ -307,7 +340,7 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     default_t = next((t for t, _, c in results if key(c) == key(default)), None)
     plan.close()
     return {"M": M, "N": N, "K": K, "best": best.as_dict(), "us": best_t * 1e3, "default_us": None if default_t is None else default_t * 1e3,
-            "torch_us": t_torch * 1e3, "ok": ok, "tried": len(results), "dev_us": dev_us,
+            "torch_us": t_torch * 1e3, "ok": ok, "tried": len(results), "dev_us": dev_us, "cold_us": cold_us,
             "all": [list(key(c)) + [round(t * 1e3, 3)] for t, _, c in results]}   # every first-pass timing: key fields, us
 
 
@@ -359,7 +392,7 @@ def main():
     ap.add_argument("--resume", action="store_true")
     ap.add_argument("--explore", type=int, default=0, help="also time this many randomly drawn candidates per shape")
     ap.add_argument("--device-metric", action="store_true",
-                    help="for kernels under 30 us: among the configurations that tie back to back, pick the shortest on the device")
+                    help="for kernels under 8 us: among the configurations that tie back to back, pick the shortest on the device")
     ap.add_argument("--max-us", type=float, default=0.0, help="with --resume-from: only shapes whose recorded time is below this")
     ap.add_argument("--from-log", metavar="JSONL", help="take the shape list (and --max-us times) from an earlier tune.jsonl")
     ap.add_argument("--grid10", action="store_true", help="the 271 shapes of the ten-value grid that contain 16384")
@@ -386,9 +419,12 @@ def main():
     mx_mk = max(max(M * K, N * K) for M, N, K in shapes)
     mx_mn = max(M * N for M, N, K in shapes)
     stream = torch.cuda.current_stream()
-    A_all = inputs.draw(1, inputs.TAG_A, 1, mx_mk, "uniform", "cuda").view(-1)
-    B_all = inputs.draw(1, inputs.TAG_B, 1, mx_mk, "uniform", "cuda").view(-1)
-    C_all = torch.empty(mx_mn, dtype=torch.float16, device="cuda")
+    # pools: the largest operand of the run, plus room for the rotating buffer sets of the cold-regime timing (> 2x L2)
+    room = 132 << 20
+    cols = 4096
+    A_all = inputs.draw(1, inputs.TAG_A, -(-(mx_mk + room) // cols), cols, "uniform", "cuda").view(-1)
+    B_all = inputs.draw(1, inputs.TAG_B, -(-(mx_mk + room) // cols), cols, "uniform", "cuda").view(-1)
+    C_all = torch.empty(mx_mn + room, dtype=torch.float16, device="cuda")
     rng = random.Random(2512)
     rows = []
     import time

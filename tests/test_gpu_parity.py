@@ -549,6 +549,7 @@ def test_static_operand_promise_keeps_the_other_operand_ordered(ctx, gu):
         hgemm.Config.make(family=F2, block_n=256, stages=3, raster_group=1, epilogue=TMA, block_k=128),
         hgemm.Config.make(family=F1, block_n=128, stages=6, split_k=4, raster_group=1, epilogue=DIRECT, block_k=64, split_mode=CLUSTER),
         hgemm.Config.make(family=F2, block_n=256, stages=4, raster_group=1, epilogue=TMA, block_k=64, swap_ab=1),
+        hgemm.Config.make(family=F2, block_n=512, stages=4, raster_group=1, epilogue=TMA, block_k=64),          # the double tile
     ]
     for cfg in configs:
         for plan in (p1, p2):
