@@ -97,7 +97,8 @@ enum {
 
 enum {
     HGEMM_TAIL_K = 0,
-    HGEMM_TAIL_N = 1
+    HGEMM_TAIL_N = 1,
+    HGEMM_TAIL_STREAM = 2
 };
 
 enum {
@@ -138,7 +139,13 @@ typedef struct {
                              every SM works until the end; otherwise ignored */
     int32_t tail_mode;    /* how tail_split cuts those tiles: HGEMM_TAIL_K (0) as above; HGEMM_TAIL_N (1): into
                              tail_split (2 or 4) column pieces of block_n / tail_split columns (a multiple of 32),
-                             each an independent narrower tile -- no partial sums, no workspace */
+                             each an independent narrower tile -- no partial sums, no workspace;
+                             HGEMM_TAIL_STREAM (2): stream-K.  The tiles beyond the last full wave (all tiles when there are
+                             fewer tiles than SMs) are taken as one sequence of k-blocks in tile order and dealt out in equal
+                             contiguous shares to min(SMs, tiles_left * tail_split) CTAs, so a CTA works on the end of one
+                             tile and the start of the next; the pieces of a tile are summed in K order through the workspace
+                             (deterministic).  Unlike the two other modes it applies whenever such tiles exist and K has at
+                             least twice as many k-blocks as a share; needs block_n <= 256, no swap_ab, fp32 accumulators, not the wide epilogue */
     int32_t accumulate;   /* HGEMM_ACC_F32 (0): fp32 accumulators, the paper's main setting and this library's default;
                              HGEMM_ACC_F16 (1): fp16 accumulators in tensor memory (the paper's other valid setting for
                              fp16 inputs, section 1): every 16-wide K step rounds the running sums to fp16, so
@@ -341,6 +348,14 @@ hgemm_status_t hgemm_ctx_last_device_status(hgemm_ctx_t *ctx, uint32_t *code);
 /* Wait budget of the bounded waits, in SM clock cycles (default 2e9, about a
  * second).  Affects plans created afterwards and later hgemm_run calls. */
 hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles);
+
+/* Test hook for the stream-K tail (HGEMM_TAIL_STREAM): work item `h` (0 or 1) of CTA position `position` under
+ * configuration `cfg` on a device with `num_sms` SMs, as the kernel decodes it.  out[0..5] = tile index, first
+ * k-block, number of k-blocks (0: no such item), slice (the item's place among the pieces of its tile, in K
+ * order), slices (pieces of that tile), positions in use.  HGEMM_ERR_UNSUPPORTED when the configuration has no
+ * stream-K tail on this shape.  Host arithmetic only; no device is touched. */
+hgemm_status_t hgemm_debug_stream_item(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg, int32_t num_sms,
+                                       int32_t position, int32_t h, int32_t out[6]);
 
 /* hgemm_run launches with programmatic stream serialisation (on by default): the
  * kernel may become resident, and run the set-up that touches no global memory,

@@ -234,6 +234,13 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         p.fd_last_group = hgemm_dev::make_fast_div(uint32_t(last));
         p.fd_split = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.split_k)));
         p.fd_pieces = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.tail_pieces)));
+        // stream-K tail: positions, k-blocks of the tail, k-blocks of a tile
+        p.stream_units = int32_t(layout.stream_units);
+        p.stream_q = int32_t((layout.tiles - layout.first_split_tile) * p.kblocks);
+        p.grid_units = std::max(1, ctx->num_sms / cg);
+        p.fd_stream_units = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.stream_units)));
+        p.fd_stream_q = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.stream_q)));
+        p.fd_kblocks = hgemm_dev::make_fast_div(uint32_t(std::max(1, p.kblocks)));
     }
     p.tmem_cols = cfg.block_n == 512 ? 512 : pow2_at_least(2 * cfg.block_n);   // two accumulators either way
     if (cfg.family == HGEMM_FAMILY_LIGHT) p.tmem_cols = pow2_at_least(cfg.block_n);   // ... except in the light kernel: one
@@ -310,6 +317,15 @@ const void *dual_kernel_of(bool wide)
                 : reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, 0, PLAIN, false, SUBS, false, true>);
 }
 
+// The stream-K tail (HGEMM_TAIL_STREAM): 32-column store boxes or direct stores, no transposed stores, no instrumentation.
+template <bool PLAIN, int SUBS>
+const void *stream_kernel_of(int cg)
+{
+    using namespace hgemm_dev;
+    return cg == 1 ? reinterpret_cast<const void *>(hgemm_umma_kernel<1, false, 3, PLAIN, false, SUBS, false, false>)
+                   : reinterpret_cast<const void *>(hgemm_umma_kernel<2, false, 3, PLAIN, false, SUBS, false, false>);
+}
+
 // `subs`: 64-wide sub-tiles per stage (block_k / 64); the plain instantiations are compiled for each value.
 // `xpose`: the instantiations that store the tile transposed (swapped operands); they exist without instrumentation.
 // `dual`: the instantiations for block_n == 512.
@@ -318,6 +334,10 @@ const void *kernel_for(int cg, bool wide, int split, bool plain, bool trace, int
     if (dual) {
         if (!plain) return dual_kernel_of<false, 0>(wide);
         return subs == 2 ? dual_kernel_of<true, 2>(wide) : dual_kernel_of<true, 1>(wide);
+    }
+    if (split == 3) {
+        if (!plain) return stream_kernel_of<false, 0>(cg);
+        return subs == 2 ? stream_kernel_of<true, 2>(cg) : stream_kernel_of<true, 1>(cg);
     }
     if (xpose) {
         if (!plain) return kernel_of<false, false, 0, true>(cg, false, split);
@@ -440,6 +460,11 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+        for (int k = 0; k < 6 && e == cudaSuccess; ++k) {           // the stream-K instantiations
+            const void *fn_k = kernel_for(1 + (k & 1), false, 3, k >= 2, false, k >= 4 ? 2 : 1);
+            e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        }
         for (int k = 0; k < 6 && e == cudaSuccess; ++k) {           // the double-accumulator instantiations
             const void *fn_k = kernel_for(2, (k & 1) != 0, 0, k >= 2, false, k >= 4 ? 2 : 1, false, true);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
@@ -528,7 +553,7 @@ int64_t hgemm_config_smem_bytes(const hgemm_config_t *cfg)
 
 int64_t hgemm_config_workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg)
 {
-    return cfg ? hgemm_host::workspace_bytes(M, N, K, *cfg) + hgemm_host::counter_bytes(M, N, *cfg) : -1;
+    return cfg ? hgemm_host::workspace_bytes(M, N, K, *cfg) + hgemm_host::counter_bytes(M, N, *cfg, 148, K) : -1;
 }
 
 hgemm_status_t hgemm_plan(hgemm_ctx_t *ctx, int64_t M, int64_t N, int64_t K, hgemm_plan_t **out)
@@ -867,7 +892,8 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     const bool light = plan->cfg.family == HGEMM_FAMILY_LIGHT;
     if (trace && (kp.transposed || kp.block_n == 512)) return HGEMM_ERR_UNSUPPORTED;   // no instrumented kernels for these
     if (light && kp.debug_skip != 0) return HGEMM_ERR_UNSUPPORTED;                       // the light kernel has stamps, no skip mask
-    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
+    if (trace && kp.stream_units > 0) return HGEMM_ERR_UNSUPPORTED;                      // ... nor for the stream-K tail
+    const void *fn = kernel_for(cg, plan->cfg.epilogue == HGEMM_EPILOGUE_TMA_WIDE, kp.stream_units > 0 ? 3 : kp.split_k > 1 ? (kp.cluster_split ? 2 : 1) : 0, plain,
                                 trace, kp.block_k / 64, kp.transposed != 0, kp.block_n == 512);
     void *args[5] = {&me->tmap_a, &me->tmap_b, &me->tmap_c, &me->tmap_bt, &plan->params};
     if (light) {
@@ -1003,6 +1029,26 @@ hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles)
 {
     if (!ctx || cycles < 1) return HGEMM_ERR_INVALID_ARG;
     ctx->wait_budget = cycles;
+    return HGEMM_OK;
+}
+
+hgemm_status_t hgemm_debug_stream_item(int64_t M, int64_t N, int64_t K, const hgemm_config_t *cfg, int32_t num_sms,
+                                       int32_t position, int32_t h, int32_t out[6])
+{
+    if (!cfg || !out || position < 0 || (h != 0 && h != 1)) return HGEMM_ERR_INVALID_ARG;
+    if (hgemm_host::validate(M, N, K, *cfg) != HGEMM_OK) return HGEMM_ERR_UNSUPPORTED;
+    const hgemm_host::SplitLayout L = hgemm_host::split_layout(M, N, K, num_sms, *cfg);
+    if (L.stream_units <= 0) return HGEMM_ERR_UNSUPPORTED;
+    const int32_t kb = int32_t((K + cfg->block_k - 1) / cfg->block_k);
+    const int32_t q = int32_t((L.tiles - L.first_split_tile) * kb);
+    const hgemm_dev::StreamItem si = hgemm_dev::stream_item(position, h, int32_t(L.stream_units), q, kb, hgemm_dev::make_fast_div(uint32_t(L.stream_units)),
+                                                            hgemm_dev::make_fast_div(uint32_t(q)), hgemm_dev::make_fast_div(uint32_t(kb)));
+    out[0] = int32_t(L.first_split_tile) + si.tile_rel;
+    out[1] = si.kb_begin;
+    out[2] = si.kb_count;
+    out[3] = si.slice;
+    out[4] = si.slices;
+    out[5] = int32_t(L.stream_units);
     return HGEMM_OK;
 }
 

@@ -73,9 +73,56 @@ __host__ __device__ inline FastDiv make_fast_div(uint32_t d)
     return f;
 }
 
-__device__ __forceinline__ int32_t fast_div(int32_t x, const FastDiv &f)
+__host__ __device__ __forceinline__ int32_t fast_div(int32_t x, const FastDiv &f)
 {
+#ifdef __CUDA_ARCH__
     return f.d == 1u ? x : static_cast<int32_t>(__umulhi(static_cast<uint32_t>(x), f.mul) >> f.shr);
+#else
+    return static_cast<int32_t>(static_cast<uint32_t>(x) / f.d);      // the host's copy (layout computations, tests)
+#endif
+}
+
+// Stream-K tail (paper section 5.2 picks a tile shape per problem; a tile count that does not fill the last wave of
+// SMs is what this evens out): the `rem` tiles that remain after the full waves are `q = rem * kblocks` k-blocks in
+// tile-major order, dealt out as `gs` contiguous ranges [floor(j q / gs), floor((j + 1) q / gs)), one per CTA
+// position j.  rem <= gs, so a range is at most one tile long and crosses at most one tile boundary: position j has
+// up to two work items, h = 0 (the part in the tile where its range starts) and h = 1 (the part in the next tile).
+// The positions that share a tile are consecutive; the item's slice is its place among them, and the tile's
+// partial sums are added in that order.
+struct StreamItem {
+    int32_t tile_rel;    // tile, counted from the first tile of the tail
+    int32_t kb_begin, kb_count;
+    int32_t slice, slices;
+};
+
+__host__ __device__ __forceinline__ StreamItem stream_item(int32_t j, int32_t h, int32_t gs, int32_t q, int32_t kblocks,
+                                                           const FastDiv &fd_gs, const FastDiv &fd_q, const FastDiv &fd_kblocks)
+{
+    StreamItem s;
+    s.tile_rel = 0; s.kb_begin = 0; s.kb_count = 0; s.slice = 0; s.slices = 1;
+    if (j >= gs) return s;                                            // a position without a share of the tail
+    const int32_t b0 = fast_div(j * q, fd_gs), b1 = fast_div((j + 1) * q, fd_gs);
+    const int32_t t0 = fast_div(b0, fd_kblocks);
+    const int32_t edge = (t0 + 1) * kblocks;                          // first k-block of the next tile
+    if (h == 0) {
+        s.tile_rel = t0;
+        s.kb_begin = b0 - t0 * kblocks;
+        s.kb_count = (b1 < edge ? b1 : edge) - b0;
+    } else {
+        s.tile_rel = t0 + 1;
+        s.kb_count = b1 - edge;
+    }
+    if (s.kb_count <= 0) {
+        s.tile_rel = 0;
+        s.kb_count = 0;
+        return s;
+    }
+    // positions whose ranges meet this tile: the largest j' with floor(j' q / gs) <= x is floor(((x + 1) gs - 1) / q)
+    const int32_t x = s.tile_rel * kblocks;
+    const int32_t j_lo = fast_div((x + 1) * gs - 1, fd_q), j_hi = fast_div((x + kblocks) * gs - 1, fd_q);
+    s.slice = j - j_lo;
+    s.slices = j_hi - j_lo + 1;
+    return s;
 }
 
 struct KernelParams {
@@ -118,6 +165,13 @@ struct KernelParams {
     int32_t raster_serpentine;    // 1: odd raster groups sweep the n-tiles from last to first
     uint32_t early_ops;           // bit 0 / bit 1: the kernel's A / B operand is static (no kernel ahead in the stream writes
                                   // it): its first loads may leave before the stream dependency is resolved
+    // stream-K tail (see stream_item): 0 positions = none.  Then split_k is the largest number of slices of a tile
+    // (the stride of a tile's workspace slots) and the work items from first_split_tile on are numbered
+    // first_split_tile + h * grid_units + j.
+    int32_t stream_units;         // positions that share the tail's k-blocks
+    int32_t stream_q;             // k-blocks of the tail: (tiles - first_split_tile) * kblocks
+    int32_t grid_units;           // CTAs (pairs) of the grid
+    FastDiv fd_stream_units, fd_stream_q, fd_kblocks;
 };
 
 template <bool OFF = false>
@@ -327,6 +381,7 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     // partly filled wave, whose tiles are cut along K (slices, summed afterwards) or into column
     // pieces (independent narrower tiles) so that every SM has work until the end.
     int32_t n_off = 0;
+    bool own_k_range = false;
     it.bn = p.block_n;
     if (w < p.first_split_tile) {
         it.tile = w;
@@ -347,6 +402,18 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
         it.slice = 0;
         it.slices = 1;
         it.split_index = 0;
+    } else if (p.stream_units > 0) {
+        const int32_t idx = w - p.first_split_tile;
+        const int32_t h = idx >= p.grid_units ? 1 : 0;
+        const StreamItem si = stream_item(idx - h * p.grid_units, h, p.stream_units, p.stream_q, p.kblocks, p.fd_stream_units,
+                                          p.fd_stream_q, p.fd_kblocks);
+        it.tile = p.first_split_tile + si.tile_rel;
+        it.slice = si.slice;
+        it.slices = si.slices;
+        it.split_index = si.tile_rel * p.split_k + si.slice;
+        it.kb_begin = si.kb_begin;
+        it.kb_count = si.kb_count;                       // 0: this position has no such item; every role skips it
+        own_k_range = true;
     } else {
         it.split_index = w - p.first_split_tile;
         const int32_t t = fast_div(it.split_index, p.fd_split);
@@ -366,7 +433,9 @@ __device__ __forceinline__ WorkItem decode_work(int32_t w, const KernelParams &p
     const int32_t tn_at = (p.raster_serpentine && (g & 1)) ? p.tiles_n - 1 - tn : tn;
     it.m0 = tm * block_m_total;
     it.n0 = tn_at * p.block_n + n_off;
-    if (!SPLIT || it.slices == 1) {
+    if (SPLIT && own_k_range) {
+        // (a stream-K item brought its own range)
+    } else if (!SPLIT || it.slices == 1) {
         it.kb_begin = 0;
         it.kb_count = p.kblocks;
     } else {
@@ -399,7 +468,8 @@ __device__ __forceinline__ WorkItem warp_uniform(const WorkItem &it)
 // the kernel
 
 // SPLIT: 0 for configurations without K slices (split_k == 1, no tail cut along K), 1 for slices summed through the
-// global workspace, 2 for slices summed inside a cluster; each instantiation carries only its own reduction, which
+// global workspace, 2 for slices summed inside a cluster, 3 for the stream-K tail (pieces of a tile parked in the
+// workspace and added by the CTA that finishes the tile); each instantiation carries only its own reduction, which
 // saves registers and shortens the start-up of every call.
 // PLAIN: the instantiation for the plain call -- C = A B^T with fp32 accumulators, K-contiguous B, rows of C that are
 // multiples of 16 bytes, whole-width tail tiles: all of those branches are compiled out.
@@ -689,6 +759,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             bool ok = true;
             for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
                 const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
+                if (SPLIT == 3 && it.kb_count <= 0) {      // a stream-K position without this item: it takes no accumulator
+                    --local_tile;                          // (the loop's increment puts it back)
+                    continue;
+                }
                 const uint32_t acc = DUAL ? 0u : (local_tile & 1u);            // DUAL: one work item fills both accumulators
                 const uint32_t acc_ph = DUAL ? (local_tile & 1u) : ((local_tile >> 1) & 1u);
                 if constexpr (DUAL) {
@@ -877,6 +951,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         grid_dependency_wait();                            // before the first store to C, workspace or counters
         for (int32_t w = unit; ok && w < p.total_work; w += num_units, ++local_tile) {
             const WorkItem it = decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal);
+            if (SPLIT == 3 && it.kb_count <= 0) {          // a stream-K position without this item (see the MMA issuer)
+                --local_tile;
+                continue;
+            }
             const uint32_t acc = DUAL ? 0u : (local_tile & 1u);
             const uint32_t acc_ph = DUAL ? (local_tile & 1u) : ((local_tile >> 1) & 1u);
             // first column, within the tile, of 32-column accumulator chunk c (DUAL: see the template comment)
@@ -1072,11 +1150,44 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (box_lo + static_cast<int32_t>(first_chunk) >= boxes) release_accumulator(rel);    // nothing to load
                 }
                 if (!ok) break;
-            } else if (SPLIT == 0 || it.slices == 1) {
+            } else if (SPLIT == 0 || it.slices == 1 || (SPLIT == 3 && it.slice == 0)) {
                 // one 32-column chunk at a time: a tensor-memory load takes ~100 cycles, and keeping a second
                 // chunk in flight costs more in registers than it hides
                 uint32_t v[32];
                 const int32_t all_chunks = live_rows ? live_chunks : 0;
+                // Stream-K: the piece that holds a tile's first k-block finishes the tile.  The tile's later pieces
+                // belong to the positions after this one, which computed them FIRST (a position works through its
+                // range in K order, so the end of the tile it starts in comes before the start of the next tile) and
+                // parked them in the workspace long ago: wait for their arrivals (8 per piece, one per epilogue warp;
+                // the counter is never reset, launch number e sees e times as many), then add them to this piece's
+                // accumulator chunk by chunk, in K order, on the way to the ordinary stores.
+                const bool add_pieces = SPLIT == 3 && it.slices > 1;
+                const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
+                // this CTA's half of the tile's second piece (slice 1)
+                const float *piece1 = p.workspace + (static_cast<size_t>(it.split_index + 1) * CTA_GROUP + cta_rank) * slot_floats;
+                if (add_pieces) {
+                    const uint32_t *ctr = p.counters + (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2;
+                    const uint32_t target = p.epoch * 8u * static_cast<uint32_t>(it.slices - 1);
+                    if (lane == 0) {
+                        const long long t0 = clock64();
+                        while (true) {
+                            uint32_t seen;
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(ctr) : "memory");
+                            if (static_cast<int32_t>(seen - target) >= 0) break;
+                            if (*abort_flag) { ok = false; break; }
+                            if (clock64() - t0 > p.wait_budget) {
+                                *abort_flag = 1u;
+                                atomicCAS(p.status, 0u, status_code(kRoleEpilogue, 3, it.slice));
+                                ok = false;
+                                break;
+                            }
+                            __nanosleep(40);
+                        }
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    __threadfence();
+                }
                 for (uint32_t hf = 0; ok && hf < kHalves; ++hf) {
                 const uint32_t rel = DUAL ? hf : acc;
                 if constexpr (DUAL) {
@@ -1096,6 +1207,22 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             v[j] = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(v[j] & 0xffffu))));
                     }
                     if (c + 2 >= chunks) release_accumulator(rel);    // every load of this warp (from this accumulator) has completed
+                    if (add_pieces) {
+                        // this thread's row of the chunk in every later piece (layout: see the parking below)
+                        const float4 *src = reinterpret_cast<const float4 *>(piece1) + static_cast<size_t>(c) * 8 * kBlockM + row_in_tile;
+                        for (int32_t sl = 1; sl < it.slices; ++sl, src += static_cast<size_t>(CTA_GROUP) * slot_floats / 4) {
+                            float4 x[8];
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) x[g] = __ldcg(src + g * kBlockM);
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) {
+                                v[4 * g + 0] = __float_as_uint(__uint_as_float(v[4 * g + 0]) + x[g].x);
+                                v[4 * g + 1] = __float_as_uint(__uint_as_float(v[4 * g + 1]) + x[g].y);
+                                v[4 * g + 2] = __float_as_uint(__uint_as_float(v[4 * g + 2]) + x[g].z);
+                                v[4 * g + 3] = __float_as_uint(__uint_as_float(v[4 * g + 3]) + x[g].w);
+                            }
+                        }
+                    }
                     if ((!PLAIN && p.scaled) && grow < p.M) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
@@ -1106,6 +1233,34 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (chunk_lo + static_cast<int32_t>(first_chunk) >= chunks) release_accumulator(rel);   // nothing to load
                 }
                 if (!ok) break;
+            } else if (SPLIT == 3) {
+                // ---- stream-K: a piece that does not hold its tile's first k-block is parked for the one that does ----
+                // The slot holds this CTA's 128 rows of the piece as float4 units: columns 4 g .. 4 g + 3 of chunk c, row r,
+                // at unit (c * 8 + g) * 128 + r -- rows innermost, so the 32 lanes of a warp (32 consecutive rows, the
+                // tensor-memory load's layout) write 512 consecutive bytes per instruction, and the finishing thread,
+                // which holds the same rows, reads them back the same way.  (Row-major units -- 32 lanes 128 bytes
+                // apart -- measured 15 us for the reads of a 128 x 256 piece.)  Only the part that holds elements of C
+                // is written.
+                const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
+                float *slot = p.workspace + (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank) * slot_floats;
+                const int32_t park_chunks = live_rows ? live_chunks : 0;
+                for (int32_t c = static_cast<int32_t>(first_chunk); c < park_chunks; c += 2) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
+                    tmem_ld_wait();
+                    float4 *dst = reinterpret_cast<float4 *>(slot) + static_cast<size_t>(c) * 8 * kBlockM + row_in_tile;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        __stcg(dst + g * kBlockM, make_float4(__uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]), __uint_as_float(v[4 * g + 2]),
+                                                    __uint_as_float(v[4 * g + 3])));
+                }
+                release_accumulator(acc);
+                // announce this warp's part: its stores, made visible to the GPU, then one arrival
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(p.counters + (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2, 1u);
+                }
             } else if (SPLIT == 2) {
                 // split-K inside a cluster: the accumulator is complete; the exchange below needs every
                 // thread of the CTA, so it happens after the role branches

@@ -72,9 +72,31 @@ SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const
     L.first_split_tile = L.tiles;
     L.slices = 1;
     L.pieces = 1;
+    L.stream_units = 0;
     if (c.split_k > 1) {
         L.first_split_tile = 0;
         L.slices = c.split_k;
+    } else if (c.tail_split >= 2 && c.tail_mode == HGEMM_TAIL_STREAM) {
+        const int64_t units = std::max(1, num_sms / cg);
+        const int64_t rem = L.tiles % units;                     // the tiles beyond the full waves
+        const int64_t kb = ceil_div(K, c.block_k);
+        const int64_t gs = std::min(units, rem * c.tail_split);  // positions that share them
+        // worth it only if a share is at least two k-blocks and no tile is cut into more pieces than may wait for each other
+        if (rem > 0 && gs > rem && rem * kb >= 2 * gs && rem * kb * gs < (int64_t(1) << 30)) {
+            const int64_t q = rem * kb;
+            int64_t most = 1;
+            for (int64_t t = 0; t < rem; ++t) {
+                const int64_t j_lo = ((t * kb + 1) * gs - 1) / q, j_hi = ((t * kb + kb) * gs - 1) / q;
+                most = std::max(most, j_hi - j_lo + 1);
+            }
+            if (most >= 2 && most <= kMaxSplitK && rem * most * cg * 128 * int64_t(c.block_n) * 4 <= kMaxWorkspaceBytes) {
+                L.first_split_tile = L.tiles - rem;
+                L.slices = most;
+                L.stream_units = gs;
+                L.work_items = L.first_split_tile + 2 * units;
+                return L;
+            }
+        }
     } else if (c.tail_split >= 2) {
         const int64_t units = std::max(1, num_sms / cg);
         const int64_t tail = L.tiles % units;
@@ -181,9 +203,12 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
         if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
     if (c.accumulate != HGEMM_ACC_F32 && c.accumulate != HGEMM_ACC_F16) return HGEMM_ERR_UNSUPPORTED;
     // fp16 accumulators: no fp16 partial sums are exchanged, so no split along K
-    if (c.accumulate == HGEMM_ACC_F16 && (c.split_k != 1 || (c.tail_split >= 2 && c.tail_mode == HGEMM_TAIL_K))) return HGEMM_ERR_UNSUPPORTED;
+    if (c.accumulate == HGEMM_ACC_F16 && (c.split_k != 1 || (c.tail_split >= 2 && c.tail_mode != HGEMM_TAIL_N))) return HGEMM_ERR_UNSUPPORTED;
     if (c.tail_split < 0 || c.tail_split > 16 || (c.tail_split >= 2 && c.split_k != 1)) return HGEMM_ERR_UNSUPPORTED;
-    if (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N) return HGEMM_ERR_UNSUPPORTED;
+    if (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N && c.tail_mode != HGEMM_TAIL_STREAM) return HGEMM_ERR_UNSUPPORTED;
+    // stream-K: partial sums in fp32 through the workspace; the transposed stores and the light kernel have no such path
+    if (c.tail_mode == HGEMM_TAIL_STREAM && (c.swap_ab || c.family == HGEMM_FAMILY_LIGHT || c.block_n > 256 || c.epilogue == HGEMM_EPILOGUE_TMA_WIDE))
+        return HGEMM_ERR_UNSUPPORTED;
     if (c.tail_mode == HGEMM_TAIL_N && c.tail_split >= 2) {
         // column pieces: whole 32-column chunks, and for a pair a whole number of 8-row groups of B per CTA
         if ((c.tail_split != 2 && c.tail_split != 4) || (c.block_n % (32 * c.tail_split)) != 0) return HGEMM_ERR_UNSUPPORTED;
@@ -242,6 +267,7 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
     // 1 / pieces (narrower tiles run below the wide ones' rate)
     double wave_count;
     if (c.split_k > 1) wave_count = double(ceil_div(work, units));
+    else if (L.stream_units > 0) wave_count = double(L.first_split_tile) / double(units) + double(L.tiles - L.first_split_tile) / double(L.stream_units);
     else if (L.slices > 1) wave_count = double(L.first_split_tile) / double(units) + 1.0 / double(L.slices);
     else if (L.pieces > 1) wave_count = double(L.first_split_tile) / double(units) + 1.52 / double(L.pieces);
     else wave_count = double(ceil_div(L.tiles, units));
@@ -260,7 +286,7 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
                             (c.epilogue == HGEMM_EPILOGUE_DIRECT ? kDirectStores : c.epilogue == HGEMM_EPILOGUE_TMA_WIDE ? kWideStores : 1.0);
     double t = wave_count * (double(kb_per) * t_kb + 0.25 * kFillLatency) + 0.75 * kFillLatency + epilogue + (cg - 1) * kPairExtra;
     const double partial = 128.0 * c.block_n * 4.0;
-    if (c.split_k == 1 && L.slices > 1) t += partial / 26.4 + 10069.4;   // the tail's reduction
+    if (c.split_k == 1 && L.slices > 1) t += (partial / 26.4 + 10069.4) * (L.stream_units > 0 ? 1.5 : 1.0);   // the tail's reduction (stream-K: two items)
     double bytes = 2.0 * (double(M) * K + double(N) * K + double(M) * N);
     if (c.split_k > 1) {
         if (c.split_mode == HGEMM_SPLIT_CLUSTER) {

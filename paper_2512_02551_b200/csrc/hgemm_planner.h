@@ -29,6 +29,10 @@ int32_t max_stages_of(const hgemm_config_t &c);                         // with 
 struct SplitLayout {
     int64_t tiles, first_split_tile, slices, work_items;
     int64_t pieces;   // > 1: the tiles from first_split_tile on are cut into this many column pieces (slices == 1)
+    // stream-K tail (HGEMM_TAIL_STREAM): stream_units > 0 CTA positions share the k-blocks of the tiles from
+    // first_split_tile on; `slices` is then the largest number of pieces any of those tiles is cut into, and
+    // work_items = first_split_tile + 2 * grid units (two items per position, possibly empty).
+    int64_t stream_units;
 };
 SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const hgemm_config_t &c);
 int64_t workspace_bytes(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c, int32_t num_sms = 148);

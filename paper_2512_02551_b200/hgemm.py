@@ -17,7 +17,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT
 FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA, FAMILY_LIGHT, FAMILY_SMALL = 0, 1, 2, 3
 EPILOGUE_DIRECT, EPILOGUE_TMA, EPILOGUE_TMA_WIDE = 0, 1, 2
 SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
-TAIL_K, TAIL_N = 0, 1
+TAIL_K, TAIL_N, TAIL_STREAM = 0, 1, 2
 ACC_F32, ACC_F16 = 0, 1
 LAYOUT_TN, LAYOUT_NN = 0, 1
 RASTER_SWEEP, RASTER_SERPENTINE = 0, 1
@@ -28,7 +28,7 @@ EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_plan_set_static_operands", "hgemm_plan_autotune", "hgemm_candidate_configs", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
-    "hgemm_last_device_status", "hgemm_ctx_last_device_status", "hgemm_debug_fail_allocs", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
+    "hgemm_last_device_status", "hgemm_ctx_last_device_status", "hgemm_debug_fail_allocs", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_stream_item", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
 ]
 
@@ -120,6 +120,7 @@ def lib() -> ctypes.CDLL:
             "hgemm_set_wait_budget": (i32, [p, i64]),
             "hgemm_set_dependent_launch": (i32, [p, i32]),
             "hgemm_debug_timeout_probe": (i32, [p, p]),
+            "hgemm_debug_stream_item": (i32, [i64, i64, i64, cfgp, i32, i32, i32, ctypes.POINTER(ctypes.c_int32)]),
             "hgemm_debug_set_trace": (i32, [p, p]),
             "hgemm_debug_set_skip": (i32, [p, ctypes.c_uint32]),
             "hgemm_last_cuda_error": (i32, [p]),
@@ -168,6 +169,17 @@ def candidate_configs(M: int, N: int, K: int, max_count: int = 64, num_sms: int 
 
 def validate_config(M: int, N: int, K: int, cfg: Config) -> int:
     return int(lib().hgemm_validate_config(M, N, K, ctypes.byref(cfg)))
+
+
+def stream_item(M: int, N: int, K: int, cfg: "Config", position: int, h: int, num_sms: int = 148):
+    """Work item `h` of CTA position `position` of a stream-K tail, as the kernel decodes it:
+    (tile, kb_begin, kb_count, slice, slices, positions), or None when the configuration has no such tail here."""
+    out = (ctypes.c_int32 * 6)()
+    st = lib().hgemm_debug_stream_item(M, N, K, ctypes.byref(cfg), num_sms, position, h, out)
+    if st == ERR_UNSUPPORTED:
+        return None
+    _check(st, "hgemm_debug_stream_item")
+    return tuple(out)
 
 
 def estimate_config(M: int, N: int, K: int, cfg: Config, num_sms: int = 148) -> float:
@@ -340,3 +352,9 @@ class Plan:
         if self._h and self.ctx._h:
             lib().hgemm_plan_destroy(self._h)
         self._h = ctypes.c_void_p()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()

@@ -99,6 +99,19 @@ def _candidates(M: int, N: int, K: int, swap: int):
                                 out.append(c)
                             if swap or light:
                                 continue                      # no tail cuts in the swapped orientation or the light kernel
+                            if split == 1 and epi != hgemm.EPILOGUE_TMA_WIDE and tiles % units:
+                                # stream-K: the tiles beyond the full waves (all of them when there are fewer tiles than SMs)
+                                # as one sequence of k-blocks in equal shares, each tile cut into about `pieces` pieces
+                                seen_units = set()
+                                for pieces in (2, 4, 8):
+                                    c4 = hgemm.Config.make(family=family, block_n=bn, stages=st, split_k=1, raster_group=rg, epilogue=epi,
+                                                           block_k=bk, tail_split=pieces, tail_mode=hgemm.TAIL_STREAM)
+                                    if hgemm.validate_config(M, N, K, c4) != hgemm.OK:
+                                        continue
+                                    item = hgemm.stream_item(M, N, K, c4, 0, 0, NUM_SMS)
+                                    if item is not None and item[5] not in seen_units:      # (more pieces, same number of positions: the same schedule)
+                                        seen_units.add(item[5])
+                                        out.append(c4)
                             tail = tiles % units
                             if split == 1 and tiles > units and 0 < tail <= units // 2:
                                 ts = min(units // tail, 8, -(-K // bk))
@@ -168,7 +181,7 @@ def device_times(plan, configs, run, reps: int = 5) -> dict:
 
 
 def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, stream, explore: int = 0,
-               device_metric: bool = False) -> dict:
+               device_metric: bool = False, only_specials: bool = False) -> dict:
     A = A_all.view(-1)[:M * K].view(M, K)
     B = B_all.view(-1)[:N * K].view(N, K)
     C = C_all[:M * N].view(M, N)
@@ -182,7 +195,16 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
     wide += [c for c in cands if c.block_n == 512 and c.epilogue != hgemm.EPILOGUE_TMA_WIDE][:4]
     wide += [c for c in cands if c.family == hgemm.FAMILY_LIGHT][:8]
     wide += [c for c in cands if c.family == hgemm.FAMILY_SMALL]
-    cands = [c for c in cands if c.epilogue != hgemm.EPILOGUE_TMA_WIDE and c.block_n != 512 and c.family not in (hgemm.FAMILY_LIGHT, hgemm.FAMILY_SMALL)]
+    is_stream = lambda c: c.tail_mode == hgemm.TAIL_STREAM and c.tail_split >= 2   # noqa: E731
+    wide += [c for c in cands if is_stream(c)][:12]
+    cands = [c for c in cands if c.epilogue != hgemm.EPILOGUE_TMA_WIDE and c.block_n != 512 and c.family not in (hgemm.FAMILY_LIGHT, hgemm.FAMILY_SMALL)
+             and not is_stream(c)]
+    if only_specials:                          # a challenge run: the plan's current configuration against the separately ranked groups
+        if not any(is_stream(c) for c in wide):
+            plan.close()
+            return None
+        wide = [c for c in wide if is_stream(c)]
+        cands = []
     chosen, seen = [], set()
     extra = rng.sample(cands[top:], min(explore, max(0, len(cands) - top))) if explore > 0 else []   # for refitting the cost model
     for c in [default] + cands[:top] + wide + extra:
@@ -395,6 +417,9 @@ def main():
                     help="for kernels under 8 us: among the configurations that tie back to back, pick the shortest on the device")
     ap.add_argument("--max-us", type=float, default=0.0, help="with --resume-from: only shapes whose recorded time is below this")
     ap.add_argument("--from-log", metavar="JSONL", help="take the shape list (and --max-us times) from an earlier tune.jsonl")
+    ap.add_argument("--challenge-stream", action="store_true",
+                    help="time only the plan's current configuration against the stream-K candidates (shapes without any are skipped)")
+    ap.add_argument("--min-us", type=float, default=0.0, help="with --from-log: only shapes whose recorded time is at least this")
     ap.add_argument("--grid10", action="store_true", help="the 271 shapes of the ten-value grid that contain 16384")
     ap.add_argument("--time-limit", type=float, default=0.0, help="stop starting new shapes after this many seconds (resume later)")
     ap.add_argument("--merge-into", metavar="TABLE", help="replace these shapes' rows in an existing table file, keep its other rows")
@@ -409,7 +434,7 @@ def main():
         shapes = [(M, N, K) for M in GRID for N in GRID for K in GRID]
     if args.from_log:
         earlier = [json.loads(line) for line in open(args.from_log)]
-        shapes = [(r["M"], r["N"], r["K"]) for r in earlier if args.max_us <= 0 or r["us"] < args.max_us]
+        shapes = [(r["M"], r["N"], r["K"]) for r in earlier if (args.max_us <= 0 or r["us"] < args.max_us) and r["us"] >= args.min_us]
     log_path = os.path.join(args.out, "tune.jsonl")
     done = {}
     if args.resume and os.path.exists(log_path):
@@ -435,7 +460,9 @@ def main():
             if r is None:
                 if args.time_limit > 0 and time.time() - started > args.time_limit:
                     continue                                   # out of time: left for a later --resume run
-                r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream, args.explore, args.device_metric)
+                r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream, args.explore, args.device_metric, args.challenge_stream)
+                if r is None:                                  # a challenge run on a shape without challengers
+                    continue
                 log.write(json.dumps(r) + "\n")
                 log.flush()
             rows.append(r)

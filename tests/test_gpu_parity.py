@@ -589,6 +589,104 @@ def test_tail_split(ctx, gu, family, bn, bk, stages, tail, M, N, K):
     plan.close()
 
 
+# ---- stream-K tail: the tiles beyond the full waves as one sequence of k-blocks, dealt out in equal shares ------
+
+STREAM_CASES = [
+    # family, block_n, block_k, stages, tail_split, epilogue, M, N, K
+    (F1, 256, 64, 4, 2, TMA, 12288, 256, 2048),        # 96 tiles on 148 SMs: no full wave, every tile in two or three pieces
+    (F2, 256, 64, 6, 2, TMA, 12288, 256, 2048),        # the same as 48 pair tiles on 74 pairs
+    (F1, 128, 128, 3, 4, DIRECT, 128, 12288, 4096),    # 96 tiles of a skinny problem, 128-wide stages
+    (F1, 128, 64, 6, 16, TMA, 512, 512, 4096),         # 16 tiles cut into up to 16 pieces each
+    (F2, 128, 64, 8, 3, TMA, 4096, 4096, 512),         # full waves first, then a stream-K tail of 68 tiles
+    (F1, 256, 64, 4, 2, DIRECT, 4096, 4096, 512),      # ... with direct stores
+    (F1, 96, 64, 6, 5, DIRECT, 2000, 4104, 520),       # ragged M, N and K
+    (F2, 192, 128, 3, 2, TMA, 2100, 3000, 300),        # ragged, K not a multiple of the stage width, pairs
+    (F1, 64, 64, 8, 2, TMA, 100, 1000, 1000),          # fewer positions than SMs
+]
+
+
+@pytest.mark.parametrize("case", STREAM_CASES, ids=lambda c: f"f{c[0]}bn{c[1]}bk{c[2]}t{c[4]}e{c[5]}-{c[6]}x{c[7]}x{c[8]}")
+def test_stream_k_tail(ctx, gu, case):
+    """HGEMM_TAIL_STREAM against the oracle: uniform inputs at the contract tolerance, small integers exactly, the same
+    bits run after run with other work in flight, and the same bits as the configuration without the tail cut
+    wherever a tile was left whole."""
+    import oracle
+    family, bn, bk, stages, tail, epi, M, N, K = case
+    cfg = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=epi, block_k=bk, tail_split=tail,
+                            tail_mode=hgemm.TAIL_STREAM)
+    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+    first = hgemm.stream_item(M, N, K, cfg, 0, 0, torch.cuda.get_device_properties(0).multi_processor_count)
+    assert first is not None and first[4] >= 2, "the case is meant to cut tiles"
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    gu.assert_close_full(C, A, B, f"stream-K {cfg.as_dict()}") if M * N * K <= gu.FULL_CHECK_VOLUME else \
+        gu.assert_close_sampled(C, A, B, "uniform", inputs.shape_seed(M, N, K), f"stream-K {cfg.as_dict()}")
+    bits0 = C.view(torch.int16).clone()
+    noise = torch.empty(1 << 24, device="cuda")
+    side = torch.cuda.Stream()
+    for it in range(4):                                  # the cut tiles reproduce their bits
+        C2 = torch.empty_like(C)
+        with torch.cuda.stream(side):
+            for _ in range(it % 3 + 1):
+                noise.normal_()
+        plan.run(A, B, C2)
+        torch.cuda.synchronize()
+        assert torch.equal(C2.view(torch.int16), bits0), f"run {it} differs"
+    st, code = plan.last_device_status()
+    assert st == hgemm.OK, hex(code)
+    # whole tiles (the full waves) are computed exactly as without the tail cut
+    plain = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=4, epilogue=epi, block_k=bk)
+    C_plain, _, _ = gu.run_gemm(ctx, A, B, plain, plan=plan)
+    cg = 2 if family == F2 else 1
+    tiles_m, tiles_n = -(-M // (128 * cg)), -(-N // bn)
+    whole = first[0]                                     # index of the first cut tile = number of whole tiles
+    if whole > 0:
+        # tiles are numbered along the raster: compare the rows of the first raster group that is entirely whole
+        group_tiles = min(4, tiles_m) * tiles_n
+        whole_groups = whole // group_tiles
+        rows = min(M, whole_groups * min(4, tiles_m) * 128 * cg)
+        if rows > 0:
+            assert torch.equal(C[:rows].view(torch.int16), C_plain[:rows].view(torch.int16))
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    if M * N * K <= gu.FULL_CHECK_VOLUME:
+        plan.set_config(cfg)
+        Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+        gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"stream-K, integers {cfg.as_dict()}")
+    plan.close()
+
+
+def test_stream_k_tail_with_other_features(ctx, gu):
+    """The stream-K tail under the scaled form, the NN layout and a K that needs padding."""
+    import oracle
+    M, N, K = 384, 1024, 2056
+    cfg = hgemm.Config.make(family=F1, block_n=128, stages=4, raster_group=2, epilogue=TMA, block_k=64, tail_split=4, tail_mode=hgemm.TAIL_STREAM)
+    A, B = inputs.make_ab(M, N, K, "int5", "cuda")
+    with ctx.plan(M, N, K) as plan:
+        plan.set_config(cfg)
+        assert hgemm.stream_item(M, N, K, cfg, 0, 0, torch.cuda.get_device_properties(0).multi_processor_count)[4] >= 2
+        C0 = inputs.draw(11, 0xC, M, N, "int5", "cuda")
+        C = C0.clone()
+        plan.run_scaled(0.5, 2.0, A, B, C)
+        torch.cuda.synchronize()
+        ref = oracle.hgemm_scaled_full(inputs.bits(A), inputs.bits(B), inputs.bits(C0), 0.5, 2.0)
+        gu.assert_exact(C, ref, "stream-K, scaled form")
+    Bt = B.T.contiguous()                                # K x N row-major
+    with ctx.plan(M, N, K, layout=hgemm.LAYOUT_NN) as plan:
+        plan.set_config(cfg)
+        C = torch.empty(M, N, dtype=torch.float16, device="cuda")
+        plan.run(A, Bt, C)
+        torch.cuda.synchronize()
+        gu.assert_exact(C, oracle.hgemm_full(inputs.bits(A), inputs.bits(B)), "stream-K, NN layout")
+    # rules: no transposed stores, no double tile, no light kernel, no fp16 accumulators
+    bad = [hgemm.Config.make(family=F1, block_n=128, stages=4, tail_split=4, tail_mode=hgemm.TAIL_STREAM, swap_ab=1),
+           hgemm.Config.make(family=F2, block_n=512, stages=3, tail_split=4, tail_mode=hgemm.TAIL_STREAM, epilogue=TMA),
+           hgemm.Config.make(family=F1, block_n=128, stages=3, tail_split=4, tail_mode=hgemm.TAIL_STREAM, epilogue=WIDE),
+           hgemm.Config.make(family=hgemm.FAMILY_LIGHT, block_n=128, stages=4, tail_split=4, tail_mode=hgemm.TAIL_STREAM),
+           hgemm.Config.make(family=F1, block_n=128, stages=4, tail_split=4, tail_mode=hgemm.TAIL_STREAM, accumulate=hgemm.ACC_F16)]
+    for c in bad:
+        assert hgemm.validate_config(1024, 1024, 1024, c) == hgemm.ERR_UNSUPPORTED, c.as_dict()
+
+
 # ---- tail split along N: the last wave's tiles as independent narrower tiles ---------------------------------
 
 @pytest.mark.parametrize("family,bn,bk,stages,pieces", [(F2, 256, 128, 3, 2), (F2, 256, 64, 6, 4), (F1, 256, 64, 4, 2), (F1, 128, 128, 3, 4),

@@ -211,3 +211,65 @@ def test_every_table_row_is_what_the_planner_returns(lib):
         rows += 1
         families.add(family)
     assert rows >= 1000 and families == {0, 1, 2, 3}
+
+
+def _stream_partition(M, N, K, family, bn, bk, tail, sms):
+    """Brute-force check of one stream-K tail: returns None where the configuration has none on this shape."""
+    cfg = hgemm.Config.make(family=family, block_n=bn, stages=3, block_k=bk, tail_split=tail, tail_mode=hgemm.TAIL_STREAM,
+                            epilogue=hgemm.EPILOGUE_TMA)
+    if hgemm.validate_config(M, N, K, cfg) != hgemm.OK or hgemm.stream_item(M, N, K, cfg, 0, 0, sms) is None:
+        return None
+    cg = 2 if family == hgemm.FAMILY_UMMA_2CTA else 1
+    units = sms // cg
+    tiles = -(-M // (128 * cg)) * -(-N // bn)
+    kb = -(-K // bk)
+    rem = tiles % units
+    cover, per_tile, positions = {}, {}, None
+    for j in range(units):
+        for h in (0, 1):
+            t, k0, n, sl, sls, gs = hgemm.stream_item(M, N, K, cfg, j, h, sms)
+            positions = gs
+            if n == 0:
+                continue
+            assert j < gs and tiles - rem <= t < tiles and 0 <= k0 and k0 + n <= kb
+            for k in range(k0, k0 + n):
+                assert (t, k) not in cover, "a k-block is computed twice"
+                cover[(t, k)] = j
+            per_tile.setdefault(t, []).append((sl, sls, k0, j, h))
+    assert len(cover) == rem * kb, "a k-block of the tail is computed by no one"
+    for t, frags in per_tile.items():
+        frags.sort()
+        sls = frags[0][1]
+        assert [f[0] for f in frags] == list(range(sls)) and all(f[1] == sls for f in frags), "slices 0..S-1, once each"
+        assert [f[2] for f in frags] == sorted(f[2] for f in frags), "slices are in K order"
+        assert [f[3] for f in frags] == list(range(frags[0][3], frags[0][3] + sls)), "consecutive positions"
+        assert all(f[4] == 0 for f in frags[1:]), "only a tile's first piece can be a position's second item"
+    shares = [sum(1 for v in cover.values() if v == j) for j in range(positions)]
+    assert max(shares) - min(shares) <= 1, "equal shares"
+    most = max(len(v) for v in per_tile.values())
+    # the workspace holds `most` slots per cut tile
+    assert hgemm.config_workspace_bytes(M, N, K, cfg) >= 0
+    return positions, most
+
+
+def test_stream_k_tail_partition(lib):
+    """The arithmetic that deals the tail's k-blocks out (the kernel decodes its work items with the same function):
+    every k-block of every cut tile exactly once, equal shares, a tile's pieces on consecutive positions in K order."""
+    import itertools
+    checked = 0
+    shapes = [(12288, 256, 12288), (128, 12288, 12288), (512, 4096, 8192), (4096, 4096, 4096), (640, 640, 640), (100, 1000, 1000),
+              (2048, 2048, 256), (256, 256, 12288), (64, 64, 16384), (12288, 12288, 128)]
+    for (M, N, K) in shapes:
+        for family, bn, bk, tail in itertools.product((0, 1), (32, 128, 192, 256), (64, 128), (2, 3, 8, 16)):
+            checked += _stream_partition(M, N, K, family, bn, bk, tail, 148) is not None
+    for sms in (2, 4, 7, 16, 132):                       # other SM counts (the layout is a function of the device)
+        for family, bn, tail in itertools.product((0, 1), (64, 256), (2, 5, 16)):
+            checked += _stream_partition(3000, 1000, 2000, family, bn, 64, tail, sms) is not None
+    assert checked > 300
+    # 96 tiles of 128 x 256 on 148 SMs: all 148 positions, each tile in two or three pieces
+    assert _stream_partition(12288, 256, 12288, 0, 256, 64, 2, 148) == (148, 3)
+    # a whole number of waves, or too few k-blocks to share: no tail, the configuration runs as if tail_split were off
+    cfg = hgemm.Config.make(family=0, block_n=128, stages=3, tail_split=2, tail_mode=hgemm.TAIL_STREAM, epilogue=hgemm.EPILOGUE_TMA)
+    assert hgemm.stream_item(148 * 128, 128, 4096, cfg, 0, 0, 148) is None
+    assert hgemm.stream_item(4096, 4096, 64, cfg, 0, 0, 148) is None
+    assert hgemm.config_workspace_bytes(4096, 4096, 64, cfg) == 0
