@@ -2,7 +2,7 @@
 
     python -m paper_2512_02551_b200.run_case 8192x8192x8192 [--iters 3] [--warmup 2]
         [--family 0|1|2|3 --block-n 256 --block-k 64|128 --stages 4 --split-k 1 --split-mode 0|1 --raster 8
-         --raster-mode 0|1 --epilogue 0|1|2 --swap-ab 0|1]
+         --raster-mode 0|1 --epilogue 0|1|2 --swap-ab 0|1 --tail-split 2 --tail-mode 0|1|2]
 
 Small enough to sit under a profiler: it draws the inputs, plans, warms up and launches
 `iters` times.  Without the configuration flags the library's own plan is used; with --family the
@@ -32,6 +32,8 @@ def main() -> None:
     ap.add_argument("--split-mode", type=int)
     ap.add_argument("--raster-mode", type=int)
     ap.add_argument("--swap-ab", type=int)
+    ap.add_argument("--tail-split", type=int)
+    ap.add_argument("--tail-mode", type=int)
     args = ap.parse_args()
     M, N, K = (int(v) for v in args.shape.lower().split("x"))
     with hgemm.Context(0) as ctx:
@@ -45,7 +47,7 @@ def main() -> None:
                 family=args.family, block_n=128, stages=4, raster_group=1, epilogue=hgemm.EPILOGUE_TMA)
         for name, attr in (("family", "family"), ("block_n", "block_n"), ("stages", "stages"), ("split_k", "split_k"),
                            ("raster", "raster_group"), ("epilogue", "epilogue"), ("block_k", "block_k"), ("split_mode", "split_mode"),
-                           ("raster_mode", "raster_mode"), ("swap_ab", "swap_ab")):
+                           ("raster_mode", "raster_mode"), ("swap_ab", "swap_ab"), ("tail_split", "tail_split"), ("tail_mode", "tail_mode")):
             v = getattr(args, name)
             if v is not None:
                 setattr(cfg, attr, v)
