@@ -68,9 +68,11 @@ enum {
                                    tail_split, no swap_ab, fp32 accumulators, the TN layout, HGEMM_EPILOGUE_DIRECT or HGEMM_EPILOGUE_TMA */
     HGEMM_FAMILY_SMALL = 3      /* the register-accumulator kernel for the smallest problems: 64 x 64 or 32 x 32 tiles, cp.async +
                                    ldmatrix + mma.sync with fp32 accumulators in registers -- no tensor memory to allocate
-                                   (0.7 us on B200), no tensor maps, no mbarriers.  Two fixed configurations: block_m = block_n
-                                   = 64 or 32, block_k = 64, stages = 3, split_k = 1, HGEMM_EPILOGUE_DIRECT.  Needs K % 8 == 0
-                                   and N % 8 == 0, no tail_split, no swap_ab, fp32 accumulators, the TN layout */
+                                   (0.7 us on B200), no tensor maps, no mbarriers.  Two tiles: block_m = block_n = 64 or 32,
+                                   with block_k = 64, stages = 3, HGEMM_EPILOGUE_DIRECT; split_k in 1..16 (at most one slice per
+                                   64-wide k-block), and with split_k > 1 split_mode = HGEMM_SPLIT_CLUSTER: the slices of a tile are
+                                   the CTAs of one cluster and sum their partial tiles through its shared memory in slice order.
+                                   Needs K % 8 == 0 and N % 8 == 0, no tail_split, no swap_ab, fp32 accumulators, the TN layout */
 };
 
 /* Where the fp32 partial sums of a split-K tile meet.  Both sum the slices in slice

@@ -132,7 +132,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     if (pl->layout == HGEMM_LAYOUT_NN && cfg.tail_mode == HGEMM_TAIL_N && cfg.tail_split >= 2 &&
         ((cfg.block_n / cfg.tail_split) % (64 * cg)) != 0)
         return HGEMM_ERR_UNSUPPORTED;
-    const bool cluster_split = cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER;
+    // (the small family's K slices are a cluster of its own kernel: at most 16 CTAs of 128 threads and 48 KB, placed anywhere)
+    const bool cluster_split = cfg.split_k > 1 && cfg.split_mode == HGEMM_SPLIT_CLUSTER && cfg.family != HGEMM_FAMILY_SMALL;
     if (cluster_split) {
         // can the device place a cluster of split_k CTAs of this kernel at all?
         cudaLaunchConfig_t lc;
@@ -272,8 +273,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
         // 64 x 64 or 32 x 32 tiles, one CTA each, static shared memory, no tensor maps
         p.tiles_m = int32_t((pl->M + cfg.block_n - 1) / cfg.block_n);
         p.tiles_n = int32_t((pl->N + cfg.block_n - 1) / cfg.block_n);
-        pl->grid = p.tiles_m * p.tiles_n;
-        pl->cluster_dim = 1;
+        pl->grid = p.tiles_m * p.tiles_n * std::max(1, cfg.split_k);
+        pl->cluster_dim = std::max(1, cfg.split_k);
         pl->smem = 0;
     }
     if (cfg.family == HGEMM_FAMILY_LIGHT) {
@@ -460,6 +461,8 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(hgemm_dev::hgemm_light_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(hgemm_dev::hgemm_small_kernel<32>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(hgemm_dev::hgemm_small_kernel<64>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         for (int k = 0; k < 6 && e == cudaSuccess; ++k) {           // the stream-K instantiations
             const void *fn_k = kernel_for(1 + (k & 1), false, 3, k >= 2, false, k >= 4 ? 2 : 1);
             e = cudaFuncSetAttribute(fn_k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(hgemm_host::kSmemOptInBytes));
@@ -787,16 +790,28 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         sp.scaled = scaled ? 1u : 0u;
         sp.alpha = alpha;
         sp.beta = beta;
+        sp.split_k = plan->cluster_dim;
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof(lc));
         lc.gridDim = dim3(unsigned(plan->grid), 1, 1);
         lc.blockDim = dim3(hgemm_dev::kSmallThreads, 1, 1);
         lc.stream = static_cast<cudaStream_t>(stream);
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchAttribute attr[2];
+        int na = 0;
+        if (plan->cluster_dim > 1) {                     // the K slices of a tile are one cluster
+            attr[na].id = cudaLaunchAttributeClusterDimension;
+            attr[na].val.clusterDim.x = unsigned(plan->cluster_dim);
+            attr[na].val.clusterDim.y = 1;
+            attr[na].val.clusterDim.z = 1;
+            ++na;
+        }
+        if (ctx->dependent_launch) {
+            attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[na].val.programmaticStreamSerializationAllowed = 1;
+            ++na;
+        }
         lc.attrs = attr;
-        lc.numAttrs = ctx->dependent_launch ? 1 : 0;
+        lc.numAttrs = unsigned(na);
         void *sargs[1] = {&sp};
         cudaError_t e = cudaLaunchKernelExC(&lc, cfg.block_n == 32 ? reinterpret_cast<const void *>(hgemm_dev::hgemm_small_kernel<32>)
                                                                    : reinterpret_cast<const void *>(hgemm_dev::hgemm_small_kernel<64>), sargs);

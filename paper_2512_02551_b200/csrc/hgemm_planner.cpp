@@ -62,7 +62,8 @@ SplitLayout split_layout(int64_t M, int64_t N, int64_t K, int32_t num_sms, const
         S.first_split_tile = S.tiles;
         S.slices = 1;
         S.pieces = 1;
-        S.work_items = S.tiles;
+        S.stream_units = 0;
+        S.work_items = S.tiles * std::max(1, c.split_k);          // one CTA per (tile, K slice)
         return S;
     }
     if (c.swap_ab) std::swap(M, N);   // the kernel tiles the transposed problem
@@ -162,12 +163,14 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
         // two fixed configurations: 64 x 64 or 32 x 32 tiles
         for (int i = 0; i < 2; ++i)
             if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
-        if ((c.block_n != 64 && c.block_n != 32) || c.block_m != c.block_n || c.block_k != 64 || c.stages != 3 || c.split_k != 1 || c.tail_split >= 2 || c.swap_ab ||
+        // K slices: the CTAs of one cluster (at most 16), summed through its shared memory
+        if (c.split_k < 1 || c.split_k > 16 || c.split_k > ceil_div(K, 64) || (c.split_k > 1 && c.split_mode != HGEMM_SPLIT_CLUSTER)) return HGEMM_ERR_UNSUPPORTED;
+        if ((c.block_n != 64 && c.block_n != 32) || c.block_m != c.block_n || c.block_k != 64 || c.stages != 3 || c.tail_split >= 2 || c.swap_ab ||
             c.accumulate != HGEMM_ACC_F32 || c.epilogue != HGEMM_EPILOGUE_DIRECT || c.raster_mode != HGEMM_RASTER_SWEEP || c.raster_group < 1 ||
             (c.split_mode != HGEMM_SPLIT_WORKSPACE && c.split_mode != HGEMM_SPLIT_CLUSTER) || (c.tail_mode != HGEMM_TAIL_K && c.tail_mode != HGEMM_TAIL_N) ||
             (K % 8) != 0 || (N % 8) != 0)
             return HGEMM_ERR_UNSUPPORTED;
-        if (ceil_div(M, c.block_n) * ceil_div(N, c.block_n) >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
+        if (ceil_div(M, c.block_n) * ceil_div(N, c.block_n) * c.split_k >= (int64_t(1) << 30)) return HGEMM_ERR_UNSUPPORTED;
         return HGEMM_OK;
     }
     if (c.family != HGEMM_FAMILY_UMMA_1CTA && c.family != HGEMM_FAMILY_UMMA_2CTA && c.family != HGEMM_FAMILY_LIGHT) return HGEMM_ERR_UNSUPPORTED;
@@ -236,8 +239,10 @@ double estimate_cycles(int64_t M, int64_t N, int64_t K, int32_t num_sms, const h
         // Not fitted: a ranking hint.  Per 64-wide k-block a CTA with 64 x 64 tiles moves 16 KB into shared memory and
         // issues 128 MMAs of 16 x 8 x 16 (a quarter of both with 32 x 32 tiles); a few CTAs share an SM; a short fixed part.
         const double t = c.block_n == 32 ? 0.3 : 1.0;
-        const double waves = std::ceil(double(ceil_div(M, c.block_n) * ceil_div(N, c.block_n)) / ((c.block_n == 32 ? 8.0 : 4.0) * std::max(1, num_sms)));
-        return 1400.0 + waves * (double(ceil_div(K, 64)) * 600.0 * t + 600.0);
+        const int32_t S = std::max(1, c.split_k);
+        const double waves = std::ceil(double(ceil_div(M, c.block_n) * ceil_div(N, c.block_n) * S) / ((c.block_n == 32 ? 8.0 : 4.0) * std::max(1, num_sms)));
+        // K slices run side by side; their sum costs a cluster barrier and S reads per element
+        return 1400.0 + waves * (double(ceil_div(ceil_div(K, 64), S)) * 600.0 * t + 600.0) + (S > 1 ? 900.0 + 40.0 * S : 0.0);
     }
     // Rough machine model, in SM clock cycles: a ranking aid, not a prediction.  Its form follows the kernel
     // (waves of tiles, k-blocks bounded by the tensor pipe, the stage hand-off, the fill rate of one SM, the
@@ -391,6 +396,13 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
         add(c);                                                     // (validate() keeps it to K % 8 == 0 and N % 8 == 0)
         c.block_m = c.block_n = 32;
         add(c);
+        c.split_mode = HGEMM_SPLIT_CLUSTER;                         // the same with the K loop cut into the CTAs of a cluster
+        for (int32_t tile = 64; tile >= 32; tile -= 32)
+            for (int32_t split = 2; split <= 16; split *= 2) {
+                c.block_m = c.block_n = tile;
+                c.split_k = split;
+                if (ceil_div(M, tile) * ceil_div(N, tile) * split <= 8 * int64_t(num_sms)) add(c);
+            }
     }
     // swap == 1: the operands trade places (few rows, many columns: the rows of B fill the MMA's 128-row side)
     for (int swap = 0; swap < 2; ++swap) {

@@ -19,6 +19,13 @@
 // Same arithmetic as the tcgen05 kernels: exact fp16 products, fp32 accumulation, one rounding to fp16 (or the
 // alpha / beta form before it).  Needs K % 8 == 0 and N % 8 == 0; rows and columns beyond M, N and K are
 // zero-filled on the way in and never stored.
+//
+// Split-K (split_k = S > 1): the S CTAs of a cluster share one tile, each with a contiguous range of the k-blocks;
+// the short K loops run side by side instead of one after the other, which is what a problem of a few tiles with
+// K in the thousands wants.  Afterwards every CTA lays its fp32 partial tile out in its own shared memory, the
+// cluster meets at a barrier, and CTA s adds share s of the tile -- its own copy and the S - 1 others, read through
+// the cluster's shared-memory network in slice order 0 .. S - 1, so the result does not depend on who finishes
+// first -- and stores it; a second barrier keeps every CTA alive while its memory may still be read.
 #pragma once
 
 #include <cuda_fp16.h>
@@ -37,9 +44,10 @@ struct SmallParams {
     const __half *B;                  // N x K, K-contiguous
     __half *C;                        // M x N row-major
     int32_t M, N, K;
-    int32_t tiles_m;                  // ceil(M / T): CTA b computes tile (b % tiles_m, b / tiles_m)
+    int32_t tiles_m;                  // ceil(M / T): cluster b computes tile (b % tiles_m, b / tiles_m)
     uint32_t scaled;                  // 1: C = alpha A B^T + beta C
     float alpha, beta;
+    int32_t split_k;                  // CTAs per cluster = K slices per tile (1: none); blockIdx.x = tile * split_k + slice
 };
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
@@ -72,10 +80,16 @@ hgemm_small_kernel(const SmallParams p)
     const uint32_t smem_base = smem_addr(smem);
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const uint32_t wm = warp & 1u, wn = warp >> 1;                      // this warp's quarter of the tile
-    const int32_t tile = static_cast<int32_t>(blockIdx.x);
+    const int32_t S = p.split_k;
+    const int32_t slice = S > 1 ? static_cast<int32_t>(cluster_ctarank()) : 0;
+    const int32_t tile = S > 1 ? static_cast<int32_t>(blockIdx.x) / S : static_cast<int32_t>(blockIdx.x);
     const int32_t tn = tile / p.tiles_m, tm = tile - tn * p.tiles_m;
     const int32_t m0 = tm * kSmallTile, n0 = tn * kSmallTile;
-    const int32_t kblocks = (p.K + kSmallBk - 1) / kSmallBk;
+    // this CTA's k-blocks: the first (all mod S) slices take one more
+    const int32_t kb_all = (p.K + kSmallBk - 1) / kSmallBk;
+    const int32_t kb_base = kb_all / S, kb_rem = kb_all - kb_base * S;
+    const int32_t kb_first = slice * kb_base + min(slice, kb_rem);
+    const int32_t kblocks = kb_base + (slice < kb_rem ? 1 : 0);
     constexpr uint32_t kTileBytes = kSmallTile * kSmallBk * 2;          // 8 KB
 
     grid_launch_dependents();          // the next kernel in the stream may start its own set-up
@@ -85,7 +99,7 @@ hgemm_small_kernel(const SmallParams p)
     auto load_stage = [&](int32_t kb, int32_t s) {
         const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * 2u * kTileBytes;
         const uint32_t b_dst = a_dst + kTileBytes;
-        const int32_t k0 = kb * kSmallBk;
+        const int32_t k0 = (kb_first + kb) * kSmallBk;
 #pragma unroll
         for (int i = 0; i < T / 16; ++i) {
             const uint32_t piece = tid + static_cast<uint32_t>(i) * kSmallThreads;       // 0 .. 8 T - 1
@@ -148,6 +162,56 @@ hgemm_small_kernel(const SmallParams p)
 #pragma unroll
                 for (int j = 0; j < NI; ++j) mma_m16n8k16(acc[i][j], a[i], b[j][0], b[j][1]);
         }
+    }
+
+    if (S > 1) {
+        // ---- split-K: the partial tiles meet in shared memory ------------------------------------------------
+        // (every thread of every CTA of the cluster takes both barriers: nothing above or below returns early)
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        __syncthreads();                                              // the ring is free: it now holds the partial tile,
+        const uint32_t part = smem_base;                              // row-major fp32, T floats per row (T * T * 4 <= 16 KB)
+#pragma unroll
+        for (int i = 0; i < MI; ++i)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int j = 0; j < NI; ++j) {
+                    const uint32_t r = wm * (T / 2) + i * 16u + h * 8u + (lane >> 2), c = wn * (T / 2) + j * 8u + (lane & 3u) * 2u;
+                    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(part + (r * T + c) * 4u), "f"(acc[i][j][2 * h]), "f"(acc[i][j][2 * h + 1]) : "memory");
+                }
+        cluster_arrive();                                             // release: this CTA's partial is written
+        cluster_wait();                                               // acquire: so is everyone's
+        // share `slice` of the tile's float4 units (four consecutive columns of one row), one unit per thread and pass
+        constexpr int32_t kUnits = T * T / 4;
+        const int32_t cap = (kUnits + S - 1) / S;
+        const int32_t u_end = min(kUnits, (slice + 1) * cap);
+        for (int32_t u = slice * cap + static_cast<int32_t>(tid); u < u_end; u += kSmallThreads) {
+            float4 sum = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            for (int32_t sl = 0; sl < S; ++sl) {                      // slice order: the same sum whoever arrives first
+                const float4 x = ld_shared_cluster_v4(mapa(part + static_cast<uint32_t>(u) * 16u, static_cast<uint32_t>(sl)));
+                sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+            }
+            const int32_t row = m0 + (u * 4) / T, col = n0 + (u * 4) % T;
+            if (row >= p.M || col >= p.N) continue;                   // N % 8 == 0 and col % 4 == 0: the unit is inside or outside
+            __half2 *dst = reinterpret_cast<__half2 *>(p.C + static_cast<size_t>(row) * p.N + col);
+            if (p.scaled) {
+                float2 o0 = make_float2(0.0f, 0.0f), o1 = make_float2(0.0f, 0.0f);
+                if (p.beta != 0.0f) {
+                    o0 = __half22float2(dst[0]);
+                    o1 = __half22float2(dst[1]);
+                }
+                sum.x = fmaf(p.beta, o0.x, p.alpha * sum.x);
+                sum.y = fmaf(p.beta, o0.y, p.alpha * sum.y);
+                sum.z = fmaf(p.beta, o1.x, p.alpha * sum.z);
+                sum.w = fmaf(p.beta, o1.y, p.alpha * sum.w);
+            }
+            dst[0] = __floats2half2_rn(sum.x, sum.y);
+            dst[1] = __floats2half2_rn(sum.z, sum.w);
+        }
+        __syncwarp();                                                 // (the loop above ends at different times within a warp)
+        cluster_arrive_relaxed();                                     // no CTA leaves while another may still read its memory
+        cluster_wait();
+        return;
     }
 
     // epilogue: accumulator element pairs (row l / 4 [+ 8], columns 2 (l % 4), + 1) -> half2 -> 4-byte stores

@@ -48,9 +48,11 @@ class Config(ctypes.Structure):
                 ("swap_ab", ctypes.c_int32), ("raster_mode", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
 
     @classmethod
-    def small(cls, tile: int = 64) -> "Config":
-        """A configuration of the register-accumulator kernel for the smallest problems (tile = 64 or 32)."""
-        c = cls.make(family=FAMILY_SMALL, block_n=tile, stages=3, split_k=1, raster_group=1, epilogue=EPILOGUE_DIRECT, block_k=64)
+    def small(cls, tile: int = 64, split_k: int = 1) -> "Config":
+        """A configuration of the register-accumulator kernel for the smallest problems (tile = 64 or 32; split_k > 1:
+        that many K slices per tile, summed inside a cluster)."""
+        c = cls.make(family=FAMILY_SMALL, block_n=tile, stages=3, split_k=split_k, raster_group=1, epilogue=EPILOGUE_DIRECT, block_k=64,
+                     split_mode=SPLIT_CLUSTER if split_k > 1 else SPLIT_WORKSPACE)
         c.block_m = tile
         return c
 

@@ -43,7 +43,7 @@ def main() -> None:
         cfg = plan.config
         if args.family is not None:
             # an explicit family starts from a clean configuration instead of the plan's own (whose other fields may not apply)
-            cfg = hgemm.Config.small() if args.family == hgemm.FAMILY_SMALL else hgemm.Config.make(
+            cfg = hgemm.Config.small(split_k=args.split_k or 1) if args.family == hgemm.FAMILY_SMALL else hgemm.Config.make(
                 family=args.family, block_n=128, stages=4, raster_group=1, epilogue=hgemm.EPILOGUE_TMA)
         for name, attr in (("family", "family"), ("block_n", "block_n"), ("stages", "stages"), ("split_k", "split_k"),
                            ("raster", "raster_group"), ("epilogue", "epilogue"), ("block_k", "block_k"), ("split_mode", "split_mode"),

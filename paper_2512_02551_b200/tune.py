@@ -42,10 +42,12 @@ def max_stages(family: int, bn: int, bk: int, epilogue: int = hgemm.EPILOGUE_TMA
 
 def candidates(M: int, N: int, K: int):
     out = []
-    for tile in (64, 32):                                         # the register-accumulator kernel's two configurations
-        small = hgemm.Config.small(tile)
-        if hgemm.validate_config(M, N, K, small) == hgemm.OK and M * N * K <= (1 << 31):
-            out.append(small)
+    for tile in (64, 32):                                         # the register-accumulator kernel: two tiles, K slices in a cluster
+        for split in (1, 2, 4, 8, 16):
+            small = hgemm.Config.small(tile, split)
+            if hgemm.validate_config(M, N, K, small) == hgemm.OK and M * N * K <= (1 << 31) and \
+                    -(-M // tile) * -(-N // tile) * split <= 8 * NUM_SMS:
+                out.append(small)
     for swap in (0, 1):
         if swap and not (M <= 256 and N >= 512 and N % 8 == 0):
             continue

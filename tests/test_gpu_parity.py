@@ -482,10 +482,60 @@ def test_small_family(ctx, gu, shape, tile):
     plan.close()
 
 
+SMALL_SPLIT_CASES = [
+    # M, N, K, tile, K slices
+    (64, 64, 1024, 32, 8), (64, 64, 1024, 64, 16), (256, 64, 1024, 32, 4), (128, 128, 2048, 64, 2), (100, 136, 1000, 32, 16),
+    (200, 72, 328, 64, 4), (1024, 64, 1024, 32, 2), (64, 64, 128, 32, 2), (96, 40, 200, 64, 3), (512, 512, 2048, 64, 8),
+]
+
+
+@pytest.mark.parametrize("case", SMALL_SPLIT_CASES, ids=lambda c: f"{c[0]}x{c[1]}x{c[2]}-t{c[3]}s{c[4]}")
+def test_small_family_split_k(ctx, gu, case):
+    """The register-accumulator kernel with the K loop cut into the CTAs of a cluster: exact on integers, the contract on
+    random inputs, the scaled form, ragged edges, uneven slices (K blocks not a multiple of the slices), and the same
+    bits run after run with other work in flight."""
+    import oracle
+    M, N, K, tile, split = case
+    cfg = hgemm.Config.small(tile, split)
+    assert hgemm.validate_config(M, N, K, cfg) == hgemm.OK
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C, _, plan = gu.run_gemm(ctx, A, B, cfg)
+    assert plan.config.family == hgemm.FAMILY_SMALL and plan.config.split_k == split
+    gu.assert_close_full(C, A, B, f"small split {case}")
+    bits0 = C.view(torch.int16).clone()
+    noise = torch.empty(1 << 22, device="cuda")
+    side = torch.cuda.Stream()
+    for it in range(4):
+        C2 = torch.empty_like(C)
+        with torch.cuda.stream(side):
+            for _ in range(it % 3 + 1):
+                noise.normal_()
+        plan.run(A, B, C2)
+        torch.cuda.synchronize()
+        assert torch.equal(C2.view(torch.int16), bits0), f"run {it} differs"
+    Ai, Bi = inputs.make_ab(M, N, K, "int5", "cuda")
+    Ci, _, _ = gu.run_gemm(ctx, Ai, Bi, plan=plan)
+    gu.assert_exact(Ci, oracle.hgemm_full(inputs.bits(Ai), inputs.bits(Bi)), f"small split {case} integers")
+    Ab, Bb = inputs.make_ab(M, N, K, "binary", "cuda")
+    C0 = inputs.draw(39, inputs.TAG_A, M, N, "int5", "cuda")
+    for alpha, beta in ((2.0, -1.0), (0.5, 0.0)):
+        buf, Cs = gu.alloc_c_with_guards(M, N)
+        if beta != 0.0:
+            Cs.copy_(C0)
+        plan.run_scaled(alpha, beta, Ab, Bb, Cs)
+        assert ctx.last_device_status() == (hgemm.OK, 0) and gu.guards_intact(buf, M, N)
+        gu.assert_exact(Cs, oracle.hgemm_scaled_full(inputs.bits(Ab), inputs.bits(Bb), inputs.bits(C0), alpha, beta), f"small split {case} scaled")
+    plan.close()
+
+
 def test_small_family_rules(ctx, gu):
     ok = hgemm.Config.small()
     assert hgemm.validate_config(256, 256, 256, ok) == hgemm.OK
     assert hgemm.validate_config(256, 260, 256, ok) == hgemm.ERR_UNSUPPORTED and hgemm.validate_config(256, 256, 260, ok) == hgemm.ERR_UNSUPPORTED
+    # K slices: at most 16, at most one per 64-wide k-block, and only inside a cluster
+    assert hgemm.validate_config(256, 256, 256, hgemm.Config.small(32, 4)) == hgemm.OK
+    assert hgemm.validate_config(256, 256, 256, hgemm.Config.small(32, 8)) == hgemm.ERR_UNSUPPORTED
+    assert hgemm.validate_config(256, 256, 4096, hgemm.Config.small(32, 32)) == hgemm.ERR_UNSUPPORTED
     for field, value in (("block_n", 128), ("stages", 4), ("split_k", 2), ("epilogue", TMA), ("swap_ab", 1), ("block_m", 128), ("accumulate", 1)):
         c = hgemm.Config.small()
         setattr(c, field, value)

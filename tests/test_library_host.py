@@ -159,7 +159,9 @@ def test_candidate_configs_are_legal_ranked_and_distinct(lib):
     # all three families, both stage widths, split-K and the wide epilogue all occur among the candidates of a shape that admits them
     pool = hgemm.candidate_configs(512, 512, 4096, max_count=256)
     assert {c.family for c in pool} == {0, 1, 2, 3} and {c.block_k for c in pool} == {64, 128}
-    assert 1 <= sum(c.family == hgemm.FAMILY_SMALL for c in pool) <= 2                        # its two fixed configurations (64 and 32 tiles)
+    small = [c for c in pool if c.family == hgemm.FAMILY_SMALL]                               # its two tiles, whole or in 2..16 K slices
+    assert {c.block_n for c in small} <= {32, 64} and 1 <= len(small) <= 10
+    assert all(c.split_mode == hgemm.SPLIT_CLUSTER for c in small if c.split_k > 1) and {c.split_k for c in small} <= {1, 2, 4, 8, 16}
     tiny = hgemm.candidate_configs(128, 128, 128, max_count=256)
     assert {c.block_n for c in tiny if c.family == hgemm.FAMILY_SMALL} == {32, 64}
     assert all(c.split_k == 1 and c.epilogue != hgemm.EPILOGUE_TMA_WIDE for c in pool if c.family == hgemm.FAMILY_LIGHT)
