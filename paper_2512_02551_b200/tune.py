@@ -303,7 +303,7 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
             b2b[key(c)] = min(b2b.get(key(c), t), t)
         ranked = sorted(results, key=lambda r: r[0])
         pool, seen_k = [], set()
-        for t, _, c in ranked[:10] + [r for r in ranked if r[2].family in (hgemm.FAMILY_LIGHT, hgemm.FAMILY_SMALL)][:9]:
+        for t, _, c in ranked[:10] + [r for r in ranked if r[2].family == hgemm.FAMILY_LIGHT][:6] + [r for r in ranked if r[2].family == hgemm.FAMILY_SMALL]:
             if key(c) not in seen_k:
                 seen_k.add(key(c))
                 pool.append(c)
