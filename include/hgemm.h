@@ -54,7 +54,8 @@ typedef enum {
     HGEMM_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (see hgemm_last_cuda_error) */
     HGEMM_ERR_ARCH = 5,        /* the device is not compute capability 10.0 */
     HGEMM_ERR_TIMEOUT = 6,     /* a bounded device-side wait ran out (see hgemm_last_device_status) */
-    HGEMM_ERR_SCRATCH_LIMIT = 7 /* hgemm_run_splitk_static: the call needs more scratch than the built-in buffer holds */
+    HGEMM_ERR_SCRATCH_LIMIT = 7, /* hgemm_run_splitk_static: the call needs more scratch than the built-in buffer holds */
+    HGEMM_ERR_CHECK = 8         /* the checked build (see hgemm_build_is_checked) found one of its invariants violated */
 } hgemm_status_t;
 
 /* Kernel families (section 5.1 of the paper picks a different kernel structure
@@ -350,6 +351,21 @@ hgemm_status_t hgemm_ctx_last_device_status(hgemm_ctx_t *ctx, uint32_t *code);
 /* Wait budget of the bounded waits, in SM clock cycles (default 2e9, about a
  * second).  Affects plans created afterwards and later hgemm_run calls. */
 hgemm_status_t hgemm_set_wait_budget(hgemm_ctx_t *ctx, int64_t cycles);
+
+/* 1 when this library was compiled as the checked build (-DHGEMM_CHECKED=1, `python -m paper_2512_02551_b200.build
+ * --checked` writes it beside the ordinary one as libhgemm_checked.so), else 0.  The checked build tests, where they are
+ * used, the invariants the kernels otherwise rely on: a work item inside the tile grid and the K range, TMA coordinates on
+ * 16-byte boundaries, reduced units and the small family's stores inside C, parked partial sums inside the workspace and
+ * their arrival counters inside their array, accumulator columns inside the tensor-memory allocation.  A violation is
+ * recorded in the plan's status word -- code (7 << 24) | (site << 8) -- the access is skipped, and
+ * hgemm_last_device_status / hgemm_ctx_last_device_status return HGEMM_ERR_CHECK.  Same ABI, same results, a few
+ * per cent slower; meant for the test suite and for chasing a suspected library bug, not for production. */
+int32_t hgemm_build_is_checked(void);
+
+/* Test hook: a one-thread kernel that evaluates an invariant that is false by construction, so that the reporting path
+ * can be exercised without any bad access.  In the checked build the context's status word then reads HGEMM_ERR_CHECK with
+ * code (7 << 24) | (99 << 8); in the ordinary build nothing is recorded. */
+hgemm_status_t hgemm_debug_check_probe(hgemm_ctx_t *ctx, void *stream);
 
 /* Test hook for the stream-K tail (HGEMM_TAIL_STREAM): work item `h` (0 or 1) of CTA position `position` under
  * configuration `cfg` on a device with `num_sms` SMs, as the kernel decodes it.  out[0..5] = tile index, first

@@ -255,6 +255,8 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
                               cfg.accumulate == HGEMM_ACC_F16);
     p.b_row_major = pl->layout == HGEMM_LAYOUT_NN ? 1 : 0;
     p.workspace = static_cast<float *>(pl->workspace);
+    p.workspace_floats = static_cast<unsigned long long>(pl->workspace_bytes / 4);
+    p.counter_words = static_cast<unsigned long long>(pl->counter_bytes / 4);
     p.counters = pl->counters;
     p.status = ctx->d_status + pl->status_slot;
     p.cluster_split = cluster_split ? 1 : 0;
@@ -400,6 +402,7 @@ const char *hgemm_status_string(hgemm_status_t s)
     case HGEMM_ERR_ARCH: return "device is not compute capability 10.0";
     case HGEMM_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case HGEMM_ERR_SCRATCH_LIMIT: return "the call needs more scratch memory than the library's built-in buffer holds";
+    case HGEMM_ERR_CHECK: return "the checked build found an invariant violated";
     }
     return "unknown status";
 }
@@ -791,6 +794,7 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
         sp.alpha = alpha;
         sp.beta = beta;
         sp.split_k = plan->cluster_dim;
+        sp.status = ctx->d_status + plan->status_slot;
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof(lc));
         lc.gridDim = dim3(unsigned(plan->grid), 1, 1);
@@ -1003,7 +1007,7 @@ hgemm_status_t hgemm_last_device_status(hgemm_plan_t *plan, uint32_t *code)
         if (s != HGEMM_OK) return s;
     }
     *code = v;
-    return v ? HGEMM_ERR_TIMEOUT : HGEMM_OK;
+    return v == 0 ? HGEMM_OK : (v >> 24) == hgemm_dev::kRoleCheck ? HGEMM_ERR_CHECK : HGEMM_ERR_TIMEOUT;
 }
 
 hgemm_status_t hgemm_ctx_last_device_status(hgemm_ctx_t *ctx, uint32_t *code)
@@ -1029,7 +1033,7 @@ hgemm_status_t hgemm_ctx_last_device_status(hgemm_ctx_t *ctx, uint32_t *code)
         if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
     *code = v;
-    return v ? HGEMM_ERR_TIMEOUT : HGEMM_OK;
+    return v == 0 ? HGEMM_OK : (v >> 24) == hgemm_dev::kRoleCheck ? HGEMM_ERR_CHECK : HGEMM_ERR_TIMEOUT;
 }
 
 hgemm_status_t hgemm_debug_fail_allocs(hgemm_ctx_t *ctx, int32_t after, int32_t count)
@@ -1078,6 +1082,20 @@ hgemm_status_t hgemm_debug_timeout_probe(hgemm_ctx_t *ctx, void *stream)
 {
     if (!ctx) return HGEMM_ERR_INVALID_ARG;
     hgemm_dev::hgemm_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status, ctx->wait_budget);   // slot 0
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return HGEMM_OK;
+}
+
+int32_t hgemm_build_is_checked(void)
+{
+    return HGEMM_CHECKED;
+}
+
+hgemm_status_t hgemm_debug_check_probe(hgemm_ctx_t *ctx, void *stream)
+{
+    if (!ctx) return HGEMM_ERR_INVALID_ARG;
+    hgemm_dev::hgemm_check_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_status);   // slot 0
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return HGEMM_OK;

@@ -50,6 +50,17 @@ constexpr int kCtrlBytes = 512;       // barriers, tensor-memory base, abort fla
 
 // Status-word roles
 constexpr uint32_t kRoleProducer = 1, kRoleMma = 2, kRoleEpilogue = 3, kRoleProbe = 4;
+// The checked build (-DHGEMM_CHECKED=1, a second library beside the ordinary one): invariants that the ordinary build relies
+// on without testing them -- a work item inside the tile grid and the K range, TMA coordinates on 16-byte boundaries, stores
+// of reduced units inside C, parked pieces inside the workspace, arrival counters inside their array, accumulator columns
+// inside the allocation -- are tested where they are used.  A violation records (kRoleCheck, site) in the plan's status
+// word and the access is skipped; hgemm_last_device_status then reports HGEMM_ERR_CHECK.
+#ifndef HGEMM_CHECKED
+#define HGEMM_CHECKED 0
+#endif
+constexpr uint32_t kRoleCheck = 7;
+constexpr uint32_t kCheckWorkItem = 1, kCheckLoadCoord = 2, kCheckUnitStore = 3, kCheckSlot = 4, kCheckCounter = 5, kCheckStoreCoord = 6,
+                   kCheckTmemColumn = 7, kCheckSmallStore = 8, kCheckProbe = 99;
 
 // x / d for x < 2^31 without a division instruction: q = umulhi(x, mul) >> shr (d == 1: q = x).
 // mul = ceil(2^(31 + ceil(log2 d)) / d), shr = ceil(log2 d) - 1.
@@ -168,6 +179,8 @@ struct KernelParams {
     // stream-K tail (see stream_item): 0 positions = none.  Then split_k is the largest number of slices of a tile
     // (the stride of a tile's workspace slots) and the work items from first_split_tile on are numbered
     // first_split_tile + h * grid_units + j.
+    unsigned long long workspace_floats;   // capacity of `workspace` and of `counters` (32-bit words): what the checked build
+    unsigned long long counter_words;      // tests parked pieces and arrivals against
     int32_t stream_units;         // positions that share the tail's k-blocks
     int32_t stream_q;             // k-blocks of the tail: (tiles - first_split_tile) * kblocks
     int32_t grid_units;           // CTAs (pairs) of the grid
@@ -228,6 +241,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
 __device__ __forceinline__ uint32_t status_code(uint32_t role, uint32_t barrier_index, uint32_t stage)
 {
     return (role << 24) | ((barrier_index & 0xffffu) << 8) | (stage & 0xffu);
+}
+
+// Checked build: `holds` is an invariant of site `site`; false records it and tells the caller to skip the access.
+// Ordinary build: always true, and the test of `holds` is compiled out with it.
+__device__ __forceinline__ bool checked(uint32_t *status, bool holds, uint32_t site)
+{
+#if HGEMM_CHECKED
+    if (!holds) {
+        atomicCAS(status, 0u, status_code(kRoleCheck, site, 0));
+        return false;
+    }
+#endif
+    return true;
 }
 
 // -------------------------------------------------------------------------------------
@@ -623,6 +649,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         };
         for (int32_t w = unit; ok && w < p.total_work; w += num_units) {
             const WorkItem it = warp_uniform(decode_work<SPLIT != 0, PLAIN>(w, p, kBlockMTotal));
+            if (HGEMM_CHECKED && !checked(p.status, it.tile >= 0 && it.tile < p.tiles_m * p.tiles_n && it.m0 >= 0 && it.m0 < p.M && it.n0 >= 0 &&
+                                                        it.n0 < p.tiles_n * p.block_n && it.kb_begin >= 0 && it.kb_count >= 0 && it.kb_begin + it.kb_count <= p.kblocks &&
+                                                        it.slice >= 0 && it.slice < it.slices, kCheckWorkItem))
+                break;                                         // (the other roles then run into their bounded waits)
             const int32_t a_row = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;
             // this CTA's rows of B: its share of the work item's columns
             const int32_t b_row = it.n0 + static_cast<int32_t>(cta_rank) * (it.bn / CTA_GROUP);
@@ -635,6 +665,11 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const uint32_t a_dst = smem_base + static_cast<uint32_t>(s) * stage_bytes;
                 const uint32_t b_dst = a_dst + a_stage_bytes;
                 const int32_t k0 = (it.kb_begin + kb) * p.block_k;
+                if (HGEMM_CHECKED && !checked(p.status, (k0 & 7) == 0 && k0 >= 0 && k0 < p.kblocks * p.block_k && a_row >= 0 && b_row >= 0 && s >= 0 &&
+                                                            s < p.stages, kCheckLoadCoord)) {
+                    ok = false;
+                    break;
+                }
                 const uint32_t fb = full_leader + 8 * s;      // the (leader's) full barrier of this stage
                 if (!dependencies_met) {
                     // Operands the caller declared static (KernelParams::early_ops: no kernel ahead of this call in the
@@ -976,6 +1011,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int32_t row0 = it.m0 + static_cast<int32_t>(cta_rank) * kBlockM;  // first row of this CTA's 128
             const int32_t grow = row0 + static_cast<int32_t>(row_in_tile);          // this thread's global row
             const uint32_t t_addr = tmem_base + ((q * 32u) << 16) + acc * static_cast<uint32_t>(p.block_n);
+            if (HGEMM_CHECKED && !checked(p.status, static_cast<int32_t>(acc) * p.block_n + (DUAL ? 512 : p.block_n) <= p.tmem_cols, kCheckTmemColumn)) {
+                ok = false;
+                break;
+            }
 
             // One 32-column chunk of this thread's row, converted and sent to C.
             auto emit_chunk = [&](const uint32_t (&v)[32], int32_t c) {
@@ -1030,7 +1069,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         // warp-uniform code: the store is predicated inside its asm block, the commit is executed
                         // by every lane (an empty group for all but lane 0)
                         const int32_t box_row = row0 + static_cast<int32_t>(q) * 32;
-                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((TRACE ? p.debug_skip : 0u) & 4u);
+                        const bool go = lane == 0 && box_row < p.M && col0 < p.N && !((TRACE ? p.debug_skip : 0u) & 4u) &&
+                                        checked(p.status, (col0 & 7) == 0 && col0 >= 0 && box_row >= 0, kCheckStoreCoord);
                         tma_store_2d_if(go ? 1u : 0u, &tmap_c, col0, box_row, buf);
                         bulk_commit_group();
                     }
@@ -1243,7 +1283,10 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 // is written.
                 const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
                 float *slot = p.workspace + (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank) * slot_floats;
-                const int32_t park_chunks = live_rows ? live_chunks : 0;
+                const bool slot_ok = checked(p.status, (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank + 1) * slot_floats <= p.workspace_floats &&
+                                                           (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2 + 2 <= p.counter_words,
+                                             kCheckSlot);
+                const int32_t park_chunks = (live_rows && slot_ok) ? live_chunks : 0;
                 for (int32_t c = static_cast<int32_t>(first_chunk); c < park_chunks; c += 2) {
                     uint32_t v[32];
                     tmem_ld_32x32b_x32(t_addr + static_cast<uint32_t>(c) * 32u, v);
@@ -1257,7 +1300,7 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 release_accumulator(acc);
                 // announce this warp's part: its stores, made visible to the GPU, then one arrival
                 __syncwarp();
-                if (lane == 0) {
+                if (lane == 0 && slot_ok) {
                     __threadfence();
                     atomicAdd(p.counters + (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2, 1u);
                 }
@@ -1276,6 +1319,13 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 //    its store buffer and sends them with one bulk copy.
                 const size_t slot_floats = static_cast<size_t>(kBlockM) * p.block_n;
                 float *slot = p.workspace + (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank) * slot_floats;
+                const bool slot_ok = checked(p.status, (static_cast<size_t>(it.split_index) * CTA_GROUP + cta_rank + 1) * slot_floats <= p.workspace_floats &&
+                                                           (static_cast<size_t>(it.tile - p.first_split_tile) * CTA_GROUP + cta_rank) * 2 + 2 <= p.counter_words,
+                                             kCheckSlot);
+                if (HGEMM_CHECKED && !slot_ok) {               // (its tile then never completes: the other slices' waits run out)
+                    ok = false;
+                    break;
+                }
                 const int32_t park_chunks = live_rows ? live_chunks : 0;
                 for (int32_t c = static_cast<int32_t>(first_chunk); c < park_chunks; c += 2) {
                     uint32_t v[32];
@@ -1388,7 +1438,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         uint2 o;
                         o.x = pack_half2_rn(__float_as_uint(sum[j].x), __float_as_uint(sum[j].y));
                         o.y = pack_half2_rn(__float_as_uint(sum[j].z), __float_as_uint(sum[j].w));
-                        *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
+                        if (checked(p.status, orow >= 0 && orow < p.M && col >= 0 && col + 4 <= p.N && (col & 3) == 0, kCheckUnitStore))
+                            *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                     }
                 }
                 if (w == unit && threadIdx.x == 64) trace_stamp<!TRACE>(p, 18);
@@ -1521,7 +1572,8 @@ hgemm_umma_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         uint2 o;
                         o.x = pack_half2_rn(__float_as_uint(sum[j].x), __float_as_uint(sum[j].y));
                         o.y = pack_half2_rn(__float_as_uint(sum[j].z), __float_as_uint(sum[j].w));
-                        *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
+                        if (checked(p.status, orow >= 0 && orow < p.M && col >= 0 && col + 4 <= p.N && (col & 3) == 0, kCheckUnitStore))
+                            *reinterpret_cast<uint2 *>(p.C + static_cast<size_t>(orow) * p.N + col) = o;   // N % 8 == 0: in bounds
                     }
                 }
             }
@@ -1580,6 +1632,12 @@ __global__ void hgemm_timeout_probe_kernel(uint32_t *status, long long budget)
         WaitCtl ctl{&abort_flag, status, budget};
         (void)mbar_wait(smem_addr(&bar), 0u, ctl, status_code(kRoleProbe, 0xffff, 0xff));
     }
+}
+
+// The reporting path of the checked build without any bad access: an invariant that is false by construction.
+__global__ void hgemm_check_probe_kernel(uint32_t *status)
+{
+    if (threadIdx.x == 0) (void)checked(status, false, kCheckProbe);
 }
 
 } // namespace hgemm_dev

@@ -39,6 +39,10 @@ constexpr int kSmallBk = 64;          // K extent of a stage
 constexpr int kSmallStages = 3;
 constexpr int kSmallThreads = 128;
 
+#ifndef HGEMM_CHECKED
+#define HGEMM_CHECKED 0        // the checked build: see hgemm_kernel.cuh
+#endif
+
 struct SmallParams {
     const __half *A;                  // M x K, K-contiguous
     const __half *B;                  // N x K, K-contiguous
@@ -48,7 +52,20 @@ struct SmallParams {
     uint32_t scaled;                  // 1: C = alpha A B^T + beta C
     float alpha, beta;
     int32_t split_k;                  // CTAs per cluster = K slices per tile (1: none); blockIdx.x = tile * split_k + slice
+    uint32_t *status;                 // the plan's status word (written by the checked build only)
 };
+
+// Checked build: a store of `width` elements at (row, col) must lie inside C on a 4-byte boundary.
+__device__ __forceinline__ bool small_store_ok(const SmallParams &p, int32_t row, int32_t col, int32_t width)
+{
+#if HGEMM_CHECKED
+    if (!(row >= 0 && row < p.M && col >= 0 && col + width <= p.N && (col & 1) == 0)) {
+        atomicCAS(p.status, 0u, (7u << 24) | (8u << 8));          // (kRoleCheck, kCheckSmallStore) of the main kernel's encoding
+        return false;
+    }
+#endif
+    return true;
+}
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes)
 {
@@ -205,6 +222,7 @@ hgemm_small_kernel(const SmallParams p)
                 sum.z = fmaf(p.beta, o1.x, p.alpha * sum.z);
                 sum.w = fmaf(p.beta, o1.y, p.alpha * sum.w);
             }
+            if (!small_store_ok(p, row, col, 4)) continue;
             dst[0] = __floats2half2_rn(sum.x, sum.y);
             dst[1] = __floats2half2_rn(sum.z, sum.w);
         }
@@ -237,7 +255,7 @@ hgemm_small_kernel(const SmallParams p)
                     x = fmaf(p.beta, ox, p.alpha * x);
                     y = fmaf(p.beta, oy, p.alpha * y);
                 }
-                *dst = __floats2half2_rn(x, y);
+                if (small_store_ok(p, row, col, 2)) *dst = __floats2half2_rn(x, y);
             }
         }
     }

@@ -211,6 +211,8 @@ extern "C" hgemm_status_t hgemm_run_splitk_static(int64_t M, int64_t N, int64_t 
     p.idesc = (1u << 4) | (uint32_t(block_n >> 3) << 17) | (uint32_t(128 >> 4) << 24);   // fp32 accumulate, fp16 A/B, K-major
     p.idesc_tail = p.idesc;
     p.workspace = reinterpret_cast<float *>(d->scratch + kControlBytes);
+    p.workspace_floats = static_cast<unsigned long long>(kScratchBytes / 4);
+    p.counter_words = static_cast<unsigned long long>(kStatusOffset / 4);
     p.counters = reinterpret_cast<uint32_t *>(d->scratch);
     p.status = reinterpret_cast<uint32_t *>(d->scratch + kStatusOffset);
     p.C = static_cast<__half *>(C);

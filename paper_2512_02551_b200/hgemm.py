@@ -11,9 +11,9 @@ import ctypes
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libhgemm.so")
+LIB_PATH = os.environ.get("HGEMM_LIB") or os.path.join(HERE, "libhgemm.so")      # HGEMM_LIB: another build of the library (the checked one)
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_SCRATCH_LIMIT = range(8)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_ARCH, ERR_TIMEOUT, ERR_SCRATCH_LIMIT, ERR_CHECK = range(9)
 FAMILY_UMMA_1CTA, FAMILY_UMMA_2CTA, FAMILY_LIGHT, FAMILY_SMALL = 0, 1, 2, 3
 EPILOGUE_DIRECT, EPILOGUE_TMA, EPILOGUE_TMA_WIDE = 0, 1, 2
 SPLIT_WORKSPACE, SPLIT_CLUSTER = 0, 1
@@ -28,7 +28,7 @@ EXPORTS = [
     "hgemm_create", "hgemm_destroy", "hgemm_plan", "hgemm_plan_layout", "hgemm_run", "hgemm_run_host", "hgemm_run_scaled", "hgemm_run_splitk_static", "hgemm_plan_destroy",
     "hgemm_plan_get_config", "hgemm_plan_set_config", "hgemm_plan_set_static_operands", "hgemm_plan_autotune", "hgemm_candidate_configs", "hgemm_heuristic_config", "hgemm_planned_config", "hgemm_validate_config", "hgemm_estimate_config",
     "hgemm_config_smem_bytes", "hgemm_config_workspace_bytes", "hgemm_plan_launches_per_run",
-    "hgemm_last_device_status", "hgemm_ctx_last_device_status", "hgemm_debug_fail_allocs", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_stream_item", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
+    "hgemm_last_device_status", "hgemm_ctx_last_device_status", "hgemm_debug_fail_allocs", "hgemm_set_wait_budget", "hgemm_set_dependent_launch", "hgemm_debug_timeout_probe", "hgemm_debug_check_probe", "hgemm_build_is_checked", "hgemm_debug_stream_item", "hgemm_debug_set_trace", "hgemm_debug_set_skip",
     "hgemm_last_cuda_error", "hgemm_status_string",
 ]
 
@@ -122,6 +122,8 @@ def lib() -> ctypes.CDLL:
             "hgemm_set_wait_budget": (i32, [p, i64]),
             "hgemm_set_dependent_launch": (i32, [p, i32]),
             "hgemm_debug_timeout_probe": (i32, [p, p]),
+            "hgemm_debug_check_probe": (i32, [p, p]),
+            "hgemm_build_is_checked": (i32, []),
             "hgemm_debug_stream_item": (i32, [i64, i64, i64, cfgp, i32, i32, i32, ctypes.POINTER(ctypes.c_int32)]),
             "hgemm_debug_set_trace": (i32, [p, p]),
             "hgemm_debug_set_skip": (i32, [p, ctypes.c_uint32]),
@@ -171,6 +173,11 @@ def candidate_configs(M: int, N: int, K: int, max_count: int = 64, num_sms: int 
 
 def validate_config(M: int, N: int, K: int, cfg: Config) -> int:
     return int(lib().hgemm_validate_config(M, N, K, ctypes.byref(cfg)))
+
+
+def build_is_checked() -> bool:
+    """True when the loaded library is the checked build (``HGEMM_LIB`` names it)."""
+    return bool(lib().hgemm_build_is_checked())
 
 
 def stream_item(M: int, N: int, K: int, cfg: "Config", position: int, h: int, num_sms: int = 148):
@@ -232,6 +239,9 @@ class Context:
 
     def debug_timeout_probe(self, stream: int = 0) -> None:
         _check(lib().hgemm_debug_timeout_probe(self._h, ctypes.c_void_p(stream)), "hgemm_debug_timeout_probe")
+
+    def debug_check_probe(self, stream: int = 0) -> None:
+        _check(lib().hgemm_debug_check_probe(self._h, ctypes.c_void_p(stream)), "hgemm_debug_check_probe")
 
     def last_cuda_error(self) -> int:
         return int(lib().hgemm_last_cuda_error(self._h))

@@ -207,3 +207,43 @@ def test_paper_grid_with_16384_default_plans(ctx, gu):
                 worst = max(worst, rep["max_err_over_bound"])
                 count += 1
     assert count == 271 and worst < 1.0
+
+
+# ---- the checked build: the same tests under a library that verifies its own invariants on the device ---------------
+
+def _run_under_checked_build(args, timeout):
+    import subprocess
+    import sys
+    from paper_2512_02551_b200 import build as hbuild
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, HGEMM_LIB=hbuild.build(checked=True), PYTHONPATH=root)
+    return subprocess.run([sys.executable] + args, env=env, cwd=root, capture_output=True, text=True, timeout=timeout)
+
+
+def test_checked_build_reports_a_violated_invariant(ctx):
+    """The reporting path, exercised by a probe whose invariant is false by construction (no bad access anywhere): the
+    checked build records (role 7, site 99) and the status calls return HGEMM_ERR_CHECK; the ordinary build records nothing."""
+    ctx.debug_check_probe()
+    assert ctx.last_device_status() == (hgemm.OK, 0) and not hgemm.build_is_checked()
+    code = ("from paper_2512_02551_b200 import hgemm\n"
+            "assert hgemm.build_is_checked()\n"
+            "with hgemm.Context(0) as ctx:\n"
+            "    ctx.debug_check_probe()\n"
+            "    st, code = ctx.last_device_status()\n"
+            "    again = ctx.last_device_status()\n"
+            "    print(st, code, again[0], again[1])\n")
+    r = _run_under_checked_build(["-c", code], 300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    st, code, st2, code2 = (int(v) for v in r.stdout.split())
+    assert st == hgemm.ERR_CHECK and code == (7 << 24) | (99 << 8)
+    assert (st2, code2) == (hgemm.OK, 0)                     # reading the status clears it
+
+
+def test_checked_build_finds_nothing_in_the_parity_cases():
+    """Every kernel family, reduction and tail mode of the parity suite under the checked build: same results, and no
+    invariant violated (each of those tests asserts a clean status word after every call)."""
+    r = _run_under_checked_build(["-m", "pytest", "tests/test_gpu_parity.py", "-x", "-q", "-m", "gpu", "-k",
+                                  "unit_shapes or stream_k or tail_split or swapped_operands or small_family or light_family or "
+                                  "double_accumulator or split_k_is_deterministic or nn_layout or scaled_form or serpentine"], 1500)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-1000:]
+    assert " passed" in r.stdout and "failed" not in r.stdout

@@ -275,3 +275,23 @@ def test_stream_k_tail_partition(lib):
     assert hgemm.stream_item(148 * 128, 128, 4096, cfg, 0, 0, 148) is None
     assert hgemm.stream_item(4096, 4096, 64, cfg, 0, 0, 148) is None
     assert hgemm.config_workspace_bytes(4096, 4096, 64, cfg) == 0
+
+
+def test_checked_build_exports_the_same_abi(lib):
+    """The checked build (-DHGEMM_CHECKED=1) is a second library with the same exports; which one is loaded is the
+    environment's choice (HGEMM_LIB), and each says which it is."""
+    import ctypes
+    import subprocess
+    import sys
+    path = hbuild.build(checked=True)
+    assert os.path.basename(path) == "libhgemm_checked.so" and os.path.exists(path)
+    L = ctypes.CDLL(path)
+    for name in hgemm.EXPORTS:
+        assert hasattr(L, name), name
+    L.hgemm_build_is_checked.restype = ctypes.c_int32
+    assert L.hgemm_build_is_checked() == 1 and lib.hgemm_build_is_checked() == 0
+    code = "from paper_2512_02551_b200 import hgemm; print(int(hgemm.build_is_checked()), hgemm.LIB_PATH)"
+    out = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, HGEMM_LIB=path, PYTHONPATH=ROOT), capture_output=True, text=True,
+                         check=True).stdout.split()
+    assert out == ["1", path]
+    assert hgemm.status_string(hgemm.ERR_CHECK) == "the checked build found an invariant violated"
