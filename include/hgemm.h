@@ -163,7 +163,12 @@ typedef struct {
                              padding, and a CTA pair splits the small operand instead of re-reading all of it.
                              Needs N % 8 == 0, fp32 accumulators, the TN layout, no tail_split and not the wide epilogue */
     int32_t raster_mode;  /* HGEMM_RASTER_* : the order in which raster groups sweep the n-tiles */
-    int32_t reserved[2];  /* must be zero */
+    int32_t wave_pace;    /* 0 or 1.  1: the CTAs of the persistent grid start their r-th tile together -- a producer holds its
+                             first load of a tile until every CTA has issued the last load of its previous tile (a counter in
+                             device memory; the wait gives up after 50 us, nothing depends on it).  With many equal tiles per
+                             CTA the CTAs otherwise drift apart and stop finding each other's operand panels in L2.  Same
+                             arithmetic, same bits.  Needs the 1-CTA or CTA-pair family, split_k == 1 and no tail_split */
+    int32_t reserved[1];  /* must be zero */
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the

@@ -57,6 +57,7 @@ struct hgemm_plan_s {
     uint32_t *counters = nullptr;
     int64_t counter_bytes = 0;
     uint32_t epoch = 0;            // launches that have used `counters` since they were last cleared
+    uint32_t wave_total = 0;       // arrivals that earlier launches have added to this plan's pacing counter (modulo 2^32)
     int status_slot = 0;           // this plan's word in the context's status array
     // tensor maps depend on the pointers: a small cache keyed by (A, B, C), round-robin replacement
     struct MapEntry {
@@ -263,6 +264,13 @@ hgemm_status_t apply_config(hgemm_plan_s *pl, const hgemm_config_t &cfg)
     p.tma_3d = (cfg.block_k == 128 && (pl->K % 64) == 0 && ctx->tma_3d && pl->layout == HGEMM_LAYOUT_TN && cfg.family != HGEMM_FAMILY_LIGHT) ? 1 : 0;
     p.C = nullptr;
     p.wait_budget = ctx->wait_budget;
+    {
+        // wave pacing needs at least two tiles per CTA (pair) to have anything to pace
+        const int pace_units = std::max(1, ctx->num_sms / cg);
+        p.wave_rounds = (p.total_work + pace_units - 1) / pace_units;
+        p.wave_pace = (cfg.wave_pace && p.wave_rounds >= 2) ? 1 : 0;
+        p.wave_counter = ctx->d_status + kStatusSlots + pl->status_slot;
+    }
     const int units = std::max(1, ctx->num_sms / cg);
     // cluster split-K is not persistent: one CTA per (tile, slice), the hardware schedules the clusters
     pl->grid = cluster_split ? cg * p.total_work : cg * std::min(p.total_work, units);
@@ -437,13 +445,13 @@ hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device)
             break;
         }
         ctx->encode = reinterpret_cast<encode_tiled_fn>(fn);
-        e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), kStatusSlots * sizeof(uint32_t));
+        e = cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 2 * kStatusSlots * sizeof(uint32_t));   // status words, then the plans' pacing counters
         if (e != cudaSuccess) {
             cuda_fail(ctx, e);
             st = HGEMM_ERR_ALLOC;
             break;
         }
-        e = cudaMemset(ctx->d_status, 0, kStatusSlots * sizeof(uint32_t));
+        e = cudaMemset(ctx->d_status, 0, 2 * kStatusSlots * sizeof(uint32_t));
         if (e != cudaSuccess) {
             st = cuda_fail(ctx, e);
             break;
@@ -883,6 +891,11 @@ static hgemm_status_t run_impl(hgemm_plan_t *plan, float alpha, float beta, bool
     plan->params.alpha = alpha;
     plan->params.beta = beta;
     if (plan->counters) plan->params.epoch = ++plan->epoch;   // the arrival counters count on from launch to launch
+    if (plan->params.wave_pace) {
+        // wave pacing: this launch's arrivals count on from where the plan's earlier launches left the counter
+        plan->params.wave_base = plan->wave_total;
+        plan->wave_total += uint32_t(plan->params.wave_rounds) * uint32_t(plan->grid / cg);
+    }
 
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof(lc));

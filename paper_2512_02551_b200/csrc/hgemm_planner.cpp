@@ -161,8 +161,7 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
     }
     if (c.family == HGEMM_FAMILY_SMALL) {
         // two fixed configurations: 64 x 64 or 32 x 32 tiles
-        for (int i = 0; i < 2; ++i)
-            if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+        if (c.reserved[0] != 0 || c.wave_pace != 0) return HGEMM_ERR_UNSUPPORTED;
         // K slices: the CTAs of one cluster (at most 16), summed through its shared memory
         if (c.split_k < 1 || c.split_k > 16 || c.split_k > ceil_div(K, 64) || (c.split_k > 1 && c.split_mode != HGEMM_SPLIT_CLUSTER)) return HGEMM_ERR_UNSUPPORTED;
         if ((c.block_n != 64 && c.block_n != 32) || c.block_m != c.block_n || c.block_k != 64 || c.stages != 3 || c.tail_split >= 2 || c.swap_ab ||
@@ -202,8 +201,9 @@ hgemm_status_t validate(int64_t M, int64_t N, int64_t K, const hgemm_config_t &c
         if (c.split_k != 1 || (c.block_n % 64) != 0) return HGEMM_ERR_UNSUPPORTED;
         if (c.tail_split >= 2 && c.tail_mode == HGEMM_TAIL_N && (c.block_n % (64 * c.tail_split)) != 0) return HGEMM_ERR_UNSUPPORTED;
     }
-    for (int i = 0; i < 2; ++i)
-        if (c.reserved[i] != 0) return HGEMM_ERR_UNSUPPORTED;
+    if (c.reserved[0] != 0) return HGEMM_ERR_UNSUPPORTED;
+    // wave pacing: whole, equal tiles of the persistent kernel
+    if (c.wave_pace != 0 && (c.wave_pace != 1 || c.family == HGEMM_FAMILY_LIGHT || c.split_k != 1 || c.tail_split >= 2)) return HGEMM_ERR_UNSUPPORTED;
     if (c.accumulate != HGEMM_ACC_F32 && c.accumulate != HGEMM_ACC_F16) return HGEMM_ERR_UNSUPPORTED;
     // fp16 accumulators: no fp16 partial sums are exchanged, so no split along K
     if (c.accumulate == HGEMM_ACC_F16 && (c.split_k != 1 || (c.tail_split >= 2 && c.tail_mode != HGEMM_TAIL_N))) return HGEMM_ERR_UNSUPPORTED;

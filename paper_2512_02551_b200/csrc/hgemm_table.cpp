@@ -18,10 +18,11 @@ struct Entry {
     int32_t tail_mode;   // after the original columns, so that rows written before it existed still read as 0
     float us;            // time the tuner measured (0 in rows written before the column existed)
     int32_t swap_ab, raster_mode;   // later columns again: absent from older rows, which then read 0
+    int32_t wave_pace;              // and again
 };
 const Entry kTable[] = {
 #include "hgemm_table.inc"
-    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0.0f, 0, 0}   // sentinel
+    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0.0f, 0, 0, 0}   // sentinel
 };
 // Rows read at run time from the file named by the environment variable HGEMM_TABLE (same row syntax as
 // hgemm_table.inc, as the tuner writes it; lines that do not start with '{' are skipped): they take precedence over
@@ -42,9 +43,9 @@ void load_file_rows()
         if (*p != '{') continue;
         Entry e;
         std::memset(&e, 0, sizeof(e));
-        const int n = std::sscanf(p, "{%d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %ff, %d, %d", &e.M, &e.N, &e.K, &e.family, &e.block_n,
+        const int n = std::sscanf(p, "{%d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %d, %ff, %d, %d, %d", &e.M, &e.N, &e.K, &e.family, &e.block_n,
                                   &e.block_k, &e.stages, &e.split_k, &e.split_mode, &e.tail_split, &e.raster_group, &e.epilogue, &e.tail_mode,
-                                  &e.us, &e.swap_ab, &e.raster_mode);
+                                  &e.us, &e.swap_ab, &e.raster_mode, &e.wave_pace);
         if (n >= 12 && e.M > 0 && e.N > 0 && e.K > 0) g_file_rows.push_back(e);
     }
     std::fclose(f);
@@ -75,6 +76,7 @@ hgemm_config_t config_of(const Entry &e)
     c.epilogue = e.epilogue;
     c.swap_ab = e.swap_ab;
     c.raster_mode = e.raster_mode;
+    c.wave_pace = e.wave_pace;
     return c;
 }
 

@@ -45,7 +45,8 @@ class Config(ctypes.Structure):
                 ("block_k", ctypes.c_int32), ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32),
                 ("raster_group", ctypes.c_int32), ("epilogue", ctypes.c_int32), ("split_mode", ctypes.c_int32),
                 ("tail_split", ctypes.c_int32), ("tail_mode", ctypes.c_int32), ("accumulate", ctypes.c_int32),
-                ("swap_ab", ctypes.c_int32), ("raster_mode", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
+                ("swap_ab", ctypes.c_int32), ("raster_mode", ctypes.c_int32), ("wave_pace", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 1)]
 
     @classmethod
     def small(cls, tile: int = 64, split_k: int = 1) -> "Config":
@@ -62,7 +63,7 @@ class Config(ctypes.Structure):
     @classmethod
     def make(cls, family=FAMILY_UMMA_1CTA, block_n=128, stages=4, split_k=1, raster_group=8,
              epilogue=EPILOGUE_DIRECT, block_k=64, split_mode=0, tail_split=0, tail_mode=0, accumulate=0, swap_ab=0,
-             raster_mode=0) -> "Config":
+             raster_mode=0, wave_pace=0) -> "Config":
         c = cls()
         c.family = family
         c.block_m = 256 if family == FAMILY_UMMA_2CTA else 64 if family == FAMILY_SMALL else 128
@@ -78,6 +79,7 @@ class Config(ctypes.Structure):
         c.accumulate = accumulate
         c.swap_ab = swap_ab
         c.raster_mode = raster_mode
+        c.wave_pace = wave_pace
         return c
 
 

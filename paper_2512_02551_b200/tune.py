@@ -152,7 +152,7 @@ def ctypes_copy(dst: hgemm.Config, src: hgemm.Config) -> None:
 def key(c: hgemm.Config):
     d = c.as_dict()
     return tuple(d[k] for k in ("family", "block_n", "block_k", "stages", "split_k", "split_mode", "tail_split", "tail_mode", "raster_group", "epilogue",
-                                "swap_ab", "raster_mode"))
+                                "swap_ab", "raster_mode", "wave_pace"))
 
 
 def device_times(plan, configs, run, reps: int = 5) -> dict:
@@ -372,17 +372,62 @@ def tune_shape(ctx, M, N, K, A_all, B_all, C_all, top: int, rng: random.Random, 
             "all": [list(key(c)) + [round(t * 1e3, 3)] for t, _, c in results]}   # every first-pass timing: key fields, us
 
 
+def challenge_pace(ctx, M, N, K, A_all, B_all, C_all, rng: random.Random, stream):
+    """The plan's configuration with and without wave pacing, timed alternately in sustained runs (about a quarter of a second
+    each, three rounds); returns a row like tune_shape's with pacing switched on if it is at least 0.5 % faster, else None."""
+    A = A_all.view(-1)[:M * K].view(M, K)
+    B = B_all.view(-1)[:N * K].view(N, K)
+    C = C_all[:M * N].view(M, N)
+    plan = ctx.plan(M, N, K)
+    base = plan.config
+    paced = hgemm.Config()
+    ctypes_copy(paced, base)
+    paced.wave_pace = 1
+    if base.wave_pace or hgemm.validate_config(M, N, K, paced) != hgemm.OK:
+        plan.close()
+        return None
+    cg = 2 if base.family == hgemm.FAMILY_UMMA_2CTA else 1
+    tiles = -(-M // (128 * cg)) * -(-N // base.block_n)
+    if tiles <= NUM_SMS // cg:                               # one tile per CTA: nothing to pace
+        plan.close()
+        return None
+    a, b, cptr, s = A.data_ptr(), B.data_ptr(), C.data_ptr(), stream.cuda_stream
+    run = lambda: plan.run_ptr(a, b, cptr, s)   # noqa: E731
+    times = {0: [], 1: []}
+    plan.set_config(base)
+    for _ in range(3):
+        run()
+    est = max(batch_ms(run, 3, stream), 1e-3)
+    n = max(5, min(2000, int(250.0 / est)))
+    for _ in range(3):
+        order = [(0, base), (1, paced)]
+        rng.shuffle(order)
+        for which, cfg in order:
+            plan.set_config(cfg)
+            run()
+            times[which].append(batch_ms(run, n, stream))
+    st, code = ctx.last_device_status()
+    plan.close()
+    if st != hgemm.OK:
+        raise RuntimeError(f"device status {st} code {code:#x} while timing {M}x{N}x{K}")
+    t0, t1 = statistics.median(times[0]), statistics.median(times[1])
+    if t1 > 0.995 * t0:
+        return None
+    return {"M": M, "N": N, "K": K, "best": paced.as_dict(), "us": t1 * 1e3, "default_us": t0 * 1e3, "default_final_us": t0 * 1e3, "torch_us": t0 * 1e3,
+            "ok": True, "tried": 2, "dev_us": None, "cold_us": None, "all": []}
+
+
 def write_table(rows, path):
     with open(path, "w") as f:
         f.write("// Tuned per-shape configurations for B200, written by tune.py on the GPU box.\n")
-        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode, measured us, swap_ab, raster_mode}\n")
+        f.write("// {M, N, K, family, block_n, block_k, stages, split_k, split_mode, tail_split, raster_group, epilogue, tail_mode, measured us, swap_ab, raster_mode, wave_pace}\n")
         for r in rows:
             if not r["ok"]:
                 continue
             b = r["best"]
             f.write(f"{{{r['M']}, {r['N']}, {r['K']}, {b['family']}, {b['block_n']}, {b['block_k']}, {b['stages']}, "
                     f"{b['split_k']}, {b['split_mode']}, {b.get('tail_split', 0)}, {b['raster_group']}, {b['epilogue']}, {b.get('tail_mode', 0)}, {r['us']:.2f}f, "
-                    f"{b.get('swap_ab', 0)}, {b.get('raster_mode', 0)}}},\n")
+                    f"{b.get('swap_ab', 0)}, {b.get('raster_mode', 0)}, {b.get('wave_pace', 0)}}},\n")
 
 
 def merge_table(new_rows, path):
@@ -425,6 +470,8 @@ def main():
     ap.add_argument("--from-log", metavar="JSONL", help="take the shape list (and --max-us times) from an earlier tune.jsonl")
     ap.add_argument("--challenge-stream", action="store_true",
                     help="time only the plan's current configuration against the stream-K candidates (shapes without any are skipped)")
+    ap.add_argument("--challenge-pace", action="store_true",
+                    help="time only the plan's current configuration with and without wave pacing; rows only where pacing wins")
     ap.add_argument("--min-us", type=float, default=0.0, help="with --from-log: only shapes whose recorded time is at least this")
     ap.add_argument("--grid10", action="store_true", help="the 271 shapes of the ten-value grid that contain 16384")
     ap.add_argument("--time-limit", type=float, default=0.0, help="stop starting new shapes after this many seconds (resume later)")
@@ -466,7 +513,10 @@ def main():
             if r is None:
                 if args.time_limit > 0 and time.time() - started > args.time_limit:
                     continue                                   # out of time: left for a later --resume run
-                r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream, args.explore, args.device_metric, args.challenge_stream)
+                if args.challenge_pace:
+                    r = challenge_pace(ctx, M, N, K, A_all, B_all, C_all, rng, stream)
+                else:
+                    r = tune_shape(ctx, M, N, K, A_all, B_all, C_all, args.top, rng, stream, args.explore, args.device_metric, args.challenge_stream)
                 if r is None:                                  # a challenge run on a shape without challengers
                     continue
                 log.write(json.dumps(r) + "\n")
@@ -476,9 +526,10 @@ def main():
     if args.merge_into:
         merge_table(rows, args.merge_into)
     import math
-    g = math.exp(sum(math.log(r["torch_us"] / r["us"]) for r in rows) / len(rows))
+    g = math.exp(sum(math.log(r["torch_us"] / r["us"]) for r in rows) / len(rows)) if rows else float("nan")
     bad = [r for r in rows if not r["ok"]]
-    print(f"tuned {len(rows)} shapes; geomean torch/ours = {g:.3f}; failed checks: {len(bad)}")
+    what = "geomean time without / with pacing" if args.challenge_pace else "geomean torch/ours"
+    print(f"tuned {len(rows)} shapes; {what} = {g:.3f}; failed checks: {len(bad)}")
 
 
 if __name__ == "__main__":

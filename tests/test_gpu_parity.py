@@ -639,6 +639,56 @@ def test_tail_split(ctx, gu, family, bn, bk, stages, tail, M, N, K):
     plan.close()
 
 
+# ---- wave pacing: the CTAs of the persistent grid start their r-th tile together -------------------------------
+
+PACE_CASES = [
+    # family, block_n, block_k, stages, epilogue, raster group, raster mode, M, N, K
+    (F2, 256, 64, 6, TMA, 4, 0, 4096, 4096, 512),        # 256 pair tiles on 74 pairs: four rounds, the last one partly filled
+    (F1, 128, 128, 3, DIRECT, 8, 1, 4096, 4096, 256),    # 1024 tiles on 148 SMs: seven rounds, serpentine sweep
+    (F2, 512, 64, 4, TMA, 8, 1, 4096, 4096, 256),        # the 256 x 512 tile: 128 tiles, two rounds
+    (F1, 96, 64, 6, TMA, 3, 0, 3000, 2008, 520),         # ragged in every dimension
+    (F2, 192, 64, 5, WIDE, 2, 0, 2048, 6144, 128),       # the wide epilogue
+    (F1, 256, 64, 4, TMA, 1, 0, 512, 512, 1024),         # fewer tiles than SMs: one round, nothing to pace
+]
+
+
+@pytest.mark.parametrize("case", PACE_CASES, ids=lambda c: f"f{c[0]}bn{c[1]}bk{c[2]}e{c[4]}-{c[7]}x{c[8]}x{c[9]}")
+def test_wave_pacing(ctx, gu, case):
+    """wave_pace = 1 changes when tiles start, not what they compute: the same bits as without it, launch after launch
+    (the arrival counter counts on from one launch to the next), also with other plans and other work in between."""
+    family, bn, bk, stages, epi, rg, rm, M, N, K = case
+    base = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=rg, epilogue=epi, block_k=bk, raster_mode=rm)
+    paced = hgemm.Config.make(family=family, block_n=bn, stages=stages, raster_group=rg, epilogue=epi, block_k=bk, raster_mode=rm, wave_pace=1)
+    assert hgemm.validate_config(M, N, K, paced) == hgemm.OK
+    A, B = inputs.make_ab(M, N, K, "uniform", "cuda")
+    C0, _, plan = gu.run_gemm(ctx, A, B, base)
+    gu.assert_close_full(C0, A, B, f"{base.as_dict()}") if M * N * K <= gu.FULL_CHECK_VOLUME else \
+        gu.assert_close_sampled(C0, A, B, "uniform", inputs.shape_seed(M, N, K), f"{base.as_dict()}")
+    ref_bits = C0.view(torch.int16).clone()
+    C1, _, _ = gu.run_gemm(ctx, A, B, paced, plan=plan)
+    assert plan.config.wave_pace == 1
+    assert torch.equal(C1.view(torch.int16), ref_bits)
+    other = ctx.plan(256, 256, 256)
+    Ao, Bo = inputs.make_ab(256, 256, 256, "int5", "cuda")
+    Co = torch.empty(256, 256, dtype=torch.float16, device="cuda")
+    noise = torch.empty(1 << 22, device="cuda")
+    side = torch.cuda.Stream()
+    for it in range(12):                                 # back to back: a launch starts while the one before it drains
+        C = torch.empty_like(C0)
+        if it % 3 == 0:
+            other.run(Ao, Bo, Co)
+        if it % 4 == 1:
+            with torch.cuda.stream(side):
+                noise.normal_()
+        plan.run(A, B, C)
+        plan.run(A, B, C)
+        torch.cuda.synchronize()
+        assert torch.equal(C.view(torch.int16), ref_bits), f"launch {it} differs"
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    other.close()
+    plan.close()
+
+
 # ---- stream-K tail: the tiles beyond the full waves as one sequence of k-blocks, dealt out in equal shares ------
 
 STREAM_CASES = [

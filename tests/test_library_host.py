@@ -72,8 +72,18 @@ def test_validate_rejects_illegal_configs(lib):
     c.block_m = 256                           # wrong for the 1-CTA family
     assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
     c = hgemm.Config.make(block_n=128, stages=4)
-    c.reserved[1] = 1
+    c.reserved[0] = 1
     assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED
+    # wave pacing: 0 or 1, whole equal tiles of the persistent kernel only
+    assert hgemm.validate_config(M, N, K, hgemm.Config.make(block_n=128, stages=4, wave_pace=1)) == hgemm.OK
+    assert hgemm.validate_config(M, N, K, hgemm.Config.make(family=1, block_n=512, stages=4, epilogue=hgemm.EPILOGUE_TMA, wave_pace=1)) == hgemm.OK
+    for kw in [dict(wave_pace=2), dict(wave_pace=1, split_k=2), dict(wave_pace=1, tail_split=2), dict(wave_pace=1, tail_split=2, tail_mode=hgemm.TAIL_STREAM),
+               dict(wave_pace=1, family=hgemm.FAMILY_LIGHT)]:
+        c = hgemm.Config.make(**{**dict(block_n=128, stages=4), **kw})
+        assert hgemm.validate_config(M, N, K, c) == hgemm.ERR_UNSUPPORTED, kw
+    small = hgemm.Config.small()
+    small.wave_pace = 1
+    assert hgemm.validate_config(M, N, K, small) == hgemm.ERR_UNSUPPORTED
     # cluster split-K: at most 16 CTAs per cluster (16 slices, 8 for CTA pairs), the ring must hold the fp32 partial
     assert hgemm.validate_config(M, N, 4096, hgemm.Config.make(block_n=128, stages=4, split_k=8, split_mode=1)) == hgemm.OK
     assert hgemm.validate_config(M, N, 4096, hgemm.Config.make(family=1, block_n=128, stages=4, split_k=8, split_mode=1)) == hgemm.OK
@@ -182,16 +192,17 @@ def test_table_file_overrides_the_built_in_table(lib, tmp_path):
     import sys
     table = tmp_path / "table.inc"
     table.write_text("// a comment line\n"
-                     "{4096, 4096, 4096, 0, 96, 64, 5, 1, 0, 0, 7, 0, 0, 123.00f, 0, 1},\n"      # a tabulated shape, overridden
+                     "{4096, 4096, 4096, 0, 96, 64, 5, 1, 0, 0, 7, 0, 0, 123.00f, 0, 1, 1},\n"   # a tabulated shape, overridden (newest row format)
                      "{1000, 2000, 3000, 1, 128, 128, 3, 1, 0, 0, 4, 1, 0, 50.00f},\n"            # an off-grid shape, old row format
                      "{64, 64, 64, 0, 48, 64, 2, 1, 0, 0, 1, 0, 0, 1.00f, 0, 0},\n")              # an illegal row: ignored
     code = ("from paper_2512_02551_b200 import hgemm\n"
             "a = hgemm.planned_config(4096, 4096, 4096); b = hgemm.planned_config(1000, 2000, 3000); c = hgemm.planned_config(64, 64, 64)\n"
-            "print(a.family, a.block_n, a.stages, a.raster_group, a.raster_mode, b.family, b.block_n, b.block_k, c.block_n)")
+            "print(a.family, a.block_n, a.stages, a.raster_group, a.raster_mode, b.family, b.block_n, b.block_k, c.block_n, a.wave_pace, b.wave_pace)")
     env = dict(os.environ, HGEMM_TABLE=str(table), PYTHONPATH=ROOT)
     out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, check=True).stdout.split()
     assert out[:8] == ["0", "96", "5", "7", "1", "1", "128", "128"]
     assert out[8] != "48"
+    assert out[9:11] == ["1", "0"]
 
 
 def test_every_table_row_is_what_the_planner_returns(lib):
@@ -206,10 +217,11 @@ def test_every_table_row_is_what_the_planner_returns(lib):
         v = [x.strip().rstrip("f") for x in line.strip().rstrip(",").strip("{}").split(",")]
         M, N, K, family, bn, bk, stages, split, mode, tail, rg, epi, tail_mode = (int(x) for x in v[:13])
         swap, raster_mode = (int(v[14]), int(v[15])) if len(v) >= 16 else (0, 0)
+        pace = int(v[16]) if len(v) >= 17 else 0
         c = hgemm.planned_config(M, N, K)
         got = (c.family, c.block_n, c.block_k, c.stages, c.split_k, c.split_mode, c.tail_split, c.raster_group, c.epilogue, c.tail_mode,
-               c.swap_ab, c.raster_mode)
-        assert got == (family, bn, bk, stages, split, mode, tail, rg, epi, tail_mode, swap, raster_mode), (M, N, K, got, line)
+               c.swap_ab, c.raster_mode, c.wave_pace)
+        assert got == (family, bn, bk, stages, split, mode, tail, rg, epi, tail_mode, swap, raster_mode, pace), (M, N, K, got, line)
         rows += 1
         families.add(family)
     assert rows >= 1000 and families == {0, 1, 2, 3}
