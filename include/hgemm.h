@@ -172,8 +172,9 @@ typedef struct {
 } hgemm_config_t;
 
 /* Create a context on CUDA device `device` (>= 0).  HGEMM_ERR_ARCH unless the
- * device has compute capability 10.0.  Allocates 16 KB of device status words
- * (one for the context, one per live plan: at most 4095 plans at a time). */
+ * device has compute capability 10.0.  Allocates 32 KB of device memory: status words
+ * (one for the context, one per live plan: at most 4095 plans at a time) and, behind
+ * them, one wave-pacing counter per plan (see hgemm_config_t::wave_pace). */
 hgemm_status_t hgemm_create(hgemm_ctx_t **out, int device);
 
 /* Free the context, every plan it still owns and their workspaces. */
