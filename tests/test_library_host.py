@@ -307,3 +307,45 @@ def test_checked_build_exports_the_same_abi(lib):
                          check=True).stdout.split()
     assert out == ["1", path]
     assert hgemm.status_string(hgemm.ERR_CHECK) == "the checked build found an invariant violated"
+
+
+def test_tuner_candidates_and_table_round_trip(lib, tmp_path):
+    """The tuner's host side: every candidate it would time is legal, every kernel family and mode is among them where the
+    shape admits it, and a row it writes reads back as the same configuration (through the HGEMM_TABLE file path)."""
+    import subprocess
+    import sys
+    from paper_2512_02551_b200 import tune
+    for (M, N, K) in [(64, 64, 64), (256, 64, 1024), (128, 12288, 4096), (4096, 4096, 4096), (12288, 256, 12288), (8192, 8192, 8192)]:
+        cands = tune.candidates(M, N, K)
+        assert cands and all(hgemm.validate_config(M, N, K, c) == hgemm.OK for c in cands), (M, N, K)
+        assert len({tune.key(c) for c in cands}) == len(cands), "duplicates"
+    small = tune.candidates(256, 64, 1024)
+    assert {c.split_k for c in small if c.family == hgemm.FAMILY_SMALL} >= {1, 2, 4, 8, 16}
+    skinny = tune.candidates(128, 12288, 4096)
+    assert any(c.swap_ab for c in skinny) and any(c.family == hgemm.FAMILY_LIGHT for c in skinny)
+    big = tune.candidates(8192, 8192, 8192)
+    assert any(c.block_n == 512 for c in big) and any(c.epilogue == hgemm.EPILOGUE_TMA_WIDE for c in big)
+    odd = tune.candidates(12288, 256, 12288)
+    assert any(c.tail_mode == hgemm.TAIL_STREAM and c.tail_split >= 2 for c in odd)
+    # a row written by the tuner, read back by the library in a child process
+    cfg = hgemm.Config.make(family=1, block_n=256, stages=6, raster_group=9, epilogue=hgemm.EPILOGUE_TMA, tail_split=2, tail_mode=hgemm.TAIL_STREAM)
+    cfg2 = hgemm.Config.make(family=1, block_n=512, stages=4, raster_group=12, epilogue=hgemm.EPILOGUE_TMA, raster_mode=1, wave_pace=1)
+    cfg3 = hgemm.Config.small(32, 8)
+    rows = [{"M": 12288, "N": 256, "K": 12288, "best": cfg.as_dict(), "us": 75.9, "ok": True},
+            {"M": 8192, "N": 8192, "K": 8192, "best": cfg2.as_dict(), "us": 700.0, "ok": True},
+            {"M": 256, "N": 64, "K": 1024, "best": cfg3.as_dict(), "us": 3.3, "ok": True},
+            {"M": 64, "N": 64, "K": 64, "best": cfg3.as_dict(), "us": 1.0, "ok": False}]          # a failed check is not written
+    path = tmp_path / "table.inc"
+    tune.write_table(rows, str(path))
+    text = path.read_text()
+    assert text.count("\n{") == 3 and "{64, 64, 64," not in text
+    tune.merge_table([{"M": 256, "N": 64, "K": 1024, "best": hgemm.Config.small(64, 4).as_dict(), "us": 3.0, "ok": True}], str(path))
+    code = ("from paper_2512_02551_b200 import hgemm\n"
+            "for s in ((12288, 256, 12288), (8192, 8192, 8192), (256, 64, 1024)):\n"
+            "    c = hgemm.planned_config(*s)\n"
+            "    print(c.family, c.block_n, c.stages, c.split_k, c.split_mode, c.tail_split, c.tail_mode, c.raster_group, c.raster_mode, c.wave_pace)")
+    out = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, HGEMM_TABLE=str(path), PYTHONPATH=ROOT), capture_output=True, text=True,
+                         check=True).stdout.strip().split("\n")
+    assert out[0].split() == ["1", "256", "6", "1", "0", "2", "2", "9", "0", "0"]
+    assert out[1].split() == ["1", "512", "4", "1", "0", "0", "0", "12", "1", "1"]
+    assert out[2].split() == ["3", "64", "3", "4", "1", "0", "0", "1", "0", "0"]             # the merged row replaced the first one
