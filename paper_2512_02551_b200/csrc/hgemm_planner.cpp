@@ -385,7 +385,7 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
     auto add = [&](const hgemm_config_t &c) {
         if (validate(M, N, K, c) == HGEMM_OK) all.emplace_back(estimate_cycles(M, N, K, num_sms, c), c);
     };
-    {
+    if (double(M) * double(N) * double(K) <= 2147483648.0) {        // the register-accumulator kernel: small problems only
         hgemm_config_t c;
         std::memset(&c, 0, sizeof(c));
         c.family = HGEMM_FAMILY_SMALL;
@@ -446,6 +446,13 @@ int32_t ranked_candidates(int64_t M, int64_t N, int64_t K, int32_t num_sms, hgem
                             if (c.stages < 1) continue;
                             c.raster_group = light ? 1 : raster_group_for(Mk, num_sms, c);
                             add(c);
+                            if (split == 1 && !swap && !light && epi != HGEMM_EPILOGUE_TMA_WIDE && (tiles % units) != 0) {
+                                // the tiles beyond the full waves as a stream-K tail (where the layout applies to this shape)
+                                hgemm_config_t t = c;
+                                t.tail_split = 2;
+                                t.tail_mode = HGEMM_TAIL_STREAM;
+                                if (split_layout(M, N, K, num_sms, t).stream_units > 0) add(t);
+                            }
                             if (split == 1 && !swap && !light && tiles > units && tail > 0 && tail <= units / 2) {
                                 const int32_t ts = int32_t(std::min<int64_t>(std::min<int64_t>(units / tail, 8), kb));
                                 if (ts >= 2) {
