@@ -214,12 +214,22 @@ hgemm_status_t hgemm_run_scaled(hgemm_plan_t *plan, float alpha, float beta, con
                                 void *stream);
 
 /* The same operation on HOST buffers (paper section 2.3 builds its inputs on the
- * CPU): copies A and B to device staging owned by the plan, runs, copies C back,
- * all enqueued on `stream`.  A_host, B_host, C_host are HOST pointers with the
- * layouts above; with page-locked memory the call is asynchronous and the result
- * is in C_host once the stream has been synchronised, with pageable memory the
- * copies block.  The first call on a plan allocates the staging (cudaMalloc,
- * synchronising): make it outside timed regions.  HGEMM_ERR_ALLOC if that fails. */
+ * CPU): copies A and B to device staging owned by the plan, runs, copies C back.
+ * A_host, B_host, C_host are HOST pointers with the layouts above; with page-locked
+ * memory the call is asynchronous and the result is in C_host once `stream` has been
+ * synchronised (work enqueued on `stream` after the call is ordered after the result
+ * copy); with pageable memory the copies block.
+ * The product runs on `stream`; the two operand copies and the result copy run on two
+ * streams owned by the context, tied to it by events, so that over a sequence of calls
+ * the inbound copies of one call overlap the product and the outbound copy of the calls
+ * before it (PCIe carries both directions at once).  Consequence for the caller: A_host
+ * and B_host are read from the moment of the call on -- NOT after the work queued on
+ * `stream` before it -- so they must be complete when the call is made and stay
+ * untouched until the call's work has finished.  Calls on one plan are ordered among
+ * themselves (its staging is reused).
+ * The first call on a context creates the two streams, the first call on a plan
+ * allocates the staging and three events (cudaMalloc, synchronising): make it outside
+ * timed regions.  HGEMM_ERR_ALLOC if the allocation fails. */
 hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void *B_host, void *C_host, void *stream);
 
 /* Split-K GEMM for callers that must not allocate.  (The paper has no counterpart:

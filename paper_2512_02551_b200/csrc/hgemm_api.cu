@@ -36,6 +36,9 @@ struct hgemm_ctx_s {
     bool dependent_launch = true;
     bool tma_3d = true;
     std::vector<hgemm_plan_s *> plans;
+    // hgemm_run_host: the operand copies and the result copy run on streams of their own (created by its first call), so that
+    // one call's copies overlap the compute and the opposite-direction copy of the calls around it
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
 };
 
 struct hgemm_plan_s {
@@ -71,6 +74,9 @@ struct hgemm_plan_s {
     int maps_used = 0, maps_next = 0;
     // device staging of hgemm_run_host (allocated by its first call)
     void *stage_a = nullptr, *stage_b = nullptr, *stage_c = nullptr;
+    // ... and its hand-offs: operands on the device / product computed / result on the host (of the plan's latest call)
+    cudaEvent_t ev_in = nullptr, ev_gemm = nullptr, ev_out = nullptr;
+    bool host_call_in_flight = false;   // the events above have been recorded at least once
 };
 
 namespace {
@@ -515,6 +521,9 @@ hgemm_status_t hgemm_plan_destroy(hgemm_plan_t *plan)
     if (plan->stage_a) cudaFree(plan->stage_a);
     if (plan->stage_b) cudaFree(plan->stage_b);
     if (plan->stage_c) cudaFree(plan->stage_c);
+    if (plan->ev_in) cudaEventDestroy(plan->ev_in);
+    if (plan->ev_gemm) cudaEventDestroy(plan->ev_gemm);
+    if (plan->ev_out) cudaEventDestroy(plan->ev_out);
     delete plan;
     return HGEMM_OK;
 }
@@ -524,6 +533,8 @@ hgemm_status_t hgemm_destroy(hgemm_ctx_t *ctx)
     if (!ctx) return HGEMM_ERR_INVALID_ARG;
     while (!ctx->plans.empty()) hgemm_plan_destroy(ctx->plans.back());
     if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     delete ctx;
     return HGEMM_OK;
 }
@@ -948,8 +959,18 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
     hgemm_ctx_s *ctx = plan->ctx;
     const size_t a_bytes = size_t(plan->M) * size_t(plan->K_user) * 2, b_bytes = size_t(plan->N) * size_t(plan->K_user) * 2,
                  c_bytes = size_t(plan->M) * size_t(plan->N) * 2;
+    cudaError_t e = cudaSuccess;
+    if (!ctx->copy_in) {
+        e = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking);
+        if (e != cudaSuccess) {
+            if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+            ctx->copy_in = ctx->copy_out = nullptr;
+            return cuda_fail(ctx, e);
+        }
+    }
     if (!plan->stage_a) {
-        cudaError_t e = ctx_malloc(ctx, &plan->stage_a, a_bytes);
+        e = ctx_malloc(ctx, &plan->stage_a, a_bytes);
         if (e == cudaSuccess) e = ctx_malloc(ctx, &plan->stage_b, b_bytes);
         if (e == cudaSuccess) e = ctx_malloc(ctx, &plan->stage_c, c_bytes);
         if (e != cudaSuccess) {
@@ -960,15 +981,38 @@ hgemm_status_t hgemm_run_host(hgemm_plan_t *plan, const void *A_host, const void
             return HGEMM_ERR_ALLOC;
         }
     }
+    if (!plan->ev_in) {
+        e = cudaEventCreateWithFlags(&plan->ev_in, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->ev_gemm, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&plan->ev_out, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(plan->stage_a, A_host, a_bytes, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = cudaMemcpyAsync(plan->stage_b, B_host, b_bytes, cudaMemcpyHostToDevice, st);
+    // operands: host -> staging on the inbound copy stream, as soon as the staging is free (the plan's previous product has
+    // been computed from it); they do not queue behind the caller's stream
+    if (plan->host_call_in_flight) {
+        e = cudaStreamWaitEvent(ctx->copy_in, plan->ev_gemm, 0);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    e = cudaMemcpyAsync(plan->stage_a, A_host, a_bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(plan->stage_b, B_host, b_bytes, cudaMemcpyHostToDevice, ctx->copy_in);
+    if (e == cudaSuccess) e = cudaEventRecord(plan->ev_in, ctx->copy_in);
+    // the product: on the caller's stream, once the operands are there and the staging of C is free (the plan's previous
+    // result has left it)
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, plan->ev_in, 0);
+    if (e == cudaSuccess && plan->host_call_in_flight) e = cudaStreamWaitEvent(st, plan->ev_out, 0);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     const hgemm_status_t s = hgemm_run(plan, plan->stage_a, plan->stage_b, plan->stage_c, stream);
     if (s != HGEMM_OK) return s;
-    e = cudaMemcpyAsync(C_host, plan->stage_c, c_bytes, cudaMemcpyDeviceToHost, st);
+    e = cudaEventRecord(plan->ev_gemm, st);
+    // the result: staging -> host on the outbound copy stream; the caller's stream then waits for it, so whatever the caller
+    // enqueues next -- and a synchronisation of the stream -- comes after C_host is complete
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, plan->ev_gemm, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(C_host, plan->stage_c, c_bytes, cudaMemcpyDeviceToHost, ctx->copy_out);
+    if (e == cudaSuccess) e = cudaEventRecord(plan->ev_out, ctx->copy_out);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, plan->ev_out, 0);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+    plan->host_call_in_flight = true;
     return HGEMM_OK;
 }
 

@@ -247,3 +247,68 @@ def test_checked_build_finds_nothing_in_the_parity_cases():
                                   "double_accumulator or split_k_is_deterministic or nn_layout or scaled_form or serpentine"], 1500)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-1000:]
     assert " passed" in r.stdout and "failed" not in r.stdout
+
+
+# ---- hgemm_run_host: host buffers, copies on the context's own streams ------------------------------------------------
+
+def test_run_host_sequences(ctx, gu):
+    """hgemm_run_host over sequences of calls: several plans in a row on one stream, the same plan twice without a
+    synchronisation in between (its staging is reused: the calls must stay ordered), a side stream, new host data after
+    a synchronisation, pageable memory -- every result equal to the device-resident run, bit for bit."""
+    import oracle
+    shapes = [(512, 384, 256), (1024, 1024, 512), (96, 200, 72), (2048, 512, 1024)]
+    plans, host, want = [], [], []
+    for i, (M, N, K) in enumerate(shapes):
+        A, B = inputs.make_ab(M, N, K, "int5" if i % 2 == 0 else "uniform", "cuda")
+        plan = ctx.plan(M, N, K)
+        C = torch.empty(M, N, dtype=torch.float16, device="cuda")
+        plan.run(A, B, C)
+        torch.cuda.synchronize()
+        plans.append(plan)
+        want.append(C.cpu())
+        host.append((A.cpu().pin_memory(), B.cpu().pin_memory(), torch.zeros(M, N, dtype=torch.float16).pin_memory()))
+    s = torch.cuda.current_stream().cuda_stream
+    for rep in range(3):                                           # the second and third pass reuse every plan's staging
+        for hA, hB, hC in host:
+            hC.zero_()
+        for plan, (hA, hB, hC) in zip(plans, host):
+            plan.run_host(hA, hB, hC, s)
+        torch.cuda.synchronize()
+        for (hA, hB, hC), w in zip(host, want):
+            assert torch.equal(hC, w), f"pass {rep}"
+    gu.assert_exact(host[0][2].cuda(), oracle.hgemm_full(inputs.bits(host[0][0].cuda()), inputs.bits(host[0][1].cuda())), "run_host, integers")
+    # the same plan twice in a row with different host buffers, no synchronisation in between
+    M, N, K = shapes[1]
+    A2, B2 = inputs.make_ab(M, N, K, "int5", "cuda")
+    C2 = torch.empty(M, N, dtype=torch.float16, device="cuda")
+    plans[1].run(A2, B2, C2)
+    torch.cuda.synchronize()
+    hA2, hB2, hC2 = A2.cpu().pin_memory(), B2.cpu().pin_memory(), torch.zeros(M, N, dtype=torch.float16).pin_memory()
+    host[1][2].zero_()
+    plans[1].run_host(host[1][0], host[1][1], host[1][2], s)
+    plans[1].run_host(hA2, hB2, hC2, s)
+    plans[1].run_host(host[1][0], host[1][1], host[1][2], s)
+    torch.cuda.synchronize()
+    assert torch.equal(hC2, C2.cpu()) and torch.equal(host[1][2], want[1])
+    # a side stream; work enqueued on it after the call sees the finished result copy
+    side = torch.cuda.Stream()
+    host[3][2].zero_()
+    with torch.cuda.stream(side):
+        plans[3].run_host(host[3][0], host[3][1], host[3][2], side.cuda_stream)
+    side.synchronize()
+    assert torch.equal(host[3][2], want[3])
+    # new host data after a synchronisation; pageable memory (blocking copies)
+    hA, hB, hC = host[2]
+    A3, B3 = inputs.make_ab(*shapes[2], "int5", "cuda")
+    hA.copy_(A3.cpu())
+    hB.copy_(B3.cpu())
+    plans[2].run_host(hA, hB, hC, s)
+    torch.cuda.synchronize()
+    assert torch.equal(hC.float(), (A3.float() @ B3.float().T).cpu())
+    pA, pB, pC = A3.cpu(), B3.cpu(), torch.zeros(shapes[2][0], shapes[2][1], dtype=torch.float16)
+    plans[2].run_host(pA, pB, pC, s)
+    torch.cuda.synchronize()
+    assert torch.equal(pC, hC)
+    assert ctx.last_device_status() == (hgemm.OK, 0)
+    for plan in plans:
+        plan.close()
