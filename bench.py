@@ -212,10 +212,13 @@ def run_ours(args) -> None:
         work.append({"S": S, "plan": ctx.plan(S, S, S), "bufs": bufs})
     step_flops = sum(flops(S, S, S) for S in SWEEP)
 
-    def one_step(i, events=None):
+    # Inside the timed region only the dominant launch (the largest shape) is bracketed by events -- its duration is what the
+    # roofline figure is computed from; events around every launch would put a record between each pair of kernels, which is
+    # instrumentation, not workload.  The other shapes' durations come from a separate pass (`every=True`) after the timed one.
+    def one_step(i, events=None, every=False):
         for w in work:
             A, B, C = w["bufs"][i % len(w["bufs"])]
-            if events is not None:
+            if events is not None and (every or w["S"] == SWEEP[-1]):
                 e0 = torch.cuda.Event(enable_timing=True)
                 e1 = torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
@@ -225,10 +228,10 @@ def run_ours(args) -> None:
             else:
                 w["plan"].run_ptr(A.data_ptr(), B.data_ptr(), C.data_ptr(), stream.cuda_stream)
 
-    def torch_step(i, events=None):
+    def torch_step(i, events=None, every=False):
         for w in work:
             A, B, C = w["bufs"][i % len(w["bufs"])]
-            if events is not None:
+            if events is not None and (every or w["S"] == SWEEP[-1]):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
                 torch.matmul(A, B.T, out=C)
@@ -267,8 +270,15 @@ def run_ours(args) -> None:
     ms_per_step = ms_total / args.steps
     value = replicas.job_throughput(step_flops, world, ms_per_step) / 1e12
     per_launch = {}
-    for S, e0, e1 in events[-4 * args.steps:]:
+    for S, e0, e1 in events[-args.steps:]:                       # the dominant launch, inside the timed region
         per_launch.setdefault(S, []).append(e0.elapsed_time(e1))
+    side_events = []                                             # every shape, in a pass of its own (not part of `value`)
+    for i in range(min(args.steps, 50)):
+        one_step(args.warmup + args.steps + i, side_events, every=True)
+    torch.cuda.synchronize()
+    for S, e0, e1 in side_events:
+        if S != SWEEP[-1]:
+            per_launch.setdefault(S, []).append(e0.elapsed_time(e1))
     per_shape = {}
     for S, v in per_launch.items():
         ms = statistics.mean(v)
@@ -308,8 +318,12 @@ def run_ours(args) -> None:
         e1.record(stream)
         torch.cuda.synchronize()
         tms = e0.elapsed_time(e1) / args.steps
+        tside = []
+        for i in range(min(args.steps, 50)):
+            torch_step(args.warmup + args.steps + i, tside, every=True)
+        torch.cuda.synchronize()
         tps = {}
-        for S, a, b in tev:
+        for S, a, b in tev + [t for t in tside if t[0] != SWEEP[-1]]:
             tps.setdefault(S, []).append(a.elapsed_time(b))
         torch_cmp = {"value": step_flops / (tms * 1e-3) / 1e12, "unit": "TFLOP/s",
                      "per_shape_tflops": {str(S): flops(S, S, S) / (statistics.mean(v) * 1e-3) / 1e12 for S, v in tps.items()}}
@@ -407,6 +421,8 @@ def run_ours(args) -> None:
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "accumulate": "f32", "inputs": "uniform[-1,1) rounded to fp16, seeded per shape",
                        "l2": "inputs larger than L2: buffer sets rotate so that each shape's footprint exceeds 2x the 126 MB L2",
+                       "events": "inside the timed region only the dominant launch (8192^3) is bracketed by CUDA events; the other shapes' "
+                                 "durations in per_shape come from a separate pass after it; torch.matmul is timed the same way",
                        "parallelism": "replicas" if world > 1 else "single GPU"},
             "pct_of_spec_peak": 100.0 * value / world / SPEC_TFLOPS,
             "variants": variants, "skinny": skinny, "grid": grid, "torch_matmul": torch_cmp, "sustained": sustained,
